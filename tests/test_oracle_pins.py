@@ -1,0 +1,330 @@
+"""Pins for the CPU oracle: each part is checked against something other than itself
+(facts fixed by Eq. 1 / Eq. 2 / Eq. 3 / Eq. 4, brute force, closed forms, library
+autograd).  These run without a GPU."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mrem_oracle as O
+from paper_2109_15082_b200 import synth
+from tests import torch_ste_ref as R
+
+
+# ----------------------------------------------------------------------------- Eq. 1 quantizer
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_code_range_is_omega_b(bits):
+    # Omega(b) = {-2^(b-1)+1 .. 2^(b-1)-1}: the most negative two's-complement code never appears
+    x = synth.normal(1, "rng", (20000,), 3.0)
+    q, _ = O.quantize_sym(x, np.float32(0.01), bits)
+    qmax = 2 ** (bits - 1) - 1
+    assert q.min() == -qmax and q.max() == qmax
+    assert set(np.unique(q)).issubset(set(range(-qmax, qmax + 1)))
+
+
+def test_omega_2_is_ternary_and_printed_ranges():
+    assert O.sym_qmax(2) == 1 and O.sym_qmax(4) == 7 and O.sym_qmax(8) == 127
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_grid_points_ties_and_error_bound(bits):
+    s = np.float32(0.125)                          # power of two: x = s*k is exact
+    qmax = 2 ** (bits - 1) - 1
+    k = np.arange(-qmax - 3, qmax + 4)
+    q, _ = O.quantize_sym((s * k).astype(np.float32), s, bits)
+    assert np.array_equal(q, np.clip(k, -qmax, qmax))            # grid points map to themselves, then clip
+    halves = np.array([0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5], np.float32) * s
+    q, _ = O.quantize_sym(halves, s, bits)
+    assert q.tolist() == [0, 2, 2, 0, -2, -2, 4]                 # closest integer, ties to even
+    x = synth.normal(2, "err", (5000,), 0.3)
+    q, z = O.quantize_sym(x, s, bits)
+    inside = np.abs(x / s) <= qmax
+    assert np.all(np.abs(s * q - x)[inside] <= s / 2 + 1e-7)     # closest integer => |x_hat - x| <= s/2
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_idempotence(bits):
+    x = synth.normal(3, "idem", (4096,), 1.0)
+    s = np.float32(0.037)
+    q1, _ = O.quantize_sym(x, s, bits)
+    q2, _ = O.quantize_sym((s * q1).astype(np.float32), s, bits)
+    assert np.array_equal(q1, q2)
+    qa, _ = O.quantize_asym(np.abs(x), s, np.float32(-0.17), 8)
+    xa = (s * qa.astype(np.float32) + np.float32(-0.17)).astype(np.float32)
+    qb, _ = O.quantize_asym(xa, s, np.float32(-0.17), 8)
+    assert np.array_equal(qa, qb) and qa.min() >= 0 and qa.max() <= 255
+
+
+def test_half_integer_2bit_grid_is_nearest_level():
+    s = np.float32(0.25)
+    x = synth.normal(4, "w2", (4000,), 0.4)
+    c, scale, _ = O.quantize_weight(x.reshape(1, -1), np.array([[s]], np.float32), 2, 1)
+    what = (scale * c).reshape(-1)
+    levels = np.array([-1.5, -0.5, 0.5, 1.5]) * s
+    nearest = levels[np.abs(x[:, None].astype(np.float64) - levels[None, :]).argmin(1)]
+    assert set(np.unique(c)) == {-3, -1, 1, 3}
+    assert np.allclose(what, nearest)
+
+
+def test_initial_weight_steps_clip_nothing():
+    wl = synth.workloads()["tiny"]
+    params = synth.teacher_params(wl, 0)
+    desc = O.ModuleDesc(1, wl.hidden, wl.n_heads, wl.ffn, 4, 8)
+    s = O.init_weight_steps(desc, params, 0)[0]
+    for k in O.WEIGHTS:
+        q, _, z = O.quantize_weight(params[0][k], s[k].reshape(-1, 1), 4, 0)
+        assert np.all(np.abs(q).max(-1) == 7)                    # each row's largest weight gets code +-7
+        assert np.all(np.abs(z) <= 7 * (1 + 1e-6))               # and nothing is clipped
+
+
+# ----------------------------------------------------------------------------- integer products, Eq. 2
+
+def test_int_matmul_brute_force():
+    rng = np.random.default_rng(0)
+    qa = rng.integers(-127, 128, (5, 19))
+    qw = rng.integers(-7, 8, (7, 19))
+    ref = [[sum(int(qa[m, k]) * int(qw[n, k]) for k in range(19)) for n in range(7)] for m in range(5)]
+    assert O.int_matmul(qa, qw).tolist() == ref
+
+
+@pytest.mark.parametrize("asym", [False, True])
+def test_student_linear_is_quantized_product_of_eq2(asym):
+    # y = w_hat^T a_hat (+ bias): integer accumulate + scales must equal the float product
+    x = np.abs(synth.normal(5, "a", (6, 24), 1.0)) if asym else synth.normal(5, "a", (6, 24), 1.0)
+    w = synth.normal(5, "w", (10, 24), 0.02)
+    b = synth.normal(5, "b", (10,), 0.1).astype(np.float64)
+    desc = O.ModuleDesc(1, 24, 1, 10, 4, 8, act_dtype="f32", asym_g=asym)
+    sw = O.init_weight_steps(desc, [dict(Wqkv=w, Wo=w, W1=w, W2=w)])[0]["W1"]
+    steps = dict(a=np.full(8, 0.02, np.float32), a_off=np.full(8, 0.11, np.float32))
+    qa = O._q_act(desc, x, steps, O.SITE_G if asym else O.SITE_A)
+    qw = O._q_w(desc, w, sw)
+    y = O.student_linear(qa, qw, b)
+    assert np.allclose(y, qa["xhat"] @ qw["what"].T + b, rtol=1e-12, atol=1e-12)
+    if asym:
+        assert qa["beta"] != 0.0 and qa["q"].min() >= 0
+
+
+# ----------------------------------------------------------------------------- module vs library autograd
+
+def _tiny(n_layers=2, H=16, h=2, Fd=32, B=2, S=5, seed=0, **kw):
+    wl = synth.Workload("pin", n_layers, H, h, Fd, S, B, act_dtype="f64", outlier_channels=0)
+    params = synth.teacher_params(wl, seed, bias_std=0.1)
+    for p in params:                                   # larger weights: every term matters
+        for k in O.WEIGHTS:
+            p[k] = (p[k] * 10).astype(np.float32)
+    x = synth.hidden_states(wl, B, seed)
+    desc = O.ModuleDesc(n_layers, H, h, Fd, act_dtype="f64", **kw)
+    return wl, desc, params, x
+
+
+def _to_torch(params, steps):
+    tp = [{k: torch.tensor(np.asarray(v, np.float64), requires_grad=True) for k, v in p.items()} for p in params]
+    ts = [dict(w={k: torch.tensor(np.asarray(s["w"][k], np.float64), requires_grad=True) for k in O.WEIGHTS},
+               a=torch.tensor(np.asarray(s["a"], np.float64), requires_grad=True),
+               a_off=torch.tensor(np.asarray(s["a_off"], np.float64), requires_grad=True)) for s in steps]
+    return tp, ts
+
+
+def _cfg(desc):
+    return dict(n_heads=desc.n_heads, a_bits=desc.a_bits, w_bits=desc.w_bits, w_grid=desc.w_grid,
+                asym_p=desc.asym_p, asym_g=desc.asym_g, ln_eps=desc.ln_eps)
+
+
+def test_unquantized_module_matches_torch_layers():
+    wl, desc, params, x = _tiny(w_bits=0, a_bits=0)
+    vl = np.array([5, 3], np.int32)
+    outs = O.teacher_forward(desc, params, x, vl)
+    tp, _ = _to_torch(params, [])
+    ref = R.module(torch.tensor(x, dtype=torch.float64), tp, [None] * len(tp), _cfg(desc), vl, quant=False)
+    for a, b in zip(outs, ref):
+        assert np.allclose(a, b.detach().numpy(), rtol=1e-10, atol=1e-12)
+
+
+CASES = [dict(w_bits=4, a_bits=8), dict(w_bits=2, a_bits=8, w_grid=1), dict(w_bits=2, a_bits=8, w_grid=0),
+         dict(w_bits=4, a_bits=8, w_per_row=False), dict(w_bits=4, a_bits=8, asym_p=False, asym_g=False),
+         dict(w_bits=4, a_bits=4)]
+
+
+@pytest.mark.parametrize("kw", CASES)
+@pytest.mark.parametrize("loss_mean", [True, False])
+def test_ste_forward_backward_matches_torch_autograd(kw, loss_mean):
+    wl, desc, params, x = _tiny(loss_mean=loss_mean, **kw)
+    vl = np.array([4, 5], np.int32)
+    teacher = [{k: v.copy() for k, v in p.items()} for p in params]
+    student = [{k: (v + synth.normal(7, k + str(i), v.shape, 0.01)).astype(np.float32) for k, v in p.items()}
+               for i, p in enumerate(params)]
+    rule = 1 if desc.w_bits == 2 else 0
+    ws = O.init_weight_steps(desc, student, rule)
+    if not desc.w_per_row:
+        ws = [{k: v.reshape(1) for k, v in d.items()} for d in ws]
+    a, off = O.init_act_steps(desc, student, x, vl)
+    a = (a * 0.8).astype(np.float32)                    # shrink: some activations clip, masks matter
+    steps = O.make_steps(ws, a, off)
+    x_t = x + synth.normal(8, "xt", x.shape, 0.05)
+    r = O.forward_loss_backward(desc, teacher, student, steps, x_t, x, vl, lam=0.3)
+
+    tp, ts = _to_torch(student, steps)
+    tt, _ = _to_torch(teacher, [])
+    xs = torch.tensor(x, dtype=torch.float64)
+    xt = torch.tensor(x_t, dtype=torch.float64)
+    f_t = R.module(xt, tt, [None] * len(tt), _cfg(desc), vl, quant=False)
+    f_s = R.module(0.3 * xt + 0.7 * xs, tp, ts, _cfg(desc), vl, quant=True)
+    c = 1.0 / f_s[0].numel() if loss_mean else 1.0
+    loss = sum(c * ((a_ - b_.detach()) ** 2).sum() for a_, b_ in zip(f_s, f_t))
+    loss.backward()
+
+    for a_, b_ in zip(r["f_s"], f_s):
+        assert np.allclose(a_, b_.detach().numpy(), rtol=1e-9, atol=1e-11)
+    assert np.isclose(r["loss"], loss.item(), rtol=1e-10)
+    clipped = 0
+    for l, g in enumerate(r["grads"]):
+        for k in O.PARAMS:
+            ref = tp[l][k].grad.numpy()
+            assert np.allclose(g[k], ref, rtol=1e-7, atol=1e-9 * np.abs(ref).max()), (l, k)
+        for k in O.WEIGHTS:
+            ref = ts[l]["w"][k].grad.numpy()
+            assert np.allclose(g["w"][k], ref, rtol=1e-7, atol=1e-9 * np.abs(ref).max()), (l, "s", k)
+        ref = ts[l]["a"].grad.numpy()
+        assert np.allclose(g["a"], ref, rtol=1e-7, atol=1e-9 * np.abs(ref).max()), (l, "a")
+        if desc.asym_g:
+            ref = ts[l]["a_off"].grad.numpy()
+            assert np.allclose(g["a_off"][O.SITE_G], ref[O.SITE_G], rtol=1e-7, atol=1e-12), (l, "a_off")
+        else:
+            assert g["a_off"][O.SITE_G] == 0.0
+        clipped += int((np.abs(r["caches"][l]["qx"]["z"]) > r["caches"][l]["qx"]["hi"]).sum())
+    assert clipped > 0                                   # the case really exercises the clip masks
+
+
+def test_bypass_gives_zero_loss_and_zero_grads():
+    wl, desc, params, x = _tiny(w_bits=0, a_bits=0)
+    steps = O.make_steps([{k: np.ones(1) for k in O.WEIGHTS}] * 2, np.ones((2, 8)), np.zeros((2, 8)))
+    r = O.forward_loss_backward(desc, params, params, steps, x, x)
+    assert r["loss"] == 0.0
+    assert all(np.all(g[k] == 0) for g in r["grads"] for k in O.PARAMS)
+
+
+def test_high_bit_width_gives_vanishing_error_and_4x_per_bit():
+    wl, desc, params, x = _tiny(n_layers=1, H=32, Fd=64, B=4, S=8)
+    losses = {}
+    for bits in (4, 5, 6, 7, 8, 16):
+        d = O.ModuleDesc(1, 32, 2, 64, bits, bits, act_dtype="f64")
+        ws = O.init_weight_steps(d, params, 0)
+        a, off = O.init_act_steps(d, params, x)
+        r = O.forward_loss_backward(d, params, params, O.make_steps(ws, a, off), x, x)
+        losses[bits] = r["loss"]
+    norm = float((r["f_t"][0] ** 2).mean())
+    assert losses[16] < 1e-6 * norm
+    vals = [losses[b] for b in (4, 5, 6, 7, 8)]
+    assert all(a > b for a, b in zip(vals, vals[1:]))            # monotone in the bit width
+    ratios = [a / b for a, b in zip(vals, vals[1:])]
+    assert all(2.0 < r_ < 8.0 for r_ in ratios), ratios          # ~4x per bit (uniform-noise model)
+
+
+# ----------------------------------------------------------------------------- finite differences
+
+def test_unquantized_backward_matches_central_differences():
+    wl, desc, params, x = _tiny(n_layers=1, H=8, h=2, Fd=12, B=2, S=3, w_bits=0, a_bits=0)
+    teacher = [{k: (v + synth.normal(9, k, v.shape, 0.05)).astype(np.float32) for k, v in params[0].items()}]
+    steps = O.make_steps([{k: np.ones(1) for k in O.WEIGHTS}], np.ones((1, 8)), np.zeros((1, 8)))
+    student = [{k: v.astype(np.float64) for k, v in params[0].items()}]
+    g = O.forward_loss_backward(desc, teacher, student, steps, x, x)["grads"][0]
+    for k in O.PARAMS:
+        flat = student[0][k].reshape(-1)
+        for i in range(0, flat.size, max(1, flat.size // 5)):
+            old = flat[i]
+            flat[i] = old + 1e-5
+            lp = O.forward_loss_backward(desc, teacher, student, steps, x, x)["loss"]
+            flat[i] = old - 1e-5
+            lm = O.forward_loss_backward(desc, teacher, student, steps, x, x)["loss"]
+            flat[i] = old
+            fd = (lp - lm) / 2e-5
+            assert np.isclose(g[k].reshape(-1)[i], fd, rtol=2e-5, atol=1e-9), (k, i)
+
+
+def test_single_linear_ste_matches_surrogate_differences():
+    # REM special case (Eq. 2): one product.  Hold the rounding residual r = q - z and the clip
+    # masks fixed; the surrogate x_hat(x, s) = x + s*r (inside) | s*q (clipped) is smooth, and
+    # the STE gradient is its exact gradient.
+    x = synth.normal(10, "x", (7, 12), 1.0).astype(np.float64)
+    w = synth.normal(10, "w", (5, 12), 0.3).astype(np.float64)
+    tgt = synth.normal(10, "t", (7, 5), 1.0).astype(np.float64)
+    sa, sw = 0.012, np.full((5, 1), 0.06)
+    qa, za = O.quantize_sym(x, sa, 8, "f64")
+    qw, _, zw = O.quantize_weight(w, sw, 4, 0, "f64")
+    ia, iw = (np.abs(za) <= 127), (np.abs(zw) <= 7)
+    ra, rw = qa - za, qw - zw
+    assert (~ia).sum() > 0 and (~iw).sum() > 0
+
+    def loss(x_, w_, sa_, sw_):
+        xh = np.where(ia, x_ + sa_ * ra, sa_ * qa)
+        wh = np.where(iw, w_ + sw_ * rw, sw_ * qw)
+        return float(((xh @ wh.T - tgt) ** 2).sum())
+
+    dy = 2 * ((sa * qa) @ (sw * qw).T - tgt)
+    dwhat = dy.T @ (sa * qa)
+    dxhat = dy @ (sw * qw)
+    ins_w, dw_ds = O.weight_ste(zw, qw, 4, 0)
+    ins_a, da_ds = O.act_ste(za, qa, -127, 127)
+    e = 1e-6
+    assert np.isclose((dxhat * da_ds).sum(), (loss(x, w, sa + e, sw) - loss(x, w, sa - e, sw)) / (2 * e), rtol=1e-6)
+    for n in range(5):
+        d = np.zeros((5, 1)); d[n] = e
+        fd = (loss(x, w, sa, sw + d) - loss(x, w, sa, sw - d)) / (2 * e)
+        assert np.isclose((dwhat * dw_ds).sum(-1)[n], fd, rtol=1e-6)
+    for (i, j) in itertools.product(range(0, 5, 2), range(0, 12, 5)):
+        d = np.zeros_like(w); d[i, j] = e
+        fd = (loss(x, w + d, sa, sw) - loss(x, w - d, sa, sw)) / (2 * e)
+        assert np.isclose((dwhat * ins_w)[i, j], fd, rtol=1e-6, atol=1e-9)
+
+
+# ----------------------------------------------------------------------------- Eq. 4, AdamW, storage
+
+def test_teacher_forcing_mix_endpoints():
+    f = synth.normal(11, "f", (3, 4), 1.0)
+    fh = synth.normal(11, "fh", (3, 4), 1.0)
+    assert np.array_equal(O.teacher_forcing_mix(f, fh, 1.0), f.astype(np.float64))
+    assert np.array_equal(O.teacher_forcing_mix(f, fh, 0.0), fh.astype(np.float64))
+    assert O.teacher_forcing_lambda(0, 10) == 1.0 and O.teacher_forcing_lambda(5, 10) == 0.5
+    assert O.teacher_forcing_lambda(12, 10) == 0.0
+
+
+def test_adamw_first_step_closed_form_and_library():
+    p0 = synth.normal(12, "p", (50,), 1.0).astype(np.float64)
+    g = synth.normal(12, "g", (50,), 0.3).astype(np.float64)
+    lr, wd, eps = 1e-2, 0.1, 1e-8
+    p1, m, v = O.adamw_update(p0, g, 0 * p0, 0 * p0, 1, lr, 0.9, 0.999, eps, wd)
+    assert np.allclose(p1, p0 * (1 - lr * wd) - lr * g / (np.abs(g) + eps), rtol=1e-12)
+    tp = torch.tensor(p0.copy(), requires_grad=True)
+    opt = torch.optim.AdamW([tp], lr=lr, betas=(0.9, 0.999), eps=eps, weight_decay=wd)
+    p, m, v = p0, 0 * p0, 0 * p0
+    for t in range(1, 4):
+        gt = g * t
+        tp.grad = torch.tensor(gt.copy())
+        opt.step()
+        p, m, v = O.adamw_update(p, gt, m, v, t, lr, 0.9, 0.999, eps, wd)
+        assert np.allclose(p, tp.detach().numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_bf16_rounding_matches_library_conversion():
+    x = np.concatenate([synth.normal(13, "r", (20000,), 3.0),
+                        np.array([1.00390625, 1.01171875, -1.00390625, 0.0], np.float32)])
+    ref = torch.tensor(x).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(O.round_bf16(x), ref)
+
+
+def test_recon_step_reduces_loss_on_repeated_batch():
+    # qualitative fact of the paper's training-loss curves: the reconstruction loss goes down
+    wl = synth.workloads()["tiny"]
+    wl = synth.shrink(wl, hidden=32, ffn=64, seq=8, batch=4)
+    params = synth.teacher_params(wl, 0)
+    x = synth.hidden_states(wl, 4, 0)
+    desc = O.ModuleDesc(1, 32, 2, 64, 4, 8, act_dtype="f32")
+    student = [{k: v.copy() for k, v in params[0].items()}]
+    ws = O.init_weight_steps(desc, student, 0)
+    a, off = O.init_act_steps(desc, student, x)
+    steps, state, losses = O.make_steps(ws, a, off), {}, []
+    for t in range(40):
+        losses.append(O.recon_step(desc, params, student, steps, state, x, x, lr=3e-5)["loss"])
+    assert np.mean(losses[-5:]) < 0.7 * losses[0]
