@@ -1,0 +1,222 @@
+/*
+ * libmrem — the reconstruction step of module-wise reconstruction error minimization
+ * (MREM) for post-training quantization of BERT-style encoders, on one B200 (sm_100a).
+ *
+ * One step (Algorithm 2 of the paper): a full-precision teacher module (a block of
+ * encoder layers) and its fake-quantized student run on the same calibration batch; the
+ * squared error between their layer outputs (Eq. 3) is back-propagated through the
+ * quantizers (Eq. 1) with the straight-through estimator; AdamW updates the latent
+ * weights and the quantization step sizes.
+ *
+ * Conventions
+ *  - Every function returns an int32 status: 0 = MREM_OK, negative = error.  No exceptions,
+ *    no exit, nothing printed.  mrem_last_error() returns text for the last failing call.
+ *  - The library allocates NO device memory.  Tensors, parameters and the workspace are
+ *    caller-owned DEVICE pointers (unless a parameter is named h_*: HOST pointer) that must
+ *    stay valid while the context uses them and be 256-byte aligned.
+ *  - All work is enqueued on the CUDA stream given at creation (a cudaStream_t passed as
+ *    void*); calls do not block unless stated.  Scalars such as the loss are written to
+ *    device addresses given by the caller.
+ *  - Conditions detected on the device (a bounded wait that ran out, a non-finite loss) are
+ *    recorded in a sticky device status word; mrem_poll_status() reads it.
+ *  - A context is not thread-safe; independent contexts are independent.
+ *  - Layouts are row-major.  Activations are [batch, seq, hidden]; a linear layer's weight
+ *    is [out_features, in_features] (so y = x W^T + b).
+ */
+#ifndef MREM_H_
+#define MREM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MREM_OK = 0,
+  MREM_ERR_ARG = -1,          /* null pointer, value out of range */
+  MREM_ERR_ALIGN = -2,        /* pointer or stride not aligned as required */
+  MREM_ERR_SHAPE = -3,        /* batch/seq/hidden combination not supported */
+  MREM_ERR_WORKSPACE = -4,    /* workspace too small */
+  MREM_ERR_ORDER = -5,        /* call made before the calls it depends on */
+  MREM_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed */
+  MREM_ERR_TIMEOUT = -7,      /* device status: a bounded wait ran out */
+  MREM_ERR_NONFINITE = -8,    /* device status: non-finite loss */
+  MREM_ERR_UNSUPPORTED = -9
+};
+
+typedef struct mrem_ctx mrem_ctx;
+
+typedef enum { MREM_TEACHER = 0, MREM_STUDENT = 1 } mrem_role;
+typedef enum { MREM_F32 = 0, MREM_BF16 = 1 } mrem_dtype;
+
+/* Parameter tensors of one encoder layer (post-LayerNorm BERT layout). */
+enum {
+  MREM_WQKV = 0, MREM_BQKV = 1,   /* [3H, H], [3H]: rows 0..H-1 query, H..2H-1 key, 2H..3H-1 value */
+  MREM_WO = 2, MREM_BO = 3,       /* [H, H], [H]   attention output projection */
+  MREM_LN1_G = 4, MREM_LN1_B = 5, /* [H]           LayerNorm after attention + skip */
+  MREM_W1 = 6, MREM_B1 = 7,       /* [F, H], [F]   first FFN layer (GELU follows) */
+  MREM_W2 = 8, MREM_B2 = 9,       /* [H, F], [H]   second FFN layer */
+  MREM_LN2_G = 10, MREM_LN2_B = 11,
+  MREM_N_PARAMS = 12
+};
+
+/* Quantizers of one layer.  0..3: weight steps of Wqkv, Wo, W1, W2 ([rows] or [1]).
+ * 4..11: activation sites in forward order, one step each (a quantizer sits on both
+ * operands of every matrix product, Sec. 3.1): layer input, Q, K, V, softmax output,
+ * attention context, FFN input, GELU output. */
+enum {
+  MREM_Q_WQKV = 0, MREM_Q_WO = 1, MREM_Q_W1 = 2, MREM_Q_W2 = 3,
+  MREM_Q_X = 4, MREM_Q_Q = 5, MREM_Q_K = 6, MREM_Q_V = 7, MREM_Q_P = 8, MREM_Q_C = 9, MREM_Q_A = 10, MREM_Q_G = 11,
+  MREM_N_QUANTIZERS = 12
+};
+/* ids for mrem_get_grad: parameter ids 0..11; MREM_GRAD_STEP + quantizer id;
+ * MREM_GRAD_OFFSET + quantizer id (only the GELU site has a learnable offset). */
+enum { MREM_GRAD_STEP = 100, MREM_GRAD_OFFSET = 200 };
+
+enum { MREM_TRAIN_WEIGHTS = 1, MREM_TRAIN_BIASES = 2, MREM_TRAIN_LAYERNORM = 4, MREM_TRAIN_W_STEPS = 8,
+       MREM_TRAIN_A_STEPS = 16, MREM_TRAIN_ALL = 31 };
+
+typedef struct {
+  uint32_t struct_size;        /* sizeof(mrem_module_desc) */
+  int32_t n_layers, hidden, n_heads, ffn;
+  int32_t max_seq, max_batch;  /* the workspace is sized for max_batch * max_seq tokens */
+  int32_t w_bits;              /* 2, 4 or 8 */
+  int32_t a_bits;              /* 8 or 4 */
+  int32_t w_grid;              /* 0: integer codes Omega(b) of Eq. 1; 1: 2-bit levels {-1.5,-.5,.5,1.5}*step */
+  int32_t w_step_per_row;      /* 1: one step per output row; 0: one per matrix */
+  int32_t act_asym_sites;      /* bit 0: softmax output unsigned (offset 0); bit 1: GELU output unsigned with
+                                  learnable offset (Sec. 3.1: asymmetric for these two) */
+  int32_t act_dtype;           /* mrem_dtype: storage type of activations (bf16: tensor cores; f32: exact path
+                                  for small checks) */
+  int32_t loss_mean;           /* 1: each layer's squared error divided by batch*seq*hidden; 0: plain sum (Eq. 3) */
+  int32_t trainable_mask;      /* MREM_TRAIN_* */
+  float ln_eps;
+} mrem_module_desc;
+
+typedef struct {
+  float lr;                    /* learning rate of this step, or the initial one when decay_total_steps > 0 */
+  float beta1, beta2, eps, weight_decay;   /* decay applies to the four weight matrices only */
+  int32_t step;                /* 1-based step index t for the bias correction; 0: use and advance the
+                                  context's device-side counter */
+  int32_t decay_total_steps;   /* > 0: lr_t = lr * (1 - (t-1)/decay_total_steps), computed on the device (Sec. 5.1:
+                                  linear decay) */
+} mrem_optim;
+
+/* ---- context ------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a context of this shape needs. */
+int32_t mrem_workspace_bytes(const mrem_module_desc* desc, size_t* out_bytes);
+
+/* Creates a context on the current device.  `workspace` (device, 256-byte aligned, at least
+ * mrem_workspace_bytes) holds codes, stashed activations, gradients and optimizer moments;
+ * it is zero-filled here (asynchronously).  Errors: ARG, ALIGN, SHAPE (hidden % n_heads != 0,
+ * head size != 64 for bf16, hidden/ffn not multiples of 16), WORKSPACE, UNSUPPORTED. */
+int32_t mrem_create(const mrem_module_desc* desc, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                    mrem_ctx** out);
+int32_t mrem_destroy(mrem_ctx* ctx);
+/* Text of the last error on this context (or of the last failed mrem_create when ctx is NULL).  Host string
+ * owned by the library. */
+const char* mrem_last_error(const mrem_ctx* ctx);
+
+/* Binds caller-owned parameter storage.  Teacher: matrices in act_dtype, vectors float32, read-only.
+ * Student: all float32 ("latent" full-precision values), updated in place by mrem_step. */
+int32_t mrem_bind_param(mrem_ctx* ctx, int32_t role, int32_t layer, int32_t tensor_id, void* d_ptr, int32_t dtype);
+/* Binds the step size(s) of one quantizer (float32, read-write) and, for MREM_Q_G, its offset
+ * (float32 [1]; may be NULL for other sites). */
+int32_t mrem_bind_steps(mrem_ctx* ctx, int32_t layer, int32_t quantizer_id, float* d_steps, float* d_offset);
+
+/* Copies the teacher's parameters into the student's latent ones; zeroes the optimizer state. */
+int32_t mrem_init_student_from_teacher(mrem_ctx* ctx);
+/* rule 0: step = max|w| / qmax over the group (nothing clipped at the start); rule 1: mean|w| over the group. */
+int32_t mrem_init_weight_steps(mrem_ctx* ctx, int32_t rule);
+/* One unquantized pass of the student over the batch; each site's step = max|x|/qmax (symmetric) or
+ * (max - min)/(2^b - 1) with offset min (GELU site) / max/(2^b-1) with offset 0 (softmax site). */
+int32_t mrem_init_act_steps(mrem_ctx* ctx, const void* d_x, const int32_t* d_valid_len, int32_t batch, int32_t seq);
+
+/* ---- one reconstruction step (Algorithm 2), in this order ------------------------------ */
+
+/* Eq. 1 on every weight matrix of the student: latent weights + steps -> int8 codes, int32 row
+ * sums of the codes, and the dequantized matrices used by the backward products. */
+int32_t mrem_quantize_weights(mrem_ctx* ctx);
+/* Borrowed pointers to the codes [rows, cols] and row sums [rows] of one matrix (valid until destroy). */
+int32_t mrem_get_weight_codes(mrem_ctx* ctx, int32_t layer, int32_t tensor_id, const int8_t** d_codes,
+                              const int32_t** d_rowsum);
+
+/* Runs one module forward.  d_x: [batch, seq, hidden] in act_dtype, this role's own input.
+ * STUDENT with lambda != 0: the input becomes lambda * d_x_other + (1 - lambda) * d_x (Eq. 4, d_x_other =
+ * the teacher-side input); otherwise d_x_other may be NULL.  d_valid_len: [batch] int32 key lengths
+ * (positions >= length are masked out of the attention) or NULL.  d_layer_outputs:
+ * [n_layers, batch, seq, hidden] act_dtype, written; the last slice is the module output.
+ * The student pass needs mrem_quantize_weights first (ERR_ORDER) and keeps d_x and d_layer_outputs
+ * borrowed until mrem_module_backward has run. */
+int32_t mrem_module_forward(mrem_ctx* ctx, int32_t role, const void* d_x, const void* d_x_other, float lambda,
+                            const int32_t* d_valid_len, int32_t batch, int32_t seq, void* d_layer_outputs);
+/* Eq. 3 over the layer outputs of the last teacher and student passes.  Writes the total to
+ * d_loss_total (float32 [1]) and, when non-NULL, each layer's term to d_loss_per_layer
+ * ([n_layers]); stores d loss / d f_hat_l for the backward. */
+int32_t mrem_recon_loss(mrem_ctx* ctx, float* d_loss_total, float* d_loss_per_layer);
+/* Straight-through backward through the student module (gradient local to the module). */
+int32_t mrem_module_backward(mrem_ctx* ctx);
+/* Borrowed pointer to a gradient (float32, same shape as the parameter / step tensor). */
+int32_t mrem_get_grad(mrem_ctx* ctx, int32_t layer, int32_t id, const float** d_grad);
+/* AdamW on everything in trainable_mask, steps clamped to >= 1e-8. */
+int32_t mrem_step(mrem_ctx* ctx, const mrem_optim* optim);
+
+/* The whole step from HOST buffers: copies h_x_teacher / h_x_student ([batch, seq, hidden] act_dtype;
+ * h_x_student may equal h_x_teacher) and h_valid_len (may be NULL) to the device, runs quantize_weights,
+ * both forwards, loss, backward and step, copies the loss back to *h_loss and blocks until it is there. */
+int32_t mrem_recon_step_host(mrem_ctx* ctx, const void* h_x_teacher, const void* h_x_student,
+                             const int32_t* h_valid_len, int32_t batch, int32_t seq, float lambda,
+                             const mrem_optim* optim, float* h_loss);
+
+/* Reads the device status word (blocks on the stream): MREM_OK, MREM_ERR_TIMEOUT or MREM_ERR_NONFINITE in
+ * *h_status; the word is cleared. */
+int32_t mrem_poll_status(mrem_ctx* ctx, int32_t* h_status);
+
+/* Optimizer state (moments of every trainable tensor and the step counter) as one blob. */
+int32_t mrem_state_bytes(mrem_ctx* ctx, size_t* out_bytes);
+int32_t mrem_export_state(mrem_ctx* ctx, void* d_blob, size_t bytes);
+int32_t mrem_import_state(mrem_ctx* ctx, const void* d_blob, size_t bytes);
+
+/* Captures quantize_weights .. step on fixed buffers into a CUDA graph owned by the context and
+ * replays it.  Between replays the caller only rewrites the contents of the input buffers. */
+int32_t mrem_graph_capture_step(mrem_ctx* ctx, const void* d_x_teacher, const void* d_x_student, float lambda,
+                                const int32_t* d_valid_len, int32_t batch, int32_t seq, void* d_teacher_outputs,
+                                void* d_student_outputs, float* d_loss_total, const mrem_optim* optim);
+int32_t mrem_graph_launch(mrem_ctx* ctx);
+
+/* out[i] = src[idx[i]] for i < n_rows (rows of row_bytes bytes, a multiple of 16): draws a batch from a
+ * calibration set resident on the device (Sec. 5.1). */
+int32_t mrem_gather_rows(const void* d_src, const int32_t* d_idx, int32_t n_rows, size_t row_bytes, void* d_out,
+                         void* cuda_stream);
+
+/* ---- single operations (the building blocks above, exposed for verification) ----------- */
+
+/* Eq. 1 on an activation tensor of n elements: z = (x - offset) / step (offset NULL = symmetric),
+ * code = nearest integer (ties to even) of clip(z, lo, hi).  Writes 8-bit codes (d_codes8, may be
+ * NULL) and/or the codes as numbers of type dtype (d_codes_t, may be NULL). */
+int32_t mrem_quantize_act(const void* d_x, int32_t dtype, int64_t n, const float* d_step, const float* d_offset,
+                          int32_t lo, int32_t hi, int8_t* d_codes8, void* d_codes_t, void* cuda_stream);
+/* Eq. 1 on a weight matrix [rows, cols]; outputs as in mrem_quantize_weights (d_what may be NULL). */
+int32_t mrem_quantize_weight(const float* d_w, int32_t rows, int32_t cols, const float* d_steps, int32_t per_row,
+                             int32_t bits, int32_t grid, int8_t* d_codes, int32_t* d_rowsum, float* d_scale,
+                             void* d_what, int32_t dtype, void* cuda_stream);
+/* acc[m, n] = sum_k a[m, k] * b[n, k] in exact int32 on the int8 tensor cores.  a: [M, K] int8 (or uint8
+ * when a_unsigned), b: [N, K] int8, K % 16 == 0, acc: [M, N] int32.  block_n 0 = automatic tile width.
+ * d_status: device int32 receiving a DeviceStatus code on a bounded-wait timeout (0 otherwise). */
+int32_t mrem_gemm_i8(const int8_t* d_a, int32_t a_unsigned, const int8_t* d_b, int32_t M, int32_t N, int32_t K,
+                     int32_t* d_acc, int32_t block_n, int32_t* d_status, void* cuda_stream);
+/* out[b, m, n] = alpha * sum_k A[b, m, k] * B[b, n, k] (float32 out).  dtype BF16: tcgen05 bf16 tensor
+ * cores with fp32 accumulation; F32: CUDA cores.  a_mn / b_mn = 1 when the operand is stored with its
+ * m / n index contiguous (lda/ldb then stride k), 0 when k is contiguous.  Batch strides in elements. */
+int32_t mrem_gemm(int32_t dtype, const void* d_a, int32_t a_mn, int64_t lda, int64_t a_batch_stride, const void* d_b,
+                  int32_t b_mn, int64_t ldb, int64_t b_batch_stride, int32_t M, int32_t N, int32_t K, int32_t batches,
+                  float alpha, float* d_out, int64_t ldc, int64_t c_batch_stride, int32_t block_n, int32_t* d_status,
+                  void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MREM_H_ */

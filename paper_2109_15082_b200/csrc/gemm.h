@@ -1,0 +1,19 @@
+// Internal interface of the two GEMM back ends.
+#pragma once
+#include "mrem_common.cuh"
+
+namespace mrem {
+
+enum GemmRc : int { GEMM_OK = 0, GEMM_ERR_ARG = -1, GEMM_ERR_ALIGN = -2, GEMM_ERR_CUDA = -6 };
+
+// Tensor-core path (tcgen05).  kind 0: bf16 x bf16 -> fp32; kind 1: (u8|s8) x s8 -> int32 (exact).
+// block_n 0 picks the tile width.  Operands need 16-byte aligned bases and strides.
+int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
+            const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream);
+
+// Plain fp32 SIMT path, used when activations are stored in float32 (small correctness
+// configurations); same operand and epilogue conventions, no alignment requirements.
+int simt_gemm_f32(const OperandDesc& A, const OperandDesc& B, const GemmShape& g, const Epilogue& epi,
+                  cudaStream_t stream);
+
+}  // namespace mrem

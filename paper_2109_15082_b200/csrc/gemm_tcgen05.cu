@@ -1,0 +1,513 @@
+// Tensor-core GEMM for sm_100a: C[b][m][n] = epilogue( sum_k A[b][m][k] * B[b][n][k] ).
+//
+// One persistent CTA per SM.  Warp 0 streams operand tiles into a ring of shared-memory
+// stages with TMA (128-byte swizzle), warp 1 issues tcgen05.mma (bf16 -> fp32, or
+// int8 -> int32 with exact accumulation) into one of two TMEM accumulator buffers, and
+// warps 2..5 drain the other buffer with tcgen05.ld, apply the epilogue and write the
+// result, so the epilogue of tile i overlaps the main loop of tile i+1.
+// Either operand may be stored k-contiguous ("K-major") or m/n-contiguous ("MN-major");
+// the second form serves the backward products (dX = dY * W_hat, dW = dY^T * X_hat) and
+// the attention products without any transposed copy.
+//
+// Every wait on an mbarrier is bounded in time; when one runs out the kernel records a
+// code in the status word, stops issuing work, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "gemm.h"
+
+namespace mrem {
+
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
+constexpr int TILE_SMEM_BUDGET = 196608;              // bytes of operand stages per CTA
+constexpr int MAX_STAGES = 8;
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait
+
+struct TcParams {
+  int M, N, K, nb0, nb1;
+  int m_tiles, n_tiles, k_blocks, num_tiles;
+  int block_n, block_k, num_stages, stage_bytes;
+  int a_mn, b_mn;
+  uint32_t idesc;
+  Epilogue epi;
+  int* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when the phase did not complete within WAIT_NS.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > WAIT_NS) return false;
+  }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+template <int KIND>
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  if constexpr (KIND == 0) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(lbo >> 4) << 16;
+  d |= (uint64_t)(sbo >> 4) << 32;
+  d |= 1ull << 46;   // descriptor version of this architecture
+  d |= 2ull << 61;   // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ void fail(const TcParams& p, int code, volatile int* abort_flag) {
+  atomicCAS(p.status, 0, code);
+  *abort_flag = 1;
+}
+
+struct TileCoord { int m0, n0, b0, b1; };
+__device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int tile) {
+  TileCoord t;
+  const int per_batch = p.m_tiles * p.n_tiles;
+  const int z = tile / per_batch, r = tile - z * per_batch;
+  t.n0 = (r / p.m_tiles) * p.block_n;      // consecutive tiles walk down one column block
+  t.m0 = (r % p.m_tiles) * BLOCK_M;
+  t.b0 = z % p.nb0;
+  t.b1 = z / p.nb0;
+  return t;
+}
+
+// ------------------------------------------------------------------ epilogue of 32 columns of one row
+template <int KIND>
+__device__ __forceinline__ void epilogue_chunk(const TcParams& p, const uint32_t* r, float alpha, long long row_off,
+                                               int row, int col0, bool row_ok, bool vec_ok) {
+  const Epilogue& e = p.epi;
+  if (!row_ok) return;
+  const int ncol = min(32, p.N - col0);
+  if (ncol <= 0) return;
+  if (e.out_kind == OUT_I32) {
+    int* out = reinterpret_cast<int*>(e.out) + row_off + col0;
+    if (vec_ok && ncol == 32) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4)
+        *reinterpret_cast<uint4*>(out + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+    } else {
+      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) out[j] = (int)r[j];
+    }
+    return;
+  }
+  float v[32];
+  const float rb = e.row_bias ? e.row_bias[row] : 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const int n = min(col0 + j, p.N - 1);
+    const float acc = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
+    const float sc = e.col_scale ? alpha * e.col_scale[n] : alpha;
+    v[j] = acc * sc + (e.col_bias ? e.col_bias[n] : 0.f) + rb;
+  }
+  const bool full = vec_ok && ncol == 32;
+  if (e.residual) {
+    if (e.out_kind == OUT_BF16) {
+      const bf16* res = reinterpret_cast<const bf16*>(e.residual) + row_off + col0;
+      if (full) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          const uint4 u = *reinterpret_cast<const uint4*>(res + j);
+          const bf16* h = reinterpret_cast<const bf16*>(&u);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) v[j + t] += __bfloat162float(h[t]);
+        }
+      } else {
+        _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) v[j] += __bfloat162float(res[j]);
+      }
+    } else {
+      const float* res = reinterpret_cast<const float*>(e.residual) + row_off + col0;
+      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) v[j] += res[j];
+    }
+  }
+  if (e.act == 1) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+  }
+  if (e.out_kind == OUT_BF16) {
+    bf16* out = reinterpret_cast<bf16*>(e.out) + row_off + col0;
+    if (full) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint4 u;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(v[j + 2 * t], v[j + 2 * t + 1]);
+        *reinterpret_cast<uint4*>(out + j) = u;
+      }
+    } else {
+      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) out[j] = __float2bfloat16_rn(v[j]);
+    }
+  } else {
+    float* out = reinterpret_cast<float*>(e.out) + row_off + col0;
+    if (full) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(out + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+    } else {
+      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) out[j] = v[j];
+    }
+  }
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int KIND>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t tfull_bar[2];
+  __shared__ __align__(8) uint64_t tempty_bar[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.num_stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&tfull_bar[a]), 1);
+      mbar_init(smem_u32(&tempty_bar[a]), 4);
+    }
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  volatile int* vabort = &abort_flag;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        const TileCoord t = decode_tile(p, tile);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (*vabort || !mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u)) {
+            if (!*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
+            ok = false;
+            break;
+          }
+          const uint32_t bar = smem_u32(&full_bar[stage]);
+          const uint32_t sa = tiles_base + stage * p.stage_bytes, sb = sa + A_STAGE_BYTES;
+          mbar_expect_tx(bar, (uint32_t)p.stage_bytes);
+          const int k0 = kb * p.block_k;
+          if (!p.a_mn) {
+            tma_load_4d(sa, &map_a, bar, k0, t.m0, t.b0, t.b1);
+          } else {
+            for (int j = 0; j < BLOCK_M / 64; ++j) tma_load_4d(sa + j * 8192, &map_a, bar, t.m0 + 64 * j, k0, t.b0, t.b1);
+          }
+          if (!p.b_mn) {
+            tma_load_4d(sb, &map_b, bar, k0, t.n0, t.b0, t.b1);
+          } else {
+            for (int j = 0; j < p.block_n / 64; ++j) tma_load_4d(sb + j * 8192, &map_b, bar, t.n0 + 64 * j, k0, t.b0, t.b1);
+          }
+          if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // let the copies already in flight land before the CTA may exit
+        for (int s = 0; s < p.num_stages; ++s) {
+          const unsigned long long t0 = global_ns();
+          while (global_ns() - t0 < 1000000ull) { }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      const uint32_t adv_a = p.a_mn ? 2048u : 32u, adv_b = p.b_mn ? 2048u : 32u;
+      const uint32_t lbo_a = p.a_mn ? 8192u : 16u, lbo_b = p.b_mn ? 8192u : 16u;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        if (*vabort || !mbar_wait(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u)) {
+          if (!*vabort) fail(p, DEV_TIMEOUT_EPI, vabort);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * p.block_n);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (*vabort || !mbar_wait(smem_u32(&full_bar[stage]), phase)) {
+            if (!*vabort) fail(p, DEV_TIMEOUT_TMA, vabort);
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + stage * p.stage_bytes, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t da = smem_desc(sa + k * adv_a, lbo_a, 1024u);
+            const uint64_t db = smem_desc(sb + k * adv_b, lbo_b, 1024u);
+            tc_mma<KIND>(tmem_d, da, db, p.idesc, (uint32_t)((kb | k) != 0));
+          }
+          tc_commit(smem_u32(&empty_bar[stage]));
+          if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&tfull_bar[acc]));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ---------------- epilogue warps (TMEM lane quadrant = warp % 4)
+    const int quad = warp & 3;
+    const Epilogue& e = p.epi;
+    float alpha = e.alpha_const;
+    if (e.alpha_p0) alpha *= *e.alpha_p0;
+    if (e.alpha_p1) alpha *= *e.alpha_p1;
+    const int esz = (e.out_kind == OUT_BF16) ? 2 : 4;
+    const int vec_elems = 16 / esz;
+    bool vec_ok = (e.ldc % vec_elems == 0) && (e.c_b0 % vec_elems == 0) && (e.c_b1 % vec_elems == 0) &&
+                  ((reinterpret_cast<uintptr_t>(e.out) & 15) == 0);
+    if (e.residual) vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(e.residual) & 15) == 0);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      const TileCoord t = decode_tile(p, tile);
+      // every lane polls; the decision is made warp-uniform before any .sync.aligned instruction
+      const bool got = !*vabort && mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase);
+      if (!__all_sync(0xffffffffu, got)) {
+        if (lane == 0 && !*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
+        break;
+      }
+      tc_fence_after();
+      const int row = t.m0 + quad * 32 + lane;
+      const bool row_ok = row < p.M;
+      const long long row_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1 + (long long)row * e.ldc;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * p.block_n);
+      for (int c = 0; c < p.block_n; c += 32) {
+        if (t.n0 + c >= p.N) break;                    // warp-uniform
+        uint32_t r[32];
+        tmem_ld32(taddr + (uint32_t)c, r);
+        epilogue_chunk<KIND>(p, r, alpha, row_off, row, t.n0 + c, row_ok, vec_ok);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Tensor map of one operand: 4-D (contiguous index, strided index, batch0, batch1).
+int make_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,
+             int tile_mn, int block_k) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return GEMM_ERR_CUDA;
+  const cuuint64_t inner = op.mn_contig ? (cuuint64_t)mn_extent : (cuuint64_t)K;
+  const cuuint64_t rows = op.mn_contig ? (cuuint64_t)K : (cuuint64_t)mn_extent;
+  cuuint64_t dims[4] = {inner, rows, (cuuint64_t)nb0, (cuuint64_t)nb1};
+  cuuint64_t s1 = (cuuint64_t)op.ld * elem_bytes;
+  cuuint64_t s2 = nb0 > 1 ? (cuuint64_t)op.s_b0 * elem_bytes : s1 * rows;
+  cuuint64_t s3 = nb1 > 1 ? (cuuint64_t)op.s_b1 * elem_bytes : s2 * (cuuint64_t)nb0;
+  if ((reinterpret_cast<uintptr_t>(op.ptr) & 15) || (s1 & 15) || (s2 & 15) || (s3 & 15)) return GEMM_ERR_ALIGN;
+  if (s1 < inner * elem_bytes) return GEMM_ERR_ARG;
+  cuuint64_t strides[3] = {s1, s2, s3};
+  cuuint32_t box[4];
+  if (op.mn_contig) {
+    box[0] = 128 / elem_bytes;
+    box[1] = (cuuint32_t)block_k;
+  } else {
+    box[0] = (cuuint32_t)block_k;
+    box[1] = (cuuint32_t)tile_mn;
+  }
+  box[2] = box[3] = 1;
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  CUresult r = fn(map, dt, 4, const_cast<void*>(op.ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? GEMM_OK : GEMM_ERR_CUDA;
+}
+
+int pick_block_n(int M, int N, int batches, int sm_count) {
+  const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
+  int best = 64;
+  double best_cost = 1e30;
+  for (int bn = 64; bn <= 256; bn *= 2) {
+    if (bn > 64 && bn / 2 >= N) break;
+    const long long tiles = (long long)m_tiles * ((N + bn - 1) / bn) * batches;
+    const long long waves = (tiles + sm_count - 1) / sm_count;
+    const double cost = (double)waves * (bn + 40.0);     // 40: fixed per-tile cost in units of columns
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
+  }
+  return best;
+}
+
+}  // namespace
+
+int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
+            const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream) {
+  if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.nb0 <= 0 || g.nb1 <= 0) return GEMM_ERR_ARG;
+  const int es = kind == 0 ? 2 : 1;
+  if (kind == 1 && (A.mn_contig || B.mn_contig)) return GEMM_ERR_ARG;
+  TcParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.nb0 = g.nb0; p.nb1 = g.nb1;
+  p.block_n = block_n > 0 ? block_n : pick_block_n(g.M, g.N, g.nb0 * g.nb1, sm_count);
+  if (p.block_n != 64 && p.block_n != 128 && p.block_n != 256) return GEMM_ERR_ARG;
+  p.block_k = 128 / es;
+  p.m_tiles = (g.M + BLOCK_M - 1) / BLOCK_M;
+  p.n_tiles = (g.N + p.block_n - 1) / p.block_n;
+  p.k_blocks = (g.K + p.block_k - 1) / p.block_k;
+  p.num_tiles = p.m_tiles * p.n_tiles * g.nb0 * g.nb1;
+  p.stage_bytes = A_STAGE_BYTES + p.block_n * 128;
+  p.num_stages = TILE_SMEM_BUDGET / p.stage_bytes;
+  if (p.num_stages > MAX_STAGES) p.num_stages = MAX_STAGES;
+  p.a_mn = A.mn_contig; p.b_mn = B.mn_contig;
+  p.epi = epi;
+  p.status = d_status;
+  // instruction descriptor: D format, A/B formats, majors, N >> 3, M >> 4
+  uint32_t idesc = 0;
+  if (kind == 0) {
+    idesc |= 1u << 4;                          // fp32 accumulate
+    idesc |= 1u << 7;                          // A = bf16
+    idesc |= 1u << 10;                         // B = bf16
+  } else {
+    idesc |= 2u << 4;                          // int32 accumulate
+    idesc |= (a_unsigned ? 0u : 1u) << 7;      // A = u8 / s8
+    idesc |= 1u << 10;                         // B = s8
+  }
+  idesc |= (uint32_t)(A.mn_contig ? 1 : 0) << 15;
+  idesc |= (uint32_t)(B.mn_contig ? 1 : 0) << 16;
+  idesc |= (uint32_t)(p.block_n >> 3) << 17;
+  idesc |= (uint32_t)(BLOCK_M >> 4) << 24;
+  p.idesc = idesc;
+
+  CUtensorMap ma, mb;
+  int rc = make_map(&ma, A, es, g.M, g.K, g.nb0, g.nb1, BLOCK_M, p.block_k);
+  if (rc != GEMM_OK) return rc;
+  rc = make_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k);
+  if (rc != GEMM_OK) return rc;
+
+  const int smem = p.num_stages * p.stage_bytes + 1024;
+  static bool attr_set[2] = {false, false};
+  auto kern = kind == 0 ? tc_gemm_kernel<0> : tc_gemm_kernel<1>;
+  if (!attr_set[kind]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TILE_SMEM_BUDGET + 1024) != cudaSuccess)
+      return GEMM_ERR_CUDA;
+    attr_set[kind] = true;
+  }
+  const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
+  kern<<<grid, GEMM_THREADS, smem, stream>>>(ma, mb, p);
+  return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
+}
+
+}  // namespace mrem

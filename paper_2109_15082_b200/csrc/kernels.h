@@ -1,0 +1,120 @@
+// Launchers of the HBM-bound kernels of the reconstruction step.  `dt` is the storage type
+// of activations: 0 = float32, 1 = bfloat16.  All launches are asynchronous on `st`.
+#pragma once
+#include "mrem_common.cuh"
+
+namespace mrem {
+
+constexpr int RED_BLOCKS = 296;     // grid of every kernel that emits per-block partial sums (2 x 148 SMs)
+
+// ---- quantizers (Eq. 1)
+// Weight quantizer: latent w[rows, cols] fp32 and steps (one per row, or one in all) ->
+// int8 codes, int32 row sums of the codes, per-row dequantization scale (s, or s/2 on the
+// half-integer 2-bit grid) and the dequantized matrix in the storage type.
+void launch_quantize_weight(const float* w, int rows, int cols, const float* steps, int per_row, int bits, int grid,
+                            int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt, cudaStream_t st);
+
+// Activation quantizer over a 2-D view x[rows, cols] with row stride ld_x:
+// z = (x - offset) / step, q = rne(clip(z, lo, hi)).  Writes int8/uint8 codes (row stride
+// ld_q8) and/or the codes as storage-type numbers (row stride ld_qt); either may be null.
+void launch_quantize_act(const void* x, int dt, long long rows, int cols, long long ld_x, const float* step,
+                         const float* offset, int lo, int hi, int8_t* q8, long long ld_q8, void* qt,
+                         long long ld_qt, cudaStream_t st);
+
+// dst[i] = (float)src[i] for a bfloat16 source
+void launch_widen_bf16(const void* src, float* dst, long long n, cudaStream_t st);
+
+// dst[i] = src[i] converted to the storage type
+void launch_narrow(const float* src, void* dst, long long n, int dt, cudaStream_t st);
+
+// Eq. 4: out = lam * f + (1 - lam) * f_hat
+void launch_mix(const void* f, const void* f_hat, float lam, void* out, long long n, int dt, cudaStream_t st);
+
+// ---- forward layer kernels
+// out = LayerNorm(y) * gamma + beta (row-wise over `cols`), mean / rstd saved when non-null; with a
+// step pointer the symmetric codes of the stored output are emitted as well.
+void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, float eps, long long rows, int cols,
+                          void* out, float* mean, float* rstd, const float* step, int qmax, int8_t* q8, void* qt,
+                          int dt, cudaStream_t st);
+
+// g = stored(gelu(u)); codes of g (asymmetric when offset != null) as int8/uint8 and storage-type numbers.
+void launch_gelu_quant(const void* u, long long n, const float* step, const float* offset, int lo, int hi,
+                       int8_t* q8, void* qt, int dt, cudaStream_t st);
+
+// P = softmax(scores) over the last axis with keys >= valid_len[b] masked out; scores fp32
+// [B, h, S, S]; optional codes of P as storage-type numbers.
+void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,
+                        const float* offset, int lo, int hi, void* qt, int dt, cudaStream_t st);
+
+// ---- loss (Eq. 3)
+// partial[l][block] = sum (f_hat - f)^2 over the block's share; dF = 2 c (f_hat - f).
+void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per_layer, float c, void* dF,
+                 float* partial, int* status, int dt, cudaStream_t st);
+void launch_loss_finalize(const float* partial, int n_layers, float c, float* loss_total, float* loss_per_layer,
+                          cudaStream_t st);
+
+// ---- backward kernels
+// Straight-through backward of an activation quantizer on a 2-D view:
+// dx = dxhat * 1[lo <= z <= hi] (+ add), per-block partials of d l/d step (and d l/d offset).
+void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long ld_d, const void* add,
+                    long long ld_add, void* dx, long long ld_dx, long long rows, int cols, const float* step,
+                    const float* offset, int lo, int hi, float* part_s, float* part_o, int dt, cudaStream_t st);
+
+// GELU-site backward: recompute g = stored(gelu(u)), STE of its quantizer, dU = dGhat * inside * gelu'(u).
+void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, const float* step, const float* offset,
+                     int lo, int hi, int quantized, float* part_s, float* part_o, int dt, cudaStream_t st);
+
+// Softmax-site backward: STE of the P quantizer, then dS = P * (dP - sum_j dP * P) per row.
+void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long rows, int S, const float* step,
+                        int lo, int hi, int quantized, float* part_s, int dt, cudaStream_t st);
+
+// LayerNorm backward: dy (storage type) from dout (+ dout2 when non-null).
+void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, const float* mean, const float* rstd,
+                          const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
+                          cudaStream_t st);
+
+// Column sums over rows: out0[c] = sum_r a[r,c]; with y/mean/rstd also out1[c] = sum_r a[r,c]*(y[r,c]-mean[r])*rstd[r].
+// Two kernels (per-chunk partials in `scratch`, then a fixed-order sum).  scratch >= 2*COL_CHUNKS*cols floats.
+constexpr int COL_CHUNKS = 64;
+void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
+                       long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st);
+
+// Weight STE: dW = dWhat * inside (in place), ds[row] = sum_k dWhat * d what/d s.
+void launch_ste_weight(const float* w, const float* steps, int per_row, int bits, int grid, float* dw, int rows,
+                       int cols, float* ds_rows, cudaStream_t st);
+
+// dst[i] = sum_j src_i[j], j in fixed order, for a table of reductions (one block each).
+struct ReduceEntry { const float* src; int count; float* dst; };
+void launch_reduce_table(const ReduceEntry* d_table, int n_entries, cudaStream_t st);
+
+// out[i] = scale[0] * in[i]  (small vectors)
+void launch_scale_vec(const float* in, const float* scale, float* out, int n, cudaStream_t st);
+// beff[n] = b[n] + beta[0] * wscale[n] * rowsum[n]
+void launch_effective_bias(const float* b, const float* beta, const float* wscale, const int32_t* rowsum, float* beff,
+                           int n, cudaStream_t st);
+
+// ---- optimizer (AdamW)
+struct OptimScalars { float lr, beta1, beta2, eps, bc1, bc2, weight_decay; };   // bc = 1 - beta^t
+struct AdamEntry { float* p; const float* g; float* m; float* v; long long n; float wd; float min_value; };   // wd: 1 = decayed
+// Computes the scalars of this step on the device: t = ++(*d_t) (or host_t when >= 1),
+// lr = lr0 * (1 - (t-1)/total) when total > 0 else lr0.
+void launch_optim_prepare(OptimScalars* d_out, int* d_t, int host_t, float lr0, int total_steps, float beta1,
+                          float beta2, float eps, float weight_decay, cudaStream_t st);
+void launch_adamw_table(const AdamEntry* d_table, int n_entries, const OptimScalars* d_sc, cudaStream_t st);
+
+// ---- step-size initialisation
+// Per-row max|w| or mean|w| -> steps (per row, or one value when !per_row: two passes).
+void launch_init_weight_steps(const float* w, int rows, int cols, int per_row, int rule, float qmax, float* steps,
+                              float* scratch, cudaStream_t st);
+// min and max of a 2-D view -> out[0] = min, out[1] = max (two kernels; scratch >= 2*RED_BLOCKS floats).
+void launch_minmax(const void* x, long long ld, long long rows, int cols, float* out, float* scratch, int dt,
+                   cudaStream_t st);
+// step/offset from (min, max): mode 0 symmetric s = max|x|/qmax; 1 unsigned s = max/qmax, offset 0;
+// 2 unsigned s = (max-min)/qmax, offset = min.
+void launch_step_from_minmax(const float* minmax, int mode, float qmax, float* step, float* offset, cudaStream_t st);
+
+// Gather rows of a calibration set: out[i] = src[idx[i]] for i < n_rows, row_bytes each (16-byte multiple).
+void launch_gather_rows(const void* src, const int* d_idx, int n_rows, long long row_bytes, void* out,
+                        cudaStream_t st);
+
+}  // namespace mrem

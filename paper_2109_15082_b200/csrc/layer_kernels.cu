@@ -1,0 +1,568 @@
+// LayerNorm, softmax, loss and straight-through backward kernels of the reconstruction step.
+// All are HBM/L2-bound passes: 16-byte vector access where the view allows it, one warp per
+// row for row-wise ops, warp-shuffle reductions, and fixed-order two-stage sums (per-block
+// partials, then one block adds them in index order) so results are reproducible run to run.
+#include "kernels.h"
+#include "vec.cuh"
+
+namespace mrem {
+
+namespace {
+
+__device__ __forceinline__ float qz(float x, float s, float off, bool has_off) {
+  return __fdiv_rn(has_off ? __fsub_rn(x, off) : x, s);
+}
+__device__ __forceinline__ int qcode(float z, float lo, float hi) { return __float2int_rn(fminf(fmaxf(z, lo), hi)); }
+
+// ------------------------------------------------------------------ LayerNorm forward (one warp per row)
+template <typename T, int V>
+__global__ void __launch_bounds__(128) ln_fwd_kernel(const T* __restrict__ y, const float* __restrict__ gamma,
+                                                     const float* __restrict__ beta, float eps, long long rows,
+                                                     int cols, T* __restrict__ out, float* __restrict__ mean,
+                                                     float* __restrict__ rstd, const float* __restrict__ step,
+                                                     float qmax, int8_t* __restrict__ q8, T* __restrict__ qt) {
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const T* yr = y + row * cols;
+  float sum = 0.f;
+  for (int c = lane * V; c < cols; c += 32 * V) {
+    float v[V];
+    load_vec<T, V>(yr + c, v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) sum += v[j];
+  }
+  const float mu = warp_sum(sum) / (float)cols;
+  float sq = 0.f;
+  for (int c = lane * V; c < cols; c += 32 * V) {
+    float v[V];
+    load_vec<T, V>(yr + c, v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) sq += (v[j] - mu) * (v[j] - mu);
+  }
+  const float rs = 1.f / sqrtf(warp_sum(sq) / (float)cols + eps);
+  if (lane == 0) {
+    if (mean) mean[row] = mu;
+    if (rstd) rstd[row] = rs;
+  }
+  const float s = step ? *step : 1.f;
+  for (int c = lane * V; c < cols; c += 32 * V) {
+    float v[V];
+    load_vec<T, V>(yr + c, v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) v[j] = (v[j] - mu) * rs * gamma[c + j] + beta[c + j];
+    store_vec<T, V>(out + row * cols + c, v);
+    if (step) {
+      int q[V];
+#pragma unroll
+      for (int j = 0; j < V; ++j) q[j] = qcode(__fdiv_rn(stored<T>(v[j]), s), -qmax, qmax);
+      if (q8) store_codes<V>(q8 + row * cols + c, q);
+      if (qt) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) v[j] = (float)q[j];
+        store_vec<T, V>(qt + row * cols + c, v);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ LayerNorm backward (one warp per row)
+template <typename T, int V>
+__global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ dout2,
+                                                     const T* __restrict__ y, const float* __restrict__ mean,
+                                                     const float* __restrict__ rstd, const float* __restrict__ gamma,
+                                                     long long rows, int cols, T* __restrict__ dy,
+                                                     T* __restrict__ dsum) {
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float mu = mean[row], rs = rstd[row];
+  const long long base = row * cols;
+  float s1 = 0.f, s2 = 0.f;
+  for (int c = lane * V; c < cols; c += 32 * V) {
+    float d[V], v[V];
+    load_vec<T, V>(dout + base + c, d);
+    if (dout2) {
+      float e[V];
+      load_vec<T, V>(dout2 + base + c, e);
+#pragma unroll
+      for (int j = 0; j < V; ++j) d[j] += e[j];
+      if (dsum) store_vec<T, V>(dsum + base + c, d);
+    }
+    load_vec<T, V>(y + base + c, v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const float dxn = (dout2 && dsum ? stored<T>(d[j]) : d[j]) * gamma[c + j];
+      s1 += dxn;
+      s2 += dxn * (v[j] - mu) * rs;
+    }
+  }
+  s1 = warp_sum(s1) / (float)cols;
+  s2 = warp_sum(s2) / (float)cols;
+  for (int c = lane * V; c < cols; c += 32 * V) {
+    float d[V], v[V];
+    load_vec<T, V>((dout2 && dsum ? dsum : dout) + base + c, d);
+    if (dout2 && !dsum) {
+      float e[V];
+      load_vec<T, V>(dout2 + base + c, e);
+#pragma unroll
+      for (int j = 0; j < V; ++j) d[j] += e[j];
+    }
+    load_vec<T, V>(y + base + c, v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const float xn = (v[j] - mu) * rs;
+      d[j] = rs * (d[j] * gamma[c + j] - s1 - xn * s2);
+    }
+    store_vec<T, V>(dy + base + c, d);
+  }
+}
+
+// ------------------------------------------------------------------ column sums over rows (bias and LayerNorm parameter gradients)
+template <typename T>
+__global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a, long long ld_a,
+                                                         const T* __restrict__ y, const float* __restrict__ mean,
+                                                         const float* __restrict__ rstd, long long rows, int cols,
+                                                         float* __restrict__ scratch) {
+  __shared__ float sh0[8][33], sh1[8][33];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + tx;
+  const long long per = (rows + COL_CHUNKS - 1) / COL_CHUNKS;
+  const long long r0 = blockIdx.y * per, r1 = r0 + per < rows ? r0 + per : rows;
+  float a0 = 0.f, a1 = 0.f;
+  if (c < cols) {
+    for (long long r = r0 + ty; r < r1; r += 8) {
+      const float v = to_f<T>(a[r * ld_a + c]);
+      a0 += v;
+      if (y) a1 += v * (to_f<T>(y[r * cols + c]) - mean[r]) * rstd[r];
+    }
+  }
+  sh0[ty][tx] = a0;
+  sh1[ty][tx] = a1;
+  __syncthreads();
+  if (ty == 0 && c < cols) {
+    float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { t0 += sh0[k][tx]; t1 += sh1[k][tx]; }
+    scratch[(long long)blockIdx.y * cols + c] = t0;
+    if (y) scratch[((long long)COL_CHUNKS + blockIdx.y) * cols + c] = t1;
+  }
+}
+__global__ void col_reduce_final_kernel(const float* __restrict__ scratch, int cols, float* __restrict__ out0,
+                                        float* __restrict__ out1) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  float t0 = 0.f, t1 = 0.f;
+  for (int k = 0; k < COL_CHUNKS; ++k) {
+    t0 += scratch[(long long)k * cols + c];
+    if (out1) t1 += scratch[((long long)COL_CHUNKS + k) * cols + c];
+  }
+  out0[c] = t0;
+  if (out1) out1[c] = t1;
+}
+
+// ------------------------------------------------------------------ softmax forward (one warp per row)
+template <typename T>
+__global__ void __launch_bounds__(128) softmax_fwd_kernel(const float* __restrict__ scores,
+                                                          const int* __restrict__ valid_len, int h, int S,
+                                                          long long rows, T* __restrict__ P,
+                                                          const float* __restrict__ step,
+                                                          const float* __restrict__ offset, float lo, float hi,
+                                                          T* __restrict__ qt) {
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int b = (int)(row / ((long long)h * S));
+  int len = valid_len ? valid_len[b] : S;
+  len = len < 1 ? 1 : (len > S ? S : len);
+  const float* sr = scores + row * S;
+  float mx = -INFINITY;
+  for (int j = lane; j < len; j += 32) mx = fmaxf(mx, sr[j]);
+  mx = warp_max(mx);
+  float sum = 0.f;
+  for (int j = lane; j < len; j += 32) sum += expf(sr[j] - mx);
+  sum = warp_sum(sum);
+  const float s = step ? *step : 1.f;
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  for (int j = lane; j < S; j += 32) {
+    const float p = j < len ? __fdiv_rn(expf(sr[j] - mx), sum) : 0.f;
+    P[row * S + j] = from_f<T>(p);
+    if (qt) qt[row * S + j] = from_f<T>((float)qcode(qz(stored<T>(p), s, off, has_off), lo, hi));
+  }
+}
+
+// ------------------------------------------------------------------ softmax backward with the STE of the P quantizer
+template <typename T>
+__global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ P, const T* __restrict__ dphat,
+                                                          T* __restrict__ dS, long long rows, int S,
+                                                          const float* __restrict__ step, float lo, float hi,
+                                                          int quantized, float* __restrict__ part_s) {
+  __shared__ float sh[32];
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = blockIdx.x * 8ll + (threadIdx.x >> 5), nwarps = gridDim.x * 8ll;
+  const float s = quantized ? *step : 1.f;
+  float ds = 0.f;
+  for (long long row = warp0; row < rows; row += nwarps) {
+    const long long base = row * S;
+    float dot = 0.f;
+    for (int j = lane; j < S; j += 32) {
+      const float p = to_f<T>(P[base + j]);
+      float d = to_f<T>(dphat[base + j]);
+      if (quantized) {
+        const float z = __fdiv_rn(p, s);
+        const bool in = z >= lo && z <= hi;
+        ds += d * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+        d = in ? d : 0.f;
+      }
+      dot += d * p;
+    }
+    dot = warp_sum(dot);
+    for (int j = lane; j < S; j += 32) {
+      const float p = to_f<T>(P[base + j]);
+      float d = to_f<T>(dphat[base + j]);
+      if (quantized) {
+        const float z = __fdiv_rn(p, s);
+        d = (z >= lo && z <= hi) ? d : 0.f;
+      }
+      dS[base + j] = from_f<T>(p * (d - dot));
+    }
+  }
+  ds = block_sum(ds, sh);
+  if (threadIdx.x == 0 && part_s) part_s[blockIdx.x] = ds;
+}
+
+// ------------------------------------------------------------------ loss (Eq. 3) and its gradient
+template <typename T, int V>
+__global__ void __launch_bounds__(256) loss_kernel(const T* __restrict__ fh, const T* __restrict__ f,
+                                                   long long n, float c, T* __restrict__ dF,
+                                                   float* __restrict__ partial, int* __restrict__ status) {
+  __shared__ float sh[32];
+  const long long base = (long long)blockIdx.y * n;
+  float acc = 0.f;
+  for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
+    float a[V], b[V];
+    load_vec<T, V>(fh + base + i, a);
+    load_vec<T, V>(f + base + i, b);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const float d = a[j] - b[j];
+      acc += d * d;
+      a[j] = 2.f * c * d;
+    }
+    store_vec<T, V>(dF + base + i, a);
+  }
+  acc = block_sum(acc, sh);
+  if (threadIdx.x == 0) {
+    partial[blockIdx.y * gridDim.x + blockIdx.x] = acc;
+    if (!isfinite(acc) && status) atomicCAS(status, 0, (int)DEV_NONFINITE);
+  }
+}
+__global__ void loss_final_kernel(const float* __restrict__ partial, int n_layers, int nb, float c,
+                                  float* __restrict__ total, float* __restrict__ per_layer) {
+  __shared__ float sh[32];
+  float tot = 0.f;
+  for (int l = 0; l < n_layers; ++l) {
+    float a = 0.f;
+    for (int i = threadIdx.x; i < nb; i += blockDim.x) a += partial[l * nb + i];
+    a = block_sum(a, sh) * c;
+    if (threadIdx.x == 0 && per_layer) per_layer[l] = a;
+    tot += a;
+  }
+  if (threadIdx.x == 0 && total) *total = tot;
+}
+
+// ------------------------------------------------------------------ STE of an activation quantizer on a 2-D view
+template <typename T, int V>
+__global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, long long ld_x,
+                                                      const T* __restrict__ dxhat, long long ld_d,
+                                                      const T* __restrict__ add, long long ld_add,
+                                                      T* __restrict__ dx, long long ld_dx, long long rows, int cols,
+                                                      const float* __restrict__ step,
+                                                      const float* __restrict__ offset, float lo, float hi,
+                                                      float* __restrict__ part_s, float* __restrict__ part_o) {
+  __shared__ float sh[32];
+  const float s = *step;
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  const int vcols = cols / V;
+  const long long total = rows * vcols;
+  float ds = 0.f, dofs = 0.f;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / vcols;
+    const int c = (int)(i - r * vcols) * V;
+    float xv[V], d[V];
+    load_vec<T, V>(x + r * ld_x + c, xv);
+    load_vec<T, V>(dxhat + r * ld_d + c, d);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const float z = qz(xv[j], s, off, has_off);
+      const bool in = z >= lo && z <= hi;
+      ds += d[j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+      dofs += in ? 0.f : d[j];
+      d[j] = in ? d[j] : 0.f;
+    }
+    if (add) {
+      float e[V];
+      load_vec<T, V>(add + r * ld_add + c, e);
+#pragma unroll
+      for (int j = 0; j < V; ++j) d[j] += e[j];
+    }
+    store_vec<T, V>(dx + r * ld_dx + c, d);
+  }
+  ds = block_sum(ds, sh);
+  dofs = block_sum(dofs, sh);
+  if (threadIdx.x == 0) {
+    part_s[blockIdx.x] = ds;
+    if (part_o) part_o[blockIdx.x] = dofs;
+  }
+}
+
+// ------------------------------------------------------------------ GELU backward with the STE of its output quantizer
+template <typename T, int V>
+__global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, const T* __restrict__ dghat,
+                                                       T* __restrict__ du, long long n,
+                                                       const float* __restrict__ step,
+                                                       const float* __restrict__ offset, float lo, float hi,
+                                                       int quantized, float* __restrict__ part_s,
+                                                       float* __restrict__ part_o) {
+  __shared__ float sh[32];
+  const float s = quantized ? *step : 1.f;
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  float ds = 0.f, dofs = 0.f;
+  for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
+    float uv[V], d[V];
+    load_vec<T, V>(u + i, uv);
+    load_vec<T, V>(dghat + i, d);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      if (quantized) {
+        const float z = qz(stored<T>(gelu_erf(uv[j])), s, off, has_off);
+        const bool in = z >= lo && z <= hi;
+        ds += d[j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+        dofs += in ? 0.f : d[j];
+        d[j] = in ? d[j] : 0.f;
+      }
+      d[j] *= gelu_erf_grad(uv[j]);
+    }
+    store_vec<T, V>(du + i, d);
+  }
+  ds = block_sum(ds, sh);
+  dofs = block_sum(dofs, sh);
+  if (threadIdx.x == 0) {
+    if (part_s) part_s[blockIdx.x] = ds;
+    if (part_o) part_o[blockIdx.x] = dofs;
+  }
+}
+
+// ------------------------------------------------------------------ STE of the weight quantizer (one block per row)
+__global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict__ w, const float* __restrict__ steps,
+                                                         int per_row, int bits, int grid, float* __restrict__ dw,
+                                                         int cols, float* __restrict__ ds_rows) {
+  __shared__ float sh[32];
+  const int row = blockIdx.x;
+  const float s = steps[per_row ? row : 0];
+  const float qmax = (float)((1 << (bits - 1)) - 1);
+  const float* wr = w + (long long)row * cols;
+  float* dr = dw + (long long)row * cols;
+  float ds = 0.f;
+  for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+    const float z = __fdiv_rn(wr[c], s);
+    const float d = dr[c];
+    bool in;
+    float level;
+    if (grid == 0) {
+      in = z >= -qmax && z <= qmax;
+      level = (float)__float2int_rn(fminf(fmaxf(z, -qmax), qmax));
+    } else {
+      in = z >= -2.f && z < 2.f;
+      level = fminf(fmaxf(floorf(z), -2.f), 1.f) + 0.5f;
+    }
+    ds += d * (level - (in ? z : 0.f));
+    dr[c] = in ? d : 0.f;
+  }
+  ds = block_sum(ds, sh);
+  if (threadIdx.x == 0) ds_rows[row] = ds;
+}
+
+__global__ void __launch_bounds__(256) reduce_table_kernel(const ReduceEntry* __restrict__ table) {
+  __shared__ float sh[32];
+  const ReduceEntry e = table[blockIdx.x];
+  float a = 0.f;
+  for (int i = threadIdx.x; i < e.count; i += blockDim.x) a += e.src[i];
+  a = block_sum(a, sh);
+  if (threadIdx.x == 0) *e.dst = a;
+}
+
+__global__ void scale_vec_kernel(const float* __restrict__ in, const float* __restrict__ scale, float* __restrict__ out, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = scale[0] * in[i];
+}
+__global__ void effective_bias_kernel(const float* __restrict__ b, const float* __restrict__ beta,
+                                      const float* __restrict__ wscale, const int32_t* __restrict__ rowsum,
+                                      float* __restrict__ beff, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) beff[i] = b[i] + beta[0] * wscale[i] * (float)rowsum[i];
+}
+
+// ------------------------------------------------------------------ AdamW
+__global__ void optim_prepare_kernel(OptimScalars* out, int* d_t, int host_t, float lr0, int total, float b1, float b2,
+                                     float eps, float wd) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int t = host_t >= 1 ? host_t : (*d_t + 1);
+  *d_t = t;
+  OptimScalars o;
+  o.lr = total > 0 ? lr0 * fmaxf(1.f - (float)(t - 1) / (float)total, 0.f) : lr0;
+  o.beta1 = b1;
+  o.beta2 = b2;
+  o.eps = eps;
+  o.weight_decay = wd;
+  o.bc1 = (float)(1.0 - pow((double)b1, (double)t));
+  o.bc2 = (float)(1.0 - pow((double)b2, (double)t));
+  *out = o;
+}
+
+__global__ void __launch_bounds__(256) adamw_table_kernel(const AdamEntry* __restrict__ table,
+                                                          const OptimScalars* __restrict__ sc) {
+  const AdamEntry e = table[blockIdx.y];
+  const OptimScalars o = *sc;
+  const float decay = 1.f - o.lr * e.wd * o.weight_decay;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < e.n; i += (long long)gridDim.x * blockDim.x) {
+    const float g = e.g[i];
+    const float m = o.beta1 * e.m[i] + (1.f - o.beta1) * g;
+    const float v = o.beta2 * e.v[i] + (1.f - o.beta2) * g * g;
+    e.m[i] = m;
+    e.v[i] = v;
+    const float upd = o.lr * (m / o.bc1) / (sqrtf(v / o.bc2) + o.eps);
+    e.p[i] = fmaxf(e.p[i] * decay - upd, e.min_value);
+  }
+}
+
+inline int grid_for(long long work_items, int threads = 256, int cap = 148 * 8) {
+  long long b = (work_items + threads - 1) / threads;
+  if (b < 1) b = 1;
+  return (int)(b < cap ? b : cap);
+}
+inline bool al16(const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+#define MREM_DT(dt, T, ...)            \
+  do {                                 \
+    if ((dt) == 1) { using T = bf16; __VA_ARGS__; } else { using T = float; __VA_ARGS__; } \
+  } while (0)
+
+void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, float eps, long long rows, int cols,
+                          void* out, float* mean, float* rstd, const float* step, int qmax, int8_t* q8, void* qt,
+                          int dt, cudaStream_t st) {
+  if (rows <= 0) return;
+  const int grid = (int)((rows + 3) / 4);
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool v = cols % V == 0 && al16(y) && al16(out) && al16(qt) && (reinterpret_cast<uintptr_t>(q8) % V) == 0;
+    if (v) ln_fwd_kernel<T, V><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
+    else ln_fwd_kernel<T, 1><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
+  });
+}
+
+void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, const float* mean, const float* rstd,
+                          const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
+                          cudaStream_t st) {
+  if (rows <= 0) return;
+  const int grid = (int)((rows + 3) / 4);
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool v = cols % V == 0 && al16(dout) && al16(dout2) && al16(y) && al16(dy) && al16(dsum);
+    if (v) ln_bwd_kernel<T, V><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
+    else ln_bwd_kernel<T, 1><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
+  });
+}
+
+void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
+                       long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st) {
+  dim3 grid((cols + 31) / 32, COL_CHUNKS);
+  MREM_DT(dt, T, { col_reduce_kernel<T><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch); });
+  col_reduce_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, cols, out0, y ? out1 : nullptr);
+}
+
+void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,
+                        const float* offset, int lo, int hi, void* qt, int dt, cudaStream_t st) {
+  const long long rows = (long long)B * h * S;
+  if (rows <= 0) return;
+  const int grid = (int)((rows + 3) / 4);
+  MREM_DT(dt, T, { softmax_fwd_kernel<T><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt); });
+}
+
+void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long rows, int S, const float* step,
+                        int lo, int hi, int quantized, float* part_s, int dt, cudaStream_t st) {
+  MREM_DT(dt, T, { softmax_bwd_kernel<T><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s); });
+}
+
+void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per_layer, float c, void* dF,
+                 float* partial, int* status, int dt, cudaStream_t st) {
+  dim3 grid(RED_BLOCKS, n_layers);
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    if (n_per_layer % V == 0 && al16(f_hat) && al16(f) && al16(dF))
+      loss_kernel<T, V><<<grid, 256, 0, st>>>((const T*)f_hat, (const T*)f, n_per_layer, c, (T*)dF, partial, status);
+    else
+      loss_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)f_hat, (const T*)f, n_per_layer, c, (T*)dF, partial, status);
+  });
+}
+void launch_loss_finalize(const float* partial, int n_layers, float c, float* loss_total, float* loss_per_layer,
+                          cudaStream_t st) {
+  loss_final_kernel<<<1, 256, 0, st>>>(partial, n_layers, RED_BLOCKS, c, loss_total, loss_per_layer);
+}
+
+void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long ld_d, const void* add,
+                    long long ld_add, void* dx, long long ld_dx, long long rows, int cols, const float* step,
+                    const float* offset, int lo, int hi, float* part_s, float* part_o, int dt, cudaStream_t st) {
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool v = cols % V == 0 && ld_x % V == 0 && ld_d % V == 0 && ld_dx % V == 0 && (!add || ld_add % V == 0) &&
+                   al16(x) && al16(dxhat) && al16(add) && al16(dx);
+    if (v) ste_act_kernel<T, V><<<RED_BLOCKS, 256, 0, st>>>((const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
+    else ste_act_kernel<T, 1><<<RED_BLOCKS, 256, 0, st>>>((const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
+  });
+}
+
+void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, const float* step, const float* offset,
+                     int lo, int hi, int quantized, float* part_s, float* part_o, int dt, cudaStream_t st) {
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    if (n % V == 0 && al16(u) && al16(dghat) && al16(du))
+      gelu_bwd_kernel<T, V><<<RED_BLOCKS, 256, 0, st>>>((const T*)u, (const T*)dghat, (T*)du, n, step, offset, (float)lo, (float)hi, quantized, part_s, part_o);
+    else
+      gelu_bwd_kernel<T, 1><<<RED_BLOCKS, 256, 0, st>>>((const T*)u, (const T*)dghat, (T*)du, n, step, offset, (float)lo, (float)hi, quantized, part_s, part_o);
+  });
+}
+
+void launch_ste_weight(const float* w, const float* steps, int per_row, int bits, int grid, float* dw, int rows,
+                       int cols, float* ds_rows, cudaStream_t st) {
+  ste_weight_kernel<<<rows, 256, 0, st>>>(w, steps, per_row, bits, grid, dw, cols, ds_rows);
+}
+
+void launch_reduce_table(const ReduceEntry* d_table, int n_entries, cudaStream_t st) {
+  if (n_entries > 0) reduce_table_kernel<<<n_entries, 256, 0, st>>>(d_table);
+}
+
+void launch_scale_vec(const float* in, const float* scale, float* out, int n, cudaStream_t st) {
+  scale_vec_kernel<<<(n + 255) / 256, 256, 0, st>>>(in, scale, out, n);
+}
+void launch_effective_bias(const float* b, const float* beta, const float* wscale, const int32_t* rowsum, float* beff,
+                           int n, cudaStream_t st) {
+  effective_bias_kernel<<<(n + 255) / 256, 256, 0, st>>>(b, beta, wscale, rowsum, beff, n);
+}
+
+void launch_optim_prepare(OptimScalars* d_out, int* d_t, int host_t, float lr0, int total_steps, float beta1,
+                          float beta2, float eps, float weight_decay, cudaStream_t st) {
+  optim_prepare_kernel<<<1, 32, 0, st>>>(d_out, d_t, host_t, lr0, total_steps, beta1, beta2, eps, weight_decay);
+}
+void launch_adamw_table(const AdamEntry* d_table, int n_entries, const OptimScalars* d_sc, cudaStream_t st) {
+  if (n_entries <= 0) return;
+  dim3 grid(64, n_entries);
+  adamw_table_kernel<<<grid, 256, 0, st>>>(d_table, d_sc);
+}
+
+}  // namespace mrem

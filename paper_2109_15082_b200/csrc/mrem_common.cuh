@@ -1,0 +1,108 @@
+// Shared device/host helpers of the MREM reconstruction-step kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mrem {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------- status word (device, sticky)
+enum DeviceStatus : int {
+  DEV_OK = 0,
+  DEV_TIMEOUT_TMA = 1,      // a wait on a TMA-filled stage ran out
+  DEV_TIMEOUT_MMA = 2,      // a wait on a tensor-core commit ran out
+  DEV_TIMEOUT_EPI = 3,      // a wait on an accumulator hand-over ran out
+  DEV_NONFINITE = 4,        // the loss kernel met a non-finite value
+};
+
+// ---------------------------------------------------------------- storage-type access
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// value of v after a round trip through storage type T
+template <typename T> __device__ __forceinline__ float stored(float v) { return to_f<T>(from_f<T>(v)); }
+
+// ---------------------------------------------------------------- reductions
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ int warp_sum_i(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Block-wide sum in a fixed order (warp shuffles, then warp 0 over the per-warp values).
+// `sh` must hold 32 floats.  Every thread gets the result.
+__device__ __forceinline__ float block_sum(float v, float* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  float r = (lane < nw) ? sh[lane] : 0.f;
+  r = warp_sum(r);
+  return r;
+}
+__device__ __forceinline__ float block_max(float v, float* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_max(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  float r = (lane < nw) ? sh[lane] : -INFINITY;
+  r = warp_max(r);
+  return r;
+}
+
+// ---------------------------------------------------------------- math
+__device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.f + erff(u * 0.70710678118654752f)); }
+__device__ __forceinline__ float gelu_erf_grad(float u) {
+  return 0.5f * (1.f + erff(u * 0.70710678118654752f)) + u * expf(-0.5f * u * u) * 0.39894228040143268f;
+}
+
+// ---------------------------------------------------------------- GEMM interface (both back ends)
+enum OutKind : int { OUT_F32 = 0, OUT_BF16 = 1, OUT_I32 = 2 };
+
+// out[b][m][n] = act( alpha * col_scale[n] * acc + col_bias[n] + row_bias[m] + residual[b][m][n] )
+// alpha = alpha_const * (*alpha_p0) * (*alpha_p1)   (null pointers count as 1)
+struct Epilogue {
+  void* out;
+  const void* residual;        // same kind and strides as out, or null
+  long long ldc, c_b0, c_b1;   // element strides of out/residual: row, batch0, batch1
+  int out_kind;                // OutKind
+  int act;                     // 0 none, 1 erf-GELU
+  float alpha_const;
+  const float* alpha_p0;
+  const float* alpha_p1;
+  const float* col_scale;      // [N] or null
+  const float* col_bias;       // [N] or null
+  const float* row_bias;       // [M] or null
+};
+
+// One operand of C[m,n] = sum_k A[m,k] * B[n,k].  `mn_contig` = 1 when the operand is
+// stored with its M (or N) index contiguous and k strided, 0 when k is contiguous.
+struct OperandDesc {
+  const void* ptr;
+  long long ld;                // element stride of the non-contiguous index
+  long long s_b0, s_b1;        // element strides of the batch indices
+  int mn_contig;
+};
+
+struct GemmShape { int M, N, K, nb0, nb1; };
+
+}  // namespace mrem

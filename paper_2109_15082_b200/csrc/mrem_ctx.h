@@ -1,0 +1,114 @@
+// Host-side state of one reconstruction context: shapes, bound pointers and the layout of
+// the caller-provided workspace.
+#pragma once
+#include <string>
+#include <vector>
+
+#include "../../include/mrem.h"
+#include "gemm.h"
+#include "kernels.h"
+
+namespace mrem {
+
+constexpr int N_SITES = 8;              // activation quantizer sites per layer
+constexpr int N_WMAT = 4;               // weight matrices per layer
+
+struct WeightBuf {                      // quantized form of one weight matrix
+  int rows = 0, cols = 0;
+  int8_t* codes = nullptr;              // [rows, cols]
+  int32_t* rowsum = nullptr;            // [rows]
+  float* scale = nullptr;               // [rows] dequantization scale (step, or step/2 on the half-integer grid)
+  void* what = nullptr;                 // [rows, cols] dequantized, storage type
+  float* beff = nullptr;                // [rows] bias + offset term (W2 only)
+  float* ds_rows = nullptr;             // [rows] per-row step gradients before a per-matrix sum
+};
+
+struct LayerStash {                     // what the student forward keeps for the backward
+  int8_t* x_q8; void* x_qt;
+  void* qkv; void* qkv_qt;
+  void* P; void* P_qt;
+  void* ctx; int8_t* ctx_q8; void* ctx_qt;
+  void* y1; float* mean1; float* rstd1;
+  void* a; int8_t* a_q8; void* a_qt;
+  void* u; int8_t* g_q8; void* g_qt;
+  void* y2; float* mean2; float* rstd2;
+  float* part;                          // [(N_SITES + 1) * RED_BLOCKS] per-block partial sums
+};
+
+struct LayerBind {
+  void* teacher[MREM_N_PARAMS] = {};
+  float* student[MREM_N_PARAMS] = {};
+  float* w_steps[N_WMAT] = {};
+  float* a_steps[N_SITES] = {};
+  float* a_off[N_SITES] = {};
+};
+
+struct LayerGrad {
+  float* p[MREM_N_PARAMS];              // parameter gradients
+  float* ws[N_WMAT];                    // weight-step gradients
+  float* a;                             // [N_SITES]
+  float* off;                           // [N_SITES]
+  float* m_p[MREM_N_PARAMS]; float* v_p[MREM_N_PARAMS];
+  float* m_ws[N_WMAT]; float* v_ws[N_WMAT];
+  float* m_a; float* v_a; float* m_off; float* v_off;
+};
+
+struct Arena {                          // bump allocator over the workspace (base may be null: sizing pass)
+  char* base = nullptr;
+  size_t off = 0;
+  void* take(size_t bytes) {
+    off = (off + 255) & ~size_t(255);
+    void* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+}  // namespace mrem
+
+struct mrem_ctx {
+  mrem_module_desc d;
+  cudaStream_t stream = nullptr;
+  int sm_count = 148;
+  int dt = 1;                           // storage type id (0 f32, 1 bf16)
+  size_t esz = 2;
+  long long max_tokens = 0;
+  std::string err;
+  char* ws_base = nullptr;
+
+  std::vector<mrem::LayerBind> bind;
+  std::vector<mrem::LayerStash> stash;
+  std::vector<mrem::LayerGrad> grad;
+  std::vector<std::vector<mrem::WeightBuf>> wq;     // [layer][4]
+
+  // shared scratch
+  void *t_qkv, *t_P, *t_ctx, *t_y1, *t_a, *t_g, *t_y2;   // teacher activations
+  float* scores;
+  void* x_mix;                                          // Eq. 4 input of the student
+  void* dF;                                             // [L, M, H] loss gradients
+  void *d_y2, *d_ghat, *d_u, *d_ahat, *d_a, *d_y1, *d_ctxhat, *d_ctx, *d_phat, *d_s, *d_qkvhat, *d_qkv, *d_xhat,
+      *d_sum, *carry[2];
+  float* col_scratch;
+  float* rowbias;
+  float* loss_partial;
+  float* minmax;
+  int* status;
+  int* t_counter;
+  mrem::OptimScalars* optim_sc;
+  mrem::ReduceEntry* reduce_table;   int reduce_per_layer = 0;
+  mrem::AdamEntry* adam_table;       int adam_entries = 0;
+  void *h2d_xt, *h2d_xs; int32_t* h2d_len; float* d_loss_e2e;   // staging of mrem_recon_step_host
+  void *e2e_t_out, *e2e_s_out;                                  // its layer outputs [L, M, H]
+  size_t state_off = 0, state_bytes = 0;                          // optimizer moments: one contiguous range
+  bool tables_dirty = true;
+
+  // per-step state
+  bool weights_quantized = false, have_teacher = false, have_student = false, have_loss = false, have_grads = false;
+  const void* s_in = nullptr;  void* s_out = nullptr;  const void* t_out = nullptr;
+  const int32_t* cur_len = nullptr;
+  int cur_batch = 0, cur_seq = 0;
+
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t graph_exec = nullptr;
+  float* h_pinned_loss = nullptr;
+};

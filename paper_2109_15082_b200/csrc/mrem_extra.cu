@@ -1,0 +1,152 @@
+// C-ABI entry points built on the step: activation-step initialisation, the host-buffer
+// step, CUDA-graph capture of a step, and the single operations exposed for verification.
+#include "mrem_ctx.h"
+
+using namespace mrem;
+
+namespace mrem {
+int fail(mrem_ctx* c, int code, const char* msg);
+int build_tables(mrem_ctx* c);
+int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, void* outs, bool student_params,
+                  bool init_steps);
+}  // namespace mrem
+
+namespace {
+
+int enqueue_step(mrem_ctx* c, const void* xt, const void* xs, float lambda, const int32_t* len, int batch, int seq,
+                 void* t_out, void* s_out, float* d_loss, const mrem_optim* o) {
+  int rc = mrem_quantize_weights(c);
+  if (rc == MREM_OK) rc = mrem_module_forward(c, MREM_TEACHER, xt, nullptr, 0.f, len, batch, seq, t_out);
+  if (rc == MREM_OK) rc = mrem_module_forward(c, MREM_STUDENT, xs, xt, lambda, len, batch, seq, s_out);
+  if (rc == MREM_OK) rc = mrem_recon_loss(c, d_loss, nullptr);
+  if (rc == MREM_OK) rc = mrem_module_backward(c);
+  if (rc == MREM_OK) rc = mrem_step(c, o);
+  return rc;
+}
+
+int map_gemm_rc(int rc) {
+  return rc == GEMM_OK ? MREM_OK : (rc == GEMM_ERR_ALIGN ? MREM_ERR_ALIGN : (rc == GEMM_ERR_ARG ? MREM_ERR_ARG : MREM_ERR_CUDA));
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t mrem_init_act_steps(mrem_ctx* c, const void* x, const int32_t* len, int32_t batch, int32_t seq) {
+  if (!c || !x) return MREM_ERR_ARG;
+  if (batch < 1 || seq < 1 || batch > c->d.max_batch || seq > c->d.max_seq) return fail(c, MREM_ERR_SHAPE, "init_act_steps: batch/seq outside the context's maximum");
+  for (int l = 0; l < c->d.n_layers; ++l) {
+    for (int k = 0; k < N_SITES; ++k) if (!c->bind[l].a_steps[k]) return fail(c, MREM_ERR_ORDER, "init_act_steps: activation steps not bound");
+    if ((c->d.act_asym_sites & 2) && !c->bind[l].a_off[7]) return fail(c, MREM_ERR_ORDER, "init_act_steps: GELU-site offset not bound");
+  }
+  const int rc = float_forward(c, x, len, batch, seq, c->e2e_s_out, true, true);
+  c->weights_quantized = false;      // the w_hat buffers were used as scratch
+  return rc;
+}
+
+int32_t mrem_recon_step_host(mrem_ctx* c, const void* h_xt, const void* h_xs, const int32_t* h_len, int32_t batch,
+                             int32_t seq, float lambda, const mrem_optim* o, float* h_loss) {
+  if (!c || !h_xt || !h_xs || !o || !h_loss) return MREM_ERR_ARG;
+  if (batch < 1 || seq < 1 || batch > c->d.max_batch || seq > c->d.max_seq) return fail(c, MREM_ERR_SHAPE, "recon_step_host: batch/seq outside the context's maximum");
+  const size_t bytes = (size_t)batch * seq * c->d.hidden * c->esz;
+  if (cudaMemcpyAsync(c->h2d_xt, h_xt, bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
+  const void* xs = c->h2d_xt;
+  if (h_xs != h_xt) {
+    if (cudaMemcpyAsync(c->h2d_xs, h_xs, bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
+    xs = c->h2d_xs;
+  }
+  const int32_t* len = nullptr;
+  if (h_len) {
+    if (cudaMemcpyAsync(c->h2d_len, h_len, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
+    len = c->h2d_len;
+  }
+  const int rc = enqueue_step(c, c->h2d_xt, xs, lambda, len, batch, seq, c->e2e_t_out, c->e2e_s_out, c->d_loss_e2e, o);
+  if (rc != MREM_OK) return rc;
+  if (cudaMemcpyAsync(c->h_pinned_loss, c->d_loss_e2e, sizeof(float), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaStreamSynchronize(c->stream) != cudaSuccess)
+    return fail(c, MREM_ERR_CUDA, "recon_step_host: device error");
+  *h_loss = *c->h_pinned_loss;
+  return MREM_OK;
+}
+
+int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, float lambda, const int32_t* len,
+                                int32_t batch, int32_t seq, void* t_out, void* s_out, float* d_loss,
+                                const mrem_optim* o) {
+  if (!c || !xt || !xs || !t_out || !s_out || !d_loss || !o) return MREM_ERR_ARG;
+  if (o->step > 0) return fail(c, MREM_ERR_ARG, "graph_capture_step: optim.step must be 0 (device-side counter)");
+  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
+  if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+  if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_capture_step: begin capture failed");
+  const int rc = enqueue_step(c, xt, xs, lambda, len, batch, seq, t_out, s_out, d_loss, o);
+  cudaGraph_t g = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+  if (rc != MREM_OK) { if (g) cudaGraphDestroy(g); return rc; }
+  if (e != cudaSuccess || !g) return fail(c, MREM_ERR_CUDA, "graph_capture_step: end capture failed");
+  c->graph = g;
+  if (cudaGraphInstantiate(&c->graph_exec, g, 0) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_capture_step: instantiate failed");
+  return MREM_OK;
+}
+
+int32_t mrem_graph_launch(mrem_ctx* c) {
+  if (!c) return MREM_ERR_ARG;
+  if (!c->graph_exec) return fail(c, MREM_ERR_ORDER, "graph_launch: no captured step");
+  return cudaGraphLaunch(c->graph_exec, c->stream) == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "graph_launch failed");
+}
+
+// ------------------------------------------------------------------ single operations
+
+int32_t mrem_quantize_act(const void* x, int32_t dtype, int64_t n, const float* step, const float* offset, int32_t lo,
+                          int32_t hi, int8_t* q8, void* qt, void* st) {
+  if (!x || !step || n < 0 || (dtype != MREM_F32 && dtype != MREM_BF16) || lo > hi || lo < -128 || hi > 255) return MREM_ERR_ARG;
+  if (n == 0) return MREM_OK;
+  // a flat tensor is a view of `rows` rows of 2^k columns (largest power of two <= 4096 dividing n)
+  int cols = 1;
+  while (cols < 4096 && n % (cols * 2) == 0) cols *= 2;
+  const long long rows = n / cols;
+  launch_quantize_act(x, dtype, rows, cols, cols, step, offset, lo, hi, q8, cols, qt, cols, (cudaStream_t)st);
+  return cudaGetLastError() == cudaSuccess ? MREM_OK : MREM_ERR_CUDA;
+}
+
+int32_t mrem_quantize_weight(const float* w, int32_t rows, int32_t cols, const float* steps, int32_t per_row,
+                             int32_t bits, int32_t grid, int8_t* codes, int32_t* rowsum, float* scale, void* what,
+                             int32_t dtype, void* st) {
+  if (!w || !steps || !codes || !rowsum || !scale || rows < 0 || cols < 1) return MREM_ERR_ARG;
+  if ((bits != 2 && bits != 4 && bits != 8) || (grid != 0 && !(grid == 1 && bits == 2))) return MREM_ERR_UNSUPPORTED;
+  if (dtype != MREM_F32 && dtype != MREM_BF16) return MREM_ERR_ARG;
+  if (rows == 0) return MREM_OK;
+  launch_quantize_weight(w, rows, cols, steps, per_row, bits, grid, codes, rowsum, scale, what, dtype, (cudaStream_t)st);
+  return cudaGetLastError() == cudaSuccess ? MREM_OK : MREM_ERR_CUDA;
+}
+
+int32_t mrem_gemm_i8(const int8_t* a, int32_t a_unsigned, const int8_t* b, int32_t M, int32_t N, int32_t K,
+                     int32_t* acc, int32_t block_n, int32_t* d_status, void* st) {
+  if (!a || !b || !acc || !d_status || M < 0 || N < 0 || K < 1) return MREM_ERR_ARG;
+  if (K % 16) return MREM_ERR_ALIGN;
+  if (M == 0 || N == 0) return MREM_OK;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MREM_ERR_CUDA;
+  OperandDesc A{a, K, 0, 0, 0}, B{b, K, 0, 0, 0};
+  GemmShape g{M, N, K, 1, 1};
+  Epilogue e{};
+  e.out = acc; e.out_kind = OUT_I32; e.ldc = N; e.alpha_const = 1.f;
+  return map_gemm_rc(tc_gemm(1, a_unsigned, A, B, g, e, block_n, d_status, sms, (cudaStream_t)st));
+}
+
+int32_t mrem_gemm(int32_t dtype, const void* a, int32_t a_mn, int64_t lda, int64_t a_bs, const void* b, int32_t b_mn,
+                  int64_t ldb, int64_t b_bs, int32_t M, int32_t N, int32_t K, int32_t batches, float alpha, float* out,
+                  int64_t ldc, int64_t c_bs, int32_t block_n, int32_t* d_status, void* st) {
+  if (!a || !b || !out || !d_status || M < 0 || N < 0 || K < 1 || batches < 1) return MREM_ERR_ARG;
+  if (dtype != MREM_F32 && dtype != MREM_BF16) return MREM_ERR_ARG;
+  if (M == 0 || N == 0) return MREM_OK;
+  OperandDesc A{a, lda, a_bs, 0, a_mn}, B{b, ldb, b_bs, 0, b_mn};
+  GemmShape g{M, N, K, batches, 1};
+  Epilogue e{};
+  e.out = out; e.out_kind = OUT_F32; e.ldc = ldc; e.c_b0 = c_bs; e.alpha_const = alpha;
+  if (dtype == MREM_F32) return map_gemm_rc(simt_gemm_f32(A, B, g, e, (cudaStream_t)st));
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MREM_ERR_CUDA;
+  return map_gemm_rc(tc_gemm(0, 0, A, B, g, e, block_n, d_status, sms, (cudaStream_t)st));
+}
+
+}  // extern "C"

@@ -1,0 +1,381 @@
+// The reconstruction step (Algorithm 2): weight quantization, teacher and student forward,
+// loss (Eq. 3), straight-through backward and the AdamW update, as sequences of kernel
+// launches on the context's stream.  No host synchronisation, no allocation.
+#include <cmath>
+
+#include "mrem_ctx.h"
+
+using namespace mrem;
+
+namespace mrem {
+int fail(mrem_ctx* c, int code, const char* msg);
+void param_shape(const mrem_module_desc& d, int id, int* rows, int* cols);
+int build_tables(mrem_ctx* c);
+}  // namespace mrem
+
+namespace {
+
+const int kMatParam[N_WMAT] = {MREM_WQKV, MREM_WO, MREM_W1, MREM_W2};
+enum { W_QKV = 0, W_O = 1, W_1 = 2, W_2 = 3 };
+enum { S_X = 0, S_Q = 1, S_K = 2, S_V = 3, S_P = 4, S_C = 5, S_A = 6, S_G = 7 };
+
+struct View {                      // an operand: pointer, stride of the non-contiguous index, batch strides
+  const void* p; long long ld, sb0, sb1; int mn;
+};
+inline View view(const void* p, long long ld, int mn = 0, long long sb0 = 0, long long sb1 = 0) {
+  return View{p, ld, sb0, sb1, mn};
+}
+
+struct Epi {                       // shorthand builder of an Epilogue
+  Epilogue e{};
+  Epi(void* out, int kind, long long ldc, long long cb0 = 0, long long cb1 = 0) {
+    e.out = out; e.out_kind = kind; e.ldc = ldc; e.c_b0 = cb0; e.c_b1 = cb1; e.alpha_const = 1.f;
+  }
+  Epi& alpha(float a, const float* p0 = nullptr, const float* p1 = nullptr) { e.alpha_const = a; e.alpha_p0 = p0; e.alpha_p1 = p1; return *this; }
+  Epi& colscale(const float* p) { e.col_scale = p; return *this; }
+  Epi& colbias(const float* p) { e.col_bias = p; return *this; }
+  Epi& rowbias(const float* p) { e.row_bias = p; return *this; }
+  Epi& residual(const void* p) { e.residual = p; return *this; }
+  Epi& gelu() { e.act = 1; return *this; }
+};
+
+struct Runner {
+  mrem_ctx* c;
+  int rc = MREM_OK;
+  explicit Runner(mrem_ctx* ctx) : c(ctx) {}
+  int okind() const { return c->dt == 1 ? OUT_BF16 : OUT_F32; }
+  void* at(const void* p, long long elems) const { return (char*)p + elems * (long long)c->esz; }
+
+  void note(int grc, const char* what) {
+    if (grc != GEMM_OK && rc == MREM_OK) {
+      rc = grc == GEMM_ERR_ALIGN ? MREM_ERR_ALIGN : (grc == GEMM_ERR_ARG ? MREM_ERR_ARG : MREM_ERR_CUDA);
+      c->err = what;
+    }
+  }
+  // storage-type product on the tensor cores (bf16) or CUDA cores (f32)
+  void gemm(const View& A, const View& B, int M, int N, int K, int nb0, int nb1, const Epilogue& e) {
+    OperandDesc a{A.p, A.ld, A.sb0, A.sb1, A.mn}, b{B.p, B.ld, B.sb0, B.sb1, B.mn};
+    GemmShape g{M, N, K, nb0, nb1};
+    if (c->dt == 1) note(tc_gemm(0, 0, a, b, g, e, 0, c->status, c->sm_count, c->stream), "bf16 GEMM launch failed");
+    else note(simt_gemm_f32(a, b, g, e, c->stream), "f32 GEMM launch failed");
+  }
+  // integer-code product with exact int32 accumulation
+  void gemm_i8(const int8_t* A, int a_unsigned, const int8_t* B, int M, int N, int K, const Epilogue& e) {
+    OperandDesc a{A, K, 0, 0, 0}, b{B, K, 0, 0, 0};
+    GemmShape g{M, N, K, 1, 1};
+    note(tc_gemm(1, a_unsigned, a, b, g, e, 0, c->status, c->sm_count, c->stream), "int8 GEMM launch failed");
+  }
+};
+
+struct ActRange { int lo, hi; bool asym; };
+ActRange site_range(const mrem_module_desc& d, int site) {
+  const bool asym = (site == S_P && (d.act_asym_sites & 1)) || (site == S_G && (d.act_asym_sites & 2));
+  if (asym) return {0, (1 << d.a_bits) - 1, true};
+  const int q = (1 << (d.a_bits - 1)) - 1;
+  return {-q, q, false};
+}
+
+int check_io(mrem_ctx* c, const void* x, int batch, int seq, void* outs) {
+  if (!x || !outs) return fail(c, MREM_ERR_ARG, "forward: NULL tensor");
+  if (batch < 1 || seq < 1 || batch > c->d.max_batch || seq > c->d.max_seq) return fail(c, MREM_ERR_SHAPE, "forward: batch/seq outside the context's maximum");
+  if (c->dt == 1 && seq % 8) return fail(c, MREM_ERR_SHAPE, "forward: bf16 path needs seq % 8 == 0");
+  if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(outs) & 15)) return fail(c, MREM_ERR_ALIGN, "forward: tensors must be 16-byte aligned");
+  return MREM_OK;
+}
+
+// Sets one activation step (and offset) from the range of a 2-D view.
+void init_site(mrem_ctx* c, const LayerBind& b, int site, const void* x, long long ld, long long rows, int cols) {
+  const ActRange r = site_range(c->d, site);
+  launch_minmax(x, ld, rows, cols, c->minmax, c->col_scratch, c->dt, c->stream);
+  const int mode = !r.asym ? 0 : (site == S_P ? 1 : 2);
+  launch_step_from_minmax(c->minmax, mode, (float)r.hi, b.a_steps[site], mode == 2 ? b.a_off[site] : nullptr, c->stream);
+}
+
+}  // namespace
+
+namespace mrem {
+// ------------------------------------------------------------------ full-precision forward
+// The teacher pass.  With `student_params` the same graph runs on the student's latent
+// parameters (matrices narrowed to the storage type in the w_hat buffers) and, with
+// `init_steps`, sets every activation step of the student from the ranges it sees.
+int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, void* outs, bool student_params,
+                  bool init_steps) {
+  const mrem_module_desc& d = c->d;
+  const int H = d.hidden, F = d.ffn, h = d.n_heads, hd = H / h;
+  const long long M = (long long)B * S;
+  Runner r(c);
+  const int ok = r.okind();
+  const void* cur = x;
+  for (int l = 0; l < d.n_layers; ++l) {
+    LayerBind b = c->bind[l];
+    if (student_params) {
+      for (int k = 0; k < MREM_N_PARAMS; ++k) {
+        if (!b.student[k]) return fail(c, MREM_ERR_ORDER, "forward: student parameters not bound");
+        b.teacher[k] = b.student[k];
+      }
+      for (int k = 0; k < N_WMAT; ++k) {
+        WeightBuf& w = c->wq[l][k];
+        launch_narrow(b.student[kMatParam[k]], w.what, (long long)w.rows * w.cols, c->dt, c->stream);
+        b.teacher[kMatParam[k]] = w.what;
+      }
+    }
+    for (int k = 0; k < MREM_N_PARAMS; ++k) if (!b.teacher[k]) return fail(c, MREM_ERR_ORDER, "forward: teacher parameters not bound");
+    void* out = r.at(outs, (long long)l * M * H);
+    if (init_steps) init_site(c, b, S_X, cur, H, M, H);
+    r.gemm(view(cur, H), view(b.teacher[MREM_WQKV], H), (int)M, 3 * H, H, 1, 1,
+           Epi(c->t_qkv, ok, 3 * H).colbias((float*)b.teacher[MREM_BQKV]).e);
+    r.gemm(view(c->t_qkv, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(c->t_qkv, H), 3 * H, 0, hd, (long long)S * 3 * H),
+           S, S, hd, h, B, Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd)).e);
+    if (init_steps)
+      for (int seg = 0; seg < 3; ++seg) init_site(c, b, S_Q + seg, r.at(c->t_qkv, seg * H), 3 * H, M, H);
+    launch_softmax_fwd(c->scores, len, B, h, S, c->t_P, nullptr, nullptr, 0, 0, nullptr, c->dt, c->stream);
+    if (init_steps) init_site(c, b, S_P, c->t_P, S, (long long)B * h * S, S);
+    r.gemm(view(c->t_P, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(c->t_qkv, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
+           S, hd, S, h, B, Epi(c->t_ctx, ok, H, hd, (long long)S * H).e);
+    if (init_steps) init_site(c, b, S_C, c->t_ctx, H, M, H);
+    r.gemm(view(c->t_ctx, H), view(b.teacher[MREM_WO], H), (int)M, H, H, 1, 1,
+           Epi(c->t_y1, ok, H).colbias((float*)b.teacher[MREM_BO]).residual(cur).e);
+    launch_layernorm_fwd(c->t_y1, (float*)b.teacher[MREM_LN1_G], (float*)b.teacher[MREM_LN1_B], d.ln_eps, M, H, c->t_a,
+                         nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, c->stream);
+    if (init_steps) init_site(c, b, S_A, c->t_a, H, M, H);
+    r.gemm(view(c->t_a, H), view(b.teacher[MREM_W1], H), (int)M, F, H, 1, 1,
+           Epi(c->t_g, ok, F).colbias((float*)b.teacher[MREM_B1]).gelu().e);
+    if (init_steps) init_site(c, b, S_G, c->t_g, F, M, F);
+    r.gemm(view(c->t_g, F), view(b.teacher[MREM_W2], F), (int)M, H, F, 1, 1,
+           Epi(c->t_y2, ok, H).colbias((float*)b.teacher[MREM_B2]).residual(c->t_a).e);
+    launch_layernorm_fwd(c->t_y2, (float*)b.teacher[MREM_LN2_G], (float*)b.teacher[MREM_LN2_B], d.ln_eps, M, H, out,
+                         nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, c->stream);
+    cur = out;
+  }
+  if (r.rc != MREM_OK) return r.rc;
+  return cudaGetLastError() == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "forward: launch failed");
+}
+}  // namespace mrem
+
+namespace {
+
+// ------------------------------------------------------------------ student
+// The fake-quantized pass: a quantizer on both operands of every matrix product.
+// Linear layers run on int8 codes with exact int32 accumulation; attention products on codes held as storage-type numbers.
+int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, void* outs) {
+  const mrem_module_desc& d = c->d;
+  const int H = d.hidden, F = d.ffn, h = d.n_heads, hd = H / h;
+  const long long M = (long long)B * S;
+  Runner r(c);
+  const int ok = r.okind();
+  const void* cur = x;
+  for (int l = 0; l < d.n_layers; ++l) {
+    const LayerBind& b = c->bind[l];
+    LayerStash& s = c->stash[l];
+    std::vector<WeightBuf>& w = c->wq[l];
+    for (int k = 0; k < MREM_N_PARAMS; ++k) if (!b.student[k]) return fail(c, MREM_ERR_ORDER, "forward: student parameters not bound");
+    for (int k = 0; k < N_SITES; ++k) if (!b.a_steps[k]) return fail(c, MREM_ERR_ORDER, "forward: activation steps not bound");
+    if ((d.act_asym_sites & 2) && !b.a_off[S_G]) return fail(c, MREM_ERR_ORDER, "forward: GELU-site offset not bound");
+    void* out = r.at(outs, (long long)l * M * H);
+    const ActRange rx = site_range(d, S_X), rp = site_range(d, S_P), rg = site_range(d, S_G);
+
+    launch_quantize_act(cur, c->dt, M, H, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi, s.x_q8, H, s.x_qt, H, c->stream);
+    r.gemm_i8(s.x_q8, 0, w[W_QKV].codes, (int)M, 3 * H, H,
+              Epi(s.qkv, ok, 3 * H).alpha(1.f, b.a_steps[S_X]).colscale(w[W_QKV].scale).colbias(b.student[MREM_BQKV]).e);
+    for (int seg = 0; seg < 3; ++seg)
+      launch_quantize_act(r.at(s.qkv, seg * H), c->dt, M, H, 3 * H, b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, nullptr, 0,
+                          r.at(s.qkv_qt, seg * H), 3 * H, c->stream);
+    r.gemm(view(s.qkv_qt, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(s.qkv_qt, H), 3 * H, 0, hd, (long long)S * 3 * H),
+           S, S, hd, h, B,
+           Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd), b.a_steps[S_Q], b.a_steps[S_K]).e);
+    launch_softmax_fwd(c->scores, len, B, h, S, s.P, b.a_steps[S_P], nullptr, rp.lo, rp.hi, s.P_qt, c->dt, c->stream);
+    r.gemm(view(s.P_qt, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(s.qkv_qt, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
+           S, hd, S, h, B, Epi(s.ctx, ok, H, hd, (long long)S * H).alpha(1.f, b.a_steps[S_P], b.a_steps[S_V]).e);
+    launch_quantize_act(s.ctx, c->dt, M, H, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi, s.ctx_q8, H, s.ctx_qt, H, c->stream);
+    r.gemm_i8(s.ctx_q8, 0, w[W_O].codes, (int)M, H, H,
+              Epi(s.y1, ok, H).alpha(1.f, b.a_steps[S_C]).colscale(w[W_O].scale).colbias(b.student[MREM_BO]).residual(cur).e);
+    launch_layernorm_fwd(s.y1, b.student[MREM_LN1_G], b.student[MREM_LN1_B], d.ln_eps, M, H, s.a, s.mean1, s.rstd1,
+                         b.a_steps[S_A], rx.hi, s.a_q8, s.a_qt, c->dt, c->stream);
+    r.gemm_i8(s.a_q8, 0, w[W_1].codes, (int)M, F, H,
+              Epi(s.u, ok, F).alpha(1.f, b.a_steps[S_A]).colscale(w[W_1].scale).colbias(b.student[MREM_B1]).e);
+    launch_gelu_quant(s.u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, s.g_q8, s.g_qt, c->dt, c->stream);
+    const float* bias2 = b.student[MREM_B2];
+    if (rg.asym) {
+      launch_effective_bias(b.student[MREM_B2], b.a_off[S_G], w[W_2].scale, w[W_2].rowsum, w[W_2].beff, H, c->stream);
+      bias2 = w[W_2].beff;
+    }
+    r.gemm_i8(s.g_q8, rg.asym ? 1 : 0, w[W_2].codes, (int)M, H, F,
+              Epi(s.y2, ok, H).alpha(1.f, b.a_steps[S_G]).colscale(w[W_2].scale).colbias(bias2).residual(s.a).e);
+    launch_layernorm_fwd(s.y2, b.student[MREM_LN2_G], b.student[MREM_LN2_B], d.ln_eps, M, H, out, s.mean2, s.rstd2,
+                         nullptr, 0, nullptr, nullptr, c->dt, c->stream);
+    cur = out;
+  }
+  if (r.rc != MREM_OK) return r.rc;
+  return cudaGetLastError() == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "student forward: launch failed");
+}
+
+// ------------------------------------------------------------------ backward
+int student_backward(mrem_ctx* c) {
+  const mrem_module_desc& d = c->d;
+  const int H = d.hidden, F = d.ffn, h = d.n_heads, hd = H / h, B = c->cur_batch, S = c->cur_seq;
+  const long long M = (long long)B * S;
+  const long long sSS = (long long)S * S, sHSS = (long long)h * S * S, sQKV = (long long)S * 3 * H;
+  Runner r(c);
+  const int ok = r.okind();
+  const float inv_sqrt_d = 1.f / sqrtf((float)hd);
+  const void* carry = nullptr;
+  for (int l = d.n_layers - 1; l >= 0; --l) {
+    const LayerBind& b = c->bind[l];
+    LayerStash& s = c->stash[l];
+    LayerGrad& g = c->grad[l];
+    std::vector<WeightBuf>& w = c->wq[l];
+    const void* x_in = l == 0 ? c->s_in : r.at(c->s_out, (long long)(l - 1) * M * H);
+    const void* dF = r.at(c->dF, (long long)l * M * H);
+    const ActRange rx = site_range(d, S_X), rp = site_range(d, S_P), rg = site_range(d, S_G);
+    float* part = s.part;
+    cudaStream_t st = c->stream;
+
+    // second LayerNorm: total gradient at the layer output = loss term + what the next layer sent back
+    launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, carry ? c->d_sum : nullptr, c->dt, st);
+    launch_col_reduce(carry ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G], c->col_scratch, c->dt, st);
+    // FFN2:  y2 = G_hat W2_hat^T + b2 + a
+    launch_col_reduce(c->d_y2, H, nullptr, nullptr, nullptr, M, H, g.p[MREM_B2], nullptr, c->col_scratch, c->dt, st);
+    r.gemm(view(c->d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
+    {
+      Epi e(g.p[MREM_W2], OUT_F32, F);
+      e.alpha(1.f, b.a_steps[S_G]);
+      if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], c->rowbias, H, st); e.rowbias(c->rowbias); }
+      r.gemm(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, 1, 1, e.e);
+    }
+    launch_gelu_bwd(s.u, c->d_ghat, c->d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
+                    part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
+    // FFN1:  u = A_hat W1_hat^T + b1
+    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, M, F, g.p[MREM_B1], nullptr, c->col_scratch, c->dt, st);
+    r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
+    r.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
+    launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
+                   part + S_A * RED_BLOCKS, nullptr, c->dt, st);
+    // first LayerNorm
+    launch_layernorm_bwd(c->d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, c->d_y1, nullptr, c->dt, st);
+    launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], c->col_scratch, c->dt, st);
+    // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x
+    launch_col_reduce(c->d_y1, H, nullptr, nullptr, nullptr, M, H, g.p[MREM_BO], nullptr, c->col_scratch, c->dt, st);
+    r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
+    r.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
+    launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
+                   part + S_C * RED_BLOCKS, nullptr, c->dt, st);
+    // attention:  ctx = P_hat V_hat,  P = softmax(Q_hat K_hat^T / sqrt(d))
+    r.gemm(view(c->d_ctx, H, 0, hd, (long long)S * H), view(r.at(s.qkv_qt, 2 * H), 3 * H, 0, hd, sQKV), S, S, hd, h, B,
+           Epi(c->d_phat, ok, S, sSS, sHSS).alpha(1.f, b.a_steps[S_V]).e);
+    r.gemm(view(s.P_qt, S, 1, sSS, sHSS), view(c->d_ctx, H, 1, hd, (long long)S * H), S, hd, S, h, B,
+           Epi(r.at(c->d_qkvhat, 2 * H), ok, 3 * H, hd, sQKV).alpha(1.f, b.a_steps[S_P]).e);
+    launch_softmax_bwd(s.P, c->d_phat, c->d_s, (long long)B * h * S, S, b.a_steps[S_P], rp.lo, rp.hi, 1, part + S_P * RED_BLOCKS, c->dt, st);
+    r.gemm(view(c->d_s, S, 0, sSS, sHSS), view(r.at(s.qkv_qt, H), 3 * H, 1, hd, sQKV), S, hd, S, h, B,
+           Epi(c->d_qkvhat, ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_K]).e);
+    r.gemm(view(c->d_s, S, 1, sSS, sHSS), view(s.qkv_qt, 3 * H, 1, hd, sQKV), S, hd, S, h, B,
+           Epi(r.at(c->d_qkvhat, H), ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_Q]).e);
+    for (int seg = 0; seg < 3; ++seg)
+      launch_ste_act(r.at(s.qkv, seg * H), 3 * H, r.at(c->d_qkvhat, seg * H), 3 * H, nullptr, 0, r.at(c->d_qkv, seg * H), 3 * H, M, H,
+                     b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, part + (S_Q + seg) * RED_BLOCKS, nullptr, c->dt, st);
+    // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
+    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, M, 3 * H, g.p[MREM_BQKV], nullptr, c->col_scratch, c->dt, st);
+    r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
+    r.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
+    void* next_carry = c->carry[l & 1];
+    launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
+                   part + S_X * RED_BLOCKS, nullptr, c->dt, st);
+    carry = next_carry;
+    // weight quantizers: mask the latent-weight gradients, reduce the step gradients
+    for (int k = 0; k < N_WMAT; ++k)
+      launch_ste_weight(b.student[kMatParam[k]], b.w_steps[k], d.w_step_per_row, d.w_bits, d.w_grid, g.p[kMatParam[k]],
+                        w[k].rows, w[k].cols, d.w_step_per_row ? g.ws[k] : w[k].ds_rows, st);
+    launch_reduce_table(c->reduce_table + (size_t)l * c->reduce_per_layer, c->reduce_per_layer, st);
+  }
+  if (r.rc != MREM_OK) return r.rc;
+  return cudaGetLastError() == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "backward: launch failed");
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t mrem_quantize_weights(mrem_ctx* c) {
+  if (!c) return MREM_ERR_ARG;
+  for (int l = 0; l < c->d.n_layers; ++l)
+    for (int k = 0; k < N_WMAT; ++k) {
+      const LayerBind& b = c->bind[l];
+      if (!b.student[kMatParam[k]] || !b.w_steps[k]) return fail(c, MREM_ERR_ORDER, "quantize_weights: weights or steps not bound");
+      WeightBuf& w = c->wq[l][k];
+      launch_quantize_weight(b.student[kMatParam[k]], w.rows, w.cols, b.w_steps[k], c->d.w_step_per_row, c->d.w_bits,
+                             c->d.w_grid, w.codes, w.rowsum, w.scale, w.what, c->dt, c->stream);
+    }
+  if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "quantize_weights: launch failed");
+  c->weights_quantized = true;
+  return MREM_OK;
+}
+
+int32_t mrem_module_forward(mrem_ctx* c, int32_t role, const void* x, const void* x_other, float lambda,
+                            const int32_t* len, int32_t batch, int32_t seq, void* outs) {
+  if (!c) return MREM_ERR_ARG;
+  int rc = check_io(c, x, batch, seq, outs);
+  if (rc != MREM_OK) return rc;
+  if (c->have_teacher || c->have_student) {
+    if (batch != c->cur_batch || seq != c->cur_seq) { c->have_teacher = c->have_student = false; }
+  }
+  if (role == MREM_TEACHER) {
+    rc = float_forward(c, x, len, batch, seq, outs, false, false);
+    if (rc != MREM_OK) return rc;
+    c->t_out = outs; c->have_teacher = true;
+  } else if (role == MREM_STUDENT) {
+    if (!c->weights_quantized) return fail(c, MREM_ERR_ORDER, "forward(student): call mrem_quantize_weights first");
+    const void* in = x;
+    if (lambda != 0.f) {
+      if (!x_other) return fail(c, MREM_ERR_ARG, "forward(student): lambda != 0 needs d_x_other");
+      if (!(lambda >= 0.f && lambda <= 1.f)) return fail(c, MREM_ERR_ARG, "forward(student): lambda outside [0, 1]");
+      launch_mix(x_other, x, lambda, c->x_mix, (long long)batch * seq * c->d.hidden, c->dt, c->stream);
+      in = c->x_mix;
+    }
+    rc = student_forward(c, in, len, batch, seq, outs);
+    if (rc != MREM_OK) return rc;
+    c->s_in = in; c->s_out = outs; c->have_student = true;
+  } else {
+    return fail(c, MREM_ERR_ARG, "forward: role");
+  }
+  c->cur_batch = batch; c->cur_seq = seq; c->cur_len = len;
+  c->have_loss = false; c->have_grads = false;
+  return MREM_OK;
+}
+
+int32_t mrem_recon_loss(mrem_ctx* c, float* loss_total, float* loss_per_layer) {
+  if (!c || !loss_total) return MREM_ERR_ARG;
+  if (!c->have_teacher || !c->have_student) return fail(c, MREM_ERR_ORDER, "recon_loss: needs a teacher and a student forward of the same batch");
+  const long long n = (long long)c->cur_batch * c->cur_seq * c->d.hidden;
+  const float cc = c->d.loss_mean ? 1.f / (float)n : 1.f;
+  launch_loss(c->s_out, c->t_out, c->d.n_layers, n, cc, c->dF, c->loss_partial, c->status, c->dt, c->stream);
+  launch_loss_finalize(c->loss_partial, c->d.n_layers, cc, loss_total, loss_per_layer, c->stream);
+  if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_loss: launch failed");
+  c->have_loss = true;
+  return MREM_OK;
+}
+
+int32_t mrem_module_backward(mrem_ctx* c) {
+  if (!c) return MREM_ERR_ARG;
+  if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
+  for (int l = 0; l < c->d.n_layers; ++l)
+    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k]) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
+  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
+  const int rc = student_backward(c);
+  if (rc != MREM_OK) return rc;
+  c->have_grads = true;
+  return MREM_OK;
+}
+
+int32_t mrem_step(mrem_ctx* c, const mrem_optim* o) {
+  if (!c || !o) return MREM_ERR_ARG;
+  if (!c->have_grads) return fail(c, MREM_ERR_ORDER, "step: needs mrem_module_backward of this step");
+  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
+  launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
+                       o->weight_decay, c->stream);
+  launch_adamw_table(c->adam_table, c->adam_entries, c->optim_sc, c->stream);
+  if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "step: launch failed");
+  c->have_grads = false; c->have_loss = false; c->have_student = false; c->have_teacher = false;
+  c->weights_quantized = false;
+  return MREM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,316 @@
+// Quantizer kernels (Eq. 1 of the paper) and step-size initialisation.  HBM-bound:
+// 16-byte vector loads/stores, one pass over each tensor, warp-shuffle reductions.
+#include "kernels.h"
+#include "vec.cuh"
+
+namespace mrem {
+
+namespace {
+
+// ------------------------------------------------------------------ weight quantizer
+// One block per output row.  grid 0: q = rne(clip(w/s, -qmax, qmax)); grid 1 (2-bit,
+// levels (k+0.5)s): c = 2*clip(floor(w/s), -2, 1) + 1 with scale s/2.
+template <typename T>
+__global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __restrict__ w, int cols,
+                                                              const float* __restrict__ steps, int per_row, int bits,
+                                                              int grid, int8_t* __restrict__ codes,
+                                                              int32_t* __restrict__ rowsum, float* __restrict__ scale,
+                                                              T* __restrict__ what) {
+  __shared__ int sh[32];
+  const int row = blockIdx.x;
+  const float s = steps[per_row ? row : 0];
+  const float sc = grid == 0 ? s : 0.5f * s;
+  const float qmax = (float)((1 << (bits - 1)) - 1);
+  const float* wr = w + (long long)row * cols;
+  int8_t* cr = codes + (long long)row * cols;
+  T* hr = what ? what + (long long)row * cols : nullptr;
+  int sum = 0;
+  for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+    const float z = __fdiv_rn(wr[c], s);
+    int q;
+    if (grid == 0) q = __float2int_rn(fminf(fmaxf(z, -qmax), qmax));
+    else q = 2 * (int)fminf(fmaxf(floorf(z), -2.f), 1.f) + 1;
+    cr[c] = (int8_t)q;
+    if (hr) hr[c] = from_f<T>(sc * (float)q);
+    sum += q;
+  }
+  sum = warp_sum_i(sum);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    int v = threadIdx.x < (blockDim.x >> 5) ? sh[threadIdx.x] : 0;
+    v = warp_sum_i(v);
+    if (threadIdx.x == 0) {
+      rowsum[row] = v;
+      scale[row] = sc;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ activation quantizer
+__device__ __forceinline__ int act_code(float x, float s, float off, bool has_off, float lo, float hi) {
+  const float t = has_off ? __fsub_rn(x, off) : x;
+  const float z = __fdiv_rn(t, s);
+  return __float2int_rn(fminf(fmaxf(z, lo), hi));
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__ x, long long rows, int cols,
+                                                           long long ld_x, const float* __restrict__ step,
+                                                           const float* __restrict__ offset, float lo, float hi,
+                                                           int8_t* __restrict__ q8, long long ld_q8,
+                                                           T* __restrict__ qt, long long ld_qt) {
+  const float s = *step;
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  const int vcols = cols / V;
+  const long long total = rows * vcols;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / vcols;
+    const int c = (int)(i - r * vcols) * V;
+    float v[V];
+    load_vec<T, V>(x + r * ld_x + c, v);
+    int q[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) q[j] = act_code(v[j], s, off, has_off, lo, hi);
+    if (q8) store_codes<V>(q8 + r * ld_q8 + c, q);
+    if (qt) {
+#pragma unroll
+      for (int j = 0; j < V; ++j) v[j] = (float)q[j];
+      store_vec<T, V>(qt + r * ld_qt + c, v);
+    }
+  }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) mix_kernel(const T* __restrict__ f, const T* __restrict__ fh, float lam,
+                                                  T* __restrict__ out, long long n) {
+  for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
+    float a[V], b[V];
+    load_vec<T, V>(f + i, a);
+    load_vec<T, V>(fh + i, b);
+#pragma unroll
+    for (int j = 0; j < V; ++j) a[j] = lam * a[j] + (1.f - lam) * b[j];
+    store_vec<T, V>(out + i, a);
+  }
+}
+
+// g = stored(gelu(u)), then the quantizer of the GELU site.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) gelu_quant_kernel(const T* __restrict__ u, long long n,
+                                                         const float* __restrict__ step,
+                                                         const float* __restrict__ offset, float lo, float hi,
+                                                         int8_t* __restrict__ q8, T* __restrict__ qt) {
+  const float s = *step;
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
+    float v[V];
+    load_vec<T, V>(u + i, v);
+    int q[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) q[j] = act_code(stored<T>(gelu_erf(v[j])), s, off, has_off, lo, hi);
+    if (q8) store_codes<V>(q8 + i, q);
+    if (qt) {
+#pragma unroll
+      for (int j = 0; j < V; ++j) v[j] = (float)q[j];
+      store_vec<T, V>(qt + i, v);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ step initialisation
+// stat[row] = max|w| (rule 0) or mean|w| (rule 1) of one row; per_row: steps[row] = stat/qmax | stat.
+__global__ void __launch_bounds__(256) weight_row_stat_kernel(const float* __restrict__ w, int cols, int rule,
+                                                              float* __restrict__ stat) {
+  __shared__ float sh[32];
+  const float* wr = w + (long long)blockIdx.x * cols;
+  float acc = 0.f;
+  for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+    const float a = fabsf(wr[c]);
+    acc = rule == 0 ? fmaxf(acc, a) : acc + a;
+  }
+  acc = rule == 0 ? block_max(acc, sh) : block_sum(acc, sh);
+  if (threadIdx.x == 0) stat[blockIdx.x] = acc;
+}
+__global__ void weight_steps_from_stat_kernel(const float* __restrict__ stat, int rows, int cols, int per_row,
+                                              int rule, float qmax, float* __restrict__ steps) {
+  if (per_row) {
+    for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < rows; r += gridDim.x * blockDim.x) {
+      const float v = rule == 0 ? __fdiv_rn(stat[r], qmax) : __fdiv_rn(stat[r], (float)cols);
+      steps[r] = fmaxf(v, 1e-8f);
+    }
+  } else if (blockIdx.x == 0 && threadIdx.x == 0) {
+    float acc = 0.f;
+    for (int r = 0; r < rows; ++r) acc = rule == 0 ? fmaxf(acc, stat[r]) : acc + stat[r];
+    const float v = rule == 0 ? __fdiv_rn(acc, qmax) : __fdiv_rn(acc, (float)rows * (float)cols);
+    steps[0] = fmaxf(v, 1e-8f);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) minmax_kernel(const T* __restrict__ x, long long ld, long long rows, int cols,
+                                                     float* __restrict__ part) {
+  __shared__ float sh[32];
+  float lo = INFINITY, hi = -INFINITY;
+  const long long total = rows * cols;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / cols;
+    const float v = to_f<T>(x[r * ld + (i - r * cols)]);
+    lo = fminf(lo, v);
+    hi = fmaxf(hi, v);
+  }
+  hi = block_max(hi, sh);
+  lo = -block_max(-lo, sh);
+  if (threadIdx.x == 0) {
+    part[blockIdx.x] = lo;
+    part[gridDim.x + blockIdx.x] = hi;
+  }
+}
+__global__ void minmax_final_kernel(const float* __restrict__ part, int n, float* __restrict__ out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = 0; i < n; ++i) {
+      lo = fminf(lo, part[i]);
+      hi = fmaxf(hi, part[n + i]);
+    }
+    out[0] = lo;
+    out[1] = hi;
+  }
+}
+__global__ void step_from_minmax_kernel(const float* __restrict__ mm, int mode, float qmax, float* step, float* offset) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    float s, o = 0.f;
+    if (mode == 0) s = __fdiv_rn(fmaxf(fabsf(mm[0]), fabsf(mm[1])), qmax);
+    else if (mode == 1) s = __fdiv_rn(mm[1], qmax);
+    else { s = __fdiv_rn(__fsub_rn(mm[1], mm[0]), qmax); o = mm[0]; }
+    *step = fmaxf(s, 1e-8f);
+    if (offset) *offset = o;
+  }
+}
+
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
+                                                          long long row_vecs, uint4* __restrict__ out) {
+  const uint4* s = src + (long long)idx[blockIdx.y] * row_vecs;
+  uint4* o = out + (long long)blockIdx.y * row_vecs;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < row_vecs; i += (long long)gridDim.x * blockDim.x)
+    o[i] = s[i];
+}
+
+__global__ void __launch_bounds__(256) widen_bf16_kernel(const bf16* __restrict__ src, float* __restrict__ dst, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    dst[i] = __bfloat162float(src[i]);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) narrow_kernel(const float* __restrict__ src, T* __restrict__ dst, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    dst[i] = from_f<T>(src[i]);
+}
+
+inline int grid_for(long long work_items, int threads = 256, int cap = 148 * 8) {
+  long long b = (work_items + threads - 1) / threads;
+  if (b < 1) b = 1;
+  return (int)(b < cap ? b : cap);
+}
+
+template <typename T>
+bool vec_ok(const void* p, long long ld, int cols) {
+  constexpr int V = 16 / (int)sizeof(T);
+  return p == nullptr || ((reinterpret_cast<uintptr_t>(p) & 15) == 0 && ld % V == 0 && cols % V == 0);
+}
+
+}  // namespace
+
+void launch_quantize_weight(const float* w, int rows, int cols, const float* steps, int per_row, int bits, int grid,
+                            int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt, cudaStream_t st) {
+  if (dt == 1)
+    quantize_weight_kernel<bf16><<<rows, 256, 0, st>>>(w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (bf16*)what);
+  else
+    quantize_weight_kernel<float><<<rows, 256, 0, st>>>(w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (float*)what);
+}
+
+template <typename T>
+static void quantize_act_t(const T* x, long long rows, int cols, long long ld_x, const float* step, const float* offset,
+                           int lo, int hi, int8_t* q8, long long ld_q8, T* qt, long long ld_qt, cudaStream_t st) {
+  constexpr int V = 16 / (int)sizeof(T);
+  const bool v = vec_ok<T>(x, ld_x, cols) && vec_ok<T>(qt, ld_qt, cols) &&
+                 (q8 == nullptr || ((reinterpret_cast<uintptr_t>(q8) % V) == 0 && ld_q8 % V == 0));
+  if (v)
+    quantize_act_kernel<T, V><<<grid_for(rows * cols / V), 256, 0, st>>>(x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
+  else
+    quantize_act_kernel<T, 1><<<grid_for(rows * cols), 256, 0, st>>>(x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
+}
+
+void launch_quantize_act(const void* x, int dt, long long rows, int cols, long long ld_x, const float* step,
+                         const float* offset, int lo, int hi, int8_t* q8, long long ld_q8, void* qt,
+                         long long ld_qt, cudaStream_t st) {
+  if (rows <= 0 || cols <= 0) return;
+  if (dt == 1) quantize_act_t<bf16>((const bf16*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (bf16*)qt, ld_qt, st);
+  else quantize_act_t<float>((const float*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (float*)qt, ld_qt, st);
+}
+
+void launch_widen_bf16(const void* src, float* dst, long long n, cudaStream_t st) {
+  if (n > 0) widen_bf16_kernel<<<grid_for(n), 256, 0, st>>>((const bf16*)src, dst, n);
+}
+
+void launch_narrow(const float* src, void* dst, long long n, int dt, cudaStream_t st) {
+  if (n <= 0) return;
+  if (dt == 1) narrow_kernel<bf16><<<grid_for(n), 256, 0, st>>>(src, (bf16*)dst, n);
+  else narrow_kernel<float><<<grid_for(n), 256, 0, st>>>(src, (float*)dst, n);
+}
+
+void launch_mix(const void* f, const void* f_hat, float lam, void* out, long long n, int dt, cudaStream_t st) {
+  if (n <= 0) return;
+  if (dt == 1) {
+    if (n % 8 == 0 && vec_ok<bf16>(f, 8, 8) && vec_ok<bf16>(f_hat, 8, 8) && vec_ok<bf16>(out, 8, 8))
+      mix_kernel<bf16, 8><<<grid_for(n / 8), 256, 0, st>>>((const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
+    else
+      mix_kernel<bf16, 1><<<grid_for(n), 256, 0, st>>>((const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
+  } else {
+    if (n % 4 == 0 && vec_ok<float>(f, 4, 4) && vec_ok<float>(f_hat, 4, 4) && vec_ok<float>(out, 4, 4))
+      mix_kernel<float, 4><<<grid_for(n / 4), 256, 0, st>>>((const float*)f, (const float*)f_hat, lam, (float*)out, n);
+    else
+      mix_kernel<float, 1><<<grid_for(n), 256, 0, st>>>((const float*)f, (const float*)f_hat, lam, (float*)out, n);
+  }
+}
+
+void launch_gelu_quant(const void* u, long long n, const float* step, const float* offset, int lo, int hi,
+                       int8_t* q8, void* qt, int dt, cudaStream_t st) {
+  if (n <= 0) return;
+  if (dt == 1) {
+    const bool v = n % 8 == 0 && vec_ok<bf16>(u, 8, 8) && vec_ok<bf16>(qt, 8, 8) && (reinterpret_cast<uintptr_t>(q8) % 8) == 0;
+    if (v) gelu_quant_kernel<bf16, 8><<<grid_for(n / 8), 256, 0, st>>>((const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
+    else gelu_quant_kernel<bf16, 1><<<grid_for(n), 256, 0, st>>>((const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
+  } else {
+    const bool v = n % 4 == 0 && vec_ok<float>(u, 4, 4) && vec_ok<float>(qt, 4, 4) && (reinterpret_cast<uintptr_t>(q8) % 4) == 0;
+    if (v) gelu_quant_kernel<float, 4><<<grid_for(n / 4), 256, 0, st>>>((const float*)u, n, step, offset, (float)lo, (float)hi, q8, (float*)qt);
+    else gelu_quant_kernel<float, 1><<<grid_for(n), 256, 0, st>>>((const float*)u, n, step, offset, (float)lo, (float)hi, q8, (float*)qt);
+  }
+}
+
+void launch_init_weight_steps(const float* w, int rows, int cols, int per_row, int rule, float qmax, float* steps,
+                              float* scratch, cudaStream_t st) {
+  weight_row_stat_kernel<<<rows, 256, 0, st>>>(w, cols, rule, scratch);
+  weight_steps_from_stat_kernel<<<per_row ? (rows + 255) / 256 : 1, 256, 0, st>>>(scratch, rows, cols, per_row, rule, qmax, steps);
+}
+
+void launch_minmax(const void* x, long long ld, long long rows, int cols, float* out, float* scratch, int dt,
+                   cudaStream_t st) {
+  if (dt == 1) minmax_kernel<bf16><<<RED_BLOCKS, 256, 0, st>>>((const bf16*)x, ld, rows, cols, scratch);
+  else minmax_kernel<float><<<RED_BLOCKS, 256, 0, st>>>((const float*)x, ld, rows, cols, scratch);
+  minmax_final_kernel<<<1, 32, 0, st>>>(scratch, RED_BLOCKS, out);
+}
+
+void launch_step_from_minmax(const float* minmax, int mode, float qmax, float* step, float* offset, cudaStream_t st) {
+  step_from_minmax_kernel<<<1, 32, 0, st>>>(minmax, mode, qmax, step, offset);
+}
+
+void launch_gather_rows(const void* src, const int* d_idx, int n_rows, long long row_bytes, void* out,
+                        cudaStream_t st) {
+  const long long row_vecs = row_bytes / 16;
+  dim3 grid(grid_for(row_vecs, 256, 64), n_rows);
+  gather_rows_kernel<<<grid, 256, 0, st>>>((const uint4*)src, d_idx, row_vecs, (uint4*)out);
+}
+
+}  // namespace mrem

@@ -1,0 +1,64 @@
+// 16-byte vector access for float32 / bfloat16 tensors and packed 8-bit codes.
+#pragma once
+#include "mrem_common.cuh"
+
+namespace mrem {
+
+template <typename T, int V>
+__device__ __forceinline__ void load_vec(const T* p, float* v) {
+  if constexpr (V == 1) {
+    v[0] = to_f<T>(p[0]);
+  } else if constexpr (sizeof(T) == 4) {
+    static_assert(V == 4, "float vectors hold 4 values");
+    const float4 t = *reinterpret_cast<const float4*>(p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+    static_assert(V == 8, "bfloat16 vectors hold 8 values");
+    const uint4 t = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(h[i]);
+      v[2 * i] = f.x;
+      v[2 * i + 1] = f.y;
+    }
+  }
+}
+
+template <typename T, int V>
+__device__ __forceinline__ void store_vec(T* p, const float* v) {
+  if constexpr (V == 1) {
+    p[0] = from_f<T>(v[0]);
+  } else if constexpr (sizeof(T) == 4) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  } else {
+    uint4 t;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    *reinterpret_cast<uint4*>(p) = t;
+  }
+}
+
+// V integer codes (each fits 8 bits, signed or unsigned) packed into V bytes.
+template <int V>
+__device__ __forceinline__ void store_codes(int8_t* p, const int* q) {
+  if constexpr (V == 1) {
+    p[0] = (int8_t)q[0];
+  } else if constexpr (V == 4) {
+    uint32_t w = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w |= (uint32_t)(q[i] & 0xff) << (8 * i);
+    *reinterpret_cast<uint32_t*>(p) = w;
+  } else {
+    uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      w0 |= (uint32_t)(q[i] & 0xff) << (8 * i);
+      w1 |= (uint32_t)(q[i + 4] & 0xff) << (8 * i);
+    }
+    *reinterpret_cast<uint2*>(p) = make_uint2(w0, w1);
+  }
+}
+
+}  // namespace mrem
