@@ -77,7 +77,10 @@ int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, flo
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
   if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
-  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_capture_step: begin capture failed");
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();   // clear the sticky-until-read error: the legacy default stream cannot be captured
+    return fail(c, MREM_ERR_CUDA, "graph_capture_step: begin capture failed (the context's stream must not be the legacy default stream)");
+  }
   const int rc = enqueue_step(c, xt, xs, lambda, len, batch, seq, t_out, s_out, d_loss, o);
   cudaGraph_t g = nullptr;
   const cudaError_t e = cudaStreamEndCapture(c->stream, &g);

@@ -1,0 +1,285 @@
+"""Module-level parity of the CUDA reconstruction step with the CPU oracle (through the C-ABI).
+
+Tolerances: forward outputs 1e-3 relative L2 against the oracle in storage-emulation mode
+(bf16 configurations), 1e-4 for the float32 configuration; loss and gradients 2e-2 relative L2.
+Integer codes reaching an interior quantizer may differ in a small fraction of positions,
+because the float operations before it round differently on the two sides; the weight codes,
+which depend only on bound inputs, must match bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mrem_oracle as O
+from paper_2109_15082_b200 import binding as B
+from paper_2109_15082_b200 import synth
+from tests.gpu_util import Problem, compare_grads, rel
+
+pytestmark = pytest.mark.gpu
+
+FWD_TOL = {"f32": 1e-4, "bf16": 1e-3}
+GRAD_TOL = 2e-2
+
+
+def _wl(name, **kw):
+    return synth.shrink(synth.workloads()[name], **kw)
+
+
+CASES = {
+    # configuration 1 as stated: 1 layer, hidden 128, 2 heads, FFN 512, seq 32, batch 4, float32
+    "tiny_f32": (_wl("tiny"), dict()),
+    # float32, two layers, padding mask, per-matrix steps, some clipping
+    "f32_2layer_clip": (_wl("tiny", n_layers=2, len_lo=9, len_hi=32, batch=3), dict(step_shrink=0.7, w_per_row=False, student_noise=0.002)),
+    # bf16 tensor-core path: ragged token count (3*40 = 120 rows: one partial tile), outlier channels
+    "bf16_small": (_wl("base3_w4a8", n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40),
+                   dict(step_shrink=0.8, student_noise=0.002)),
+    # several tiles in every dimension: 2*136 = 272 tokens, hidden 256, ffn 640
+    "bf16_tiles": (_wl("base3_w4a8", n_layers=1, hidden=256, n_heads=4, ffn=640, seq=136, batch=2, len_lo=32, len_hi=136), dict()),
+    # 2-bit half-integer grid with mean|w| steps
+    "bf16_w2_halfgrid": (_wl("base3_w2a8", n_layers=2, hidden=128, n_heads=2, ffn=256, seq=32, batch=4, len_lo=8, len_hi=32), dict()),
+    # Omega(2) = {-1, 0, 1} (Eq. 1), symmetric sites only, plain-sum loss
+    "f32_w2_ternary_sym": (_wl("tiny", w_bits=2, w_step_rule=1, hidden=64, ffn=128), dict(asym=0, loss_mean=False)),
+    # 4-bit activations
+    "bf16_a4": (_wl("base3_w4a8", n_layers=1, hidden=128, n_heads=2, ffn=256, seq=32, batch=2, len_lo=0), dict(a_bits=4)),
+}
+
+
+@pytest.mark.parametrize("case", list(CASES))
+def test_forward_loss_backward_parity(case):
+    wl, kw = CASES[case]
+    p = Problem(wl, **kw)
+    try:
+        g = p.run_gpu()
+        r = p.run_oracle()
+        tol = FWD_TOL[wl.act_dtype]
+        for l in range(wl.n_layers):
+            assert rel(g["f_t"][l], r["f_t"][l]) < tol, ("teacher", l, rel(g["f_t"][l], r["f_t"][l]))
+            assert rel(g["f_s"][l], r["f_s"][l]) < tol, ("student", l, rel(g["f_s"][l], r["f_s"][l]))
+        assert abs(g["loss"] - r["loss"]) / r["loss"] < GRAD_TOL
+        assert np.allclose(g["per"], r["loss_per_layer"], rtol=GRAD_TOL)
+        # weight codes and row sums: bit exact
+        for l in range(wl.n_layers):
+            for pid, name in ((B.WQKV, "Wqkv"), (B.WO, "Wo"), (B.W1, "W1"), (B.W2, "W2")):
+                codes, rowsum = p.m.weight_codes(l, pid)
+                ref = r["caches"][l]["qw"][name]["q"]
+                assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref)
+                assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1))
+        worst = compare_grads(g["grads"], r["grads"], GRAD_TOL, check_offset=kw.get("step_shrink", 1.0) < 1.0)
+        print(case, "loss", g["loss"], r["loss"], "worst grad", worst)
+    finally:
+        p.close()
+
+
+def test_teacher_forcing_mix():
+    wl, kw = CASES["bf16_small"]
+    p = Problem(wl, **kw)
+    try:
+        for lam in (1.0, 0.35):
+            g = p.run_gpu(lam=lam, same_input=False)
+            r = p.run_oracle(lam=lam, same_input=False)
+            assert rel(g["f_s"][-1], r["f_s"][-1]) < 1e-3
+            assert abs(g["loss"] - r["loss"]) / r["loss"] < GRAD_TOL
+        # lambda = 1: the student consumes exactly the teacher-side input (Eq. 4)
+        g1 = p.run_gpu(lam=1.0, same_input=False)
+        p.xd.copy_(p.xtd)
+        g2 = p.run_gpu(lam=0.0, same_input=True)
+        assert np.array_equal(g1["f_s"], g2["f_s"])
+    finally:
+        p.close()
+
+
+def test_full_step_matches_oracle_and_is_reproducible():
+    wl, kw = CASES["tiny_f32"]
+    p = Problem(wl, **kw)
+    try:
+        m = p.m
+        opt = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+        # The update is checked on its own: the oracle's AdamW is fed the gradients the GPU
+        # produced (their parity is the business of the tests above), because Adam's first steps
+        # are ~lr * sign(g) and amplify any difference in near-zero gradients.
+        mom = {}
+        losses = []
+        for t in range(1, 4):
+            before = m.student_numpy()
+            w0, a0, off0 = m.get_steps()
+            losses.append(p.run_gpu()["loss"])
+            g = p.gpu_grads()
+            m.step(B.make_optim(step=t, **opt))
+            torch.cuda.synchronize()
+            got = m.student_numpy()
+            w1, a1, off1 = m.get_steps()
+
+            def expect(key, p0, grad, wd, clamp=None):
+                mm, vv = mom.get(key, (np.zeros_like(p0, np.float64), np.zeros_like(p0, np.float64)))
+                p1, mm, vv = O.adamw_update(p0, grad, mm, vv, t, opt["lr"], 0.9, 0.999, 1e-8, wd)
+                mom[key] = (mm, vv)
+                return np.maximum(p1, clamp) if clamp is not None else p1
+
+            for l in range(wl.n_layers):
+                for k in O.PARAMS:
+                    ref = expect((l, k), before[l][k], g[l][k], 0.01 if k in O.WEIGHTS else 0.0)
+                    assert np.allclose(got[l][k], ref, rtol=1e-5, atol=2e-3 * opt["lr"]), (t, l, k)
+                for k in O.WEIGHTS:
+                    ref = expect((l, "s", k), w0[l][k], g[l]["w"][k], 0.0, O.MIN_STEP)
+                    assert np.allclose(w1[l][k], ref, rtol=1e-5, atol=2e-3 * opt["lr"]), (t, l, "s", k)
+                ref = expect((l, "a"), a0[l], g[l]["a"], 0.0, O.MIN_STEP)
+                assert np.allclose(a1[l], ref, rtol=1e-5, atol=2e-3 * opt["lr"]), (t, l, "a")
+                ref = expect((l, "off"), off0[l, 7:8], g[l]["a_off"][7:8], 0.0)
+                assert np.allclose(off1[l, 7:8], ref, rtol=1e-5, atol=2e-3 * opt["lr"]), (t, l, "off")
+            assert not np.array_equal(got[0]["W1"], before[0]["W1"])
+        # same inputs twice: bitwise identical loss and gradients (fixed-order reductions)
+        a1 = p.run_gpu()
+        a2 = p.run_gpu()
+        assert a1["loss"] == a2["loss"]
+        for g1, g2 in zip(a1["grads"], a2["grads"]):
+            for k in O.PARAMS:
+                assert np.array_equal(g1[k], g2[k])
+            assert np.array_equal(g1["a"], g2["a"])
+    finally:
+        p.close()
+
+
+def test_step_initialisation_matches_oracle():
+    wl, _ = CASES["bf16_small"]
+    p = Problem(wl)
+    try:
+        m = p.m
+        m.init_weight_steps(0)
+        m.init_act_steps(p.xd, p.vld, wl.batch, wl.seq)
+        torch.cuda.synchronize()
+        w, a, off = m.get_steps()
+        ws = O.init_weight_steps(p.desc, p.student, 0)
+        a_ref, off_ref = O.init_act_steps(p.desc, p.student, p.x, p.vl)
+        for l in range(wl.n_layers):
+            for k in O.WEIGHTS:
+                assert np.allclose(w[l][k], ws[l][k], rtol=1e-6)
+        assert np.allclose(a, a_ref, rtol=2e-2)
+        assert np.allclose(off[:, 7], off_ref[:, 7], rtol=2e-2, atol=1e-3)
+        m.init_weight_steps(1)
+        torch.cuda.synchronize()
+        w, _, _ = m.get_steps()
+        ws = O.init_weight_steps(p.desc, p.student, 1)
+        assert np.allclose(w[0]["W1"], ws[0]["W1"], rtol=1e-5)
+    finally:
+        p.close()
+
+
+def test_graph_replay_and_host_step_equal_eager():
+    wl, kw = CASES["bf16_small"]
+    opt = B.make_optim(lr=1e-4, step=0, decay_total_steps=10)
+    results = []
+    side = torch.cuda.Stream()                 # the legacy default stream cannot be captured
+    for mode in ("eager", "graph", "host"):
+        with torch.cuda.stream(side):
+            p = Problem(wl, **kw)
+            try:
+                m = p.m
+                losses = []
+                if mode == "graph":
+                    side.synchronize()
+                    B.mrem_graph_capture_step(m.ctx, p.xd, p.xd, 0.0, p.vld, wl.batch, wl.seq, m.t_out, m.s_out,
+                                              m.loss, opt)
+                x_host = p.xd.cpu().contiguous().pin_memory()
+                vl_host = torch.from_numpy(p.vl).pin_memory()
+                for t in range(3):
+                    if mode == "eager":
+                        p.run_gpu()
+                        m.step(opt)
+                        losses.append(float(m.loss[0]))
+                    elif mode == "graph":
+                        B.mrem_graph_launch(m.ctx)
+                        torch.cuda.synchronize()
+                        losses.append(float(m.loss[0]))
+                    else:
+                        losses.append(B.mrem_recon_step_host(m.ctx, x_host, x_host, vl_host, wl.batch, wl.seq, 0.0, opt))
+                torch.cuda.synchronize()
+                assert m.poll_status() == 0
+                results.append((losses, m.student_numpy()[0]["W1"].copy()))
+            finally:
+                p.close()
+    for losses, w1 in results[1:]:
+        assert losses == results[0][0]
+        assert np.array_equal(w1, results[0][1])
+    assert results[0][0][2] != results[0][0][0]
+
+
+def test_state_export_import_resumes_bitwise():
+    wl, kw = CASES["bf16_small"]
+    opt = B.make_optim(lr=1e-4, step=0, decay_total_steps=8)
+
+    def run(n_steps, p):
+        for _ in range(n_steps):
+            p.run_gpu()
+            p.m.step(opt)
+
+    p = Problem(wl, **kw)
+    q = Problem(wl, **kw)
+    try:
+        run(4, p)
+        run(2, q)
+        nbytes = B.mrem_state_bytes(q.m.ctx)
+        blob = torch.zeros(nbytes, dtype=torch.uint8, device="cuda:0")
+        B.mrem_export_state(q.m.ctx, blob, nbytes)
+        saved_student = q.m.student_numpy()
+        saved_steps = q.m.get_steps()
+        q.close()
+        q = Problem(wl, **kw)
+        q.m.load_student(saved_student)
+        q.m.set_steps(*saved_steps)
+        B.mrem_import_state(q.m.ctx, blob, nbytes)
+        run(2, q)
+        torch.cuda.synchronize()
+        a, b = p.m.student_numpy(), q.m.student_numpy()
+        for l in range(wl.n_layers):
+            for k in O.PARAMS:
+                assert np.array_equal(a[l][k], b[l][k]), (l, k)
+    finally:
+        p.close()
+        q.close()
+
+
+def test_call_order_and_argument_errors():
+    wl, kw = CASES["bf16_small"]
+    p = Problem(wl, **kw)
+    try:
+        m = p.m
+        with pytest.raises(B.MremError) as e:
+            m.forward_student(p.xd, p.vld, wl.batch, wl.seq)          # weights not quantized yet
+        assert e.value.code == -5
+        with pytest.raises(B.MremError) as e:
+            m.backward()
+        assert e.value.code == -5
+        m.quantize_weights()
+        m.forward_student(p.xd, p.vld, wl.batch, wl.seq)
+        with pytest.raises(B.MremError) as e:
+            m.recon_loss()                                              # no teacher pass
+        assert e.value.code == -5
+        with pytest.raises(B.MremError) as e:
+            m.forward_teacher(p.xd, p.vld, wl.batch + 1, wl.seq)        # beyond max_batch
+        assert e.value.code == -3
+        with pytest.raises(B.MremError) as e:
+            m.forward_teacher(p.xd, p.vld, wl.batch, wl.seq - 1)        # bf16 needs seq % 8 == 0
+        assert e.value.code == -3
+        with pytest.raises(B.MremError) as e:
+            m.step(B.make_optim())
+        assert e.value.code == -5
+        torch.cuda.synchronize()
+        assert m.poll_status() == 0
+    finally:
+        p.close()
+
+
+def test_nonfinite_loss_is_reported_in_status():
+    wl, kw = CASES["bf16_small"]
+    p = Problem(wl, **kw)
+    try:
+        p.xd[0, 0, 0] = float("inf")
+        m = p.m
+        m.quantize_weights()
+        m.forward_teacher(p.xd, p.vld, wl.batch, wl.seq)
+        m.forward_student(p.xd, p.vld, wl.batch, wl.seq)
+        m.recon_loss()
+        torch.cuda.synchronize()
+        assert m.poll_status() == -8
+        assert m.poll_status() == 0                                     # cleared by the poll
+    finally:
+        p.close()
