@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the MREM reconstruction step.
+
+A step = one pass of the whole hot path (weight quantization, teacher forward, student
+forward, loss, straight-through backward, AdamW) over one calibration batch of one module.
+Default workload: a BERT-large module of 6 layers, W4A8, batch 32 x seq 128, bf16 storage,
+drawn from a 1024-sequence seeded synthetic calibration set that lives in HBM.
+
+    python bench.py --gpus 1 --steps 20 --warmup 3
+    python bench.py --impl reference            # the CPU oracle, as it stands, on the host cores
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "recon-step tokens/sec (fwd+bwd) per BERT-large W4A8 module"
+UNIT = "tokens/s"
+INT8_OVER_BF16 = 2.0        # nominal dense int8 : bf16 tensor throughput on this part
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for line in open(self.path):
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+
+def oracle_sample(wl, n_steps=1, warmup=0, batch=None):
+    """Times the oracle, as it stands, on ONE layer of the module with the full batch
+    (teacher forward, student forward, loss, backward, AdamW) and extrapolates to the
+    module's layer count.  Returns (tokens/s, threads used, description, seconds per sample)."""
+    from oracle import mrem_oracle as O
+    from paper_2109_15082_b200 import synth
+    batch = batch or wl.batch
+    one = synth.shrink(wl, n_layers=1, batch=batch)
+    params = synth.teacher_params(one, 0)
+    x = synth.hidden_states(one, batch, 0)
+    vl = synth.valid_lengths(one, batch, 0)
+    desc = O.ModuleDesc(1, wl.hidden, wl.n_heads, wl.ffn, wl.w_bits, wl.a_bits, wl.w_grid, act_dtype=wl.act_dtype)
+    student = [{k: v.copy() for k, v in params[0].items()}]
+    ws = O.init_weight_steps(desc, student, wl.w_step_rule)
+    a, off = O.init_act_steps(desc, student, x, vl)
+    steps, state = O.make_steps(ws, a, off), {}
+    times = []
+    for i in range(warmup + n_steps):
+        t0 = time.perf_counter()
+        O.recon_step(desc, params, student, steps, state, x, x, vl, lr=wl.lr)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = sum(times) / len(times)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    tokens = batch * wl.seq
+    desc_txt = (f"1 of {wl.n_layers} layers, batch {batch}x{wl.seq} of {wl.batch}x{wl.seq}, teacher fwd + student fwd + loss + "
+                f"backward + AdamW in float64 numpy; tokens/s extrapolated as tokens / ({wl.n_layers} x t_layer)")
+    return tokens / (wl.n_layers * sec), threads, desc_txt, sec
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    # each step is a bounded sample: the full batch for short runs, a quarter of it for long ones
+    batch = wl.batch if args.steps <= 5 else max(2, wl.batch // 4)
+    val, threads, sample, sec = oracle_sample(wl, n_steps=max(1, args.steps), warmup=min(args.warmup, 1), batch=batch)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec * wl.n_layers,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "batch": wl.batch, "seq_len": wl.seq, "note": "CPU oracle (numpy float64)"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU leg
+
+def build_problem(wl, rank, torch, calib_n):
+    from paper_2109_15082_b200 import synth
+    from paper_2109_15082_b200.session import ReconModule
+    m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, wl.a_bits, wl.w_grid,
+                    True, 3, wl.act_dtype)
+    m.load_teacher(synth.teacher_params(wl, seed=rank))
+    m.init_student_from_teacher()
+    m.init_weight_steps(wl.w_step_rule)
+    calib = torch.empty(calib_n, wl.seq, wl.hidden, dtype=m.tdtype, device=m.device)
+    chunk = 64
+    for c0 in range(0, calib_n, chunk):
+        n = min(chunk, calib_n - c0)
+        x = synth.hidden_states(wl, n, seed=rank, tag=f"calib{c0}")
+        calib[c0:c0 + n].copy_(torch.from_numpy(x).to(m.device))
+    lens = torch.from_numpy(synth.valid_lengths(wl, calib_n, seed=rank)).to(m.device)
+    return m, calib, lens
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large6_w4a8")
+    ap.add_argument("--calib", type=int, default=0, help="calibration sequences (0: the workload's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2109_15082_b200 import synth
+    wl = synth.workloads()[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2109_15082_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    W = max(3, args.warmup)
+    K = args.steps
+    calib_n = args.calib or wl.calib or wl.batch * 8
+    tokens = wl.batch * wl.seq
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        m, calib, lens = build_problem(wl, rank, torch, calib_n)
+        total = W + K
+        n_batches = calib_n // wl.batch
+        perm = np.concatenate([synth.permutation(rank, f"epoch{e}", calib_n)[: n_batches * wl.batch]
+                               for e in range((total + n_batches - 1) // n_batches + 1)])
+        idx = torch.from_numpy(perm[: total * wl.batch].reshape(total, wl.batch).astype(np.int32)).to(m.device)
+        lens_steps = lens[idx.long()].contiguous()                    # [total, batch] int32, built once, untimed
+        step_ids = torch.arange(total, dtype=torch.int32, device=m.device)
+        xbuf = torch.empty(wl.batch, wl.seq, wl.hidden, dtype=m.tdtype, device=m.device)
+        lenbuf = torch.zeros(max(wl.batch, 64), dtype=torch.int32, device=m.device)
+        row_bytes = wl.seq * wl.hidden * xbuf.element_size()
+        len_row_bytes = wl.batch * 4
+        assert len_row_bytes % 16 == 0
+        st = side.cuda_stream
+
+        def stage(t):
+            B.mrem_gather_rows(calib, idx[t], wl.batch, row_bytes, xbuf, st)
+            B.mrem_gather_rows(lens_steps, step_ids[t:t + 1], 1, len_row_bytes, lenbuf, st)
+
+        stage(0)
+        m.init_act_steps(xbuf, lenbuf, wl.batch, wl.seq)
+        opt = B.make_optim(lr=wl.lr, step=0, decay_total_steps=max(wl.steps, total))
+        side.synchronize()
+        B.mrem_graph_capture_step(m.ctx, xbuf, xbuf, 0.0, lenbuf, wl.batch, wl.seq, m.t_out, m.s_out, m.loss, opt)
+        kernels_per_step = B.mrem_graph_num_kernels(m.ctx) + 2
+
+        for t in range(W):
+            stage(t)
+            B.mrem_graph_launch(m.ctx)
+        side.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for t in range(W, W + K):
+            stage(t)
+            B.mrem_graph_launch(m.ctx)
+        e1.record(side)
+        side.synchronize()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        clocks = sampler.stop() if rank == 0 else None
+        ms = e0.elapsed_time(e1)
+        loss_last = float(m.loss[0])
+        status = m.poll_status()
+        if world > 1:
+            tt = torch.tensor([ms], dtype=torch.float64, device=m.device)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt[0])
+
+        # ---- per-kernel timing (CUDA events around every launch of a few eager steps)
+        B.mrem_trace_enable(m.ctx, 1)
+        n_trace = 3
+        for t in range(n_trace):
+            stage(t)
+            m.quantize_weights()
+            m.forward_teacher(xbuf, lenbuf, wl.batch, wl.seq)
+            m.forward_student(xbuf, lenbuf, wl.batch, wl.seq)
+            m.recon_loss()
+            m.backward()
+            m.step(opt)
+        trace = B.mrem_trace_read(m.ctx)
+        B.mrem_trace_enable(m.ctx, 0)
+
+        # ---- end to end: host buffers in, loss out, every step
+        e2e = None
+        if not args.no_e2e:
+            hb = [calib[idx[t].long()].cpu().pin_memory() for t in range(min(4, total))]
+            hl = [lens_steps[t].cpu().pin_memory() for t in range(min(4, total))]
+            ke = max(3, min(K, 10))
+            for t in range(2):
+                B.mrem_recon_step_host(m.ctx, hb[t % len(hb)], hb[t % len(hb)], hl[t % len(hl)], wl.batch, wl.seq, 0.0, opt)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for t in range(ke):
+                B.mrem_recon_step_host(m.ctx, hb[t % len(hb)], hb[t % len(hb)], hl[t % len(hl)], wl.batch, wl.seq, 0.0, opt)
+            torch.cuda.synchronize()
+            dt_e2e = time.perf_counter() - t0
+            if world > 1:
+                tt = torch.tensor([dt_e2e], dtype=torch.float64, device=m.device)
+                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+                dt_e2e = float(tt[0])
+            e2e = {"value": world * tokens * ke / dt_e2e, "unit": UNIT,
+                   "h2d_bytes_per_step": row_bytes * wl.batch + len_row_bytes, "d2h_bytes_per_step": 4,
+                   "steps": ke}
+        m.close()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    kernels = []
+    for e in sorted(trace, key=lambda e: -e["ms"]):
+        per_launch_ms = e["ms"] / max(e["launches"], 1)
+        if e["is_flops"]:
+            ach = e["work"] / (e["ms"] * 1e-3) / 1e12
+            peak = pk["bf16_sustained"] * (INT8_OVER_BF16 if "i8" in e["name"] else 1.0)
+            unit, bound = "TFLOP/s", "tensor"
+        else:
+            ach = e["work"] / (e["ms"] * 1e-3) / 1e9
+            peak, unit, bound = pk["hbm_gbs"], "GB/s", "hbm"
+        kernels.append({"name": e["name"], "launches_per_step": e["launches"] / n_trace, "ms_per_step": e["ms"] / n_trace,
+                        "us_per_launch": 1e3 * per_launch_ms, "bound": bound, "achieved": ach, "peak": peak,
+                        "unit": unit, "frac": ach / peak})
+    top = kernels[0]
+    roofline = {"kernel": top["name"], "bound": top["bound"], "achieved": top["achieved"], "peak": top["peak"],
+                "unit": top["unit"], "frac": top["frac"], "traffic": None,
+                "peak_source": pk["source"] + (" bf16 sustained" if top["bound"] == "tensor" else " copy bandwidth"),
+                "timed": f"CUDA events around each launch of {n_trace} eager steps"}
+
+    line = {"metric": METRIC, "value": world * tokens * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16+int8", "data": "synthetic",
+            "config": {"workload": wl.name, "layers": wl.n_layers, "hidden": wl.hidden, "heads": wl.n_heads,
+                       "ffn": wl.ffn, "batch": wl.batch, "seq_len": wl.seq, "bits": f"W{wl.w_bits}A{wl.a_bits}",
+                       "calibration_sequences": calib_n, "parallelism": "replicas only" if world > 1 else "1 GPU",
+                       "l2": "inputs larger than L2: calibration set, weights and optimizer state exceed 126 MB",
+                       "launch": "one CUDA-graph replay per step + 2 gather kernels"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_step * K, "roofline": roofline,
+            "kernels": kernels, "loss_last": loss_last, "device_status": status}
+    if world == 1 and not args.no_cpu_baseline:
+        val, threads, sample, sec = oracle_sample(wl)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                                "seconds": sec}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

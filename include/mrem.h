@@ -186,6 +186,16 @@ int32_t mrem_graph_capture_step(mrem_ctx* ctx, const void* d_x_teacher, const vo
                                 const int32_t* d_valid_len, int32_t batch, int32_t seq, void* d_teacher_outputs,
                                 void* d_student_outputs, float* d_loss_total, const mrem_optim* optim);
 int32_t mrem_graph_launch(mrem_ctx* ctx);
+/* Number of kernel nodes in the captured step. */
+int32_t mrem_graph_num_kernels(mrem_ctx* ctx, int32_t* n_kernels);
+
+/* Per-kernel timing of the eager calls (not of graph replays) with CUDA events on the context's stream.
+ * `work` is the algorithmic work of all launches of that kernel: FLOPs (is_flops = 1: 2*M*N*K per product)
+ * or bytes read plus written once at storage width (is_flops = 0).  mrem_trace_enable resets the totals
+ * and blocks on the stream; mrem_trace_read blocks on the stream and fills up to max_entries entries. */
+typedef struct { char name[40]; double ms; double work; int64_t launches; int32_t is_flops; int32_t reserved; } mrem_trace_entry;
+int32_t mrem_trace_enable(mrem_ctx* ctx, int32_t on);
+int32_t mrem_trace_read(mrem_ctx* ctx, mrem_trace_entry* out, int32_t max_entries, int32_t* n_entries);
 
 /* out[i] = src[idx[i]] for i < n_rows (rows of row_bytes bytes, a multiple of 16): draws a batch from a
  * calibration set resident on the device (Sec. 5.1). */

@@ -30,7 +30,8 @@ EXPORTS = (
     "mrem_get_weight_codes", "mrem_module_forward", "mrem_recon_loss", "mrem_module_backward", "mrem_get_grad",
     "mrem_step", "mrem_recon_step_host", "mrem_poll_status", "mrem_state_bytes", "mrem_export_state",
     "mrem_import_state", "mrem_graph_capture_step", "mrem_graph_launch", "mrem_gather_rows", "mrem_quantize_act",
-    "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm",
+    "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
+    "mrem_trace_read",
 )
 
 
@@ -207,6 +208,30 @@ def mrem_graph_capture_step(ctx, x_teacher, x_student, lam, valid_len, batch, se
 
 def mrem_graph_launch(ctx):
     _check(lib().mrem_graph_launch(ctx), "mrem_graph_launch", ctx)
+
+
+def mrem_graph_num_kernels(ctx) -> int:
+    n = C.c_int32(0)
+    _check(lib().mrem_graph_num_kernels(ctx, C.byref(n)), "mrem_graph_num_kernels", ctx)
+    return n.value
+
+
+class TraceEntry(C.Structure):
+    _fields_ = [("name", C.c_char * 40), ("ms", C.c_double), ("work", C.c_double), ("launches", C.c_int64),
+                ("is_flops", C.c_int32), ("reserved", C.c_int32)]
+
+
+def mrem_trace_enable(ctx, on):
+    _check(lib().mrem_trace_enable(ctx, int(on)), "mrem_trace_enable", ctx)
+
+
+def mrem_trace_read(ctx, max_entries=64):
+    """-> list of dicts name, ms, work, launches, is_flops."""
+    buf = (TraceEntry * max_entries)()
+    n = C.c_int32(0)
+    _check(lib().mrem_trace_read(ctx, buf, max_entries, C.byref(n)), "mrem_trace_read", ctx)
+    return [dict(name=buf[i].name.decode(), ms=buf[i].ms, work=buf[i].work, launches=buf[i].launches,
+                 is_flops=bool(buf[i].is_flops)) for i in range(n.value)]
 
 
 def mrem_gather_rows(src, idx, n_rows, row_bytes, out, stream):

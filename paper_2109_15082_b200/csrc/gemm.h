@@ -1,6 +1,7 @@
 // Internal interface of the two GEMM back ends.
 #pragma once
 #include "mrem_common.cuh"
+#include "trace.h"
 
 namespace mrem {
 

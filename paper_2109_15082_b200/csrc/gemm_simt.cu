@@ -81,6 +81,7 @@ int simt_gemm_f32(const OperandDesc& A, const OperandDesc& B, const GemmShape& g
   SimtParams p{A, B, g, epi};
   dim3 grid((g.N + TS - 1) / TS, (g.M + TS - 1) / TS, g.nb0 * g.nb1);
   if (grid.y > 65535 || grid.z > 65535) return GEMM_ERR_ARG;
+  Scope sc("gemm_f32_simt", 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream);
   simt_gemm_kernel<<<grid, 256, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }

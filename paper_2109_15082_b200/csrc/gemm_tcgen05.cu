@@ -506,6 +506,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
     attr_set[kind] = true;
   }
   const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
+  Scope sc(kind == 0 ? "gemm_bf16_tcgen05" : "gemm_i8_tcgen05", 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream);
   kern<<<grid, GEMM_THREADS, smem, stream>>>(ma, mb, p);
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }

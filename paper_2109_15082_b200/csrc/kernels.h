@@ -2,6 +2,7 @@
 // of activations: 0 = float32, 1 = bfloat16.  All launches are asynchronous on `st`.
 #pragma once
 #include "mrem_common.cuh"
+#include "trace.h"
 
 namespace mrem {
 
@@ -100,7 +101,8 @@ struct AdamEntry { float* p; const float* g; float* m; float* v; long long n; fl
 // lr = lr0 * (1 - (t-1)/total) when total > 0 else lr0.
 void launch_optim_prepare(OptimScalars* d_out, int* d_t, int host_t, float lr0, int total_steps, float beta1,
                           float beta2, float eps, float weight_decay, cudaStream_t st);
-void launch_adamw_table(const AdamEntry* d_table, int n_entries, const OptimScalars* d_sc, cudaStream_t st);
+void launch_adamw_table(const AdamEntry* d_table, int n_entries, long long total_elems, const OptimScalars* d_sc,
+                        cudaStream_t st);
 
 // ---- step-size initialisation
 // Per-row max|w| or mean|w| -> steps (per row, or one value when !per_row: two passes).

@@ -457,6 +457,7 @@ void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, 
                           void* out, float* mean, float* rstd, const float* step, int qmax, int8_t* q8, void* qt,
                           int dt, cudaStream_t st) {
   if (rows <= 0) return;
+  Scope sc("layernorm_fwd", (double)rows * cols * ((dt == 1 ? 2.0 : 4.0) * (qt ? 3 : 2) + (q8 ? 1 : 0)), 0, st);
   const int grid = (int)((rows + 3) / 4);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
@@ -470,6 +471,7 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
                           const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
                           cudaStream_t st) {
   if (rows <= 0) return;
+  Scope sc("layernorm_bwd", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (3 + (dout2 ? 1 : 0) + (dsum ? 1 : 0)), 0, st);
   const int grid = (int)((rows + 3) / 4);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
@@ -481,6 +483,7 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
 
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
                        long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st) {
+  Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (y ? 2 : 1), 0, st);
   dim3 grid((cols + 31) / 32, COL_CHUNKS);
   MREM_DT(dt, T, { col_reduce_kernel<T><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch); });
   col_reduce_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, cols, out0, y ? out1 : nullptr);
@@ -490,17 +493,20 @@ void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h,
                         const float* offset, int lo, int hi, void* qt, int dt, cudaStream_t st) {
   const long long rows = (long long)B * h * S;
   if (rows <= 0) return;
+  Scope sc("softmax_fwd", (double)rows * S * (4.0 + (dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1)), 0, st);
   const int grid = (int)((rows + 3) / 4);
   MREM_DT(dt, T, { softmax_fwd_kernel<T><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt); });
 }
 
 void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long rows, int S, const float* step,
                         int lo, int hi, int quantized, float* part_s, int dt, cudaStream_t st) {
+  Scope sc("softmax_bwd", (double)rows * S * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
   MREM_DT(dt, T, { softmax_bwd_kernel<T><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s); });
 }
 
 void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per_layer, float c, void* dF,
                  float* partial, int* status, int dt, cudaStream_t st) {
+  Scope sc("recon_loss", (double)n_layers * n_per_layer * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
   dim3 grid(RED_BLOCKS, n_layers);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
@@ -518,6 +524,7 @@ void launch_loss_finalize(const float* partial, int n_layers, float c, float* lo
 void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long ld_d, const void* add,
                     long long ld_add, void* dx, long long ld_dx, long long rows, int cols, const float* step,
                     const float* offset, int lo, int hi, float* part_s, float* part_o, int dt, cudaStream_t st) {
+  Scope sc("ste_act", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (add ? 4 : 3), 0, st);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
     const bool v = cols % V == 0 && ld_x % V == 0 && ld_d % V == 0 && ld_dx % V == 0 && (!add || ld_add % V == 0) &&
@@ -529,6 +536,7 @@ void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long 
 
 void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, const float* step, const float* offset,
                      int lo, int hi, int quantized, float* part_s, float* part_o, int dt, cudaStream_t st) {
+  Scope sc("gelu_bwd", (double)n * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
     if (n % V == 0 && al16(u) && al16(dghat) && al16(du))
@@ -540,6 +548,7 @@ void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, co
 
 void launch_ste_weight(const float* w, const float* steps, int per_row, int bits, int grid, float* dw, int rows,
                        int cols, float* ds_rows, cudaStream_t st) {
+  Scope sc("ste_weight", (double)rows * cols * 12.0, 0, st);
   ste_weight_kernel<<<rows, 256, 0, st>>>(w, steps, per_row, bits, grid, dw, cols, ds_rows);
 }
 
@@ -559,8 +568,10 @@ void launch_optim_prepare(OptimScalars* d_out, int* d_t, int host_t, float lr0, 
                           float beta2, float eps, float weight_decay, cudaStream_t st) {
   optim_prepare_kernel<<<1, 32, 0, st>>>(d_out, d_t, host_t, lr0, total_steps, beta1, beta2, eps, weight_decay);
 }
-void launch_adamw_table(const AdamEntry* d_table, int n_entries, const OptimScalars* d_sc, cudaStream_t st) {
+void launch_adamw_table(const AdamEntry* d_table, int n_entries, long long total_elems, const OptimScalars* d_sc,
+                        cudaStream_t st) {
   if (n_entries <= 0) return;
+  Scope sc("adamw", (double)total_elems * 28.0, 0, st);
   dim3 grid(64, n_entries);
   adamw_table_kernel<<<grid, 256, 0, st>>>(d_table, d_sc);
 }

@@ -6,6 +6,8 @@
 
 using namespace mrem;
 
+namespace mrem { thread_local Tracer* g_tracer = nullptr; }
+
 namespace {
 std::string g_create_err;
 
@@ -182,6 +184,8 @@ int build_tables(mrem_ctx* c) {
   if (cudaMemcpyAsync(c->reduce_table, red.data(), sizeof(ReduceEntry) * red.size(), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
     return fail(c, MREM_ERR_CUDA, "table upload failed");
   c->adam_entries = (int)adam.size();
+  c->adam_elems = 0;
+  for (const AdamEntry& e : adam) c->adam_elems += e.n;
   if (cudaMemcpyAsync(c->adam_table, adam.data(), sizeof(AdamEntry) * adam.size(), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
     return fail(c, MREM_ERR_CUDA, "table upload failed");
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "sync failed");
@@ -320,6 +324,7 @@ int32_t mrem_init_student_from_teacher(mrem_ctx* c) {
 
 int32_t mrem_init_weight_steps(mrem_ctx* c, int32_t rule) {
   if (!c) return MREM_ERR_ARG;
+  TracerGuard tg(nullptr);
   if (rule != 0 && rule != 1) return fail(c, MREM_ERR_ARG, "init_weight_steps: rule");
   const float qmax = c->d.w_grid == 0 ? (float)((1 << (c->d.w_bits - 1)) - 1) : 1.5f;
   for (int l = 0; l < c->d.n_layers; ++l)
@@ -364,6 +369,30 @@ int32_t mrem_import_state(mrem_ctx* c, const void* blob, size_t bytes) {
   if (cudaMemcpyAsync(c->t_counter, blob, 256, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess ||
       cudaMemcpyAsync(base + c->state_off, (const char*)blob + 256, c->state_bytes, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
     return fail(c, MREM_ERR_CUDA, "import_state: copy failed");
+  return MREM_OK;
+}
+
+int32_t mrem_trace_enable(mrem_ctx* c, int32_t on) {
+  if (!c) return MREM_ERR_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "trace_enable: sync failed");
+  c->tracer.reset();
+  c->trace_on = on != 0;
+  return MREM_OK;
+}
+
+int32_t mrem_trace_read(mrem_ctx* c, mrem_trace_entry* out, int32_t max_entries, int32_t* n_entries) {
+  if (!c || !out || !n_entries || max_entries < 0) return MREM_ERR_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "trace_read: sync failed");
+  c->tracer.collect();
+  int n = 0;
+  for (const auto& kv : c->tracer.totals()) {
+    if (n >= max_entries) break;
+    mrem_trace_entry& e = out[n++];
+    std::memset(&e, 0, sizeof(e));
+    std::strncpy(e.name, kv.first.c_str(), sizeof(e.name) - 1);
+    e.ms = kv.second.ms; e.work = kv.second.work; e.launches = kv.second.launches; e.is_flops = kv.second.is_flops;
+  }
+  *n_entries = n;
   return MREM_OK;
 }
 

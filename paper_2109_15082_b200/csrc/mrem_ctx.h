@@ -96,7 +96,8 @@ struct mrem_ctx {
   int* t_counter;
   mrem::OptimScalars* optim_sc;
   mrem::ReduceEntry* reduce_table;   int reduce_per_layer = 0;
-  mrem::AdamEntry* adam_table;       int adam_entries = 0;
+  mrem::AdamEntry* adam_table;       int adam_entries = 0;  long long adam_elems = 0;
+  mrem::Tracer tracer;               bool trace_on = false;
   void *h2d_xt, *h2d_xs; int32_t* h2d_len; float* d_loss_e2e;   // staging of mrem_recon_step_host
   void *e2e_t_out, *e2e_s_out;                                  // its layer outputs [L, M, H]
   size_t state_off = 0, state_bytes = 0;                          // optimizer moments: one contiguous range

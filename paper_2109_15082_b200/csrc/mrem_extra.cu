@@ -77,6 +77,9 @@ int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, flo
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
   if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
+  const bool was_tracing = c->trace_on;
+  c->trace_on = false;              // event pairs are not recorded inside a captured graph
+  struct Restore { mrem_ctx* c; bool v; ~Restore() { c->trace_on = v; } } restore{c, was_tracing};
   if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();   // clear the sticky-until-read error: the legacy default stream cannot be captured
     return fail(c, MREM_ERR_CUDA, "graph_capture_step: begin capture failed (the context's stream must not be the legacy default stream)");
@@ -88,6 +91,22 @@ int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, flo
   if (e != cudaSuccess || !g) return fail(c, MREM_ERR_CUDA, "graph_capture_step: end capture failed");
   c->graph = g;
   if (cudaGraphInstantiate(&c->graph_exec, g, 0) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_capture_step: instantiate failed");
+  return MREM_OK;
+}
+
+int32_t mrem_graph_num_kernels(mrem_ctx* c, int32_t* n_kernels) {
+  if (!c || !n_kernels) return MREM_ERR_ARG;
+  if (!c->graph) return fail(c, MREM_ERR_ORDER, "graph_num_kernels: no captured step");
+  size_t n = 0;
+  if (cudaGraphGetNodes(c->graph, nullptr, &n) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_num_kernels failed");
+  std::vector<cudaGraphNode_t> nodes(n);
+  if (n && cudaGraphGetNodes(c->graph, nodes.data(), &n) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_num_kernels failed");
+  int k = 0;
+  for (size_t i = 0; i < n; ++i) {
+    cudaGraphNodeType t;
+    if (cudaGraphNodeGetType(nodes[i], &t) == cudaSuccess && t == cudaGraphNodeTypeKernel) ++k;
+  }
+  *n_kernels = k;
   return MREM_OK;
 }
 

@@ -296,6 +296,7 @@ extern "C" {
 
 int32_t mrem_quantize_weights(mrem_ctx* c) {
   if (!c) return MREM_ERR_ARG;
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) {
       const LayerBind& b = c->bind[l];
@@ -312,6 +313,7 @@ int32_t mrem_quantize_weights(mrem_ctx* c) {
 int32_t mrem_module_forward(mrem_ctx* c, int32_t role, const void* x, const void* x_other, float lambda,
                             const int32_t* len, int32_t batch, int32_t seq, void* outs) {
   if (!c) return MREM_ERR_ARG;
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   int rc = check_io(c, x, batch, seq, outs);
   if (rc != MREM_OK) return rc;
   if (c->have_teacher || c->have_student) {
@@ -343,6 +345,7 @@ int32_t mrem_module_forward(mrem_ctx* c, int32_t role, const void* x, const void
 
 int32_t mrem_recon_loss(mrem_ctx* c, float* loss_total, float* loss_per_layer) {
   if (!c || !loss_total) return MREM_ERR_ARG;
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_teacher || !c->have_student) return fail(c, MREM_ERR_ORDER, "recon_loss: needs a teacher and a student forward of the same batch");
   const long long n = (long long)c->cur_batch * c->cur_seq * c->d.hidden;
   const float cc = c->d.loss_mean ? 1.f / (float)n : 1.f;
@@ -355,6 +358,7 @@ int32_t mrem_recon_loss(mrem_ctx* c, float* loss_total, float* loss_per_layer) {
 
 int32_t mrem_module_backward(mrem_ctx* c) {
   if (!c) return MREM_ERR_ARG;
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k]) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
@@ -367,11 +371,12 @@ int32_t mrem_module_backward(mrem_ctx* c) {
 
 int32_t mrem_step(mrem_ctx* c, const mrem_optim* o) {
   if (!c || !o) return MREM_ERR_ARG;
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_grads) return fail(c, MREM_ERR_ORDER, "step: needs mrem_module_backward of this step");
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
                        o->weight_decay, c->stream);
-  launch_adamw_table(c->adam_table, c->adam_entries, c->optim_sc, c->stream);
+  launch_adamw_table(c->adam_table, c->adam_entries, c->adam_elems, c->optim_sc, c->stream);
   if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "step: launch failed");
   c->have_grads = false; c->have_loss = false; c->have_student = false; c->have_teacher = false;
   c->weights_quantized = false;

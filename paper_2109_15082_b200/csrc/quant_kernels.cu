@@ -224,6 +224,7 @@ bool vec_ok(const void* p, long long ld, int cols) {
 
 void launch_quantize_weight(const float* w, int rows, int cols, const float* steps, int per_row, int bits, int grid,
                             int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt, cudaStream_t st) {
+  Scope sc("quantize_weight", (double)rows * cols * (5.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)) + rows * 8.0, 0, st);
   if (dt == 1)
     quantize_weight_kernel<bf16><<<rows, 256, 0, st>>>(w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (bf16*)what);
   else
@@ -246,6 +247,7 @@ void launch_quantize_act(const void* x, int dt, long long rows, int cols, long l
                          const float* offset, int lo, int hi, int8_t* q8, long long ld_q8, void* qt,
                          long long ld_qt, cudaStream_t st) {
   if (rows <= 0 || cols <= 0) return;
+  Scope sc("quantize_act", (double)rows * cols * ((dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1) + (q8 ? 1 : 0)), 0, st);
   if (dt == 1) quantize_act_t<bf16>((const bf16*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (bf16*)qt, ld_qt, st);
   else quantize_act_t<float>((const float*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (float*)qt, ld_qt, st);
 }
@@ -262,6 +264,7 @@ void launch_narrow(const float* src, void* dst, long long n, int dt, cudaStream_
 
 void launch_mix(const void* f, const void* f_hat, float lam, void* out, long long n, int dt, cudaStream_t st) {
   if (n <= 0) return;
+  Scope sc("teacher_forcing_mix", (double)n * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
   if (dt == 1) {
     if (n % 8 == 0 && vec_ok<bf16>(f, 8, 8) && vec_ok<bf16>(f_hat, 8, 8) && vec_ok<bf16>(out, 8, 8))
       mix_kernel<bf16, 8><<<grid_for(n / 8), 256, 0, st>>>((const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
@@ -278,6 +281,7 @@ void launch_mix(const void* f, const void* f_hat, float lam, void* out, long lon
 void launch_gelu_quant(const void* u, long long n, const float* step, const float* offset, int lo, int hi,
                        int8_t* q8, void* qt, int dt, cudaStream_t st) {
   if (n <= 0) return;
+  Scope sc("gelu_quant", (double)n * ((dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1) + (q8 ? 1 : 0)), 0, st);
   if (dt == 1) {
     const bool v = n % 8 == 0 && vec_ok<bf16>(u, 8, 8) && vec_ok<bf16>(qt, 8, 8) && (reinterpret_cast<uintptr_t>(q8) % 8) == 0;
     if (v) gelu_quant_kernel<bf16, 8><<<grid_for(n / 8), 256, 0, st>>>((const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
@@ -309,6 +313,7 @@ void launch_step_from_minmax(const float* minmax, int mode, float qmax, float* s
 void launch_gather_rows(const void* src, const int* d_idx, int n_rows, long long row_bytes, void* out,
                         cudaStream_t st) {
   const long long row_vecs = row_bytes / 16;
+  Scope sc("gather_rows", 2.0 * n_rows * (double)row_bytes, 0, st);
   dim3 grid(grid_for(row_vecs, 256, 64), n_rows);
   gather_rows_kernel<<<grid, 256, 0, st>>>((const uint4*)src, d_idx, row_vecs, (uint4*)out);
 }
