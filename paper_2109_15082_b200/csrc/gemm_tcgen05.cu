@@ -3,8 +3,10 @@
 // One persistent CTA per SM.  Warp 0 streams operand tiles into a ring of shared-memory
 // stages with TMA (128-byte swizzle), warp 1 issues tcgen05.mma (bf16 -> fp32, or
 // int8 -> int32 with exact accumulation) into one of two TMEM accumulator buffers, and
-// warps 2..5 drain the other buffer with tcgen05.ld, apply the epilogue and write the
-// result, so the epilogue of tile i overlaps the main loop of tile i+1.
+// warps 2..9 drain the other buffer with tcgen05.ld, apply the epilogue and write the
+// result through a per-warp shared-memory transpose (each store instruction then covers
+// whole 64- or 128-byte row segments), so the epilogue of tile i overlaps the main loop of
+// tile i+1.
 // Either operand may be stored k-contiguous ("K-major") or m/n-contiguous ("MN-major");
 // the second form serves the backward products (dX = dY * W_hat, dW = dY^T * X_hat) and
 // the attention products without any transposed copy.
@@ -23,7 +25,10 @@ constexpr int BLOCK_M = 128;
 constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
 constexpr int TILE_SMEM_BUDGET = 196608;              // bytes of operand stages per CTA
 constexpr int MAX_STAGES = 8;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;                    // TMA warp, MMA warp, 8 epilogue warps
+constexpr int EPI_WARPS = 8;
+constexpr int STAGING_WORDS = 32 * 33;               // per epilogue warp: 32 rows x 32 words, padded
+constexpr int STAGING_BYTES = EPI_WARPS * STAGING_WORDS * 4;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait
 
@@ -224,6 +229,99 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, const uint32_t
   }
 }
 
+// ------------------------------------------------------------------ epilogue of a 32-row x 32-word block
+// One warp, one round: 64 bf16 or 32 fp32/int32 output columns of its 32 rows.  Values go
+// through the warp's staging buffer so that global loads (residual) and stores are issued
+// as 16-byte pieces with 8 lanes covering one contiguous row segment.
+template <int KIND>
+__device__ __forceinline__ void epilogue_round(const TcParams& p, uint32_t taddr, float alpha, long long tile_off,
+                                               int row0, int col0, int lane, uint32_t* stg) {
+  const Epilogue& e = p.epi;
+  const bool is_bf16 = e.out_kind == OUT_BF16;
+  const int vec_elems = is_bf16 ? 8 : 4;
+  const int sub = lane >> 3, seg = lane & 7;             // 4 rows per instruction, 8 lanes per row
+  uint32_t res[32];
+  if (e.residual) {
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int rl = it * 4 + sub, row = row0 + rl;
+      uint4 u = make_uint4(0, 0, 0, 0);
+      if (row < p.M) {
+        const long long off = tile_off + (long long)row * e.ldc + col0 + seg * vec_elems;
+        u = is_bf16 ? *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(e.residual) + off)
+                    : *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(e.residual) + off);
+      }
+      uint32_t* d = stg + rl * 33 + seg * 4;
+      d[0] = u.x; d[1] = u.y; d[2] = u.z; d[3] = u.w;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) res[j] = stg[lane * 33 + j];
+    __syncwarp();
+  }
+  const int row = row0 + lane;
+  const float rb = (e.row_bias && row < p.M) ? e.row_bias[row] : 0.f;
+  const int n_loads = is_bf16 ? 2 : 1;
+  for (int h = 0; h < n_loads; ++h) {
+    uint32_t r[32];
+    tmem_ld32(taddr + (uint32_t)(h * 32), r);
+    if (e.out_kind == OUT_I32) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = r[j];
+      continue;
+    }
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int n = col0 + h * 32 + j;
+      const float a = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
+      const float sc = e.col_scale ? alpha * e.col_scale[n] : alpha;
+      v[j] = a * sc + (e.col_bias ? e.col_bias[n] : 0.f) + rb;
+    }
+    if (e.residual) {
+      if (is_bf16) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&res[h * 16 + j]);
+          const float2 f = __bfloat1622float2(h2);
+          v[2 * j] += f.x;
+          v[2 * j + 1] += f.y;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(res[j]);
+      }
+    }
+    if (e.act == 1) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+    }
+    if (is_bf16) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        stg[lane * 33 + h * 16 + j] = *reinterpret_cast<const uint32_t*>(&h2);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __float_as_uint(v[j]);
+    }
+  }
+  __syncwarp();
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int rl = it * 4 + sub, orow = row0 + rl;
+    if (orow < p.M) {
+      const uint32_t* sp = stg + rl * 33 + seg * 4;
+      const uint4 u = make_uint4(sp[0], sp[1], sp[2], sp[3]);
+      const long long off = tile_off + (long long)orow * e.ldc + col0 + seg * vec_elems;
+      if (is_bf16) *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(e.out) + off) = u;
+      else *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(e.out) + off) = u;
+    }
+  }
+  __syncwarp();
+}
+
 // ------------------------------------------------------------------ the kernel
 template <int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -247,7 +345,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&tfull_bar[a]), 1);
-      mbar_init(smem_u32(&tempty_bar[a]), 4);
+      mbar_init(smem_u32(&tempty_bar[a]), EPI_WARPS);
     }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -343,8 +441,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ---------------- epilogue warps (TMEM lane quadrant = warp % 4)
-    const int quad = warp & 3;
+    // ---------------- epilogue warps: TMEM lane quadrant = warp % 4, two warps per quadrant
+    const int quad = warp & 3, half = (warp - 2) >> 2;
     const Epilogue& e = p.epi;
     float alpha = e.alpha_const;
     if (e.alpha_p0) alpha *= *e.alpha_p0;
@@ -354,6 +452,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     bool vec_ok = (e.ldc % vec_elems == 0) && (e.c_b0 % vec_elems == 0) && (e.c_b1 % vec_elems == 0) &&
                   ((reinterpret_cast<uintptr_t>(e.out) & 15) == 0);
     if (e.residual) vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(e.residual) & 15) == 0);
+    uint32_t* stg = reinterpret_cast<uint32_t*>(smem_raw + (tiles_base - smem_u32(smem_raw)) +
+                                                (size_t)p.num_stages * p.stage_bytes) + (warp - 2) * STAGING_WORDS;
+    const int cols_per_round = (e.out_kind == OUT_BF16) ? 64 : 32;
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
@@ -365,15 +466,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         break;
       }
       tc_fence_after();
-      const int row = t.m0 + quad * 32 + lane;
-      const bool row_ok = row < p.M;
-      const long long row_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1 + (long long)row * e.ldc;
+      const int row0 = t.m0 + quad * 32;
+      const long long tile_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * p.block_n);
-      for (int c = 0; c < p.block_n; c += 32) {
-        if (t.n0 + c >= p.N) break;                    // warp-uniform
-        uint32_t r[32];
-        tmem_ld32(taddr + (uint32_t)c, r);
-        epilogue_chunk<KIND>(p, r, alpha, row_off, row, t.n0 + c, row_ok, vec_ok);
+      for (int round = half; round * cols_per_round < p.block_n; round += 2) {
+        const int c0 = round * cols_per_round, col0 = t.n0 + c0;
+        if (col0 >= p.N) break;                          // warp-uniform
+        const bool fast = vec_ok && col0 + cols_per_round <= p.N;
+        if (fast) {
+          epilogue_round<KIND>(p, taddr + (uint32_t)c0, alpha, tile_off, row0, col0, lane, stg);
+        } else {
+          const int row = row0 + lane;
+          const long long row_off = tile_off + (long long)row * e.ldc;
+          for (int c = c0; c < c0 + cols_per_round && t.n0 + c < p.N; c += 32) {
+            uint32_t r[32];
+            tmem_ld32(taddr + (uint32_t)c, r);
+            epilogue_chunk<KIND>(p, r, alpha, row_off, row, t.n0 + c, row < p.M, false);
+          }
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -497,11 +607,11 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   rc = make_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k);
   if (rc != GEMM_OK) return rc;
 
-  const int smem = p.num_stages * p.stage_bytes + 1024;
+  const int smem = p.num_stages * p.stage_bytes + 1024 + STAGING_BYTES;
   static bool attr_set[2] = {false, false};
   auto kern = kind == 0 ? tc_gemm_kernel<0> : tc_gemm_kernel<1>;
   if (!attr_set[kind]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TILE_SMEM_BUDGET + 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TILE_SMEM_BUDGET + 1024 + STAGING_BYTES) != cudaSuccess)
       return GEMM_ERR_CUDA;
     attr_set[kind] = true;
   }

@@ -6,7 +6,7 @@
 
 namespace mrem {
 
-constexpr int RED_BLOCKS = 296;     // grid of every kernel that emits per-block partial sums (2 x 148 SMs)
+constexpr int RED_BLOCKS = 1184;    // grid of every kernel that emits per-block partial sums (8 x 148 SMs)
 
 // ---- quantizers (Eq. 1)
 // Weight quantizer: latent w[rows, cols] fp32 and steps (one per row, or one in all) ->

@@ -14,224 +14,6 @@ __device__ __forceinline__ float qz(float x, float s, float off, bool has_off) {
 }
 __device__ __forceinline__ int qcode(float z, float lo, float hi) { return __float2int_rn(fminf(fmaxf(z, lo), hi)); }
 
-// ------------------------------------------------------------------ LayerNorm forward (one warp per row)
-template <typename T, int V>
-__global__ void __launch_bounds__(128) ln_fwd_kernel(const T* __restrict__ y, const float* __restrict__ gamma,
-                                                     const float* __restrict__ beta, float eps, long long rows,
-                                                     int cols, T* __restrict__ out, float* __restrict__ mean,
-                                                     float* __restrict__ rstd, const float* __restrict__ step,
-                                                     float qmax, int8_t* __restrict__ q8, T* __restrict__ qt) {
-  const int lane = threadIdx.x & 31;
-  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
-  if (row >= rows) return;
-  const T* yr = y + row * cols;
-  float sum = 0.f;
-  for (int c = lane * V; c < cols; c += 32 * V) {
-    float v[V];
-    load_vec<T, V>(yr + c, v);
-#pragma unroll
-    for (int j = 0; j < V; ++j) sum += v[j];
-  }
-  const float mu = warp_sum(sum) / (float)cols;
-  float sq = 0.f;
-  for (int c = lane * V; c < cols; c += 32 * V) {
-    float v[V];
-    load_vec<T, V>(yr + c, v);
-#pragma unroll
-    for (int j = 0; j < V; ++j) sq += (v[j] - mu) * (v[j] - mu);
-  }
-  const float rs = 1.f / sqrtf(warp_sum(sq) / (float)cols + eps);
-  if (lane == 0) {
-    if (mean) mean[row] = mu;
-    if (rstd) rstd[row] = rs;
-  }
-  const float s = step ? *step : 1.f;
-  for (int c = lane * V; c < cols; c += 32 * V) {
-    float v[V];
-    load_vec<T, V>(yr + c, v);
-#pragma unroll
-    for (int j = 0; j < V; ++j) v[j] = (v[j] - mu) * rs * gamma[c + j] + beta[c + j];
-    store_vec<T, V>(out + row * cols + c, v);
-    if (step) {
-      int q[V];
-#pragma unroll
-      for (int j = 0; j < V; ++j) q[j] = qcode(__fdiv_rn(stored<T>(v[j]), s), -qmax, qmax);
-      if (q8) store_codes<V>(q8 + row * cols + c, q);
-      if (qt) {
-#pragma unroll
-        for (int j = 0; j < V; ++j) v[j] = (float)q[j];
-        store_vec<T, V>(qt + row * cols + c, v);
-      }
-    }
-  }
-}
-
-// ------------------------------------------------------------------ LayerNorm backward (one warp per row)
-template <typename T, int V>
-__global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ dout2,
-                                                     const T* __restrict__ y, const float* __restrict__ mean,
-                                                     const float* __restrict__ rstd, const float* __restrict__ gamma,
-                                                     long long rows, int cols, T* __restrict__ dy,
-                                                     T* __restrict__ dsum) {
-  const int lane = threadIdx.x & 31;
-  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
-  if (row >= rows) return;
-  const float mu = mean[row], rs = rstd[row];
-  const long long base = row * cols;
-  float s1 = 0.f, s2 = 0.f;
-  for (int c = lane * V; c < cols; c += 32 * V) {
-    float d[V], v[V];
-    load_vec<T, V>(dout + base + c, d);
-    if (dout2) {
-      float e[V];
-      load_vec<T, V>(dout2 + base + c, e);
-#pragma unroll
-      for (int j = 0; j < V; ++j) d[j] += e[j];
-      if (dsum) store_vec<T, V>(dsum + base + c, d);
-    }
-    load_vec<T, V>(y + base + c, v);
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-      const float dxn = (dout2 && dsum ? stored<T>(d[j]) : d[j]) * gamma[c + j];
-      s1 += dxn;
-      s2 += dxn * (v[j] - mu) * rs;
-    }
-  }
-  s1 = warp_sum(s1) / (float)cols;
-  s2 = warp_sum(s2) / (float)cols;
-  for (int c = lane * V; c < cols; c += 32 * V) {
-    float d[V], v[V];
-    load_vec<T, V>((dout2 && dsum ? dsum : dout) + base + c, d);
-    if (dout2 && !dsum) {
-      float e[V];
-      load_vec<T, V>(dout2 + base + c, e);
-#pragma unroll
-      for (int j = 0; j < V; ++j) d[j] += e[j];
-    }
-    load_vec<T, V>(y + base + c, v);
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-      const float xn = (v[j] - mu) * rs;
-      d[j] = rs * (d[j] * gamma[c + j] - s1 - xn * s2);
-    }
-    store_vec<T, V>(dy + base + c, d);
-  }
-}
-
-// ------------------------------------------------------------------ column sums over rows (bias and LayerNorm parameter gradients)
-template <typename T>
-__global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a, long long ld_a,
-                                                         const T* __restrict__ y, const float* __restrict__ mean,
-                                                         const float* __restrict__ rstd, long long rows, int cols,
-                                                         float* __restrict__ scratch) {
-  __shared__ float sh0[8][33], sh1[8][33];
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int c = blockIdx.x * 32 + tx;
-  const long long per = (rows + COL_CHUNKS - 1) / COL_CHUNKS;
-  const long long r0 = blockIdx.y * per, r1 = r0 + per < rows ? r0 + per : rows;
-  float a0 = 0.f, a1 = 0.f;
-  if (c < cols) {
-    for (long long r = r0 + ty; r < r1; r += 8) {
-      const float v = to_f<T>(a[r * ld_a + c]);
-      a0 += v;
-      if (y) a1 += v * (to_f<T>(y[r * cols + c]) - mean[r]) * rstd[r];
-    }
-  }
-  sh0[ty][tx] = a0;
-  sh1[ty][tx] = a1;
-  __syncthreads();
-  if (ty == 0 && c < cols) {
-    float t0 = 0.f, t1 = 0.f;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) { t0 += sh0[k][tx]; t1 += sh1[k][tx]; }
-    scratch[(long long)blockIdx.y * cols + c] = t0;
-    if (y) scratch[((long long)COL_CHUNKS + blockIdx.y) * cols + c] = t1;
-  }
-}
-__global__ void col_reduce_final_kernel(const float* __restrict__ scratch, int cols, float* __restrict__ out0,
-                                        float* __restrict__ out1) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
-  float t0 = 0.f, t1 = 0.f;
-  for (int k = 0; k < COL_CHUNKS; ++k) {
-    t0 += scratch[(long long)k * cols + c];
-    if (out1) t1 += scratch[((long long)COL_CHUNKS + k) * cols + c];
-  }
-  out0[c] = t0;
-  if (out1) out1[c] = t1;
-}
-
-// ------------------------------------------------------------------ softmax forward (one warp per row)
-template <typename T>
-__global__ void __launch_bounds__(128) softmax_fwd_kernel(const float* __restrict__ scores,
-                                                          const int* __restrict__ valid_len, int h, int S,
-                                                          long long rows, T* __restrict__ P,
-                                                          const float* __restrict__ step,
-                                                          const float* __restrict__ offset, float lo, float hi,
-                                                          T* __restrict__ qt) {
-  const int lane = threadIdx.x & 31;
-  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
-  if (row >= rows) return;
-  const int b = (int)(row / ((long long)h * S));
-  int len = valid_len ? valid_len[b] : S;
-  len = len < 1 ? 1 : (len > S ? S : len);
-  const float* sr = scores + row * S;
-  float mx = -INFINITY;
-  for (int j = lane; j < len; j += 32) mx = fmaxf(mx, sr[j]);
-  mx = warp_max(mx);
-  float sum = 0.f;
-  for (int j = lane; j < len; j += 32) sum += expf(sr[j] - mx);
-  sum = warp_sum(sum);
-  const float s = step ? *step : 1.f;
-  const bool has_off = offset != nullptr;
-  const float off = has_off ? *offset : 0.f;
-  for (int j = lane; j < S; j += 32) {
-    const float p = j < len ? __fdiv_rn(expf(sr[j] - mx), sum) : 0.f;
-    P[row * S + j] = from_f<T>(p);
-    if (qt) qt[row * S + j] = from_f<T>((float)qcode(qz(stored<T>(p), s, off, has_off), lo, hi));
-  }
-}
-
-// ------------------------------------------------------------------ softmax backward with the STE of the P quantizer
-template <typename T>
-__global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ P, const T* __restrict__ dphat,
-                                                          T* __restrict__ dS, long long rows, int S,
-                                                          const float* __restrict__ step, float lo, float hi,
-                                                          int quantized, float* __restrict__ part_s) {
-  __shared__ float sh[32];
-  const int lane = threadIdx.x & 31;
-  const long long warp0 = blockIdx.x * 8ll + (threadIdx.x >> 5), nwarps = gridDim.x * 8ll;
-  const float s = quantized ? *step : 1.f;
-  float ds = 0.f;
-  for (long long row = warp0; row < rows; row += nwarps) {
-    const long long base = row * S;
-    float dot = 0.f;
-    for (int j = lane; j < S; j += 32) {
-      const float p = to_f<T>(P[base + j]);
-      float d = to_f<T>(dphat[base + j]);
-      if (quantized) {
-        const float z = __fdiv_rn(p, s);
-        const bool in = z >= lo && z <= hi;
-        ds += d * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
-        d = in ? d : 0.f;
-      }
-      dot += d * p;
-    }
-    dot = warp_sum(dot);
-    for (int j = lane; j < S; j += 32) {
-      const float p = to_f<T>(P[base + j]);
-      float d = to_f<T>(dphat[base + j]);
-      if (quantized) {
-        const float z = __fdiv_rn(p, s);
-        d = (z >= lo && z <= hi) ? d : 0.f;
-      }
-      dS[base + j] = from_f<T>(p * (d - dot));
-    }
-  }
-  ds = block_sum(ds, sh);
-  if (threadIdx.x == 0 && part_s) part_s[blockIdx.x] = ds;
-}
-
 // ------------------------------------------------------------------ loss (Eq. 3) and its gradient
 template <typename T, int V>
 __global__ void __launch_bounds__(256) loss_kernel(const T* __restrict__ fh, const T* __restrict__ f,
@@ -452,57 +234,6 @@ inline bool al16(const void* p) { return p == nullptr || (reinterpret_cast<uintp
   do {                                 \
     if ((dt) == 1) { using T = bf16; __VA_ARGS__; } else { using T = float; __VA_ARGS__; } \
   } while (0)
-
-void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, float eps, long long rows, int cols,
-                          void* out, float* mean, float* rstd, const float* step, int qmax, int8_t* q8, void* qt,
-                          int dt, cudaStream_t st) {
-  if (rows <= 0) return;
-  Scope sc("layernorm_fwd", (double)rows * cols * ((dt == 1 ? 2.0 : 4.0) * (qt ? 3 : 2) + (q8 ? 1 : 0)), 0, st);
-  const int grid = (int)((rows + 3) / 4);
-  MREM_DT(dt, T, {
-    constexpr int V = 16 / (int)sizeof(T);
-    const bool v = cols % V == 0 && al16(y) && al16(out) && al16(qt) && (reinterpret_cast<uintptr_t>(q8) % V) == 0;
-    if (v) ln_fwd_kernel<T, V><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
-    else ln_fwd_kernel<T, 1><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
-  });
-}
-
-void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, const float* mean, const float* rstd,
-                          const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
-                          cudaStream_t st) {
-  if (rows <= 0) return;
-  Scope sc("layernorm_bwd", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (3 + (dout2 ? 1 : 0) + (dsum ? 1 : 0)), 0, st);
-  const int grid = (int)((rows + 3) / 4);
-  MREM_DT(dt, T, {
-    constexpr int V = 16 / (int)sizeof(T);
-    const bool v = cols % V == 0 && al16(dout) && al16(dout2) && al16(y) && al16(dy) && al16(dsum);
-    if (v) ln_bwd_kernel<T, V><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
-    else ln_bwd_kernel<T, 1><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
-  });
-}
-
-void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
-                       long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st) {
-  Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (y ? 2 : 1), 0, st);
-  dim3 grid((cols + 31) / 32, COL_CHUNKS);
-  MREM_DT(dt, T, { col_reduce_kernel<T><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch); });
-  col_reduce_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, cols, out0, y ? out1 : nullptr);
-}
-
-void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,
-                        const float* offset, int lo, int hi, void* qt, int dt, cudaStream_t st) {
-  const long long rows = (long long)B * h * S;
-  if (rows <= 0) return;
-  Scope sc("softmax_fwd", (double)rows * S * (4.0 + (dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1)), 0, st);
-  const int grid = (int)((rows + 3) / 4);
-  MREM_DT(dt, T, { softmax_fwd_kernel<T><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt); });
-}
-
-void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long rows, int S, const float* step,
-                        int lo, int hi, int quantized, float* part_s, int dt, cudaStream_t st) {
-  Scope sc("softmax_bwd", (double)rows * S * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
-  MREM_DT(dt, T, { softmax_bwd_kernel<T><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s); });
-}
 
 void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per_layer, float c, void* dF,
                  float* partial, int* status, int dt, cudaStream_t st) {

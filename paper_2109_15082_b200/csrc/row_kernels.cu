@@ -1,0 +1,476 @@
+// Row-wise kernels: LayerNorm forward/backward, attention softmax forward/backward (with the
+// quantizer of the probabilities), and column sums over rows (bias / LayerNorm-parameter
+// gradients).  One warp owns one row and keeps it in registers (one read of each input,
+// 8- or 16-byte vector accesses, warp-shuffle reductions); a slower re-reading form covers
+// rows too long for the register cache or views that are not vector aligned.
+#include "kernels.h"
+#include "vec.cuh"
+
+namespace mrem {
+
+namespace {
+
+constexpr int MAXNV = 4;     // vectors per lane held in registers
+
+__device__ __forceinline__ float qz(float x, float s, float off, bool has_off) {
+  return __fdiv_rn(has_off ? __fsub_rn(x, off) : x, s);
+}
+__device__ __forceinline__ int qcode(float z, float lo, float hi) { return __float2int_rn(fminf(fmaxf(z, lo), hi)); }
+
+// 4 consecutive values
+template <typename T> __device__ __forceinline__ void load4(const T* p, float* v);
+template <> __device__ __forceinline__ void load4<float>(const float* p, float* v) {
+  const float4 t = *reinterpret_cast<const float4*>(p);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+template <> __device__ __forceinline__ void load4<bf16>(const bf16* p, float* v) {
+  const uint2 t = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&t);
+  const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+  v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+template <typename T> __device__ __forceinline__ void store4(T* p, const float* v);
+template <> __device__ __forceinline__ void store4<float>(float* p, const float* v) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <> __device__ __forceinline__ void store4<bf16>(bf16* p, const float* v) {
+  uint2 t;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&t);
+  h[0] = __floats2bfloat162_rn(v[0], v[1]);
+  h[1] = __floats2bfloat162_rn(v[2], v[3]);
+  *reinterpret_cast<uint2*>(p) = t;
+}
+
+// ------------------------------------------------------------------ LayerNorm forward
+// CACHED: the row sits in registers (cols <= 32 * V * MAXNV, cols % V == 0); else V == 1 and
+// the row is re-read from L1/L2 in each of the three passes.
+template <typename T, int V, bool CACHED>
+__global__ void __launch_bounds__(128) ln_fwd_kernel(const T* __restrict__ y, const float* __restrict__ gamma,
+                                                     const float* __restrict__ beta, float eps, long long rows,
+                                                     int cols, T* __restrict__ out, float* __restrict__ mean,
+                                                     float* __restrict__ rstd, const float* __restrict__ step,
+                                                     float qmax, int8_t* __restrict__ q8, T* __restrict__ qt) {
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const T* yr = y + row * cols;
+  float v[CACHED ? MAXNV : 1][V];
+  float sum = 0.f;
+  if constexpr (CACHED) {
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * V;
+      if (c < cols) {
+        load_vec<T, V>(yr + c, v[i]);
+#pragma unroll
+        for (int j = 0; j < V; ++j) sum += v[i][j];
+      }
+    }
+  } else {
+    for (int c = lane; c < cols; c += 32) sum += to_f<T>(yr[c]);
+  }
+  const float mu = warp_sum(sum) / (float)cols;
+  float sq = 0.f;
+  if constexpr (CACHED) {
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i)
+      if ((lane + 32 * i) * V < cols) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) sq += (v[i][j] - mu) * (v[i][j] - mu);
+      }
+  } else {
+    for (int c = lane; c < cols; c += 32) { const float d = to_f<T>(yr[c]) - mu; sq += d * d; }
+  }
+  const float rs = 1.f / sqrtf(warp_sum(sq) / (float)cols + eps);
+  if (lane == 0) {
+    if (mean) mean[row] = mu;
+    if (rstd) rstd[row] = rs;
+  }
+  const float s = step ? *step : 1.f;
+  auto emit = [&](int c, float* o) {
+#pragma unroll
+    for (int j = 0; j < V; ++j) o[j] = (o[j] - mu) * rs * gamma[c + j] + beta[c + j];
+    store_vec<T, V>(out + row * cols + c, o);
+    if (step) {
+      int q[V];
+#pragma unroll
+      for (int j = 0; j < V; ++j) q[j] = qcode(__fdiv_rn(stored<T>(o[j]), s), -qmax, qmax);
+      if (q8) store_codes<V>(q8 + row * cols + c, q);
+      if (qt) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) o[j] = (float)q[j];
+        store_vec<T, V>(qt + row * cols + c, o);
+      }
+    }
+  };
+  if constexpr (CACHED) {
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * V;
+      if (c < cols) emit(c, v[i]);
+    }
+  } else {
+    for (int c = lane; c < cols; c += 32) {
+      float o[V];
+      o[0] = to_f<T>(yr[c]);
+      emit(c, o);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ LayerNorm backward
+template <typename T, int V, bool CACHED>
+__global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ dout2,
+                                                     const T* __restrict__ y, const float* __restrict__ mean,
+                                                     const float* __restrict__ rstd, const float* __restrict__ gamma,
+                                                     long long rows, int cols, T* __restrict__ dy,
+                                                     T* __restrict__ dsum) {
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float mu = mean[row], rs = rstd[row];
+  const long long base = row * cols;
+  float d[CACHED ? MAXNV : 1][V], xn[CACHED ? MAXNV : 1][V];
+  float s1 = 0.f, s2 = 0.f;
+  // total incoming gradient of one vector; written to dsum (rounded to storage) when requested
+  auto fetch = [&](int c, float* dv, float* xv) {
+    load_vec<T, V>(dout + base + c, dv);
+    if (dout2) {
+      float e[V];
+      load_vec<T, V>(dout2 + base + c, e);
+#pragma unroll
+      for (int j = 0; j < V; ++j) dv[j] += e[j];
+      if (dsum) {
+        store_vec<T, V>(dsum + base + c, dv);
+#pragma unroll
+        for (int j = 0; j < V; ++j) dv[j] = stored<T>(dv[j]);
+      }
+    }
+    load_vec<T, V>(y + base + c, xv);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      xv[j] = (xv[j] - mu) * rs;
+      dv[j] *= gamma[c + j];
+    }
+  };
+  if constexpr (CACHED) {
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * V;
+      if (c < cols) {
+        fetch(c, d[i], xn[i]);
+#pragma unroll
+        for (int j = 0; j < V; ++j) { s1 += d[i][j]; s2 += d[i][j] * xn[i][j]; }
+      }
+    }
+  } else {
+    for (int c = lane; c < cols; c += 32) {
+      fetch(c, d[0], xn[0]);
+      s1 += d[0][0];
+      s2 += d[0][0] * xn[0][0];
+    }
+  }
+  s1 = warp_sum(s1) / (float)cols;
+  s2 = warp_sum(s2) / (float)cols;
+  if constexpr (CACHED) {
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * V;
+      if (c < cols) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) d[i][j] = rs * (d[i][j] - s1 - xn[i][j] * s2);
+        store_vec<T, V>(dy + base + c, d[i]);
+      }
+    }
+  } else {
+    const T* dsrc = (dout2 && dsum) ? dsum : dout;
+    for (int c = lane; c < cols; c += 32) {
+      float dv = to_f<T>(dsrc[base + c]);
+      if (dout2 && !dsum) dv += to_f<T>(dout2[base + c]);
+      const float x = (to_f<T>(y[base + c]) - mu) * rs;
+      dy[base + c] = from_f<T>(rs * (dv * gamma[c] - s1 - x * s2));
+    }
+  }
+}
+
+// ------------------------------------------------------------------ column sums over rows
+// Block (32 x 8): 32 * V columns, a chunk of rows; fixed-order tree over the 8 row groups.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a, long long ld_a,
+                                                         const T* __restrict__ y, const float* __restrict__ mean,
+                                                         const float* __restrict__ rstd, long long rows, int cols,
+                                                         float* __restrict__ scratch) {
+  __shared__ float sh0[8][32 * V + 1], sh1[8][32 * V + 1];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int c = (blockIdx.x * 32 + tx) * V;
+  const long long per = (rows + COL_CHUNKS - 1) / COL_CHUNKS;
+  const long long r0 = blockIdx.y * per, r1 = r0 + per < rows ? r0 + per : rows;
+  float a0[V], a1[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) a0[j] = a1[j] = 0.f;
+  if (c < cols) {
+    for (long long r = r0 + ty; r < r1; r += 8) {
+      float v[V];
+      load_vec<T, V>(a + r * ld_a + c, v);
+#pragma unroll
+      for (int j = 0; j < V; ++j) a0[j] += v[j];
+      if (y) {
+        float w[V];
+        load_vec<T, V>(y + r * cols + c, w);
+        const float mu = mean[r], rs = rstd[r];
+#pragma unroll
+        for (int j = 0; j < V; ++j) a1[j] += v[j] * (w[j] - mu) * rs;
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < V; ++j) { sh0[ty][tx * V + j] = a0[j]; sh1[ty][tx * V + j] = a1[j]; }
+  __syncthreads();
+  for (int i = threadIdx.x; i < 32 * V; i += 256) {
+    const int cc = blockIdx.x * 32 * V + i;
+    if (cc >= cols) continue;
+    float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { t0 += sh0[k][i]; t1 += sh1[k][i]; }
+    scratch[(long long)blockIdx.y * cols + cc] = t0;
+    if (y) scratch[((long long)COL_CHUNKS + blockIdx.y) * cols + cc] = t1;
+  }
+}
+__global__ void col_reduce_final_kernel(const float* __restrict__ scratch, int cols, float* __restrict__ out0,
+                                        float* __restrict__ out1) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  float t0 = 0.f, t1 = 0.f;
+  for (int k = 0; k < COL_CHUNKS; ++k) {
+    t0 += scratch[(long long)k * cols + c];
+    if (out1) t1 += scratch[((long long)COL_CHUNKS + k) * cols + c];
+  }
+  out0[c] = t0;
+  if (out1) out1[c] = t1;
+}
+
+// ------------------------------------------------------------------ softmax forward
+// CACHED: S % 4 == 0 and S <= 128 * MAXNV; the row of scores stays in registers.
+template <typename T, bool CACHED>
+__global__ void __launch_bounds__(128) softmax_fwd_kernel(const float* __restrict__ scores,
+                                                          const int* __restrict__ valid_len, int h, int S,
+                                                          long long rows, T* __restrict__ P,
+                                                          const float* __restrict__ step,
+                                                          const float* __restrict__ offset, float lo, float hi,
+                                                          T* __restrict__ qt) {
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int b = (int)(row / ((long long)h * S));
+  int len = valid_len ? valid_len[b] : S;
+  len = len < 1 ? 1 : (len > S ? S : len);
+  const float* sr = scores + row * S;
+  const float s = step ? *step : 1.f;
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  if constexpr (CACHED) {
+    float e[MAXNV][4];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * 4;
+      if (c < S) {
+        load4<float>(sr + c, e[i]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) if (c + j < len) mx = fmaxf(mx, e[i][j]);
+      }
+    }
+    mx = warp_max(mx);
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * 4;
+      if (c < S) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          e[i][j] = c + j < len ? expf(e[i][j] - mx) : 0.f;
+          sum += e[i][j];
+        }
+      }
+    }
+    sum = warp_sum(sum);
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * 4;
+      if (c < S) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) e[i][j] = __fdiv_rn(e[i][j], sum);
+        store4<T>(P + row * S + c, e[i]);
+        if (qt) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) e[i][j] = (float)qcode(qz(stored<T>(e[i][j]), s, off, has_off), lo, hi);
+          store4<T>(qt + row * S + c, e[i]);
+        }
+      }
+    }
+  } else {
+    float mx = -INFINITY;
+    for (int j = lane; j < len; j += 32) mx = fmaxf(mx, sr[j]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int j = lane; j < len; j += 32) sum += expf(sr[j] - mx);
+    sum = warp_sum(sum);
+    for (int j = lane; j < S; j += 32) {
+      const float p = j < len ? __fdiv_rn(expf(sr[j] - mx), sum) : 0.f;
+      P[row * S + j] = from_f<T>(p);
+      if (qt) qt[row * S + j] = from_f<T>((float)qcode(qz(stored<T>(p), s, off, has_off), lo, hi));
+    }
+  }
+}
+
+// ------------------------------------------------------------------ softmax backward with the STE of the P quantizer
+template <typename T, bool CACHED>
+__global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ P, const T* __restrict__ dphat,
+                                                          T* __restrict__ dS, long long rows, int S,
+                                                          const float* __restrict__ step, float lo, float hi,
+                                                          int quantized, float* __restrict__ part_s) {
+  __shared__ float sh[32];
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = blockIdx.x * 8ll + (threadIdx.x >> 5), nwarps = gridDim.x * 8ll;
+  const float s = quantized ? *step : 1.f;
+  float ds = 0.f;
+  for (long long row = warp0; row < rows; row += nwarps) {
+    const long long base = row * S;
+    if constexpr (CACHED) {
+      float p[MAXNV][4], d[MAXNV][4];
+      float dot = 0.f;
+#pragma unroll
+      for (int i = 0; i < MAXNV; ++i) {
+        const int c = (lane + 32 * i) * 4;
+        if (c < S) {
+          load4<T>(P + base + c, p[i]);
+          load4<T>(dphat + base + c, d[i]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (quantized) {
+              const float z = __fdiv_rn(p[i][j], s);
+              const bool in = z >= lo && z <= hi;
+              ds += d[i][j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+              d[i][j] = in ? d[i][j] : 0.f;
+            }
+            dot += d[i][j] * p[i][j];
+          }
+        }
+      }
+      dot = warp_sum(dot);
+#pragma unroll
+      for (int i = 0; i < MAXNV; ++i) {
+        const int c = (lane + 32 * i) * 4;
+        if (c < S) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) d[i][j] = p[i][j] * (d[i][j] - dot);
+          store4<T>(dS + base + c, d[i]);
+        }
+      }
+    } else {
+      float dot = 0.f;
+      for (int j = lane; j < S; j += 32) {
+        const float p = to_f<T>(P[base + j]);
+        float d = to_f<T>(dphat[base + j]);
+        if (quantized) {
+          const float z = __fdiv_rn(p, s);
+          const bool in = z >= lo && z <= hi;
+          ds += d * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+          d = in ? d : 0.f;
+        }
+        dot += d * p;
+      }
+      dot = warp_sum(dot);
+      for (int j = lane; j < S; j += 32) {
+        const float p = to_f<T>(P[base + j]);
+        float d = to_f<T>(dphat[base + j]);
+        if (quantized) {
+          const float z = __fdiv_rn(p, s);
+          d = (z >= lo && z <= hi) ? d : 0.f;
+        }
+        dS[base + j] = from_f<T>(p * (d - dot));
+      }
+    }
+  }
+  ds = block_sum(ds, sh);
+  if (threadIdx.x == 0 && part_s) part_s[blockIdx.x] = ds;
+}
+
+inline bool al16(const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+#define MREM_DT(dt, T, ...)            \
+  do {                                 \
+    if ((dt) == 1) { using T = bf16; __VA_ARGS__; } else { using T = float; __VA_ARGS__; } \
+  } while (0)
+
+void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, float eps, long long rows, int cols,
+                          void* out, float* mean, float* rstd, const float* step, int qmax, int8_t* q8, void* qt,
+                          int dt, cudaStream_t st) {
+  if (rows <= 0) return;
+  Scope sc("layernorm_fwd", (double)rows * cols * ((dt == 1 ? 2.0 : 4.0) * (qt ? 3 : 2) + (q8 ? 1 : 0)), 0, st);
+  const int grid = (int)((rows + 3) / 4);
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(y) && al16(out) && al16(qt) &&
+                   (reinterpret_cast<uintptr_t>(q8) % V) == 0;
+    if (v) ln_fwd_kernel<T, V, true><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
+    else ln_fwd_kernel<T, 1, false><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
+  });
+}
+
+void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, const float* mean, const float* rstd,
+                          const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
+                          cudaStream_t st) {
+  if (rows <= 0) return;
+  Scope sc("layernorm_bwd", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (3 + (dout2 ? 1 : 0) + (dsum ? 1 : 0)), 0, st);
+  const int grid = (int)((rows + 3) / 4);
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(dout) && al16(dout2) && al16(y) && al16(dy) && al16(dsum);
+    if (v) ln_bwd_kernel<T, V, true><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
+    else ln_bwd_kernel<T, 1, false><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
+  });
+}
+
+void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
+                       long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st) {
+  Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (y ? 2 : 1), 0, st);
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    if (cols % V == 0 && ld_a % V == 0 && al16(a) && al16(y)) {
+      dim3 grid((cols + 32 * V - 1) / (32 * V), COL_CHUNKS);
+      col_reduce_kernel<T, V><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch);
+    } else {
+      dim3 grid((cols + 31) / 32, COL_CHUNKS);
+      col_reduce_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch);
+    }
+  });
+  col_reduce_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, cols, out0, y ? out1 : nullptr);
+}
+
+void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,
+                        const float* offset, int lo, int hi, void* qt, int dt, cudaStream_t st) {
+  const long long rows = (long long)B * h * S;
+  if (rows <= 0) return;
+  Scope sc("softmax_fwd", (double)rows * S * (4.0 + (dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1)), 0, st);
+  const int grid = (int)((rows + 3) / 4);
+  const bool cached = S % 4 == 0 && S <= 128 * MAXNV && al16(scores) && al16(P) && al16(qt);
+  MREM_DT(dt, T, {
+    if (cached) softmax_fwd_kernel<T, true><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt);
+    else softmax_fwd_kernel<T, false><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt);
+  });
+}
+
+void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long rows, int S, const float* step,
+                        int lo, int hi, int quantized, float* part_s, int dt, cudaStream_t st) {
+  Scope sc("softmax_bwd", (double)rows * S * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
+  const bool cached = S % 4 == 0 && S <= 128 * MAXNV && al16(P) && al16(dphat) && al16(dS);
+  MREM_DT(dt, T, {
+    if (cached) softmax_bwd_kernel<T, true><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s);
+    else softmax_bwd_kernel<T, false><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s);
+  });
+}
+
+}  // namespace mrem
