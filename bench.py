@@ -265,7 +265,7 @@ def main():
             m.recon_loss()
             m.backward()
             m.step(opt)
-        trace = B.mrem_trace_read(m.ctx)
+        trace = B.mrem_trace_read(m.ctx, 128)
         B.mrem_trace_enable(m.ctx, 0)
 
         # ---- end to end: host buffers in, loss out, every step
@@ -297,6 +297,14 @@ def main():
         return
 
     pk = peaks()
+    # products are traced per shape ("gemm_bf16 MxNxK.."); fold them into one row per kernel, keep the shapes
+    shapes = [e for e in trace if e["name"].startswith("gemm_")]
+    folded = {}
+    for e in trace:
+        key = {"gemm_bf16": "gemm_bf16_tcgen05", "gemm_i8": "gemm_i8_tcgen05"}.get(e["name"].split(" ")[0], e["name"])
+        f = folded.setdefault(key, dict(name=key, ms=0.0, work=0.0, launches=0, is_flops=e["is_flops"]))
+        f["ms"] += e["ms"]; f["work"] += e["work"]; f["launches"] += e["launches"]
+    trace = list(folded.values())
     kernels = []
     for e in sorted(trace, key=lambda e: -e["ms"]):
         per_launch_ms = e["ms"] / max(e["launches"], 1)
@@ -325,7 +333,11 @@ def main():
                        "l2": "inputs larger than L2: calibration set, weights and optimizer state exceed 126 MB",
                        "launch": "one CUDA-graph replay per step + 2 gather kernels"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_step * K, "roofline": roofline,
-            "kernels": kernels, "loss_last": loss_last, "device_status": status}
+            "kernels": kernels,
+            "gemm_shapes": [{"shape": e["name"], "launches_per_step": e["launches"] / n_trace,
+                             "us_per_launch": 1e3 * e["ms"] / max(e["launches"], 1),
+                             "tflops": e["work"] / (e["ms"] * 1e-3) / 1e12} for e in sorted(shapes, key=lambda e: -e["ms"])],
+            "loss_last": loss_last, "device_status": status}
     if world == 1 and not args.no_cpu_baseline:
         val, threads, sample, sec = oracle_sample(wl)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,

@@ -140,6 +140,10 @@ int32_t mrem_init_act_steps(mrem_ctx* ctx, const void* d_x, const int32_t* d_val
 /* Eq. 1 on every weight matrix of the student: latent weights + steps -> int8 codes, int32 row
  * sums of the codes, and the dequantized matrices used by the backward products. */
 int32_t mrem_quantize_weights(mrem_ctx* ctx);
+/* Tells the context that the caller wrote the student's weights or weight steps itself (through its own
+ * pointers): the next mrem_quantize_weights then recomputes the codes instead of trusting the ones the
+ * last mrem_step produced. */
+int32_t mrem_invalidate_weight_codes(mrem_ctx* ctx);
 /* Borrowed pointers to the codes [rows, cols] and row sums [rows] of one matrix (valid until destroy). */
 int32_t mrem_get_weight_codes(mrem_ctx* ctx, int32_t layer, int32_t tensor_id, const int8_t** d_codes,
                               const int32_t** d_rowsum);
@@ -159,9 +163,12 @@ int32_t mrem_module_forward(mrem_ctx* ctx, int32_t role, const void* d_x, const 
 int32_t mrem_recon_loss(mrem_ctx* ctx, float* d_loss_total, float* d_loss_per_layer);
 /* Straight-through backward through the student module (gradient local to the module). */
 int32_t mrem_module_backward(mrem_ctx* ctx);
-/* Borrowed pointer to a gradient (float32, same shape as the parameter / step tensor). */
+/* Borrowed pointer to a gradient (float32, same shape as the parameter / step tensor).  Asking for a weight
+ * matrix or a weight step applies the weight quantizers' straight-through masks on the spot. */
 int32_t mrem_get_grad(mrem_ctx* ctx, int32_t layer, int32_t id, const float** d_grad);
-/* AdamW on everything in trainable_mask, steps clamped to >= 1e-8. */
+/* AdamW on everything in trainable_mask, steps clamped to >= 1e-8.  With per-row weight steps the update of
+ * each matrix also re-quantizes it (Eq. 1 with the new weights and steps), so the next
+ * mrem_quantize_weights has nothing left to do. */
 int32_t mrem_step(mrem_ctx* ctx, const mrem_optim* optim);
 
 /* The whole step from HOST buffers: copies h_x_teacher / h_x_student ([batch, seq, hidden] act_dtype;

@@ -15,6 +15,8 @@
 // code in the status word, stops issuing work, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <cstdio>
+
 #include "gemm.h"
 
 namespace mrem {
@@ -616,7 +618,12 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
     attr_set[kind] = true;
   }
   const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
-  Scope sc(kind == 0 ? "gemm_bf16_tcgen05" : "gemm_i8_tcgen05", 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream);
+  Scope sc([&] {
+    char buf[40];
+    snprintf(buf, sizeof(buf), "%s %dx%dx%d%s%s b%d", kind == 0 ? "gemm_bf16" : "gemm_i8", g.M, g.N, g.K,
+             A.mn_contig ? "T" : "N", B.mn_contig ? "N" : "T", g.nb0 * g.nb1);
+    return std::string(buf);
+  }, 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream, 0);
   kern<<<grid, GEMM_THREADS, smem, stream>>>(ma, mb, p);
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }

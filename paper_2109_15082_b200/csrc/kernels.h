@@ -74,11 +74,14 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
                           const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
                           cudaStream_t st);
 
-// Column sums over rows: out0[c] = sum_r a[r,c]; with y/mean/rstd also out1[c] = sum_r a[r,c]*(y[r,c]-mean[r])*rstd[r].
-// Two kernels (per-chunk partials in `scratch`, then a fixed-order sum).  scratch >= 2*COL_CHUNKS*cols floats.
+// Column sums over rows: out0[c] = sum_r a[r,c]; with y/mean/rstd also out1[c] = sum_r a[r,c]*(y[r,c]-mean[r])*rstd[r];
+// with a2 also out2[c] = sum_r a2[r,c].  One kernel: per-chunk partials in `scratch` (>= 3*COL_CHUNKS*cols
+// floats), summed in index order by the last block of each column group.  `counters` (>= cols/32 + 1 ints)
+// must be zero before the first launch; the kernel leaves them zero.
 constexpr int COL_CHUNKS = 64;
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
-                       long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st);
+                       const void* a2, long long ld_a2, long long rows, int cols, float* out0, float* out1,
+                       float* out2, float* scratch, int* counters, int dt, cudaStream_t st);
 
 // Weight STE: dW = dWhat * inside (in place), ds[row] = sum_k dWhat * d what/d s.
 void launch_ste_weight(const float* w, const float* steps, int per_row, int bits, int grid, float* dw, int rows,
@@ -103,6 +106,14 @@ void launch_optim_prepare(OptimScalars* d_out, int* d_t, int host_t, float lr0, 
                           float beta2, float eps, float weight_decay, cudaStream_t st);
 void launch_adamw_table(const AdamEntry* d_table, int n_entries, long long total_elems, const OptimScalars* d_sc,
                         cudaStream_t st);
+
+// Fused per-row update of a weight matrix and its per-row steps: step gradient (or ds_in when the
+// gradients were already masked), AdamW on step and weights, re-quantization (codes, row sums,
+// scale, dequantized row).
+void launch_fused_weight_update(float* w, const float* g, float* m, float* v, float* steps, const float* ds_in,
+                                float* m_s, float* v_s, const OptimScalars* sc, int rows, int cols, int bits, int grid,
+                                int train_w, int train_s, int8_t* codes, int32_t* rowsum, float* scale, void* what,
+                                int dt, cudaStream_t st);
 
 // ---- step-size initialisation
 // Per-row max|w| or mean|w| -> steps (per row, or one value when !per_row: two passes).

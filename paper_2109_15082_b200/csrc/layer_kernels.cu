@@ -3,6 +3,7 @@
 // row for row-wise ops, warp-shuffle reductions, and fixed-order two-stage sums (per-block
 // partials, then one block adds them in index order) so results are reproducible run to run.
 #include "kernels.h"
+#include "optim.cuh"
 #include "vec.cuh"
 
 namespace mrem {
@@ -146,23 +147,18 @@ __global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict
   const int row = blockIdx.x;
   const float s = steps[per_row ? row : 0];
   const float qmax = (float)((1 << (bits - 1)) - 1);
-  const float* wr = w + (long long)row * cols;
-  float* dr = dw + (long long)row * cols;
+  const float4* wr = reinterpret_cast<const float4*>(w + (long long)row * cols);
+  float4* dr = reinterpret_cast<float4*>(dw + (long long)row * cols);
   float ds = 0.f;
-  for (int c = threadIdx.x; c < cols; c += blockDim.x) {
-    const float z = __fdiv_rn(wr[c], s);
-    const float d = dr[c];
+  for (int c = threadIdx.x; c < cols / 4; c += blockDim.x) {     // cols is a multiple of 16
+    const float4 wv = wr[c];
+    float4 d = dr[c];
     bool in;
-    float level;
-    if (grid == 0) {
-      in = z >= -qmax && z <= qmax;
-      level = (float)__float2int_rn(fminf(fmaxf(z, -qmax), qmax));
-    } else {
-      in = z >= -2.f && z < 2.f;
-      level = fminf(fmaxf(floorf(z), -2.f), 1.f) + 0.5f;
-    }
-    ds += d * (level - (in ? z : 0.f));
-    dr[c] = in ? d : 0.f;
+    ds = step_grad_acc(ds, wv.x, d.x, s, qmax, grid, in); d.x = in ? d.x : 0.f;
+    ds = step_grad_acc(ds, wv.y, d.y, s, qmax, grid, in); d.y = in ? d.y : 0.f;
+    ds = step_grad_acc(ds, wv.z, d.z, s, qmax, grid, in); d.z = in ? d.z : 0.f;
+    ds = step_grad_acc(ds, wv.w, d.w, s, qmax, grid, in); d.w = in ? d.w : 0.f;
+    dr[c] = d;
   }
   ds = block_sum(ds, sh);
   if (threadIdx.x == 0) ds_rows[row] = ds;
@@ -209,15 +205,11 @@ __global__ void __launch_bounds__(256) adamw_table_kernel(const AdamEntry* __res
                                                           const OptimScalars* __restrict__ sc) {
   const AdamEntry e = table[blockIdx.y];
   const OptimScalars o = *sc;
-  const float decay = 1.f - o.lr * e.wd * o.weight_decay;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < e.n; i += (long long)gridDim.x * blockDim.x) {
-    const float g = e.g[i];
-    const float m = o.beta1 * e.m[i] + (1.f - o.beta1) * g;
-    const float v = o.beta2 * e.v[i] + (1.f - o.beta2) * g * g;
+    float m = e.m[i], v = e.v[i];
+    e.p[i] = adam_one(e.p[i], e.g[i], m, v, o, e.wd, e.min_value);
     e.m[i] = m;
     e.v[i] = v;
-    const float upd = o.lr * (m / o.bc1) / (sqrtf(v / o.bc2) + o.eps);
-    e.p[i] = fmaxf(e.p[i] * decay - upd, e.min_value);
   }
 }
 

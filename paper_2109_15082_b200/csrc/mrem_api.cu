@@ -68,11 +68,13 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->minmax = (float*)A.take(256);
   c->d_loss_e2e = (float*)A.take(256);
   c->loss_partial = (float*)A.take(sizeof(float) * RED_BLOCKS * L);
-  c->col_scratch = (float*)A.take(sizeof(float) * 2 * COL_CHUNKS * (3 * H > F ? 3 * H : F));
+  c->col_scratch = (float*)A.take(sizeof(float) * 3 * COL_CHUNKS * (3 * H > F ? 3 * H : F));
+  c->col_counters = (int*)A.take(sizeof(int) * ((3 * H > F ? 3 * H : F) / 32 + 2));
   c->rowbias = (float*)A.take(sizeof(float) * (3 * H > F ? 3 * H : F));
   c->reduce_per_layer = N_SITES + 1 + N_WMAT;
   c->reduce_table = (ReduceEntry*)A.take(sizeof(ReduceEntry) * c->reduce_per_layer * L);
   c->adam_table = (AdamEntry*)A.take(sizeof(AdamEntry) * (MREM_N_PARAMS + N_WMAT + N_SITES + 1) * L);
+  c->adam_rest = (AdamEntry*)A.take(sizeof(AdamEntry) * (MREM_N_PARAMS + N_WMAT + N_SITES + 1) * L);
   c->h2d_xt = A.take(M * H * es);
   c->h2d_xs = A.take(M * H * es);
   c->h2d_len = (int32_t*)A.take(sizeof(int32_t) * d.max_batch);
@@ -146,7 +148,7 @@ int build_tables(mrem_ctx* c) {
   const mrem_module_desc& d = c->d;
   const int L = d.n_layers;
   std::vector<ReduceEntry> red;
-  std::vector<AdamEntry> adam;
+  std::vector<AdamEntry> adam, rest;
   for (int l = 0; l < L; ++l) {
     LayerStash& s = c->stash[l];
     LayerGrad& g = c->grad[l];
@@ -166,6 +168,7 @@ int build_tables(mrem_ctx* c) {
       if (!b.student[k]) return fail(c, MREM_ERR_ORDER, "student parameter not bound");
       int r, q; param_shape(d, k, &r, &q);
       adam.push_back({b.student[k], g.p[k], g.m_p[k], g.v_p[k], (long long)r * q, mat ? 1.f : 0.f, -INFINITY});
+      if (!mat) rest.push_back(adam.back());
     }
     if (d.trainable_mask & MREM_TRAIN_W_STEPS)
       for (int k = 0; k < N_WMAT; ++k) {
@@ -176,9 +179,10 @@ int build_tables(mrem_ctx* c) {
       for (int site = 0; site < N_SITES; ++site) {
         if (!b.a_steps[site]) return fail(c, MREM_ERR_ORDER, "activation steps not bound");
         adam.push_back({b.a_steps[site], g.a + site, g.m_a + site, g.v_a + site, 1, 0.f, 1e-8f});
+        rest.push_back(adam.back());
       }
       if ((d.act_asym_sites & 2) && b.a_off[7])
-        adam.push_back({b.a_off[7], g.off + 7, g.m_off + 7, g.v_off + 7, 1, 0.f, -INFINITY});
+        { adam.push_back({b.a_off[7], g.off + 7, g.m_off + 7, g.v_off + 7, 1, 0.f, -INFINITY}); rest.push_back(adam.back()); }
     }
   }
   if (cudaMemcpyAsync(c->reduce_table, red.data(), sizeof(ReduceEntry) * red.size(), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
@@ -186,6 +190,11 @@ int build_tables(mrem_ctx* c) {
   c->adam_entries = (int)adam.size();
   c->adam_elems = 0;
   for (const AdamEntry& e : adam) c->adam_elems += e.n;
+  c->rest_entries = (int)rest.size();
+  c->rest_elems = 0;
+  for (const AdamEntry& e : rest) c->rest_elems += e.n;
+  if (!rest.empty() && cudaMemcpyAsync(c->adam_rest, rest.data(), sizeof(AdamEntry) * rest.size(), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+    return fail(c, MREM_ERR_CUDA, "table upload failed");
   if (cudaMemcpyAsync(c->adam_table, adam.data(), sizeof(AdamEntry) * adam.size(), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
     return fail(c, MREM_ERR_CUDA, "table upload failed");
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "sync failed");
@@ -265,6 +274,7 @@ int32_t mrem_bind_param(mrem_ctx* c, int32_t role, int32_t layer, int32_t id, vo
     return fail(c, MREM_ERR_ARG, "bind_param: role");
   }
   c->tables_dirty = true;
+  c->codes_fresh = false;
   return MREM_OK;
 }
 
@@ -275,6 +285,7 @@ int32_t mrem_bind_steps(mrem_ctx* c, int32_t layer, int32_t q, float* steps, flo
   if (q < N_WMAT) c->bind[layer].w_steps[q] = steps;
   else { c->bind[layer].a_steps[q - N_WMAT] = steps; c->bind[layer].a_off[q - N_WMAT] = offset; }
   c->tables_dirty = true;
+  c->codes_fresh = false;
   return MREM_OK;
 }
 
@@ -292,6 +303,23 @@ int32_t mrem_get_grad(mrem_ctx* c, int32_t layer, int32_t id, const float** g) {
   if (!c || !g) return MREM_ERR_ARG;
   if (layer < 0 || layer >= c->d.n_layers) return fail(c, MREM_ERR_ARG, "get_grad: bad layer");
   if (!c->have_grads) return fail(c, MREM_ERR_ORDER, "get_grad: no backward has run");
+  const bool weight_id = (id >= 0 && id < MREM_N_PARAMS && kParamIsMatrix[id]) || (id >= MREM_GRAD_STEP && id < MREM_GRAD_STEP + N_WMAT);
+  if (weight_id && !c->w_ste_done) {
+    // The backward leaves the matrices' gradients unmasked for the fused update; a caller who wants
+    // to read them gets the straight-through masks and the step gradients applied now.
+    TracerGuard tg(nullptr);
+    for (int l = 0; l < c->d.n_layers; ++l)
+      for (int k = 0; k < N_WMAT; ++k) {
+        const WeightBuf& w = c->wq[l][k];
+        launch_ste_weight(c->bind[l].student[kMatParam[k]], c->bind[l].w_steps[k], c->d.w_step_per_row, c->d.w_bits,
+                          c->d.w_grid, c->grad[l].p[kMatParam[k]], w.rows, w.cols,
+                          c->d.w_step_per_row ? c->grad[l].ws[k] : w.ds_rows, c->stream);
+        if (!c->d.w_step_per_row)
+          launch_reduce_table(c->reduce_table + (size_t)l * c->reduce_per_layer + N_SITES + 1 + k, 1, c->stream);
+      }
+    if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "get_grad: launch failed");
+    c->w_ste_done = true;
+  }
   LayerGrad& G = c->grad[layer];
   if (id >= 0 && id < MREM_N_PARAMS) *g = G.p[id];
   else if (id >= MREM_GRAD_STEP && id < MREM_GRAD_STEP + N_WMAT) *g = G.ws[id - MREM_GRAD_STEP];
@@ -319,6 +347,7 @@ int32_t mrem_init_student_from_teacher(mrem_ctx* c) {
   if (cudaMemsetAsync(base + c->state_off, 0, c->state_bytes, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "memset failed");
   if (cudaMemsetAsync(c->t_counter, 0, 4, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "memset failed");
   c->weights_quantized = false;
+  c->codes_fresh = false;
   return MREM_OK;
 }
 
@@ -335,7 +364,15 @@ int32_t mrem_init_weight_steps(mrem_ctx* c, int32_t rule) {
       launch_init_weight_steps(b.student[kMatParam[k]], w.rows, w.cols, c->d.w_step_per_row, rule, qmax, b.w_steps[k], w.ds_rows, c->stream);
     }
   c->weights_quantized = false;
+  c->codes_fresh = false;
   return cudaGetLastError() == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "launch failed");
+}
+
+int32_t mrem_invalidate_weight_codes(mrem_ctx* c) {
+  if (!c) return MREM_ERR_ARG;
+  c->codes_fresh = false;
+  c->weights_quantized = false;
+  return MREM_OK;
 }
 
 int32_t mrem_poll_status(mrem_ctx* c, int32_t* h_status) {

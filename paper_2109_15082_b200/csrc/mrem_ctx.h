@@ -89,6 +89,7 @@ struct mrem_ctx {
   void *d_y2, *d_ghat, *d_u, *d_ahat, *d_a, *d_y1, *d_ctxhat, *d_ctx, *d_phat, *d_s, *d_qkvhat, *d_qkv, *d_xhat,
       *d_sum, *carry[2];
   float* col_scratch;
+  int* col_counters;
   float* rowbias;
   float* loss_partial;
   float* minmax;
@@ -96,7 +97,10 @@ struct mrem_ctx {
   int* t_counter;
   mrem::OptimScalars* optim_sc;
   mrem::ReduceEntry* reduce_table;   int reduce_per_layer = 0;
-  mrem::AdamEntry* adam_table;       int adam_entries = 0;  long long adam_elems = 0;
+  mrem::AdamEntry* adam_table;       int adam_entries = 0;  long long adam_elems = 0;   // every trainable tensor
+  mrem::AdamEntry* adam_rest;        int rest_entries = 0;  long long rest_elems = 0;   // all but matrices and their steps
+  bool w_ste_done = false;           // the weight gradients have been masked and the step gradients reduced
+  bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;
   void *h2d_xt, *h2d_xs; int32_t* h2d_len; float* d_loss_e2e;   // staging of mrem_recon_step_host
   void *e2e_t_out, *e2e_s_out;                                  // its layer outputs [L, M, H]

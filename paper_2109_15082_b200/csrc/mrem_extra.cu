@@ -41,6 +41,7 @@ int32_t mrem_init_act_steps(mrem_ctx* c, const void* x, const int32_t* len, int3
   }
   const int rc = float_forward(c, x, len, batch, seq, c->e2e_s_out, true, true);
   c->weights_quantized = false;      // the w_hat buffers were used as scratch
+  c->codes_fresh = false;
   return rc;
 }
 
@@ -77,6 +78,8 @@ int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, flo
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
   if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
+  // quantize once outside the graph: inside it the fused update keeps the codes current
+  { const int qrc = mrem_quantize_weights(c); if (qrc != MREM_OK) return qrc; }
   const bool was_tracing = c->trace_on;
   c->trace_on = false;              // event pairs are not recorded inside a captured graph
   struct Restore { mrem_ctx* c; bool v; ~Restore() { c->trace_on = v; } } restore{c, was_tracing};

@@ -232,9 +232,9 @@ int student_backward(mrem_ctx* c) {
 
     // second LayerNorm: total gradient at the layer output = loss term + what the next layer sent back
     launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, carry ? c->d_sum : nullptr, c->dt, st);
-    launch_col_reduce(carry ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G], c->col_scratch, c->dt, st);
-    // FFN2:  y2 = G_hat W2_hat^T + b2 + a
-    launch_col_reduce(c->d_y2, H, nullptr, nullptr, nullptr, M, H, g.p[MREM_B2], nullptr, c->col_scratch, c->dt, st);
+    // LayerNorm parameter gradients and the bias gradient of FFN2 (y2 = G_hat W2_hat^T + b2 + a) in one pass
+    launch_col_reduce(carry ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, c->d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
+                      g.p[MREM_B2], c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
     {
       Epi e(g.p[MREM_W2], OUT_F32, F);
@@ -245,16 +245,16 @@ int student_backward(mrem_ctx* c) {
     launch_gelu_bwd(s.u, c->d_ghat, c->d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
                     part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
     // FFN1:  u = A_hat W1_hat^T + b1
-    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, M, F, g.p[MREM_B1], nullptr, c->col_scratch, c->dt, st);
+    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
     r.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
                    part + S_A * RED_BLOCKS, nullptr, c->dt, st);
     // first LayerNorm
     launch_layernorm_bwd(c->d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, c->d_y1, nullptr, c->dt, st);
-    launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], c->col_scratch, c->dt, st);
-    // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x
-    launch_col_reduce(c->d_y1, H, nullptr, nullptr, nullptr, M, H, g.p[MREM_BO], nullptr, c->col_scratch, c->dt, st);
+    // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x  (its bias gradient rides along)
+    launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
+                      c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
     r.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
@@ -273,7 +273,7 @@ int student_backward(mrem_ctx* c) {
       launch_ste_act(r.at(s.qkv, seg * H), 3 * H, r.at(c->d_qkvhat, seg * H), 3 * H, nullptr, 0, r.at(c->d_qkv, seg * H), 3 * H, M, H,
                      b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, part + (S_Q + seg) * RED_BLOCKS, nullptr, c->dt, st);
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
-    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, M, 3 * H, g.p[MREM_BQKV], nullptr, c->col_scratch, c->dt, st);
+    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
     r.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
     void* next_carry = c->carry[l & 1];
@@ -281,9 +281,8 @@ int student_backward(mrem_ctx* c) {
                    part + S_X * RED_BLOCKS, nullptr, c->dt, st);
     carry = next_carry;
     // weight quantizers: mask the latent-weight gradients, reduce the step gradients
-    for (int k = 0; k < N_WMAT; ++k)
-      launch_ste_weight(b.student[kMatParam[k]], b.w_steps[k], d.w_step_per_row, d.w_bits, d.w_grid, g.p[kMatParam[k]],
-                        w[k].rows, w[k].cols, d.w_step_per_row ? g.ws[k] : w[k].ds_rows, st);
+    // (the weight quantizers' masks and step gradients are applied inside the fused update of mrem_step,
+    //  or on demand by mrem_get_grad)
     launch_reduce_table(c->reduce_table + (size_t)l * c->reduce_per_layer, c->reduce_per_layer, st);
   }
   if (r.rc != MREM_OK) return r.rc;
@@ -297,6 +296,7 @@ extern "C" {
 int32_t mrem_quantize_weights(mrem_ctx* c) {
   if (!c) return MREM_ERR_ARG;
   TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
+  if (c->codes_fresh) { c->weights_quantized = true; return MREM_OK; }   // the last update already re-quantized
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) {
       const LayerBind& b = c->bind[l];
@@ -307,6 +307,7 @@ int32_t mrem_quantize_weights(mrem_ctx* c) {
     }
   if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "quantize_weights: launch failed");
   c->weights_quantized = true;
+  c->codes_fresh = true;
   return MREM_OK;
 }
 
@@ -366,6 +367,7 @@ int32_t mrem_module_backward(mrem_ctx* c) {
   const int rc = student_backward(c);
   if (rc != MREM_OK) return rc;
   c->have_grads = true;
+  c->w_ste_done = false;
   return MREM_OK;
 }
 
@@ -376,10 +378,36 @@ int32_t mrem_step(mrem_ctx* c, const mrem_optim* o) {
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
                        o->weight_decay, c->stream);
-  launch_adamw_table(c->adam_table, c->adam_entries, c->adam_elems, c->optim_sc, c->stream);
+  const mrem_module_desc& d = c->d;
+  if (d.w_step_per_row) {
+    // every tensor but the matrices and their steps, then one fused pass per matrix
+    launch_adamw_table(c->adam_rest, c->rest_entries, c->rest_elems, c->optim_sc, c->stream);
+    const int train_w = (d.trainable_mask & MREM_TRAIN_WEIGHTS) != 0, train_s = (d.trainable_mask & MREM_TRAIN_W_STEPS) != 0;
+    for (int l = 0; l < d.n_layers; ++l)
+      for (int k = 0; k < N_WMAT; ++k) {
+        const int pid = kMatParam[k];
+        WeightBuf& w = c->wq[l][k];
+        LayerGrad& g = c->grad[l];
+        launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
+                                   c->w_ste_done ? g.ws[k] : nullptr, g.m_ws[k], g.v_ws[k], c->optim_sc, w.rows, w.cols,
+                                   d.w_bits, d.w_grid, train_w, train_s, w.codes, w.rowsum, w.scale, w.what, c->dt, c->stream);
+      }
+  } else {
+    if (!c->w_ste_done) {
+      for (int l = 0; l < d.n_layers; ++l)
+        for (int k = 0; k < N_WMAT; ++k) {
+          WeightBuf& w = c->wq[l][k];
+          launch_ste_weight(c->bind[l].student[kMatParam[k]], c->bind[l].w_steps[k], 0, d.w_bits, d.w_grid,
+                            c->grad[l].p[kMatParam[k]], w.rows, w.cols, w.ds_rows, c->stream);
+          launch_reduce_table(c->reduce_table + (size_t)l * c->reduce_per_layer + N_SITES + 1 + k, 1, c->stream);
+        }
+    }
+    launch_adamw_table(c->adam_table, c->adam_entries, c->adam_elems, c->optim_sc, c->stream);
+  }
   if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "step: launch failed");
   c->have_grads = false; c->have_loss = false; c->have_student = false; c->have_teacher = false;
-  c->weights_quantized = false;
+  c->codes_fresh = d.w_step_per_row != 0;
+  c->weights_quantized = c->codes_fresh;
   return MREM_OK;
 }
 

@@ -194,20 +194,27 @@ __global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout,
 }
 
 // ------------------------------------------------------------------ column sums over rows
-// Block (32 x 8): 32 * V columns, a chunk of rows; fixed-order tree over the 8 row groups.
+// out0[c] = sum_r a[r,c];  out1[c] = sum_r a[r,c] * (y[r,c] - mean[r]) * rstd[r] (when y);  out2[c] = sum_r a2[r,c]
+// (when a2).  Block (32 x 8) owns 32*V columns of one chunk of rows and adds its 8 row groups in a
+// fixed order; the last block to finish a column group (ticket counter) adds the chunks' partials in
+// index order, so the result does not depend on scheduling.
 template <typename T, int V>
 __global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a, long long ld_a,
                                                          const T* __restrict__ y, const float* __restrict__ mean,
-                                                         const float* __restrict__ rstd, long long rows, int cols,
-                                                         float* __restrict__ scratch) {
-  __shared__ float sh0[8][32 * V + 1], sh1[8][32 * V + 1];
+                                                         const float* __restrict__ rstd, const T* __restrict__ a2,
+                                                         long long ld_a2, long long rows, int cols,
+                                                         float* __restrict__ out0, float* __restrict__ out1,
+                                                         float* __restrict__ out2, float* __restrict__ scratch,
+                                                         int* __restrict__ counters) {
+  __shared__ float sh[3][8][32 * V + 1];
+  __shared__ int is_last;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int c = (blockIdx.x * 32 + tx) * V;
   const long long per = (rows + COL_CHUNKS - 1) / COL_CHUNKS;
   const long long r0 = blockIdx.y * per, r1 = r0 + per < rows ? r0 + per : rows;
-  float a0[V], a1[V];
+  float a0[V], a1[V], a2s[V];
 #pragma unroll
-  for (int j = 0; j < V; ++j) a0[j] = a1[j] = 0.f;
+  for (int j = 0; j < V; ++j) a0[j] = a1[j] = a2s[j] = 0.f;
   if (c < cols) {
     for (long long r = r0 + ty; r < r1; r += 8) {
       float v[V];
@@ -221,32 +228,48 @@ __global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a
 #pragma unroll
         for (int j = 0; j < V; ++j) a1[j] += v[j] * (w[j] - mu) * rs;
       }
+      if (a2) {
+        float w[V];
+        load_vec<T, V>(a2 + r * ld_a2 + c, w);
+#pragma unroll
+        for (int j = 0; j < V; ++j) a2s[j] += w[j];
+      }
     }
   }
 #pragma unroll
-  for (int j = 0; j < V; ++j) { sh0[ty][tx * V + j] = a0[j]; sh1[ty][tx * V + j] = a1[j]; }
+  for (int j = 0; j < V; ++j) { sh[0][ty][tx * V + j] = a0[j]; sh[1][ty][tx * V + j] = a1[j]; sh[2][ty][tx * V + j] = a2s[j]; }
   __syncthreads();
+  const long long plane = (long long)COL_CHUNKS * cols;
   for (int i = threadIdx.x; i < 32 * V; i += 256) {
     const int cc = blockIdx.x * 32 * V + i;
     if (cc >= cols) continue;
-    float t0 = 0.f, t1 = 0.f;
+    float t0 = 0.f, t1 = 0.f, t2 = 0.f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { t0 += sh0[k][i]; t1 += sh1[k][i]; }
+    for (int k = 0; k < 8; ++k) { t0 += sh[0][k][i]; t1 += sh[1][k][i]; t2 += sh[2][k][i]; }
     scratch[(long long)blockIdx.y * cols + cc] = t0;
-    if (y) scratch[((long long)COL_CHUNKS + blockIdx.y) * cols + cc] = t1;
+    if (y) scratch[plane + (long long)blockIdx.y * cols + cc] = t1;
+    if (a2) scratch[2 * plane + (long long)blockIdx.y * cols + cc] = t2;
   }
-}
-__global__ void col_reduce_final_kernel(const float* __restrict__ scratch, int cols, float* __restrict__ out0,
-                                        float* __restrict__ out1) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
-  float t0 = 0.f, t1 = 0.f;
-  for (int k = 0; k < COL_CHUNKS; ++k) {
-    t0 += scratch[(long long)k * cols + c];
-    if (out1) t1 += scratch[((long long)COL_CHUNKS + k) * cols + c];
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = atomicAdd(&counters[blockIdx.x], 1) == (int)gridDim.y - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int i = threadIdx.x; i < 32 * V; i += 256) {
+    const int cc = blockIdx.x * 32 * V + i;
+    if (cc >= cols) continue;
+    float t0 = 0.f, t1 = 0.f, t2 = 0.f;
+    for (int k = 0; k < COL_CHUNKS; ++k) {
+      t0 += scratch[(long long)k * cols + cc];
+      if (y) t1 += scratch[plane + (long long)k * cols + cc];
+      if (a2) t2 += scratch[2 * plane + (long long)k * cols + cc];
+    }
+    out0[cc] = t0;
+    if (y) out1[cc] = t1;
+    if (a2) out2[cc] = t2;
   }
-  out0[c] = t0;
-  if (out1) out1[c] = t1;
+  if (threadIdx.x == 0) counters[blockIdx.x] = 0;         // ready for the next launch on this stream
 }
 
 // ------------------------------------------------------------------ softmax forward
@@ -435,19 +458,19 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
 }
 
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
-                       long long rows, int cols, float* out0, float* out1, float* scratch, int dt, cudaStream_t st) {
-  Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (y ? 2 : 1), 0, st);
+                       const void* a2, long long ld_a2, long long rows, int cols, float* out0, float* out1,
+                       float* out2, float* scratch, int* counters, int dt, cudaStream_t st) {
+  Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (1 + (y ? 1 : 0) + (a2 ? 1 : 0)), 0, st);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
-    if (cols % V == 0 && ld_a % V == 0 && al16(a) && al16(y)) {
+    if (cols % V == 0 && ld_a % V == 0 && ld_a2 % V == 0 && al16(a) && al16(y) && al16(a2)) {
       dim3 grid((cols + 32 * V - 1) / (32 * V), COL_CHUNKS);
-      col_reduce_kernel<T, V><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch);
+      col_reduce_kernel<T, V><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
     } else {
       dim3 grid((cols + 31) / 32, COL_CHUNKS);
-      col_reduce_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, rows, cols, scratch);
+      col_reduce_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
     }
   });
-  col_reduce_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, cols, out0, y ? out1 : nullptr);
 }
 
 void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,

@@ -16,7 +16,7 @@ struct TraceTotals { double ms = 0, work = 0; long long launches = 0; int is_flo
 class Tracer {
  public:
   ~Tracer() { for (cudaEvent_t e : pool_) cudaEventDestroy(e); }
-  void begin(const char* name, double work, int is_flops, cudaStream_t st) {
+  void begin(const std::string& name, double work, int is_flops, cudaStream_t st) {
     Rec r{name, work, is_flops, next(), next()};
     cudaEventRecord(r.a, st);
     open_ = r;
@@ -40,7 +40,7 @@ class Tracer {
   const std::map<std::string, TraceTotals>& totals() const { return totals_; }
 
  private:
-  struct Rec { const char* name; double work; int is_flops; cudaEvent_t a, b; };
+  struct Rec { std::string name; double work; int is_flops; cudaEvent_t a, b; };
   cudaEvent_t next() {
     if (used_ == pool_.size()) {
       cudaEvent_t e;
@@ -63,6 +63,11 @@ struct Scope {
   bool on;
   Scope(const char* name, double work, int is_flops, cudaStream_t s) : st(s), on(g_tracer != nullptr) {
     if (on) g_tracer->begin(name, work, is_flops, st);
+  }
+  // name built only when tracing is on
+  template <class F>
+  Scope(F&& make_name, double work, int is_flops, cudaStream_t s, int) : st(s), on(g_tracer != nullptr) {
+    if (on) g_tracer->begin(make_name(), work, is_flops, st);
   }
   ~Scope() { if (on) g_tracer->end(st); }
 };

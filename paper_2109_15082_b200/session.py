@@ -87,6 +87,7 @@ class ReconModule:
         for l, p in enumerate(params):
             for pid, name in enumerate(B.PARAM_NAMES):
                 self.student[l][pid].copy_(torch.from_numpy(np.ascontiguousarray(p[name], dtype=np.float32)))
+        B.mrem_invalidate_weight_codes(self.ctx)
 
     def student_numpy(self):
         return [{name: self.student[l][pid].float().cpu().numpy() for pid, name in enumerate(B.PARAM_NAMES)}
@@ -104,6 +105,7 @@ class ReconModule:
                 self.w_steps[l][k].copy_(torch.from_numpy(v))
         self.a_steps[:, :, 0].copy_(torch.from_numpy(np.asarray(a_steps, np.float32)))
         self.a_off[:, :, 0].copy_(torch.from_numpy(np.asarray(a_off, np.float32)))
+        B.mrem_invalidate_weight_codes(self.ctx)
 
     def get_steps(self):
         w = [{B.PARAM_NAMES[pid]: self.w_steps[l][k].cpu().numpy() for k, pid in enumerate(MATRICES)}
