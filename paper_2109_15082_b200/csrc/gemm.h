@@ -1,5 +1,7 @@
 // Internal interface of the two GEMM back ends.
 #pragma once
+#include <cuda.h>
+
 #include "mrem_common.cuh"
 #include "trace.h"
 
@@ -11,6 +13,11 @@ enum GemmRc : int { GEMM_OK = 0, GEMM_ERR_ARG = -1, GEMM_ERR_ALIGN = -2, GEMM_ER
 // block_n 0 picks the tile width.  Operands need 16-byte aligned bases and strides.
 int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
             const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream);
+
+// 4-D TMA tensor map (128-byte swizzle) of an operand: (contiguous index, strided index, batch0, batch1).
+// K-major operands get boxes of block_k x tile_mn elements, MN-major ones 64 x block_k.
+int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,
+                     int tile_mn, int block_k);
 
 // Plain fp32 SIMT path, used when activations are stored in float32 (small correctness
 // configurations); same operand and epilogue conventions, no alignment requirements.

@@ -18,6 +18,7 @@
 #include <cstdio>
 
 #include "gemm.h"
+#include "tc_ptx.cuh"
 
 namespace mrem {
 
@@ -32,7 +33,6 @@ constexpr int EPI_WARPS = 8;
 constexpr int STAGING_WORDS = 32 * 33;               // per epilogue warp: 32 rows x 32 words, padded
 constexpr int STAGING_BYTES = EPI_WARPS * STAGING_WORDS * 4;
 constexpr int TMEM_COLS = 512;
-constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait
 
 struct TcParams {
   int M, N, K, nb0, nb1;
@@ -43,99 +43,6 @@ struct TcParams {
   Epilogue epi;
   int* status;
 };
-
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: false when the phase did not complete within WAIT_NS.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > WAIT_NS) return false;
-  }
-}
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            int c2, int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-      : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-template <int KIND>
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  if constexpr (KIND == 0) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  }
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
-  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)(lbo >> 4) << 16;
-  d |= (uint64_t)(sbo >> 4) << 32;
-  d |= 1ull << 46;   // descriptor version of this architecture
-  d |= 2ull << 61;   // 128-byte swizzle
-  return d;
-}
 
 __device__ __forceinline__ void fail(const TcParams& p, int code, volatile int* abort_flag) {
   atomicCAS(p.status, 0, code);
@@ -520,8 +427,10 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+}  // namespace
+
 // Tensor map of one operand: 4-D (contiguous index, strided index, batch0, batch1).
-int make_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,
+int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,
              int tile_mn, int block_k) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return GEMM_ERR_CUDA;
@@ -549,6 +458,8 @@ int make_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_ext
                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? GEMM_OK : GEMM_ERR_CUDA;
 }
+
+namespace {
 
 int pick_block_n(int M, int N, int batches, int sm_count) {
   const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
@@ -604,9 +515,9 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   p.idesc = idesc;
 
   CUtensorMap ma, mb;
-  int rc = make_map(&ma, A, es, g.M, g.K, g.nb0, g.nb1, BLOCK_M, p.block_k);
+  int rc = make_operand_map(&ma, A, es, g.M, g.K, g.nb0, g.nb1, BLOCK_M, p.block_k);
   if (rc != GEMM_OK) return rc;
-  rc = make_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k);
+  rc = make_operand_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k);
   if (rc != GEMM_OK) return rc;
 
   const int smem = p.num_stages * p.stage_bytes + 1024 + STAGING_BYTES;

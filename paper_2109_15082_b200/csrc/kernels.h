@@ -47,6 +47,15 @@ void launch_gelu_quant(const void* u, long long n, const float* step, const floa
 void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,
                         const float* offset, int lo, int hi, void* qt, int dt, cudaStream_t st);
 
+// Fused attention forward on the tensor cores (bf16 storage, head size 64, seq <= 384, seq % 8 == 0):
+// scores, masked softmax, quantizer of the probabilities, context product and (student) the context's
+// codes in one kernel.  Returns a GemmRc.  Null p_step / c_step: no quantizer.
+bool attention_fwd_supported(int S, int head_dim, int dt);
+int launch_attention_fwd(const void* qkv, int B, int S, int h, int H, const int* valid_len, float alpha_const,
+                         const float* a_p0, const float* a_p1, const float* c_p0, const float* c_p1,
+                         const float* p_step, int p_lo, int p_hi, void* P, void* P_qt, void* ctx, const float* c_step,
+                         int c_qmax, int8_t* ctx_q8, void* ctx_qt, int* status, cudaStream_t st);
+
 // ---- loss (Eq. 3)
 // partial[l][block] = sum (f_hat - f)^2 over the block's share; dF = 2 c (f_hat - f).
 void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per_layer, float c, void* dF,

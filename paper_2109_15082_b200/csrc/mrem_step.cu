@@ -124,14 +124,20 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
     if (init_steps) init_site(c, b, S_X, cur, H, M, H);
     r.gemm(view(cur, H), view(b.teacher[MREM_WQKV], H), (int)M, 3 * H, H, 1, 1,
            Epi(c->t_qkv, ok, 3 * H).colbias((float*)b.teacher[MREM_BQKV]).e);
-    r.gemm(view(c->t_qkv, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(c->t_qkv, H), 3 * H, 0, hd, (long long)S * 3 * H),
-           S, S, hd, h, B, Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd)).e);
     if (init_steps)
       for (int seg = 0; seg < 3; ++seg) init_site(c, b, S_Q + seg, r.at(c->t_qkv, seg * H), 3 * H, M, H);
-    launch_softmax_fwd(c->scores, len, B, h, S, c->t_P, nullptr, nullptr, 0, 0, nullptr, c->dt, c->stream);
+    if (attention_fwd_supported(S, hd, c->dt)) {
+      r.note(launch_attention_fwd(c->t_qkv, B, S, h, H, len, 1.f / sqrtf((float)hd), nullptr, nullptr, nullptr, nullptr,
+                                  nullptr, 0, 0, c->t_P, nullptr, c->t_ctx, nullptr, 0, nullptr, nullptr, c->status, c->stream),
+             "attention launch failed");
+    } else {
+      r.gemm(view(c->t_qkv, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(c->t_qkv, H), 3 * H, 0, hd, (long long)S * 3 * H),
+             S, S, hd, h, B, Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd)).e);
+      launch_softmax_fwd(c->scores, len, B, h, S, c->t_P, nullptr, nullptr, 0, 0, nullptr, c->dt, c->stream);
+      r.gemm(view(c->t_P, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(c->t_qkv, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
+             S, hd, S, h, B, Epi(c->t_ctx, ok, H, hd, (long long)S * H).e);
+    }
     if (init_steps) init_site(c, b, S_P, c->t_P, S, (long long)B * h * S, S);
-    r.gemm(view(c->t_P, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(c->t_qkv, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
-           S, hd, S, h, B, Epi(c->t_ctx, ok, H, hd, (long long)S * H).e);
     if (init_steps) init_site(c, b, S_C, c->t_ctx, H, M, H);
     r.gemm(view(c->t_ctx, H), view(b.teacher[MREM_WO], H), (int)M, H, H, 1, 1,
            Epi(c->t_y1, ok, H).colbias((float*)b.teacher[MREM_BO]).residual(cur).e);
@@ -180,13 +186,20 @@ int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S
     for (int seg = 0; seg < 3; ++seg)
       launch_quantize_act(r.at(s.qkv, seg * H), c->dt, M, H, 3 * H, b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, nullptr, 0,
                           r.at(s.qkv_qt, seg * H), 3 * H, c->stream);
-    r.gemm(view(s.qkv_qt, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(s.qkv_qt, H), 3 * H, 0, hd, (long long)S * 3 * H),
-           S, S, hd, h, B,
-           Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd), b.a_steps[S_Q], b.a_steps[S_K]).e);
-    launch_softmax_fwd(c->scores, len, B, h, S, s.P, b.a_steps[S_P], nullptr, rp.lo, rp.hi, s.P_qt, c->dt, c->stream);
-    r.gemm(view(s.P_qt, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(s.qkv_qt, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
-           S, hd, S, h, B, Epi(s.ctx, ok, H, hd, (long long)S * H).alpha(1.f, b.a_steps[S_P], b.a_steps[S_V]).e);
-    launch_quantize_act(s.ctx, c->dt, M, H, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi, s.ctx_q8, H, s.ctx_qt, H, c->stream);
+    if (attention_fwd_supported(S, hd, c->dt)) {
+      r.note(launch_attention_fwd(s.qkv_qt, B, S, h, H, len, 1.f / sqrtf((float)hd), b.a_steps[S_Q], b.a_steps[S_K],
+                                  b.a_steps[S_P], b.a_steps[S_V], b.a_steps[S_P], rp.lo, rp.hi, s.P, s.P_qt, s.ctx,
+                                  b.a_steps[S_C], rx.hi, s.ctx_q8, s.ctx_qt, c->status, c->stream),
+             "attention launch failed");
+    } else {
+      r.gemm(view(s.qkv_qt, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(s.qkv_qt, H), 3 * H, 0, hd, (long long)S * 3 * H),
+             S, S, hd, h, B,
+             Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd), b.a_steps[S_Q], b.a_steps[S_K]).e);
+      launch_softmax_fwd(c->scores, len, B, h, S, s.P, b.a_steps[S_P], nullptr, rp.lo, rp.hi, s.P_qt, c->dt, c->stream);
+      r.gemm(view(s.P_qt, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(s.qkv_qt, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
+             S, hd, S, h, B, Epi(s.ctx, ok, H, hd, (long long)S * H).alpha(1.f, b.a_steps[S_P], b.a_steps[S_V]).e);
+      launch_quantize_act(s.ctx, c->dt, M, H, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi, s.ctx_q8, H, s.ctx_qt, H, c->stream);
+    }
     r.gemm_i8(s.ctx_q8, 0, w[W_O].codes, (int)M, H, H,
               Epi(s.y1, ok, H).alpha(1.f, b.a_steps[S_C]).colscale(w[W_O].scale).colbias(b.student[MREM_BO]).residual(cur).e);
     launch_layernorm_fwd(s.y1, b.student[MREM_LN1_G], b.student[MREM_LN1_B], d.ln_eps, M, H, s.a, s.mean1, s.rstd1,
