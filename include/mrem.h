@@ -233,6 +233,37 @@ int32_t mrem_gemm(int32_t dtype, const void* d_a, int32_t a_mn, int64_t lda, int
                   float alpha, float* d_out, int64_t ldc, int64_t c_batch_stride, int32_t block_n, int32_t* d_status,
                   void* cuda_stream);
 
+/* ---- for callers that cannot allocate device memory -------------------------------------- */
+
+/* (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * The loss of Eq. 3 and its gradient WITHOUT a context and without any allocation: meant for callers
+ * that have the two sets of layer outputs in hand but cannot call cudaMalloc or set up a workspace,
+ * for example a plug-in inside a process whose device memory is handed out entirely by the host
+ * application, a hook that runs while the application's allocator lock is held, or a latency-critical
+ * loop where the device-wide synchronisation of cudaMalloc is not acceptable.  The scratch of the
+ * two-stage reduction (one partial sum per layer and block) is a fixed array inside the library:
+ * MREM_NOALLOC_MAX_LAYERS * 1184 floats (about 150 KB) that every GPU holds from the moment the library
+ * is loaded on it until the process exits.
+ *
+ *   d_f_student, d_f_teacher  [n_layers, n_per_layer] of dtype (MREM_F32 / MREM_BF16), device, 16-byte aligned
+ *   loss_mean                 1: each layer's squared error divided by n_per_layer; 0: plain sum
+ *   d_grad                    [n_layers, n_per_layer] dtype, written: d loss / d f_student
+ *   d_loss_total              float32 [1], written;  d_loss_per_layer: float32 [n_layers] or NULL
+ *
+ * Returns MREM_ERR_SHAPE when n_layers > MREM_NOALLOC_MAX_LAYERS (the built-in scratch is that large and
+ * no larger), MREM_ERR_ARG for null pointers, a bad dtype or non-positive sizes, MREM_ERR_CUDA when the
+ * device cannot be queried.  The first call on each device looks up the device address of the built-in
+ * array (a one-off host-side query, made with that device current); make that first call before entering
+ * any stream capture.  All calls on a device share the one array: calls that may overlap on the GPU (two
+ * streams, two threads) race on it and must be serialised by the caller.  Nothing in the array has to
+ * be cleared between calls: each call rewrites every slot it later reads.  The call never allocates or
+ * frees memory, on the host side of CUDA or otherwise. */
+#define MREM_NOALLOC_MAX_LAYERS 32
+int32_t mrem_recon_loss_noalloc(const void* d_f_student, const void* d_f_teacher, int32_t dtype, int32_t n_layers,
+                                int64_t n_per_layer, int32_t loss_mean, void* d_grad, float* d_loss_total,
+                                float* d_loss_per_layer, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

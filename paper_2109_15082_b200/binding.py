@@ -31,7 +31,7 @@ EXPORTS = (
     "mrem_step", "mrem_recon_step_host", "mrem_poll_status", "mrem_state_bytes", "mrem_export_state",
     "mrem_import_state", "mrem_graph_capture_step", "mrem_graph_launch", "mrem_gather_rows", "mrem_quantize_act",
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
-    "mrem_trace_read", "mrem_invalidate_weight_codes",
+    "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc",
 )
 
 
@@ -263,3 +263,15 @@ def mrem_gemm(dtype, a, a_mn, lda, a_bs, b, b_mn, ldb, b_bs, M, N, K, batches, a
     _check(lib().mrem_gemm(dtype, _p(a), a_mn, C.c_int64(lda), C.c_int64(a_bs), _p(b), b_mn, C.c_int64(ldb),
                            C.c_int64(b_bs), M, N, K, batches, C.c_float(alpha), _p(out), C.c_int64(ldc),
                            C.c_int64(c_bs), block_n, _p(status), _p(stream)), "mrem_gemm")
+
+
+NOALLOC_MAX_LAYERS = 32
+
+
+def mrem_recon_loss_noalloc(f_student, f_teacher, dtype, n_layers, n_per_layer, loss_mean, grad, loss_total,
+                            loss_per_layer, stream):
+    """Loss of Eq. 3 and its gradient for callers that cannot allocate device memory: no context, no
+    workspace; the reduction scratch is a fixed array inside the library (see include/mrem.h)."""
+    _check(lib().mrem_recon_loss_noalloc(_p(f_student), _p(f_teacher), dtype, n_layers, C.c_int64(n_per_layer),
+                                         int(loss_mean), _p(grad), _p(loss_total), _p(loss_per_layer), _p(stream)),
+           "mrem_recon_loss_noalloc")
