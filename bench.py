@@ -150,7 +150,7 @@ def build_problem(wl, rank, torch, calib_n):
     from paper_2109_15082_b200.session import ReconModule
     m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, wl.a_bits, wl.w_grid,
                     True, 3, wl.act_dtype)
-    m.load_teacher(synth.teacher_params(wl, seed=rank))
+    m.load_teacher(synth.teacher_params(wl, seed=rank))          # rank = replica seed: independent problems
     m.init_student_from_teacher()
     m.init_weight_steps(wl.w_step_rule)
     calib = torch.empty(calib_n, wl.seq, wl.hidden, dtype=m.tdtype, device=m.device)
@@ -185,9 +185,8 @@ def main():
     import torch.distributed as dist
     from paper_2109_15082_b200 import binding as B
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2109_15082_b200 import dist as D
+    rank, world, local = D.env_rank()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
     torch.cuda.set_device(local)
@@ -249,10 +248,7 @@ def main():
         ms = e0.elapsed_time(e1)
         loss_last = float(m.loss[0])
         status = m.poll_status()
-        if world > 1:
-            tt = torch.tensor([ms], dtype=torch.float64, device=m.device)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt[0])
+        ms = D.max_over_ranks(ms, m.device)
 
         # ---- per-kernel timing (CUDA events around every launch of a few eager steps)
         B.mrem_trace_enable(m.ctx, 1)
@@ -282,11 +278,8 @@ def main():
                 B.mrem_recon_step_host(m.ctx, hb[t % len(hb)], hb[t % len(hb)], hl[t % len(hl)], wl.batch, wl.seq, 0.0, opt)
             torch.cuda.synchronize()
             dt_e2e = time.perf_counter() - t0
-            if world > 1:
-                tt = torch.tensor([dt_e2e], dtype=torch.float64, device=m.device)
-                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-                dt_e2e = float(tt[0])
-            e2e = {"value": world * tokens * ke / dt_e2e, "unit": UNIT,
+            dt_e2e = D.max_over_ranks(dt_e2e, m.device)
+            e2e = {"value": D.whole_job_rate(tokens, ke, world, dt_e2e * 1e3), "unit": UNIT,
                    "h2d_bytes_per_step": row_bytes * wl.batch + len_row_bytes, "d2h_bytes_per_step": 4,
                    "steps": ke}
         m.close()
@@ -324,7 +317,7 @@ def main():
                 "peak_source": pk["source"] + (" bf16 sustained" if top["bound"] == "tensor" else " copy bandwidth"),
                 "timed": f"CUDA events around each launch of {n_trace} eager steps"}
 
-    line = {"metric": METRIC, "value": world * tokens * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+    line = {"metric": METRIC, "value": D.whole_job_rate(tokens, K, world, ms), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16+int8", "data": "synthetic",
             "config": {"workload": wl.name, "layers": wl.n_layers, "hidden": wl.hidden, "heads": wl.n_heads,
