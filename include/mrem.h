@@ -221,7 +221,8 @@ int32_t mrem_quantize_weight(const float* d_w, int32_t rows, int32_t cols, const
                              int32_t bits, int32_t grid, int8_t* d_codes, int32_t* d_rowsum, float* d_scale,
                              void* d_what, int32_t dtype, void* cuda_stream);
 /* acc[m, n] = sum_k a[m, k] * b[n, k] in exact int32 on the int8 tensor cores.  a: [M, K] int8 (or uint8
- * when a_unsigned), b: [N, K] int8, K % 16 == 0, acc: [M, N] int32.  block_n 0 = automatic tile width.
+ * when a_unsigned), b: [N, K] int8, K % 16 == 0, acc: [M, N] int32.  block_n 0 = automatic tile width; 64/128/256 force it;
+ * -2 selects the CTA-pair kernel (two SMs per 256 x 256 tile, tcgen05 cta_group::2).
  * d_status: device int32 receiving a DeviceStatus code on a bounded-wait timeout (0 otherwise). */
 int32_t mrem_gemm_i8(const int8_t* d_a, int32_t a_unsigned, const int8_t* d_b, int32_t M, int32_t N, int32_t K,
                      int32_t* d_acc, int32_t block_n, int32_t* d_status, void* cuda_stream);

@@ -14,6 +14,11 @@ enum GemmRc : int { GEMM_OK = 0, GEMM_ERR_ARG = -1, GEMM_ERR_ALIGN = -2, GEMM_ER
 int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
             const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream);
 
+// CTA-pair variant (cta_group::2) for single large products; tc_gemm hands eligible calls to it.
+bool tc_gemm_pair_eligible(const GemmShape& g, const Epilogue& epi, int block_n);
+int tc_gemm_pair(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
+                 const Epilogue& epi, int* d_status, int sm_count, cudaStream_t stream);
+
 // 4-D TMA tensor map (128-byte swizzle) of an operand: (contiguous index, strided index, batch0, batch1).
 // K-major operands get boxes of block_k x tile_mn elements, MN-major ones 64 x block_k.
 int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,

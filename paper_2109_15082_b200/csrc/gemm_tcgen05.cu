@@ -17,219 +17,13 @@
 
 #include <cstdio>
 
-#include "gemm.h"
-#include "tc_ptx.cuh"
+#include "gemm_epi.cuh"
 
 namespace mrem {
 
+using namespace tc;
+
 namespace {
-
-constexpr int BLOCK_M = 128;
-constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
-constexpr int TILE_SMEM_BUDGET = 196608;              // bytes of operand stages per CTA
-constexpr int MAX_STAGES = 8;
-constexpr int GEMM_THREADS = 320;                    // TMA warp, MMA warp, 8 epilogue warps
-constexpr int EPI_WARPS = 8;
-constexpr int STAGING_WORDS = 32 * 33;               // per epilogue warp: 32 rows x 32 words, padded
-constexpr int STAGING_BYTES = EPI_WARPS * STAGING_WORDS * 4;
-constexpr int TMEM_COLS = 512;
-
-struct TcParams {
-  int M, N, K, nb0, nb1;
-  int m_tiles, n_tiles, k_blocks, num_tiles;
-  int block_n, block_k, num_stages, stage_bytes;
-  int a_mn, b_mn;
-  uint32_t idesc;
-  Epilogue epi;
-  int* status;
-};
-
-__device__ __forceinline__ void fail(const TcParams& p, int code, volatile int* abort_flag) {
-  atomicCAS(p.status, 0, code);
-  *abort_flag = 1;
-}
-
-struct TileCoord { int m0, n0, b0, b1; };
-__device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int tile) {
-  TileCoord t;
-  const int per_batch = p.m_tiles * p.n_tiles;
-  const int z = tile / per_batch, r = tile - z * per_batch;
-  t.n0 = (r / p.m_tiles) * p.block_n;      // consecutive tiles walk down one column block
-  t.m0 = (r % p.m_tiles) * BLOCK_M;
-  t.b0 = z % p.nb0;
-  t.b1 = z / p.nb0;
-  return t;
-}
-
-// ------------------------------------------------------------------ epilogue of 32 columns of one row
-template <int KIND>
-__device__ __forceinline__ void epilogue_chunk(const TcParams& p, const uint32_t* r, float alpha, long long row_off,
-                                               int row, int col0, bool row_ok, bool vec_ok) {
-  const Epilogue& e = p.epi;
-  if (!row_ok) return;
-  const int ncol = min(32, p.N - col0);
-  if (ncol <= 0) return;
-  if (e.out_kind == OUT_I32) {
-    int* out = reinterpret_cast<int*>(e.out) + row_off + col0;
-    if (vec_ok && ncol == 32) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 4)
-        *reinterpret_cast<uint4*>(out + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-    } else {
-      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) out[j] = (int)r[j];
-    }
-    return;
-  }
-  float v[32];
-  const float rb = e.row_bias ? e.row_bias[row] : 0.f;
-#pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    const int n = min(col0 + j, p.N - 1);
-    const float acc = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
-    const float sc = e.col_scale ? alpha * e.col_scale[n] : alpha;
-    v[j] = acc * sc + (e.col_bias ? e.col_bias[n] : 0.f) + rb;
-  }
-  const bool full = vec_ok && ncol == 32;
-  if (e.residual) {
-    if (e.out_kind == OUT_BF16) {
-      const bf16* res = reinterpret_cast<const bf16*>(e.residual) + row_off + col0;
-      if (full) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-          const uint4 u = *reinterpret_cast<const uint4*>(res + j);
-          const bf16* h = reinterpret_cast<const bf16*>(&u);
-#pragma unroll
-          for (int t = 0; t < 8; ++t) v[j + t] += __bfloat162float(h[t]);
-        }
-      } else {
-        _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) v[j] += __bfloat162float(res[j]);
-      }
-    } else {
-      const float* res = reinterpret_cast<const float*>(e.residual) + row_off + col0;
-      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) v[j] += res[j];
-    }
-  }
-  if (e.act == 1) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-  }
-  if (e.out_kind == OUT_BF16) {
-    bf16* out = reinterpret_cast<bf16*>(e.out) + row_off + col0;
-    if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        uint4 u;
-        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
-#pragma unroll
-        for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(v[j + 2 * t], v[j + 2 * t + 1]);
-        *reinterpret_cast<uint4*>(out + j) = u;
-      }
-    } else {
-      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) out[j] = __float2bfloat16_rn(v[j]);
-    }
-  } else {
-    float* out = reinterpret_cast<float*>(e.out) + row_off + col0;
-    if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(out + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-    } else {
-      _Pragma("unroll") for (int j = 0; j < 32; ++j) if (j < ncol) out[j] = v[j];
-    }
-  }
-}
-
-// ------------------------------------------------------------------ epilogue of a 32-row x 32-word block
-// One warp, one round: 64 bf16 or 32 fp32/int32 output columns of its 32 rows.  Values go
-// through the warp's staging buffer so that global loads (residual) and stores are issued
-// as 16-byte pieces with 8 lanes covering one contiguous row segment.
-template <int KIND>
-__device__ __forceinline__ void epilogue_round(const TcParams& p, uint32_t taddr, float alpha, long long tile_off,
-                                               int row0, int col0, int lane, uint32_t* stg) {
-  const Epilogue& e = p.epi;
-  const bool is_bf16 = e.out_kind == OUT_BF16;
-  const int vec_elems = is_bf16 ? 8 : 4;
-  const int sub = lane >> 3, seg = lane & 7;             // 4 rows per instruction, 8 lanes per row
-  uint32_t res[32];
-  if (e.residual) {
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int rl = it * 4 + sub, row = row0 + rl;
-      uint4 u = make_uint4(0, 0, 0, 0);
-      if (row < p.M) {
-        const long long off = tile_off + (long long)row * e.ldc + col0 + seg * vec_elems;
-        u = is_bf16 ? *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(e.residual) + off)
-                    : *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(e.residual) + off);
-      }
-      uint32_t* d = stg + rl * 33 + seg * 4;
-      d[0] = u.x; d[1] = u.y; d[2] = u.z; d[3] = u.w;
-    }
-    __syncwarp();
-#pragma unroll
-    for (int j = 0; j < 32; ++j) res[j] = stg[lane * 33 + j];
-    __syncwarp();
-  }
-  const int row = row0 + lane;
-  const float rb = (e.row_bias && row < p.M) ? e.row_bias[row] : 0.f;
-  const int n_loads = is_bf16 ? 2 : 1;
-  for (int h = 0; h < n_loads; ++h) {
-    uint32_t r[32];
-    tmem_ld32(taddr + (uint32_t)(h * 32), r);
-    if (e.out_kind == OUT_I32) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = r[j];
-      continue;
-    }
-    float v[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int n = col0 + h * 32 + j;
-      const float a = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
-      const float sc = e.col_scale ? alpha * e.col_scale[n] : alpha;
-      v[j] = a * sc + (e.col_bias ? e.col_bias[n] : 0.f) + rb;
-    }
-    if (e.residual) {
-      if (is_bf16) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&res[h * 16 + j]);
-          const float2 f = __bfloat1622float2(h2);
-          v[2 * j] += f.x;
-          v[2 * j + 1] += f.y;
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(res[j]);
-      }
-    }
-    if (e.act == 1) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-    }
-    if (is_bf16) {
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-        stg[lane * 33 + h * 16 + j] = *reinterpret_cast<const uint32_t*>(&h2);
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __float_as_uint(v[j]);
-    }
-  }
-  __syncwarp();
-#pragma unroll
-  for (int it = 0; it < 8; ++it) {
-    const int rl = it * 4 + sub, orow = row0 + rl;
-    if (orow < p.M) {
-      const uint32_t* sp = stg + rl * 33 + seg * 4;
-      const uint4 u = make_uint4(sp[0], sp[1], sp[2], sp[3]);
-      const long long off = tile_off + (long long)orow * e.ldc + col0 + seg * vec_elems;
-      if (is_bf16) *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(e.out) + off) = u;
-      else *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(e.out) + off) = u;
-    }
-  }
-  __syncwarp();
-}
 
 // ------------------------------------------------------------------ the kernel
 template <int KIND>
@@ -480,6 +274,7 @@ int pick_block_n(int M, int N, int batches, int sm_count) {
 int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
             const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.nb0 <= 0 || g.nb1 <= 0) return GEMM_ERR_ARG;
+  if (tc_gemm_pair_eligible(g, epi, block_n)) return tc_gemm_pair(kind, a_unsigned, A, B, g, epi, d_status, sm_count, stream);
   const int es = kind == 0 ? 2 : 1;
   if (kind == 1 && (A.mn_contig || B.mn_contig)) return GEMM_ERR_ARG;
   TcParams p;
