@@ -173,6 +173,7 @@ def main():
     ap.add_argument("--calib", type=int, default=0, help="calibration sequences (0: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches (no programmatic dependent launch)")
     args = ap.parse_args()
 
     from paper_2109_15082_b200 import synth
@@ -190,6 +191,8 @@ def main():
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
     torch.cuda.set_device(local)
+    if args.no_pdl:
+        B.mrem_set_programmatic_launch(0)
     if world > 1:
         dist.init_process_group("nccl")
     W = max(3, args.warmup)

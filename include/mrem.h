@@ -178,6 +178,12 @@ int32_t mrem_recon_step_host(mrem_ctx* ctx, const void* h_x_teacher, const void*
                              const int32_t* h_valid_len, int32_t batch, int32_t seq, float lambda,
                              const mrem_optim* optim, float* h_loss);
 
+/* Process-wide switch (default on): kernels are launched with programmatic stream serialization, i.e. a
+ * kernel may be scheduled and run its set-up while its predecessor in the stream is still finishing; each
+ * kernel waits for its predecessor's results before touching global memory, so results do not change.
+ * Turn it off (0) to get plain stream-ordered launches, e.g. when comparing timings. */
+int32_t mrem_set_programmatic_launch(int32_t on);
+
 /* Reads the device status word (blocks on the stream): MREM_OK, MREM_ERR_TIMEOUT or MREM_ERR_NONFINITE in
  * *h_status; the word is cleared. */
 int32_t mrem_poll_status(mrem_ctx* ctx, int32_t* h_status);

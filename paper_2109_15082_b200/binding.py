@@ -31,7 +31,7 @@ EXPORTS = (
     "mrem_step", "mrem_recon_step_host", "mrem_poll_status", "mrem_state_bytes", "mrem_export_state",
     "mrem_import_state", "mrem_graph_capture_step", "mrem_graph_launch", "mrem_gather_rows", "mrem_quantize_act",
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
-    "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc",
+    "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
 )
 
 
@@ -136,6 +136,10 @@ def mrem_init_weight_steps(ctx, rule):
 
 def mrem_init_act_steps(ctx, x, valid_len, batch, seq):
     _check(lib().mrem_init_act_steps(ctx, _p(x), _p(valid_len), batch, seq), "mrem_init_act_steps", ctx)
+
+
+def mrem_set_programmatic_launch(on):
+    _check(lib().mrem_set_programmatic_launch(int(on)), "mrem_set_programmatic_launch")
 
 
 def mrem_invalidate_weight_codes(ctx):

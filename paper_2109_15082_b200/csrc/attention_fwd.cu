@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
   const int n_box = (p.S + 127) / 128;                       // 128-row TMA boxes of keys / values
   const uint32_t sQ = base, sK = sQ + 16384, sV = sK + n_box * 16384, sP = sV + n_box * 16384;
   uint8_t* gP = smem_raw + (sP - smem_u32(smem_raw));        // generic pointer to the P operand tile
+  pdl_trigger();
 
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bar_full), 1);
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
   const uint32_t tmem_ctx = tmem + (uint32_t)p.n16;
 
@@ -292,7 +294,7 @@ int launch_attention_fwd(const void* qkv, int B, int S, int h, int H, const int*
   const long long rows = (long long)B * h * S;
   Scope sc("attention_fwd_tcgen05", 4.0 * rows * S * HD, 1, st);
   dim3 grid((S + 127) / 128, h, B);
-  attention_fwd_kernel<<<grid, ATT_THREADS, smem, st>>>(map, p);
+  if (launch_k(attention_fwd_kernel, grid, ATT_THREADS, smem, st, map, p) != cudaSuccess) return GEMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }
 

@@ -23,6 +23,8 @@ __device__ __forceinline__ float load_op(const OperandDesc& o, long long base, i
 }
 
 __global__ void __launch_bounds__(256) simt_gemm_kernel(const SimtParams p) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sa[TK][TS + 1];
   __shared__ float sb[TK][TS + 1];
   const int z = blockIdx.z, b0 = z % p.g.nb0, b1 = z / p.g.nb0;
@@ -82,7 +84,7 @@ int simt_gemm_f32(const OperandDesc& A, const OperandDesc& B, const GemmShape& g
   dim3 grid((g.N + TS - 1) / TS, (g.M + TS - 1) / TS, g.nb0 * g.nb1);
   if (grid.y > 65535 || grid.z > 65535) return GEMM_ERR_ARG;
   Scope sc("gemm_f32_simt", 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream);
-  simt_gemm_kernel<<<grid, 256, 0, stream>>>(p);
+  launch_k(simt_gemm_kernel, grid, 256, 0, stream, p);
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }
 

@@ -40,6 +40,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  pdl_trigger();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.num_stages; ++s) {
@@ -63,6 +64,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                            // set-up done; from here on the predecessor's results are needed
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
   volatile int* vabort = &abort_flag;
 
@@ -330,7 +332,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
              A.mn_contig ? "T" : "N", B.mn_contig ? "N" : "T", g.nb0 * g.nb1);
     return std::string(buf);
   }, 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream, 0);
-  kern<<<grid, GEMM_THREADS, smem, stream>>>(ma, mb, p);
+  if (launch_k(kern, grid, GEMM_THREADS, smem, stream, ma, mb, p) != cudaSuccess) return GEMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }
 

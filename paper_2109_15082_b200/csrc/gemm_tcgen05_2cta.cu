@@ -95,6 +95,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const uint32_t rank = cluster_ctarank();
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int half_n = p.block_n >> 1;
+  pdl_trigger();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.num_stages; ++s) {
@@ -119,6 +120,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   __syncthreads();
   cluster_sync_all();                    // the peer's barriers exist before anyone signals them
   tc_fence_after();
+  pdl_wait();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
   volatile int* vabort = &abort_flag;
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
@@ -318,13 +320,15 @@ int tc_gemm_pair(int kind, int a_unsigned, const OperandDesc& A, const OperandDe
   cfg.blockDim = dim3(GEMM_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = g_programmatic_launch ? 1 : 0;
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   if (cudaLaunchKernelEx(&cfg, kern, ma, mb, p) != cudaSuccess) return GEMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }

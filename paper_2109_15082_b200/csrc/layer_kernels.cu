@@ -20,6 +20,8 @@ template <typename T, int V>
 __global__ void __launch_bounds__(256) loss_kernel(const T* __restrict__ fh, const T* __restrict__ f,
                                                    long long n, float c, T* __restrict__ dF,
                                                    float* __restrict__ partial, int* __restrict__ status) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const long long base = (long long)blockIdx.y * n;
   float acc = 0.f;
@@ -43,6 +45,8 @@ __global__ void __launch_bounds__(256) loss_kernel(const T* __restrict__ fh, con
 }
 __global__ void loss_final_kernel(const float* __restrict__ partial, int n_layers, int nb, float c,
                                   float* __restrict__ total, float* __restrict__ per_layer) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   float tot = 0.f;
   for (int l = 0; l < n_layers; ++l) {
@@ -64,6 +68,8 @@ __global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, l
                                                       const float* __restrict__ step,
                                                       const float* __restrict__ offset, float lo, float hi,
                                                       float* __restrict__ part_s, float* __restrict__ part_o) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const float s = *step;
   const bool has_off = offset != nullptr;
@@ -109,6 +115,8 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
                                                        const float* __restrict__ offset, float lo, float hi,
                                                        int quantized, float* __restrict__ part_s,
                                                        float* __restrict__ part_o) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const float s = quantized ? *step : 1.f;
   const bool has_off = offset != nullptr;
@@ -143,6 +151,8 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
 __global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict__ w, const float* __restrict__ steps,
                                                          int per_row, int bits, int grid, float* __restrict__ dw,
                                                          int cols, float* __restrict__ ds_rows) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const int row = blockIdx.x;
   const float s = steps[per_row ? row : 0];
@@ -165,6 +175,8 @@ __global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict
 }
 
 __global__ void __launch_bounds__(256) reduce_table_kernel(const ReduceEntry* __restrict__ table) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const ReduceEntry e = table[blockIdx.x];
   float a = 0.f;
@@ -174,12 +186,16 @@ __global__ void __launch_bounds__(256) reduce_table_kernel(const ReduceEntry* __
 }
 
 __global__ void scale_vec_kernel(const float* __restrict__ in, const float* __restrict__ scale, float* __restrict__ out, int n) {
+  pdl_trigger();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = scale[0] * in[i];
 }
 __global__ void effective_bias_kernel(const float* __restrict__ b, const float* __restrict__ beta,
                                       const float* __restrict__ wscale, const int32_t* __restrict__ rowsum,
                                       float* __restrict__ beff, int n) {
+  pdl_trigger();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) beff[i] = b[i] + beta[0] * wscale[i] * (float)rowsum[i];
 }
@@ -187,6 +203,8 @@ __global__ void effective_bias_kernel(const float* __restrict__ b, const float* 
 // ------------------------------------------------------------------ AdamW
 __global__ void optim_prepare_kernel(OptimScalars* out, int* d_t, int host_t, float lr0, int total, float b1, float b2,
                                      float eps, float wd) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
   int t = host_t >= 1 ? host_t : (*d_t + 1);
   *d_t = t;
@@ -203,6 +221,8 @@ __global__ void optim_prepare_kernel(OptimScalars* out, int* d_t, int host_t, fl
 
 __global__ void __launch_bounds__(256) adamw_table_kernel(const AdamEntry* __restrict__ table,
                                                           const OptimScalars* __restrict__ sc) {
+  pdl_trigger();
+  pdl_wait();
   const AdamEntry e = table[blockIdx.y];
   const OptimScalars o = *sc;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < e.n; i += (long long)gridDim.x * blockDim.x) {
@@ -234,14 +254,14 @@ void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
     if (n_per_layer % V == 0 && al16(f_hat) && al16(f) && al16(dF))
-      loss_kernel<T, V><<<grid, 256, 0, st>>>((const T*)f_hat, (const T*)f, n_per_layer, c, (T*)dF, partial, status);
+      launch_k(loss_kernel<T, V>, grid, 256, 0, st, (const T*)f_hat, (const T*)f, n_per_layer, c, (T*)dF, partial, status);
     else
-      loss_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)f_hat, (const T*)f, n_per_layer, c, (T*)dF, partial, status);
+      launch_k(loss_kernel<T, 1>, grid, 256, 0, st, (const T*)f_hat, (const T*)f, n_per_layer, c, (T*)dF, partial, status);
   });
 }
 void launch_loss_finalize(const float* partial, int n_layers, float c, float* loss_total, float* loss_per_layer,
                           cudaStream_t st) {
-  loss_final_kernel<<<1, 256, 0, st>>>(partial, n_layers, RED_BLOCKS, c, loss_total, loss_per_layer);
+  launch_k(loss_final_kernel, 1, 256, 0, st, partial, n_layers, RED_BLOCKS, c, loss_total, loss_per_layer);
 }
 
 void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long ld_d, const void* add,
@@ -252,8 +272,8 @@ void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long 
     constexpr int V = 16 / (int)sizeof(T);
     const bool v = cols % V == 0 && ld_x % V == 0 && ld_d % V == 0 && ld_dx % V == 0 && (!add || ld_add % V == 0) &&
                    al16(x) && al16(dxhat) && al16(add) && al16(dx);
-    if (v) ste_act_kernel<T, V><<<RED_BLOCKS, 256, 0, st>>>((const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
-    else ste_act_kernel<T, 1><<<RED_BLOCKS, 256, 0, st>>>((const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
+    if (v) launch_k(ste_act_kernel<T, V>, RED_BLOCKS, 256, 0, st, (const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
+    else launch_k(ste_act_kernel<T, 1>, RED_BLOCKS, 256, 0, st, (const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
   });
 }
 
@@ -263,40 +283,40 @@ void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, co
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
     if (n % V == 0 && al16(u) && al16(dghat) && al16(du))
-      gelu_bwd_kernel<T, V><<<RED_BLOCKS, 256, 0, st>>>((const T*)u, (const T*)dghat, (T*)du, n, step, offset, (float)lo, (float)hi, quantized, part_s, part_o);
+      launch_k(gelu_bwd_kernel<T, V>, RED_BLOCKS, 256, 0, st, (const T*)u, (const T*)dghat, (T*)du, n, step, offset, (float)lo, (float)hi, quantized, part_s, part_o);
     else
-      gelu_bwd_kernel<T, 1><<<RED_BLOCKS, 256, 0, st>>>((const T*)u, (const T*)dghat, (T*)du, n, step, offset, (float)lo, (float)hi, quantized, part_s, part_o);
+      launch_k(gelu_bwd_kernel<T, 1>, RED_BLOCKS, 256, 0, st, (const T*)u, (const T*)dghat, (T*)du, n, step, offset, (float)lo, (float)hi, quantized, part_s, part_o);
   });
 }
 
 void launch_ste_weight(const float* w, const float* steps, int per_row, int bits, int grid, float* dw, int rows,
                        int cols, float* ds_rows, cudaStream_t st) {
   Scope sc("ste_weight", (double)rows * cols * 12.0, 0, st);
-  ste_weight_kernel<<<rows, 256, 0, st>>>(w, steps, per_row, bits, grid, dw, cols, ds_rows);
+  launch_k(ste_weight_kernel, rows, 256, 0, st, w, steps, per_row, bits, grid, dw, cols, ds_rows);
 }
 
 void launch_reduce_table(const ReduceEntry* d_table, int n_entries, cudaStream_t st) {
-  if (n_entries > 0) reduce_table_kernel<<<n_entries, 256, 0, st>>>(d_table);
+  if (n_entries > 0) launch_k(reduce_table_kernel, n_entries, 256, 0, st, d_table);
 }
 
 void launch_scale_vec(const float* in, const float* scale, float* out, int n, cudaStream_t st) {
-  scale_vec_kernel<<<(n + 255) / 256, 256, 0, st>>>(in, scale, out, n);
+  launch_k(scale_vec_kernel, (n + 255) / 256, 256, 0, st, in, scale, out, n);
 }
 void launch_effective_bias(const float* b, const float* beta, const float* wscale, const int32_t* rowsum, float* beff,
                            int n, cudaStream_t st) {
-  effective_bias_kernel<<<(n + 255) / 256, 256, 0, st>>>(b, beta, wscale, rowsum, beff, n);
+  launch_k(effective_bias_kernel, (n + 255) / 256, 256, 0, st, b, beta, wscale, rowsum, beff, n);
 }
 
 void launch_optim_prepare(OptimScalars* d_out, int* d_t, int host_t, float lr0, int total_steps, float beta1,
                           float beta2, float eps, float weight_decay, cudaStream_t st) {
-  optim_prepare_kernel<<<1, 32, 0, st>>>(d_out, d_t, host_t, lr0, total_steps, beta1, beta2, eps, weight_decay);
+  launch_k(optim_prepare_kernel, 1, 32, 0, st, d_out, d_t, host_t, lr0, total_steps, beta1, beta2, eps, weight_decay);
 }
 void launch_adamw_table(const AdamEntry* d_table, int n_entries, long long total_elems, const OptimScalars* d_sc,
                         cudaStream_t st) {
   if (n_entries <= 0) return;
   Scope sc("adamw", (double)total_elems * 28.0, 0, st);
   dim3 grid(64, n_entries);
-  adamw_table_kernel<<<grid, 256, 0, st>>>(d_table, d_sc);
+  launch_k(adamw_table_kernel, grid, 256, 0, st, d_table, d_sc);
 }
 
 }  // namespace mrem

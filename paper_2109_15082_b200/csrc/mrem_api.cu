@@ -6,7 +6,10 @@
 
 using namespace mrem;
 
-namespace mrem { thread_local Tracer* g_tracer = nullptr; }
+namespace mrem {
+thread_local Tracer* g_tracer = nullptr;
+int g_programmatic_launch = 1;
+}
 
 namespace {
 std::string g_create_err;
@@ -372,6 +375,11 @@ int32_t mrem_invalidate_weight_codes(mrem_ctx* c) {
   if (!c) return MREM_ERR_ARG;
   c->codes_fresh = false;
   c->weights_quantized = false;
+  return MREM_OK;
+}
+
+int32_t mrem_set_programmatic_launch(int32_t on) {
+  mrem::g_programmatic_launch = on ? 1 : 0;
   return MREM_OK;
 }
 

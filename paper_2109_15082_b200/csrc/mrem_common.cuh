@@ -17,6 +17,31 @@ enum DeviceStatus : int {
   DEV_NONFINITE = 4,        // the loss kernel met a non-finite value
 };
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the library is launched so that it may start while its predecessor in the stream is
+// still draining: it announces itself (pdl_trigger) and then waits (pdl_wait) until everything the
+// predecessor wrote is visible, before it touches global memory.  What runs before the wait (barrier
+// and TMEM set-up in the tensor-core kernels) and the launch latency itself overlap the predecessor's tail.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+extern int g_programmatic_launch;      // 1: launch with programmatic stream serialization (default)
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = g_programmatic_launch ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------- storage-type access
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }

@@ -16,6 +16,8 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
                                                               int grid, int8_t* __restrict__ codes,
                                                               int32_t* __restrict__ rowsum, float* __restrict__ scale,
                                                               T* __restrict__ what) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int sh[32];
   const int row = blockIdx.x;
   const float s = steps[per_row ? row : 0];
@@ -60,6 +62,8 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
                                                            const float* __restrict__ offset, float lo, float hi,
                                                            int8_t* __restrict__ q8, long long ld_q8,
                                                            T* __restrict__ qt, long long ld_qt) {
+  pdl_trigger();
+  pdl_wait();
   const float s = *step;
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
@@ -85,6 +89,8 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
 template <typename T, int V>
 __global__ void __launch_bounds__(256) mix_kernel(const T* __restrict__ f, const T* __restrict__ fh, float lam,
                                                   T* __restrict__ out, long long n) {
+  pdl_trigger();
+  pdl_wait();
   for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
     float a[V], b[V];
     load_vec<T, V>(f + i, a);
@@ -101,6 +107,8 @@ __global__ void __launch_bounds__(256) gelu_quant_kernel(const T* __restrict__ u
                                                          const float* __restrict__ step,
                                                          const float* __restrict__ offset, float lo, float hi,
                                                          int8_t* __restrict__ q8, T* __restrict__ qt) {
+  pdl_trigger();
+  pdl_wait();
   const float s = *step;
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
@@ -123,6 +131,8 @@ __global__ void __launch_bounds__(256) gelu_quant_kernel(const T* __restrict__ u
 // stat[row] = max|w| (rule 0) or mean|w| (rule 1) of one row; per_row: steps[row] = stat/qmax | stat.
 __global__ void __launch_bounds__(256) weight_row_stat_kernel(const float* __restrict__ w, int cols, int rule,
                                                               float* __restrict__ stat) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const float* wr = w + (long long)blockIdx.x * cols;
   float acc = 0.f;
@@ -135,6 +145,8 @@ __global__ void __launch_bounds__(256) weight_row_stat_kernel(const float* __res
 }
 __global__ void weight_steps_from_stat_kernel(const float* __restrict__ stat, int rows, int cols, int per_row,
                                               int rule, float qmax, float* __restrict__ steps) {
+  pdl_trigger();
+  pdl_wait();
   if (per_row) {
     for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < rows; r += gridDim.x * blockDim.x) {
       const float v = rule == 0 ? __fdiv_rn(stat[r], qmax) : __fdiv_rn(stat[r], (float)cols);
@@ -151,6 +163,8 @@ __global__ void weight_steps_from_stat_kernel(const float* __restrict__ stat, in
 template <typename T>
 __global__ void __launch_bounds__(256) minmax_kernel(const T* __restrict__ x, long long ld, long long rows, int cols,
                                                      float* __restrict__ part) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   float lo = INFINITY, hi = -INFINITY;
   const long long total = rows * cols;
@@ -168,6 +182,8 @@ __global__ void __launch_bounds__(256) minmax_kernel(const T* __restrict__ x, lo
   }
 }
 __global__ void minmax_final_kernel(const float* __restrict__ part, int n, float* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     float lo = INFINITY, hi = -INFINITY;
     for (int i = 0; i < n; ++i) {
@@ -179,6 +195,8 @@ __global__ void minmax_final_kernel(const float* __restrict__ part, int n, float
   }
 }
 __global__ void step_from_minmax_kernel(const float* __restrict__ mm, int mode, float qmax, float* step, float* offset) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     float s, o = 0.f;
     if (mode == 0) s = __fdiv_rn(fmaxf(fabsf(mm[0]), fabsf(mm[1])), qmax);
@@ -191,6 +209,8 @@ __global__ void step_from_minmax_kernel(const float* __restrict__ mm, int mode, 
 
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
                                                           long long row_vecs, uint4* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   const uint4* s = src + (long long)idx[blockIdx.y] * row_vecs;
   uint4* o = out + (long long)blockIdx.y * row_vecs;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < row_vecs; i += (long long)gridDim.x * blockDim.x)
@@ -198,12 +218,16 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restric
 }
 
 __global__ void __launch_bounds__(256) widen_bf16_kernel(const bf16* __restrict__ src, float* __restrict__ dst, long long n) {
+  pdl_trigger();
+  pdl_wait();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
     dst[i] = __bfloat162float(src[i]);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_kernel(const float* __restrict__ src, T* __restrict__ dst, long long n) {
+  pdl_trigger();
+  pdl_wait();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
     dst[i] = from_f<T>(src[i]);
 }
@@ -226,9 +250,9 @@ void launch_quantize_weight(const float* w, int rows, int cols, const float* ste
                             int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt, cudaStream_t st) {
   Scope sc("quantize_weight", (double)rows * cols * (5.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)) + rows * 8.0, 0, st);
   if (dt == 1)
-    quantize_weight_kernel<bf16><<<rows, 256, 0, st>>>(w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (bf16*)what);
+    launch_k(quantize_weight_kernel<bf16>, rows, 256, 0, st, w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (bf16*)what);
   else
-    quantize_weight_kernel<float><<<rows, 256, 0, st>>>(w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (float*)what);
+    launch_k(quantize_weight_kernel<float>, rows, 256, 0, st, w, cols, steps, per_row, bits, grid, codes, rowsum, scale, (float*)what);
 }
 
 template <typename T>
@@ -238,9 +262,9 @@ static void quantize_act_t(const T* x, long long rows, int cols, long long ld_x,
   const bool v = vec_ok<T>(x, ld_x, cols) && vec_ok<T>(qt, ld_qt, cols) &&
                  (q8 == nullptr || ((reinterpret_cast<uintptr_t>(q8) % V) == 0 && ld_q8 % V == 0));
   if (v)
-    quantize_act_kernel<T, V><<<grid_for(rows * cols / V), 256, 0, st>>>(x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
+    launch_k(quantize_act_kernel<T, V>, grid_for(rows * cols / V), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
   else
-    quantize_act_kernel<T, 1><<<grid_for(rows * cols), 256, 0, st>>>(x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
+    launch_k(quantize_act_kernel<T, 1>, grid_for(rows * cols), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
 }
 
 void launch_quantize_act(const void* x, int dt, long long rows, int cols, long long ld_x, const float* step,
@@ -253,13 +277,13 @@ void launch_quantize_act(const void* x, int dt, long long rows, int cols, long l
 }
 
 void launch_widen_bf16(const void* src, float* dst, long long n, cudaStream_t st) {
-  if (n > 0) widen_bf16_kernel<<<grid_for(n), 256, 0, st>>>((const bf16*)src, dst, n);
+  if (n > 0) launch_k(widen_bf16_kernel, grid_for(n), 256, 0, st, (const bf16*)src, dst, n);
 }
 
 void launch_narrow(const float* src, void* dst, long long n, int dt, cudaStream_t st) {
   if (n <= 0) return;
-  if (dt == 1) narrow_kernel<bf16><<<grid_for(n), 256, 0, st>>>(src, (bf16*)dst, n);
-  else narrow_kernel<float><<<grid_for(n), 256, 0, st>>>(src, (float*)dst, n);
+  if (dt == 1) launch_k(narrow_kernel<bf16>, grid_for(n), 256, 0, st, src, (bf16*)dst, n);
+  else launch_k(narrow_kernel<float>, grid_for(n), 256, 0, st, src, (float*)dst, n);
 }
 
 void launch_mix(const void* f, const void* f_hat, float lam, void* out, long long n, int dt, cudaStream_t st) {
@@ -267,14 +291,14 @@ void launch_mix(const void* f, const void* f_hat, float lam, void* out, long lon
   Scope sc("teacher_forcing_mix", (double)n * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
   if (dt == 1) {
     if (n % 8 == 0 && vec_ok<bf16>(f, 8, 8) && vec_ok<bf16>(f_hat, 8, 8) && vec_ok<bf16>(out, 8, 8))
-      mix_kernel<bf16, 8><<<grid_for(n / 8), 256, 0, st>>>((const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
+      launch_k(mix_kernel<bf16, 8>, grid_for(n / 8), 256, 0, st, (const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
     else
-      mix_kernel<bf16, 1><<<grid_for(n), 256, 0, st>>>((const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
+      launch_k(mix_kernel<bf16, 1>, grid_for(n), 256, 0, st, (const bf16*)f, (const bf16*)f_hat, lam, (bf16*)out, n);
   } else {
     if (n % 4 == 0 && vec_ok<float>(f, 4, 4) && vec_ok<float>(f_hat, 4, 4) && vec_ok<float>(out, 4, 4))
-      mix_kernel<float, 4><<<grid_for(n / 4), 256, 0, st>>>((const float*)f, (const float*)f_hat, lam, (float*)out, n);
+      launch_k(mix_kernel<float, 4>, grid_for(n / 4), 256, 0, st, (const float*)f, (const float*)f_hat, lam, (float*)out, n);
     else
-      mix_kernel<float, 1><<<grid_for(n), 256, 0, st>>>((const float*)f, (const float*)f_hat, lam, (float*)out, n);
+      launch_k(mix_kernel<float, 1>, grid_for(n), 256, 0, st, (const float*)f, (const float*)f_hat, lam, (float*)out, n);
   }
 }
 
@@ -284,30 +308,30 @@ void launch_gelu_quant(const void* u, long long n, const float* step, const floa
   Scope sc("gelu_quant", (double)n * ((dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1) + (q8 ? 1 : 0)), 0, st);
   if (dt == 1) {
     const bool v = n % 8 == 0 && vec_ok<bf16>(u, 8, 8) && vec_ok<bf16>(qt, 8, 8) && (reinterpret_cast<uintptr_t>(q8) % 8) == 0;
-    if (v) gelu_quant_kernel<bf16, 8><<<grid_for(n / 8), 256, 0, st>>>((const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
-    else gelu_quant_kernel<bf16, 1><<<grid_for(n), 256, 0, st>>>((const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
+    if (v) launch_k(gelu_quant_kernel<bf16, 8>, grid_for(n / 8), 256, 0, st, (const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
+    else launch_k(gelu_quant_kernel<bf16, 1>, grid_for(n), 256, 0, st, (const bf16*)u, n, step, offset, (float)lo, (float)hi, q8, (bf16*)qt);
   } else {
     const bool v = n % 4 == 0 && vec_ok<float>(u, 4, 4) && vec_ok<float>(qt, 4, 4) && (reinterpret_cast<uintptr_t>(q8) % 4) == 0;
-    if (v) gelu_quant_kernel<float, 4><<<grid_for(n / 4), 256, 0, st>>>((const float*)u, n, step, offset, (float)lo, (float)hi, q8, (float*)qt);
-    else gelu_quant_kernel<float, 1><<<grid_for(n), 256, 0, st>>>((const float*)u, n, step, offset, (float)lo, (float)hi, q8, (float*)qt);
+    if (v) launch_k(gelu_quant_kernel<float, 4>, grid_for(n / 4), 256, 0, st, (const float*)u, n, step, offset, (float)lo, (float)hi, q8, (float*)qt);
+    else launch_k(gelu_quant_kernel<float, 1>, grid_for(n), 256, 0, st, (const float*)u, n, step, offset, (float)lo, (float)hi, q8, (float*)qt);
   }
 }
 
 void launch_init_weight_steps(const float* w, int rows, int cols, int per_row, int rule, float qmax, float* steps,
                               float* scratch, cudaStream_t st) {
-  weight_row_stat_kernel<<<rows, 256, 0, st>>>(w, cols, rule, scratch);
-  weight_steps_from_stat_kernel<<<per_row ? (rows + 255) / 256 : 1, 256, 0, st>>>(scratch, rows, cols, per_row, rule, qmax, steps);
+  launch_k(weight_row_stat_kernel, rows, 256, 0, st, w, cols, rule, scratch);
+  launch_k(weight_steps_from_stat_kernel, per_row ? (rows + 255) / 256 : 1, 256, 0, st, scratch, rows, cols, per_row, rule, qmax, steps);
 }
 
 void launch_minmax(const void* x, long long ld, long long rows, int cols, float* out, float* scratch, int dt,
                    cudaStream_t st) {
-  if (dt == 1) minmax_kernel<bf16><<<RED_BLOCKS, 256, 0, st>>>((const bf16*)x, ld, rows, cols, scratch);
-  else minmax_kernel<float><<<RED_BLOCKS, 256, 0, st>>>((const float*)x, ld, rows, cols, scratch);
-  minmax_final_kernel<<<1, 32, 0, st>>>(scratch, RED_BLOCKS, out);
+  if (dt == 1) launch_k(minmax_kernel<bf16>, RED_BLOCKS, 256, 0, st, (const bf16*)x, ld, rows, cols, scratch);
+  else launch_k(minmax_kernel<float>, RED_BLOCKS, 256, 0, st, (const float*)x, ld, rows, cols, scratch);
+  launch_k(minmax_final_kernel, 1, 32, 0, st, scratch, RED_BLOCKS, out);
 }
 
 void launch_step_from_minmax(const float* minmax, int mode, float qmax, float* step, float* offset, cudaStream_t st) {
-  step_from_minmax_kernel<<<1, 32, 0, st>>>(minmax, mode, qmax, step, offset);
+  launch_k(step_from_minmax_kernel, 1, 32, 0, st, minmax, mode, qmax, step, offset);
 }
 
 void launch_gather_rows(const void* src, const int* d_idx, int n_rows, long long row_bytes, void* out,
@@ -315,7 +339,7 @@ void launch_gather_rows(const void* src, const int* d_idx, int n_rows, long long
   const long long row_vecs = row_bytes / 16;
   Scope sc("gather_rows", 2.0 * n_rows * (double)row_bytes, 0, st);
   dim3 grid(grid_for(row_vecs, 256, 64), n_rows);
-  gather_rows_kernel<<<grid, 256, 0, st>>>((const uint4*)src, d_idx, row_vecs, (uint4*)out);
+  launch_k(gather_rows_kernel, grid, 256, 0, st, (const uint4*)src, d_idx, row_vecs, (uint4*)out);
 }
 
 }  // namespace mrem

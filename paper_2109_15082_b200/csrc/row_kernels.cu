@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(128) ln_fwd_kernel(const T* __restrict__ y, co
                                                      int cols, T* __restrict__ out, float* __restrict__ mean,
                                                      float* __restrict__ rstd, const float* __restrict__ step,
                                                      float qmax, int8_t* __restrict__ q8, T* __restrict__ qt) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -125,6 +127,8 @@ __global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout,
                                                      const float* __restrict__ rstd, const float* __restrict__ gamma,
                                                      long long rows, int cols, T* __restrict__ dy,
                                                      T* __restrict__ dsum) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -206,6 +210,8 @@ __global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a
                                                          float* __restrict__ out0, float* __restrict__ out1,
                                                          float* __restrict__ out2, float* __restrict__ scratch,
                                                          int* __restrict__ counters) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[3][8][32 * V + 1];
   __shared__ int is_last;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -281,6 +287,8 @@ __global__ void __launch_bounds__(128) softmax_fwd_kernel(const float* __restric
                                                           const float* __restrict__ step,
                                                           const float* __restrict__ offset, float lo, float hi,
                                                           T* __restrict__ qt) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long row = blockIdx.x * 4ll + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -352,6 +360,8 @@ __global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ 
                                                           T* __restrict__ dS, long long rows, int S,
                                                           const float* __restrict__ step, float lo, float hi,
                                                           int quantized, float* __restrict__ part_s) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const int lane = threadIdx.x & 31;
   const long long warp0 = blockIdx.x * 8ll + (threadIdx.x >> 5), nwarps = gridDim.x * 8ll;
@@ -438,8 +448,8 @@ void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, 
     constexpr int V = 16 / (int)sizeof(T);
     const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(y) && al16(out) && al16(qt) &&
                    (reinterpret_cast<uintptr_t>(q8) % V) == 0;
-    if (v) ln_fwd_kernel<T, V, true><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
-    else ln_fwd_kernel<T, 1, false><<<grid, 128, 0, st>>>((const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
+    if (v) launch_k(ln_fwd_kernel<T, V, true>, grid, 128, 0, st, (const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
+    else launch_k(ln_fwd_kernel<T, 1, false>, grid, 128, 0, st, (const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
   });
 }
 
@@ -452,8 +462,8 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
     const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(dout) && al16(dout2) && al16(y) && al16(dy) && al16(dsum);
-    if (v) ln_bwd_kernel<T, V, true><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
-    else ln_bwd_kernel<T, 1, false><<<grid, 128, 0, st>>>((const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
+    if (v) launch_k(ln_bwd_kernel<T, V, true>, grid, 128, 0, st, (const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
+    else launch_k(ln_bwd_kernel<T, 1, false>, grid, 128, 0, st, (const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
   });
 }
 
@@ -465,10 +475,10 @@ void launch_col_reduce(const void* a, long long ld_a, const void* y, const float
     constexpr int V = 16 / (int)sizeof(T);
     if (cols % V == 0 && ld_a % V == 0 && ld_a2 % V == 0 && al16(a) && al16(y) && al16(a2)) {
       dim3 grid((cols + 32 * V - 1) / (32 * V), COL_CHUNKS);
-      col_reduce_kernel<T, V><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
+      launch_k(col_reduce_kernel<T, V>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
     } else {
       dim3 grid((cols + 31) / 32, COL_CHUNKS);
-      col_reduce_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
+      launch_k(col_reduce_kernel<T, 1>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
     }
   });
 }
@@ -481,8 +491,8 @@ void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h,
   const int grid = (int)((rows + 3) / 4);
   const bool cached = S % 4 == 0 && S <= 128 * MAXNV && al16(scores) && al16(P) && al16(qt);
   MREM_DT(dt, T, {
-    if (cached) softmax_fwd_kernel<T, true><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt);
-    else softmax_fwd_kernel<T, false><<<grid, 128, 0, st>>>(scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt);
+    if (cached) launch_k(softmax_fwd_kernel<T, true>, grid, 128, 0, st, scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt);
+    else launch_k(softmax_fwd_kernel<T, false>, grid, 128, 0, st, scores, valid_len, h, S, rows, (T*)P, step, offset, (float)lo, (float)hi, (T*)qt);
   });
 }
 
@@ -491,8 +501,8 @@ void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long ro
   Scope sc("softmax_bwd", (double)rows * S * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
   const bool cached = S % 4 == 0 && S <= 128 * MAXNV && al16(P) && al16(dphat) && al16(dS);
   MREM_DT(dt, T, {
-    if (cached) softmax_bwd_kernel<T, true><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s);
-    else softmax_bwd_kernel<T, false><<<RED_BLOCKS, 256, 0, st>>>((const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s);
+    if (cached) launch_k(softmax_bwd_kernel<T, true>, RED_BLOCKS, 256, 0, st, (const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s);
+    else launch_k(softmax_bwd_kernel<T, false>, RED_BLOCKS, 256, 0, st, (const T*)P, (const T*)dphat, (T*)dS, rows, S, step, (float)lo, (float)hi, quantized, part_s);
   });
 }
 

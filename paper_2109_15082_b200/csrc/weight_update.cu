@@ -45,6 +45,8 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
     float* __restrict__ steps, const float* __restrict__ ds_in, float* __restrict__ m_s, float* __restrict__ v_s,
     const OptimScalars* __restrict__ sc, int cols, int bits, int grid, int train_w, int train_s,
     int8_t* __restrict__ codes, int32_t* __restrict__ rowsum, float* __restrict__ scale, T* __restrict__ what) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   __shared__ int shi[32];
   __shared__ float s_new_sh;
@@ -172,9 +174,9 @@ void launch_fused_weight_update(float* w, const float* g, float* m, float* v, fl
                                 int dt, cudaStream_t st) {
   Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
   if (dt == 1)
-    fused_weight_update_kernel<bf16><<<rows, 256, 0, st>>>(w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (bf16*)what);
+    launch_k(fused_weight_update_kernel<bf16>, rows, 256, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (bf16*)what);
   else
-    fused_weight_update_kernel<float><<<rows, 256, 0, st>>>(w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (float*)what);
+    launch_k(fused_weight_update_kernel<float>, rows, 256, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (float*)what);
 }
 
 }  // namespace mrem
