@@ -16,7 +16,6 @@ namespace mrem {
 
 namespace {
 
-constexpr int MAXV = 4;      // float4 vectors per thread kept in registers (256 threads: 4096 columns)
 
 __device__ __forceinline__ int weight_code(float w, float s, float qmax, int grid) {
   const float z = __fdiv_rn(w, s);
@@ -39,7 +38,8 @@ __device__ __forceinline__ void store_what4<bf16>(bf16* p, float a, float b, flo
   *reinterpret_cast<uint2*>(p) = t;
 }
 
-template <typename T>
+// NV = float4 vectors per thread kept in registers: 1 for rows up to 1024 wide, 4 up to 4096; wider rows are re-read.
+template <typename T, int NV>
 __global__ void __launch_bounds__(256) fused_weight_update_kernel(
     float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v,
     float* __restrict__ steps, const float* __restrict__ ds_in, float* __restrict__ m_s, float* __restrict__ v_s,
@@ -56,21 +56,27 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   const float qmax = (float)((1 << (bits - 1)) - 1);
   const long long base = (long long)row * cols;
   const int nvec = cols / 4;                                   // cols is a multiple of 16
-  const bool cached = nvec <= MAXV * 256;
+  const bool cached = nvec <= NV * 256;
   const float4* w4 = reinterpret_cast<const float4*>(w + base);
   const float4* g4 = reinterpret_cast<const float4*>(g + base);
-  float4 wr[MAXV], gr[MAXV];
-  // 1. step gradient of this row; the masked gradient is kept for step 3
+  float4 wr[NV], gr[NV], mr[NV], vr[NV];
+  const float4* m4c = reinterpret_cast<const float4*>(m + base);
+  const float4* v4c = reinterpret_cast<const float4*>(v + base);
+  // 1. step gradient of this row; the masked gradient is kept for step 3.  The moments are fetched now
+  //    as well, so that their latency hides behind the reduction and the step's own update.
   float ds = 0.f;
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < MAXV; ++i) {
+    for (int i = 0; i < NV; ++i) {
       const int c = threadIdx.x + i * 256;
-      if (c < nvec) { wr[i] = w4[c]; gr[i] = g4[c]; }
+      if (c < nvec) {
+        wr[i] = w4[c]; gr[i] = g4[c];
+        if (train_w) { mr[i] = m4c[c]; vr[i] = v4c[c]; }
+      }
     }
   }
 #pragma unroll
-  for (int i = 0; i < MAXV; ++i) {
+  for (int i = 0; i < NV; ++i) {
     const int c = threadIdx.x + i * 256;
     if (cached && c < nvec) {
       bool in;
@@ -114,9 +120,8 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   float4* m4 = reinterpret_cast<float4*>(m + base);
   float4* v4 = reinterpret_cast<float4*>(v + base);
   int sum = 0;
-  auto update = [&](int c, float4 wv, float4 d) {
+  auto update = [&](int c, float4 wv, float4 d, float4 mm, float4 vv) {
     if (train_w) {
-      float4 mm = m4[c], vv = v4[c];
       wv.x = adam_one(wv.x, d.x, mm.x, vv.x, o, 1.f, -INFINITY);
       wv.y = adam_one(wv.y, d.y, mm.y, vv.y, o, 1.f, -INFINITY);
       wv.z = adam_one(wv.z, d.z, mm.z, vv.z, o, 1.f, -INFINITY);
@@ -134,9 +139,9 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   };
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < MAXV; ++i) {
+    for (int i = 0; i < NV; ++i) {
       const int c = threadIdx.x + i * 256;
-      if (c < nvec) update(c, wr[i], gr[i]);
+      if (c < nvec) update(c, wr[i], gr[i], mr[i], vr[i]);
     }
   } else {
     for (int c = threadIdx.x; c < nvec; c += 256) {
@@ -150,7 +155,7 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
         weight_ste(__fdiv_rn(wv.z, s_old), qmax, grid, in, lvl); d.z = in ? d.z : 0.f;
         weight_ste(__fdiv_rn(wv.w, s_old), qmax, grid, in, lvl); d.w = in ? d.w : 0.f;
       }
-      update(c, wv, d);
+      update(c, wv, d, train_w ? m4[c] : make_float4(0, 0, 0, 0), train_w ? v4[c] : make_float4(0, 0, 0, 0));
     }
   }
   sum = warp_sum_i(sum);
@@ -173,10 +178,10 @@ void launch_fused_weight_update(float* w, const float* g, float* m, float* v, fl
                                 int train_w, int train_s, int8_t* codes, int32_t* rowsum, float* scale, void* what,
                                 int dt, cudaStream_t st) {
   Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
-  if (dt == 1)
-    launch_k(fused_weight_update_kernel<bf16>, rows, 256, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (bf16*)what);
-  else
-    launch_k(fused_weight_update_kernel<float>, rows, 256, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (float*)what);
+#define MREM_FWU(T, NV) launch_k(fused_weight_update_kernel<T, NV>, rows, 256, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (T*)what)
+  if (dt == 1) { if (cols <= 1024) MREM_FWU(bf16, 1); else MREM_FWU(bf16, 4); }
+  else { if (cols <= 1024) MREM_FWU(float, 1); else MREM_FWU(float, 4); }
+#undef MREM_FWU
 }
 
 }  // namespace mrem
