@@ -184,6 +184,14 @@ int32_t mrem_recon_step_host(mrem_ctx* ctx, const void* h_x_teacher, const void*
  * Turn it off (0) to get plain stream-ordered launches, e.g. when comparing timings. */
 int32_t mrem_set_programmatic_launch(int32_t on);
 
+/* Per context (default on): where the shapes allow it (bf16 storage, head size 64, seq <= 128, seq % 8 == 0)
+ * the backward of the attention block (Sec. 3.1: the gradients of Q, K, V through the quantized scores,
+ * softmax and context products, with the straight-through masks of the Q, K, V, P quantizers) runs as one
+ * kernel; off (0) selects the kernel-per-operation path that covers every shape.  Both compute the same
+ * quantities; they differ in where intermediates are rounded to the storage type.  Do not change it
+ * between the capture and the replay of a graph. */
+int32_t mrem_set_fused_attention_backward(mrem_ctx* ctx, int32_t on);
+
 /* Reads the device status word (blocks on the stream): MREM_OK, MREM_ERR_TIMEOUT or MREM_ERR_NONFINITE in
  * *h_status; the word is cleared. */
 int32_t mrem_poll_status(mrem_ctx* ctx, int32_t* h_status);

@@ -32,6 +32,7 @@ EXPORTS = (
     "mrem_import_state", "mrem_graph_capture_step", "mrem_graph_launch", "mrem_gather_rows", "mrem_quantize_act",
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
+    "mrem_set_fused_attention_backward",
 )
 
 
@@ -140,6 +141,10 @@ def mrem_init_act_steps(ctx, x, valid_len, batch, seq):
 
 def mrem_set_programmatic_launch(on):
     _check(lib().mrem_set_programmatic_launch(int(on)), "mrem_set_programmatic_launch")
+
+
+def mrem_set_fused_attention_backward(ctx, on):
+    _check(lib().mrem_set_fused_attention_backward(ctx, int(on)), "mrem_set_fused_attention_backward", ctx)
 
 
 def mrem_invalidate_weight_codes(ctx):

@@ -56,6 +56,16 @@ int launch_attention_fwd(const void* qkv, int B, int S, int h, int H, const int*
                          const float* p_step, int p_lo, int p_hi, void* P, void* P_qt, void* ctx, const float* c_step,
                          int c_qmax, int8_t* ctx_q8, void* ctx_qt, int* status, cudaStream_t st);
 
+// Fused attention backward of the student on the tensor cores (bf16 storage, head size 64, seq <= 128,
+// seq % 8 == 0, batch * heads <= RED_BLOCKS): from the context gradient to the masked gradients of
+// the pre-quantization Q, K, V ([B*S, 3H]) with the step-size partials of the Q, K, V, P sites
+// (RED_BLOCKS slots each; unused slots are zeroed).  Returns a GemmRc.
+bool attention_bwd_supported(int S, int head_dim, int dt, int batch_heads);
+int launch_attention_bwd(const void* qkv_codes, const void* qkv, const void* P, const void* dctx, int B, int S, int h,
+                         int H, const float* s_q, const float* s_k, const float* s_v, const float* s_p, int q_lo,
+                         int q_hi, int p_lo, int p_hi, void* dqkv, float* part_q, float* part_k, float* part_v,
+                         float* part_p, int* status, cudaStream_t st);
+
 // ---- loss (Eq. 3)
 // partial[l][block] = sum (f_hat - f)^2 over the block's share; dF = 2 c (f_hat - f).
 void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per_layer, float c, void* dF,

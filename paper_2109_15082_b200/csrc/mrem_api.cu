@@ -383,6 +383,12 @@ int32_t mrem_set_programmatic_launch(int32_t on) {
   return MREM_OK;
 }
 
+int32_t mrem_set_fused_attention_backward(mrem_ctx* c, int32_t on) {
+  if (!c) return MREM_ERR_ARG;
+  c->fused_attention_bwd = on != 0;
+  return MREM_OK;
+}
+
 int32_t mrem_poll_status(mrem_ctx* c, int32_t* h_status) {
   if (!c || !h_status) return MREM_ERR_ARG;
   int v = 0;

@@ -100,6 +100,7 @@ struct mrem_ctx {
   mrem::AdamEntry* adam_table;       int adam_entries = 0;  long long adam_elems = 0;   // every trainable tensor
   mrem::AdamEntry* adam_rest;        int rest_entries = 0;  long long rest_elems = 0;   // all but matrices and their steps
   bool w_ste_done = false;           // the weight gradients have been masked and the step gradients reduced
+  bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;
   void *h2d_xt, *h2d_xs; int32_t* h2d_len; float* d_loss_e2e;   // staging of mrem_recon_step_host

@@ -273,18 +273,25 @@ int student_backward(mrem_ctx* c) {
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
                    part + S_C * RED_BLOCKS, nullptr, c->dt, st);
     // attention:  ctx = P_hat V_hat,  P = softmax(Q_hat K_hat^T / sqrt(d))
-    r.gemm(view(c->d_ctx, H, 0, hd, (long long)S * H), view(r.at(s.qkv_qt, 2 * H), 3 * H, 0, hd, sQKV), S, S, hd, h, B,
-           Epi(c->d_phat, ok, S, sSS, sHSS).alpha(1.f, b.a_steps[S_V]).e);
-    r.gemm(view(s.P_qt, S, 1, sSS, sHSS), view(c->d_ctx, H, 1, hd, (long long)S * H), S, hd, S, h, B,
-           Epi(r.at(c->d_qkvhat, 2 * H), ok, 3 * H, hd, sQKV).alpha(1.f, b.a_steps[S_P]).e);
-    launch_softmax_bwd(s.P, c->d_phat, c->d_s, (long long)B * h * S, S, b.a_steps[S_P], rp.lo, rp.hi, 1, part + S_P * RED_BLOCKS, c->dt, st);
-    r.gemm(view(c->d_s, S, 0, sSS, sHSS), view(r.at(s.qkv_qt, H), 3 * H, 1, hd, sQKV), S, hd, S, h, B,
-           Epi(c->d_qkvhat, ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_K]).e);
-    r.gemm(view(c->d_s, S, 1, sSS, sHSS), view(s.qkv_qt, 3 * H, 1, hd, sQKV), S, hd, S, h, B,
-           Epi(r.at(c->d_qkvhat, H), ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_Q]).e);
-    for (int seg = 0; seg < 3; ++seg)
-      launch_ste_act(r.at(s.qkv, seg * H), 3 * H, r.at(c->d_qkvhat, seg * H), 3 * H, nullptr, 0, r.at(c->d_qkv, seg * H), 3 * H, M, H,
-                     b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, part + (S_Q + seg) * RED_BLOCKS, nullptr, c->dt, st);
+    if (c->fused_attention_bwd && attention_bwd_supported(S, hd, c->dt, B * h)) {
+      r.note(launch_attention_bwd(s.qkv_qt, s.qkv, s.P, c->d_ctx, B, S, h, H, b.a_steps[S_Q], b.a_steps[S_K], b.a_steps[S_V],
+                                  b.a_steps[S_P], rx.lo, rx.hi, rp.lo, rp.hi, c->d_qkv, part + S_Q * RED_BLOCKS,
+                                  part + S_K * RED_BLOCKS, part + S_V * RED_BLOCKS, part + S_P * RED_BLOCKS, c->status, st),
+             "attention backward launch failed");
+    } else {
+      r.gemm(view(c->d_ctx, H, 0, hd, (long long)S * H), view(r.at(s.qkv_qt, 2 * H), 3 * H, 0, hd, sQKV), S, S, hd, h, B,
+             Epi(c->d_phat, ok, S, sSS, sHSS).alpha(1.f, b.a_steps[S_V]).e);
+      r.gemm(view(s.P_qt, S, 1, sSS, sHSS), view(c->d_ctx, H, 1, hd, (long long)S * H), S, hd, S, h, B,
+             Epi(r.at(c->d_qkvhat, 2 * H), ok, 3 * H, hd, sQKV).alpha(1.f, b.a_steps[S_P]).e);
+      launch_softmax_bwd(s.P, c->d_phat, c->d_s, (long long)B * h * S, S, b.a_steps[S_P], rp.lo, rp.hi, 1, part + S_P * RED_BLOCKS, c->dt, st);
+      r.gemm(view(c->d_s, S, 0, sSS, sHSS), view(r.at(s.qkv_qt, H), 3 * H, 1, hd, sQKV), S, hd, S, h, B,
+             Epi(c->d_qkvhat, ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_K]).e);
+      r.gemm(view(c->d_s, S, 1, sSS, sHSS), view(s.qkv_qt, 3 * H, 1, hd, sQKV), S, hd, S, h, B,
+             Epi(r.at(c->d_qkvhat, H), ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_Q]).e);
+      for (int seg = 0; seg < 3; ++seg)
+        launch_ste_act(r.at(s.qkv, seg * H), 3 * H, r.at(c->d_qkvhat, seg * H), 3 * H, nullptr, 0, r.at(c->d_qkv, seg * H), 3 * H, M, H,
+                       b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, part + (S_Q + seg) * RED_BLOCKS, nullptr, c->dt, st);
+    }
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
     launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);

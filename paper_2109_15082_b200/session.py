@@ -143,6 +143,9 @@ class ReconModule:
     def backward(self):
         B.mrem_module_backward(self.ctx)
 
+    def set_fused_attention_backward(self, on):
+        B.mrem_set_fused_attention_backward(self.ctx, on)
+
     def step(self, optim):
         B.mrem_step(self.ctx, optim)
 
