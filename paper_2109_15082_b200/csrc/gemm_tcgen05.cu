@@ -257,7 +257,12 @@ int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, in
 
 namespace {
 
-int pick_block_n(int M, int N, int batches, int sm_count) {
+// Tile width by a cost model fitted to event timings on the encoder shapes: a persistent CTA works through
+// `waves` tiles one after the other, a tile costs k_blocks main-loop steps plus an epilogue share that is
+// not hidden.  A step of a narrow tile is cheaper, but far from proportionally (the A tile is re-fetched
+// for every column block and the shared-memory traffic per flop grows), so wide tiles win unless they
+// leave most SMs idle.
+int pick_block_n(int M, int N, int k_blocks, int batches, int sm_count) {
   const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
   int best = 64;
   double best_cost = 1e30;
@@ -265,7 +270,9 @@ int pick_block_n(int M, int N, int batches, int sm_count) {
     if (bn > 64 && bn / 2 >= N) break;
     const long long tiles = (long long)m_tiles * ((N + bn - 1) / bn) * batches;
     const long long waves = (tiles + sm_count - 1) / sm_count;
-    const double cost = (double)waves * (bn + 40.0);     // 40: fixed per-tile cost in units of columns
+    const double step_us = bn == 64 ? 0.32 : (bn == 128 ? 0.43 : 0.50);
+    const double epi_us = bn == 64 ? 0.5 : (bn == 128 ? 1.0 : 2.0);
+    const double cost = (double)waves * (k_blocks * step_us + epi_us);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
   }
   return best;
@@ -281,7 +288,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   if (kind == 1 && (A.mn_contig || B.mn_contig)) return GEMM_ERR_ARG;
   TcParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.nb0 = g.nb0; p.nb1 = g.nb1;
-  p.block_n = block_n > 0 ? block_n : pick_block_n(g.M, g.N, g.nb0 * g.nb1, sm_count);
+  p.block_n = block_n > 0 ? block_n : pick_block_n(g.M, g.N, (g.K + 128 / es - 1) / (128 / es), g.nb0 * g.nb1, sm_count);
   if (p.block_n != 64 && p.block_n != 128 && p.block_n != 256) return GEMM_ERR_ARG;
   p.block_k = 128 / es;
   p.m_tiles = (g.M + BLOCK_M - 1) / BLOCK_M;
