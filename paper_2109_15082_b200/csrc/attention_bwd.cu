@@ -61,6 +61,7 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 __device__ __forceinline__ float ste_store(const uint32_t* a, bool row_ok, const bf16* x, bf16* out, float scale,
                                            float step, float lo, float hi) {
   float acc = 0.f;
+  const float r_step = __frcp_rn(step);
   if (row_ok) {
     uint32_t xw[16], ow[16];
 #pragma unroll
@@ -69,7 +70,7 @@ __device__ __forceinline__ float ste_store(const uint32_t* a, bool row_ok, const
     for (int j = 0; j < 16; ++j) {
       const float2 xv = unpack2(xw[j]);
       const float g0 = scale * __uint_as_float(a[2 * j]), g1 = scale * __uint_as_float(a[2 * j + 1]);
-      const float z0 = __fdiv_rn(xv.x, step), z1 = __fdiv_rn(xv.y, step);
+      const float z0 = quotient(xv.x, step, r_step), z1 = quotient(xv.y, step, r_step);
       const bool in0 = z0 >= lo && z0 <= hi, in1 = z1 >= lo && z1 <= hi;
       const float q0 = (float)__float2int_rn(fminf(fmaxf(z0, lo), hi));
       const float q1 = (float)__float2int_rn(fminf(fmaxf(z1, lo), hi));
@@ -165,6 +166,7 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
     const bool row_ok = r < p.S;
     const uint32_t trow = tmem + ((uint32_t)(quad * 32) << 16);
     const float s_p = *p.s_p, s_v = *p.s_v, s_q = *p.s_q, s_k = *p.s_k;
+    const float r_p = __frcp_rn(s_p);
     const int n_chunks = (p.S + 31) / 32;
     const long long prow = (((long long)b * p.h + head) * p.S + r) * p.S;
     float ds_p = 0.f;
@@ -187,7 +189,7 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
         for (int j = 0; j < 16; ++j) {
           const float2 pv = unpack2(pw[j]);
           float d0 = s_v * __uint_as_float(a[2 * j]), d1 = s_v * __uint_as_float(a[2 * j + 1]);
-          const float z0 = __fdiv_rn(pv.x, s_p), z1 = __fdiv_rn(pv.y, s_p);
+          const float z0 = quotient(pv.x, s_p, r_p), z1 = quotient(pv.y, s_p, r_p);
           const bool in0 = z0 >= p.p_lo && z0 <= p.p_hi, in1 = z1 >= p.p_lo && z1 <= p.p_hi;
           const float q0 = (float)__float2int_rn(fminf(fmaxf(z0, p.p_lo), p.p_hi));
           const float q1 = (float)__float2int_rn(fminf(fmaxf(z1, p.p_lo), p.p_hi));

@@ -117,7 +117,8 @@ void launch_effective_bias(const float* b, const float* beta, const float* wscal
                            int n, cudaStream_t st);
 
 // ---- optimizer (AdamW)
-struct OptimScalars { float lr, beta1, beta2, eps, bc1, bc2, weight_decay; };   // bc = 1 - beta^t
+// bc = 1 - beta^t; lr_bc1 = lr / bc1, rsqrt_bc2 = 1 / sqrt(bc2)
+struct OptimScalars { float lr, beta1, beta2, eps, bc1, bc2, weight_decay, lr_bc1, rsqrt_bc2; };
 struct AdamEntry { float* p; const float* g; float* m; float* v; long long n; float wd; float min_value; };   // wd: 1 = decayed
 // Computes the scalars of this step on the device: t = ++(*d_t) (or host_t when >= 1),
 // lr = lr0 * (1 - (t-1)/total) when total > 0 else lr0.

@@ -10,8 +10,9 @@ namespace mrem {
 
 namespace {
 
-__device__ __forceinline__ float qz(float x, float s, float off, bool has_off) {
-  return __fdiv_rn(has_off ? __fsub_rn(x, off) : x, s);
+// (x - offset) / step for the straight-through factors (see quotient)
+__device__ __forceinline__ float qz(float x, float s, float r_s, float off, bool has_off) {
+  return quotient(has_off ? __fsub_rn(x, off) : x, s, r_s);
 }
 __device__ __forceinline__ int qcode(float z, float lo, float hi) { return __float2int_rn(fminf(fmaxf(z, lo), hi)); }
 
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, l
   pdl_trigger();
   pdl_wait();
   __shared__ float sh[32];
-  const float s = *step;
+  const float s = *step, r_s = __frcp_rn(s);
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
   const int vcols = cols / V;
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, l
     load_vec<T, V>(dxhat + r * ld_d + c, d);
 #pragma unroll
     for (int j = 0; j < V; ++j) {
-      const float z = qz(xv[j], s, off, has_off);
+      const float z = qz(xv[j], s, r_s, off, has_off);
       const bool in = z >= lo && z <= hi;
       ds += d[j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
       dofs += in ? 0.f : d[j];
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
   pdl_trigger();
   pdl_wait();
   __shared__ float sh[32];
-  const float s = quantized ? *step : 1.f;
+  const float s = quantized ? *step : 1.f, r_s = __frcp_rn(s);
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
   float ds = 0.f, dofs = 0.f;
@@ -128,14 +129,16 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
     load_vec<T, V>(dghat + i, d);
 #pragma unroll
     for (int j = 0; j < V; ++j) {
+      float cdf, pdf;
+      gelu_parts(uv[j], cdf, pdf);
       if (quantized) {
-        const float z = qz(stored<T>(gelu_erf(uv[j])), s, off, has_off);
+        const float z = qz(stored<T>(uv[j] * cdf), s, r_s, off, has_off);
         const bool in = z >= lo && z <= hi;
         ds += d[j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
         dofs += in ? 0.f : d[j];
         d[j] = in ? d[j] : 0.f;
       }
-      d[j] *= gelu_erf_grad(uv[j]);
+      d[j] *= fmaf(uv[j], pdf, cdf);
     }
     store_vec<T, V>(du + i, d);
   }
@@ -156,6 +159,7 @@ __global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict
   __shared__ float sh[32];
   const int row = blockIdx.x;
   const float s = steps[per_row ? row : 0];
+  const float r_s = __frcp_rn(s);
   const float qmax = (float)((1 << (bits - 1)) - 1);
   const float4* wr = reinterpret_cast<const float4*>(w + (long long)row * cols);
   float4* dr = reinterpret_cast<float4*>(dw + (long long)row * cols);
@@ -164,10 +168,10 @@ __global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict
     const float4 wv = wr[c];
     float4 d = dr[c];
     bool in;
-    ds = step_grad_acc(ds, wv.x, d.x, s, qmax, grid, in); d.x = in ? d.x : 0.f;
-    ds = step_grad_acc(ds, wv.y, d.y, s, qmax, grid, in); d.y = in ? d.y : 0.f;
-    ds = step_grad_acc(ds, wv.z, d.z, s, qmax, grid, in); d.z = in ? d.z : 0.f;
-    ds = step_grad_acc(ds, wv.w, d.w, s, qmax, grid, in); d.w = in ? d.w : 0.f;
+    ds = step_grad_acc(ds, wv.x, d.x, s, r_s, qmax, grid, in); d.x = in ? d.x : 0.f;
+    ds = step_grad_acc(ds, wv.y, d.y, s, r_s, qmax, grid, in); d.y = in ? d.y : 0.f;
+    ds = step_grad_acc(ds, wv.z, d.z, s, r_s, qmax, grid, in); d.z = in ? d.z : 0.f;
+    ds = step_grad_acc(ds, wv.w, d.w, s, r_s, qmax, grid, in); d.w = in ? d.w : 0.f;
     dr[c] = d;
   }
   ds = block_sum(ds, sh);
@@ -216,6 +220,8 @@ __global__ void optim_prepare_kernel(OptimScalars* out, int* d_t, int host_t, fl
   o.weight_decay = wd;
   o.bc1 = (float)(1.0 - pow((double)b1, (double)t));
   o.bc2 = (float)(1.0 - pow((double)b2, (double)t));
+  o.lr_bc1 = (float)((double)o.lr / (1.0 - pow((double)b1, (double)t)));
+  o.rsqrt_bc2 = (float)(1.0 / sqrt(1.0 - pow((double)b2, (double)t)));
   *out = o;
 }
 

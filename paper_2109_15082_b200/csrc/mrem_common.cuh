@@ -95,9 +95,46 @@ __device__ __forceinline__ float block_max(float v, float* sh) {
 }
 
 // ---------------------------------------------------------------- math
-__device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.f + erff(u * 0.70710678118654752f)); }
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// x / s from r_s = RN(1/s): one product, the exact residual by FMA, one correction.  Equals the correctly
+// rounded quotient except where x/s lies within ~2^-48 (relative) of the midpoint of two floats; a value
+// sitting exactly on a clipping boundary gets the same side as the quantizer's IEEE division.  Used where
+// the quotient feeds a straight-through factor (a surrogate gradient); the codes themselves are always
+// produced with the IEEE division of Eq. 1.
+__device__ __forceinline__ float quotient(float x, float s, float r_s) {
+  const float z0 = __fmul_rn(x, r_s);
+  return __fmaf_rn(__fmaf_rn(-z0, s, x), r_s, z0);
+}
+
+// GELU(u) = u * Phi(u) with the erf form.  erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x), x >= 0
+// (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7, below half a float32 ulp of 1 + erf for u > 0): one
+// exponential serves both erf and the density needed by the derivative.
+__device__ __forceinline__ void gelu_parts(float u, float& cdf, float& pdf_scaled) {
+  const float x = fabsf(u) * 0.70710678118654752f;
+  const float ex = __expf(-x * x);                          // exp(-u^2 / 2)
+  const float t = rcp_approx(fmaf(0.3275911f, x, 1.f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float tail = 0.5f * poly * t * ex;                  // (1 - erf(x)) / 2
+  cdf = u >= 0.f ? 1.f - tail : tail;
+  pdf_scaled = ex * 0.39894228040143268f;                   // exp(-u^2/2) / sqrt(2 pi)
+}
+__device__ __forceinline__ float gelu_erf(float u) {
+  float cdf, pdf;
+  gelu_parts(u, cdf, pdf);
+  return u * cdf;
+}
 __device__ __forceinline__ float gelu_erf_grad(float u) {
-  return 0.5f * (1.f + erff(u * 0.70710678118654752f)) + u * expf(-0.5f * u * u) * 0.39894228040143268f;
+  float cdf, pdf;
+  gelu_parts(u, cdf, pdf);
+  return fmaf(u, pdf, cdf);
 }
 
 // ---------------------------------------------------------------- GEMM interface (both back ends)

@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ 
   __shared__ float sh[32];
   const int lane = threadIdx.x & 31;
   const long long warp0 = blockIdx.x * 8ll + (threadIdx.x >> 5), nwarps = gridDim.x * 8ll;
-  const float s = quantized ? *step : 1.f;
+  const float s = quantized ? *step : 1.f, r_s = __frcp_rn(s);
   float ds = 0.f;
   for (long long row = warp0; row < rows; row += nwarps) {
     const long long base = row * S;
@@ -381,7 +381,7 @@ __global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ 
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             if (quantized) {
-              const float z = __fdiv_rn(p[i][j], s);
+              const float z = quotient(p[i][j], s, r_s);
               const bool in = z >= lo && z <= hi;
               ds += d[i][j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
               d[i][j] = in ? d[i][j] : 0.f;
@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ 
         const float p = to_f<T>(P[base + j]);
         float d = to_f<T>(dphat[base + j]);
         if (quantized) {
-          const float z = __fdiv_rn(p, s);
+          const float z = quotient(p, s, r_s);
           const bool in = z >= lo && z <= hi;
           ds += d * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
           d = in ? d : 0.f;
@@ -418,7 +418,7 @@ __global__ void __launch_bounds__(256) softmax_bwd_kernel(const T* __restrict__ 
         const float p = to_f<T>(P[base + j]);
         float d = to_f<T>(dphat[base + j]);
         if (quantized) {
-          const float z = __fdiv_rn(p, s);
+          const float z = quotient(p, s, r_s);
           d = (z >= lo && z <= hi) ? d : 0.f;
         }
         dS[base + j] = from_f<T>(p * (d - dot));

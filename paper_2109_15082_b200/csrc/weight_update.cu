@@ -38,9 +38,10 @@ __device__ __forceinline__ void store_what4<bf16>(bf16* p, float a, float b, flo
   *reinterpret_cast<uint2*>(p) = t;
 }
 
-// NV = float4 vectors per thread kept in registers: 1 for rows up to 1024 wide, 4 up to 4096; wider rows are re-read.
-template <typename T, int NV>
-__global__ void __launch_bounds__(256) fused_weight_update_kernel(
+// NT threads per row, NV float4 vectors per thread kept in registers: (256, 1) for rows up to 1024 wide,
+// (512, 2) up to 4096; wider rows are re-read.
+template <typename T, int NV, int NT>
+__global__ void __launch_bounds__(NT, 1024 / NT) fused_weight_update_kernel(
     float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v,
     float* __restrict__ steps, const float* __restrict__ ds_in, float* __restrict__ m_s, float* __restrict__ v_s,
     const OptimScalars* __restrict__ sc, int cols, int bits, int grid, int train_w, int train_s,
@@ -53,10 +54,11 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   const int row = blockIdx.x;
   const OptimScalars o = *sc;
   const float s_old = steps[row];
+  const float r_old = __frcp_rn(s_old);
   const float qmax = (float)((1 << (bits - 1)) - 1);
   const long long base = (long long)row * cols;
   const int nvec = cols / 4;                                   // cols is a multiple of 16
-  const bool cached = nvec <= NV * 256;
+  const bool cached = nvec <= NV * NT;
   const float4* w4 = reinterpret_cast<const float4*>(w + base);
   const float4* g4 = reinterpret_cast<const float4*>(g + base);
   float4 wr[NV], gr[NV], mr[NV], vr[NV];
@@ -68,7 +70,7 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   if (cached) {
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
-      const int c = threadIdx.x + i * 256;
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) {
         wr[i] = w4[c]; gr[i] = g4[c];
         if (train_w) { mr[i] = m4c[c]; vr[i] = v4c[c]; }
@@ -77,25 +79,25 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   }
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
-    const int c = threadIdx.x + i * 256;
+    const int c = threadIdx.x + i * NT;
     if (cached && c < nvec) {
       bool in;
       float4 d = gr[i];
-      ds = step_grad_acc(ds, wr[i].x, d.x, s_old, qmax, grid, in); d.x = (in || ds_in) ? d.x : 0.f;
-      ds = step_grad_acc(ds, wr[i].y, d.y, s_old, qmax, grid, in); d.y = (in || ds_in) ? d.y : 0.f;
-      ds = step_grad_acc(ds, wr[i].z, d.z, s_old, qmax, grid, in); d.z = (in || ds_in) ? d.z : 0.f;
-      ds = step_grad_acc(ds, wr[i].w, d.w, s_old, qmax, grid, in); d.w = (in || ds_in) ? d.w : 0.f;
+      ds = step_grad_acc(ds, wr[i].x, d.x, s_old, r_old, qmax, grid, in); d.x = (in || ds_in) ? d.x : 0.f;
+      ds = step_grad_acc(ds, wr[i].y, d.y, s_old, r_old, qmax, grid, in); d.y = (in || ds_in) ? d.y : 0.f;
+      ds = step_grad_acc(ds, wr[i].z, d.z, s_old, r_old, qmax, grid, in); d.z = (in || ds_in) ? d.z : 0.f;
+      ds = step_grad_acc(ds, wr[i].w, d.w, s_old, r_old, qmax, grid, in); d.w = (in || ds_in) ? d.w : 0.f;
       gr[i] = d;
     }
   }
   if (!cached) {
-    for (int c = threadIdx.x; c < nvec; c += 256) {
+    for (int c = threadIdx.x; c < nvec; c += NT) {
       const float4 wv = w4[c], d = g4[c];
       bool in;
-      ds = step_grad_acc(ds, wv.x, d.x, s_old, qmax, grid, in);
-      ds = step_grad_acc(ds, wv.y, d.y, s_old, qmax, grid, in);
-      ds = step_grad_acc(ds, wv.z, d.z, s_old, qmax, grid, in);
-      ds = step_grad_acc(ds, wv.w, d.w, s_old, qmax, grid, in);
+      ds = step_grad_acc(ds, wv.x, d.x, s_old, r_old, qmax, grid, in);
+      ds = step_grad_acc(ds, wv.y, d.y, s_old, r_old, qmax, grid, in);
+      ds = step_grad_acc(ds, wv.z, d.z, s_old, r_old, qmax, grid, in);
+      ds = step_grad_acc(ds, wv.w, d.w, s_old, r_old, qmax, grid, in);
     }
   }
   ds = block_sum(ds, sh);
@@ -140,20 +142,20 @@ __global__ void __launch_bounds__(256) fused_weight_update_kernel(
   if (cached) {
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
-      const int c = threadIdx.x + i * 256;
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) update(c, wr[i], gr[i], mr[i], vr[i]);
     }
   } else {
-    for (int c = threadIdx.x; c < nvec; c += 256) {
+    for (int c = threadIdx.x; c < nvec; c += NT) {
       const float4 wv = w4[c];
       float4 d = g4[c];
       if (!ds_in) {
         bool in;
         float lvl;
-        weight_ste(__fdiv_rn(wv.x, s_old), qmax, grid, in, lvl); d.x = in ? d.x : 0.f;
-        weight_ste(__fdiv_rn(wv.y, s_old), qmax, grid, in, lvl); d.y = in ? d.y : 0.f;
-        weight_ste(__fdiv_rn(wv.z, s_old), qmax, grid, in, lvl); d.z = in ? d.z : 0.f;
-        weight_ste(__fdiv_rn(wv.w, s_old), qmax, grid, in, lvl); d.w = in ? d.w : 0.f;
+        weight_ste(quotient(wv.x, s_old, r_old), qmax, grid, in, lvl); d.x = in ? d.x : 0.f;
+        weight_ste(quotient(wv.y, s_old, r_old), qmax, grid, in, lvl); d.y = in ? d.y : 0.f;
+        weight_ste(quotient(wv.z, s_old, r_old), qmax, grid, in, lvl); d.z = in ? d.z : 0.f;
+        weight_ste(quotient(wv.w, s_old, r_old), qmax, grid, in, lvl); d.w = in ? d.w : 0.f;
       }
       update(c, wv, d, train_w ? m4[c] : make_float4(0, 0, 0, 0), train_w ? v4[c] : make_float4(0, 0, 0, 0));
     }
@@ -178,9 +180,9 @@ void launch_fused_weight_update(float* w, const float* g, float* m, float* v, fl
                                 int train_w, int train_s, int8_t* codes, int32_t* rowsum, float* scale, void* what,
                                 int dt, cudaStream_t st) {
   Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
-#define MREM_FWU(T, NV) launch_k(fused_weight_update_kernel<T, NV>, rows, 256, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (T*)what)
-  if (dt == 1) { if (cols <= 1024) MREM_FWU(bf16, 1); else MREM_FWU(bf16, 4); }
-  else { if (cols <= 1024) MREM_FWU(float, 1); else MREM_FWU(float, 4); }
+#define MREM_FWU(T, NV, NT) launch_k(fused_weight_update_kernel<T, NV, NT>, rows, NT, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (T*)what)
+  if (dt == 1) { if (cols <= 1024) MREM_FWU(bf16, 1, 256); else MREM_FWU(bf16, 2, 512); }
+  else { if (cols <= 1024) MREM_FWU(float, 1, 256); else MREM_FWU(float, 2, 512); }
 #undef MREM_FWU
 }
 
