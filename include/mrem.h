@@ -170,6 +170,14 @@ int32_t mrem_get_grad(mrem_ctx* ctx, int32_t layer, int32_t id, const float** d_
  * each matrix also re-quantizes it (Eq. 1 with the new weights and steps), so the next
  * mrem_quantize_weights has nothing left to do. */
 int32_t mrem_step(mrem_ctx* ctx, const mrem_optim* optim);
+/* mrem_module_backward and mrem_step as one call (the last two lines of Algorithm 2's inner loop).  With per-row
+ * weight steps the matrices of a layer are updated, on a second stream the context owns, as soon as that
+ * layer's gradients are complete, while the backward pass continues below it; the context's stream waits
+ * for those updates before the call's work is considered done, so callers keep ordering everything on
+ * their one stream.  Same kernels on the same data as the two separate calls: bitwise the same result.
+ * The gradients are consumed: mrem_get_grad is not available afterwards.  mrem_recon_step_host and the
+ * captured step use this form. */
+int32_t mrem_backward_and_step(mrem_ctx* ctx, const mrem_optim* optim);
 
 /* The whole step from HOST buffers: copies h_x_teacher / h_x_student ([batch, seq, hidden] act_dtype;
  * h_x_student may equal h_x_teacher) and h_valid_len (may be NULL) to the device, runs quantize_weights,

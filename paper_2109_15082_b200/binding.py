@@ -32,7 +32,7 @@ EXPORTS = (
     "mrem_import_state", "mrem_graph_capture_step", "mrem_graph_launch", "mrem_gather_rows", "mrem_quantize_act",
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
-    "mrem_set_fused_attention_backward",
+    "mrem_set_fused_attention_backward", "mrem_backward_and_step",
 )
 
 
@@ -183,6 +183,10 @@ def mrem_get_grad(ctx, layer, grad_id) -> int:
 
 def mrem_step(ctx, optim):
     _check(lib().mrem_step(ctx, C.byref(optim)), "mrem_step", ctx)
+
+
+def mrem_backward_and_step(ctx, optim):
+    _check(lib().mrem_backward_and_step(ctx, C.byref(optim)), "mrem_backward_and_step", ctx)
 
 
 def mrem_recon_step_host(ctx, h_x_teacher, h_x_student, h_valid_len, batch, seq, lam, optim) -> float:

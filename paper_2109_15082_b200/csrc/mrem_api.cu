@@ -247,6 +247,14 @@ int32_t mrem_create(const mrem_module_desc* desc, void* workspace, size_t worksp
   }
   if (cudaMemsetAsync(workspace, 0, need, c->stream) != cudaSuccess) { delete c; return fail(nullptr, MREM_ERR_CUDA, "memset failed"); }
   if (cudaMallocHost((void**)&c->h_pinned_loss, 256) != cudaSuccess) { delete c; return fail(nullptr, MREM_ERR_CUDA, "pinned alloc failed"); }
+  int pri_lo = 0, pri_hi = 0;
+  if (cudaDeviceGetStreamPriorityRange(&pri_lo, &pri_hi) != cudaSuccess ||
+      cudaStreamCreateWithPriority(&c->side_stream, cudaStreamNonBlocking, pri_lo) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    mrem_destroy(c);
+    return fail(nullptr, MREM_ERR_CUDA, "stream or event creation failed");
+  }
   *out = c;
   return MREM_OK;
 }
@@ -256,6 +264,9 @@ int32_t mrem_destroy(mrem_ctx* c) {
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   if (c->graph) cudaGraphDestroy(c->graph);
   if (c->h_pinned_loss) cudaFreeHost(c->h_pinned_loss);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->side_stream) cudaStreamDestroy(c->side_stream);
   delete c;
   return MREM_OK;
 }

@@ -100,6 +100,10 @@ struct mrem_ctx {
   mrem::AdamEntry* adam_table;       int adam_entries = 0;  long long adam_elems = 0;   // every trainable tensor
   mrem::AdamEntry* adam_rest;        int rest_entries = 0;  long long rest_elems = 0;   // all but matrices and their steps
   bool w_ste_done = false;           // the weight gradients have been masked and the step gradients reduced
+  // second stream (lowest priority) and its fork/join events: the memory-bound weight updates of a layer
+  // run there while the main stream goes on with the tensor-core work of the layer below
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;

@@ -19,8 +19,7 @@ int enqueue_step(mrem_ctx* c, const void* xt, const void* xs, float lambda, cons
   if (rc == MREM_OK) rc = mrem_module_forward(c, MREM_TEACHER, xt, nullptr, 0.f, len, batch, seq, t_out);
   if (rc == MREM_OK) rc = mrem_module_forward(c, MREM_STUDENT, xs, xt, lambda, len, batch, seq, s_out);
   if (rc == MREM_OK) rc = mrem_recon_loss(c, d_loss, nullptr);
-  if (rc == MREM_OK) rc = mrem_module_backward(c);
-  if (rc == MREM_OK) rc = mrem_step(c, o);
+  if (rc == MREM_OK) rc = mrem_backward_and_step(c, o);
   return rc;
 }
 

@@ -42,7 +42,9 @@ struct Epi {                       // shorthand builder of an Epilogue
 struct Runner {
   mrem_ctx* c;
   int rc = MREM_OK;
-  explicit Runner(mrem_ctx* ctx) : c(ctx) {}
+  cudaStream_t st;
+  explicit Runner(mrem_ctx* ctx) : c(ctx), st(ctx->stream) {}
+  Runner(mrem_ctx* ctx, cudaStream_t stream) : c(ctx), st(stream) {}
   int okind() const { return c->dt == 1 ? OUT_BF16 : OUT_F32; }
   void* at(const void* p, long long elems) const { return (char*)p + elems * (long long)c->esz; }
 
@@ -56,14 +58,14 @@ struct Runner {
   void gemm(const View& A, const View& B, int M, int N, int K, int nb0, int nb1, const Epilogue& e) {
     OperandDesc a{A.p, A.ld, A.sb0, A.sb1, A.mn}, b{B.p, B.ld, B.sb0, B.sb1, B.mn};
     GemmShape g{M, N, K, nb0, nb1};
-    if (c->dt == 1) note(tc_gemm(0, 0, a, b, g, e, 0, c->status, c->sm_count, c->stream), "bf16 GEMM launch failed");
-    else note(simt_gemm_f32(a, b, g, e, c->stream), "f32 GEMM launch failed");
+    if (c->dt == 1) note(tc_gemm(0, 0, a, b, g, e, 0, c->status, c->sm_count, st), "bf16 GEMM launch failed");
+    else note(simt_gemm_f32(a, b, g, e, st), "f32 GEMM launch failed");
   }
   // integer-code product with exact int32 accumulation
   void gemm_i8(const int8_t* A, int a_unsigned, const int8_t* B, int M, int N, int K, const Epilogue& e) {
     OperandDesc a{A, K, 0, 0, 0}, b{B, K, 0, 0, 0};
     GemmShape g{M, N, K, 1, 1};
-    note(tc_gemm(1, a_unsigned, a, b, g, e, 0, c->status, c->sm_count, c->stream), "int8 GEMM launch failed");
+    note(tc_gemm(1, a_unsigned, a, b, g, e, 0, c->status, c->sm_count, st), "int8 GEMM launch failed");
   }
 };
 
@@ -222,13 +224,46 @@ int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S
   return cudaGetLastError() == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "student forward: launch failed");
 }
 
+// The fused update of one layer's four matrices and their row steps (Algorithm 2: Update(w), Update(s)).
+void enqueue_matrix_updates(mrem_ctx* c, int l, cudaStream_t st) {
+  const mrem_module_desc& d = c->d;
+  const int train_w = (d.trainable_mask & MREM_TRAIN_WEIGHTS) != 0, train_s = (d.trainable_mask & MREM_TRAIN_W_STEPS) != 0;
+  for (int k = 0; k < N_WMAT; ++k) {
+    const int pid = kMatParam[k];
+    WeightBuf& w = c->wq[l][k];
+    LayerGrad& g = c->grad[l];
+    launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
+                               c->w_ste_done ? g.ws[k] : nullptr, g.m_ws[k], g.v_ws[k], c->optim_sc, w.rows, w.cols,
+                               d.w_bits, d.w_grid, train_w, train_s, w.codes, w.rowsum, w.scale, w.what, c->dt, st);
+  }
+}
+
 // ------------------------------------------------------------------ backward
-int student_backward(mrem_ctx* c) {
+// Two streams: the weight-gradient products (tensor-core bound, results needed only by the update) are
+// issued on the side stream and run under the main stream's element-wise and row kernels (memory bound);
+// the main stream waits for them before the next layer reuses the gradient buffers they read.  With
+// `update_as_you_go` (per-row steps; the optimizer scalars of this step are already on the device) each
+// layer's matrices are also updated on the side stream as soon as their gradients are complete.  The main
+// stream joins the side stream before returning.  While kernels are being timed one by one (tracing) all
+// of it stays on the main stream.
+int student_backward(mrem_ctx* c, bool update_as_you_go) {
   const mrem_module_desc& d = c->d;
   const int H = d.hidden, F = d.ffn, h = d.n_heads, hd = H / h, B = c->cur_batch, S = c->cur_seq;
   const long long M = (long long)B * S;
   const long long sSS = (long long)S * S, sHSS = (long long)h * S * S, sQKV = (long long)S * 3 * H;
   Runner r(c);
+  const bool two_streams = c->side_stream && !c->trace_on;
+  cudaStream_t side = two_streams ? c->side_stream : c->stream;
+  Runner rw(c, side);                            // weight-gradient products
+  bool sync_failed = false;
+  auto fork = [&]() {                            // side stream: wait for what the main stream has enqueued so far
+    if (two_streams && (cudaEventRecord(c->ev_fork, c->stream) != cudaSuccess || cudaStreamWaitEvent(side, c->ev_fork, 0) != cudaSuccess))
+      sync_failed = true;
+  };
+  auto join = [&]() {                            // main stream: wait for what the side stream has enqueued so far
+    if (two_streams && (cudaEventRecord(c->ev_join, side) != cudaSuccess || cudaStreamWaitEvent(c->stream, c->ev_join, 0) != cudaSuccess))
+      sync_failed = true;
+  };
   const int ok = r.okind();
   const float inv_sqrt_d = 1.f / sqrtf((float)hd);
   const void* carry = nullptr;
@@ -253,14 +288,16 @@ int student_backward(mrem_ctx* c) {
       Epi e(g.p[MREM_W2], OUT_F32, F);
       e.alpha(1.f, b.a_steps[S_G]);
       if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], c->rowbias, H, st); e.rowbias(c->rowbias); }
-      r.gemm(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, 1, 1, e.e);
+      fork();
+      rw.gemm(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, 1, 1, e.e);
     }
     launch_gelu_bwd(s.u, c->d_ghat, c->d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
                     part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
     // FFN1:  u = A_hat W1_hat^T + b1
     launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
-    r.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
+    fork();
+    rw.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
                    part + S_A * RED_BLOCKS, nullptr, c->dt, st);
     // first LayerNorm
@@ -269,7 +306,8 @@ int student_backward(mrem_ctx* c) {
     launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
                       c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
-    r.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
+    fork();
+    rw.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
                    part + S_C * RED_BLOCKS, nullptr, c->dt, st);
     // attention:  ctx = P_hat V_hat,  P = softmax(Q_hat K_hat^T / sqrt(d))
@@ -295,7 +333,8 @@ int student_backward(mrem_ctx* c) {
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
     launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
     r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
-    r.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
+    fork();
+    rw.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
     void* next_carry = c->carry[l & 1];
     launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
                    part + S_X * RED_BLOCKS, nullptr, c->dt, st);
@@ -304,7 +343,14 @@ int student_backward(mrem_ctx* c) {
     // (the weight quantizers' masks and step gradients are applied inside the fused update of mrem_step,
     //  or on demand by mrem_get_grad)
     launch_reduce_table(c->reduce_table + (size_t)l * c->reduce_per_layer, c->reduce_per_layer, st);
+    // the layer below overwrites d_y2, d_u, d_y1, d_qkv and the bias row the weight-gradient products read
+    join();
+    // nothing below reads what the update writes: the latent weights, moments, row steps and this layer's codes
+    if (update_as_you_go) enqueue_matrix_updates(c, l, side);
   }
+  join();
+  if (sync_failed) return fail(c, MREM_ERR_CUDA, "backward: stream fork/join failed");
+  if (rw.rc != MREM_OK) { c->err = "weight-gradient GEMM launch failed"; return rw.rc; }
   if (r.rc != MREM_OK) return r.rc;
   return cudaGetLastError() == cudaSuccess ? MREM_OK : fail(c, MREM_ERR_CUDA, "backward: launch failed");
 }
@@ -384,10 +430,36 @@ int32_t mrem_module_backward(mrem_ctx* c) {
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k]) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
-  const int rc = student_backward(c);
+  const int rc = student_backward(c, false);
   if (rc != MREM_OK) return rc;
   c->have_grads = true;
   c->w_ste_done = false;
+  return MREM_OK;
+}
+
+// mrem_module_backward followed by mrem_step, with the matrix updates overlapped with the backward pass
+// (same kernels on the same data: the results are bitwise those of the two separate calls).
+int32_t mrem_backward_and_step(mrem_ctx* c, const mrem_optim* o) {
+  if (!c || !o) return MREM_ERR_ARG;
+  if (!c->d.w_step_per_row) {
+    const int rc = mrem_module_backward(c);
+    return rc != MREM_OK ? rc : mrem_step(c, o);
+  }
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
+  if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
+  for (int l = 0; l < c->d.n_layers; ++l)
+    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k]) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
+  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
+  launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
+                       o->weight_decay, c->stream);
+  c->w_ste_done = false;
+  const int rc = student_backward(c, true);
+  if (rc != MREM_OK) return rc;
+  launch_adamw_table(c->adam_rest, c->rest_entries, c->rest_elems, c->optim_sc, c->stream);
+  if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "step: launch failed");
+  c->have_grads = false; c->have_loss = false; c->have_student = false; c->have_teacher = false;
+  c->codes_fresh = true;
+  c->weights_quantized = true;
   return MREM_OK;
 }
 
@@ -402,16 +474,7 @@ int32_t mrem_step(mrem_ctx* c, const mrem_optim* o) {
   if (d.w_step_per_row) {
     // every tensor but the matrices and their steps, then one fused pass per matrix
     launch_adamw_table(c->adam_rest, c->rest_entries, c->rest_elems, c->optim_sc, c->stream);
-    const int train_w = (d.trainable_mask & MREM_TRAIN_WEIGHTS) != 0, train_s = (d.trainable_mask & MREM_TRAIN_W_STEPS) != 0;
-    for (int l = 0; l < d.n_layers; ++l)
-      for (int k = 0; k < N_WMAT; ++k) {
-        const int pid = kMatParam[k];
-        WeightBuf& w = c->wq[l][k];
-        LayerGrad& g = c->grad[l];
-        launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
-                                   c->w_ste_done ? g.ws[k] : nullptr, g.m_ws[k], g.v_ws[k], c->optim_sc, w.rows, w.cols,
-                                   d.w_bits, d.w_grid, train_w, train_s, w.codes, w.rowsum, w.scale, w.what, c->dt, c->stream);
-      }
+    for (int l = 0; l < d.n_layers; ++l) enqueue_matrix_updates(c, l, c->stream);
   } else {
     if (!c->w_ste_done) {
       for (int l = 0; l < d.n_layers; ++l)

@@ -471,16 +471,12 @@ void launch_col_reduce(const void* a, long long ld_a, const void* y, const float
                        const void* a2, long long ld_a2, long long rows, int cols, float* out0, float* out1,
                        float* out2, float* scratch, int* counters, int dt, cudaStream_t st) {
   Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (1 + (y ? 1 : 0) + (a2 ? 1 : 0)), 0, st);
-  MREM_DT(dt, T, {
-    constexpr int V = 16 / (int)sizeof(T);
-    if (cols % V == 0 && ld_a % V == 0 && ld_a2 % V == 0 && al16(a) && al16(y) && al16(a2)) {
-      dim3 grid((cols + 32 * V - 1) / (32 * V), COL_CHUNKS);
-      launch_k(col_reduce_kernel<T, V>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
-    } else {
-      dim3 grid((cols + 31) / 32, COL_CHUNKS);
-      launch_k(col_reduce_kernel<T, 1>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters);
-    }
-  });
+#define MREM_COLRED(T, V) do { dim3 grid((cols + 32 * V - 1) / (32 * V), COL_CHUNKS); \
+    launch_k(col_reduce_kernel<T, V>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters); } while (0)
+  const bool vec_ok = cols % 8 == 0 && ld_a % 8 == 0 && ld_a2 % 8 == 0 && al16(a) && al16(y) && al16(a2);
+  if (dt == 1) { if (vec_ok) MREM_COLRED(bf16, 8); else MREM_COLRED(bf16, 1); }
+  else { if (vec_ok) MREM_COLRED(float, 4); else MREM_COLRED(float, 1); }
+#undef MREM_COLRED
 }
 
 void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h, int S, void* P, const float* step,

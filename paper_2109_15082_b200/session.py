@@ -149,6 +149,9 @@ class ReconModule:
     def step(self, optim):
         B.mrem_step(self.ctx, optim)
 
+    def backward_and_step(self, optim):
+        B.mrem_backward_and_step(self.ctx, optim)
+
     def grad(self, layer, grad_id, shape):
         ptr = B.mrem_get_grad(self.ctx, layer, grad_id)
         n = int(np.prod(shape))
