@@ -104,6 +104,7 @@ struct mrem_ctx {
   // run there while the main stream goes on with the tensor-core work of the layer below
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaStream_t teacher_stream = nullptr;   // set for the duration of a step that runs the teacher pass beside the student's
   bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;

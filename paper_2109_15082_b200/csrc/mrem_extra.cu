@@ -16,8 +16,21 @@ namespace {
 int enqueue_step(mrem_ctx* c, const void* xt, const void* xs, float lambda, const int32_t* len, int batch, int seq,
                  void* t_out, void* s_out, float* d_loss, const mrem_optim* o) {
   int rc = mrem_quantize_weights(c);
+  // Without teacher forcing the two passes are independent until the loss: the teacher's runs on the side
+  // stream beside the student's (its tensor-core products under the student's quantizer kernels).  Only
+  // with the fused attention kernel, whose path shares no scratch between the passes.
+  const bool beside = lambda == 0.f && c->side_stream && !c->trace_on && c->d.n_heads > 0 &&
+                      attention_fwd_supported(seq, c->d.hidden / c->d.n_heads, c->dt);
+  if (rc == MREM_OK && beside) {
+    if (cudaEventRecord(c->ev_fork, c->stream) != cudaSuccess || cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess)
+      return fail(c, MREM_ERR_CUDA, "step: stream fork failed");
+    c->teacher_stream = c->side_stream;
+  }
   if (rc == MREM_OK) rc = mrem_module_forward(c, MREM_TEACHER, xt, nullptr, 0.f, len, batch, seq, t_out);
+  c->teacher_stream = nullptr;
   if (rc == MREM_OK) rc = mrem_module_forward(c, MREM_STUDENT, xs, xt, lambda, len, batch, seq, s_out);
+  if (beside && (cudaEventRecord(c->ev_join, c->side_stream) != cudaSuccess || cudaStreamWaitEvent(c->stream, c->ev_join, 0) != cudaSuccess))
+    return fail(c, MREM_ERR_CUDA, "step: stream join failed");
   if (rc == MREM_OK) rc = mrem_recon_loss(c, d_loss, nullptr);
   if (rc == MREM_OK) rc = mrem_backward_and_step(c, o);
   return rc;

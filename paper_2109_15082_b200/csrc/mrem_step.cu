@@ -105,7 +105,8 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
   const mrem_module_desc& d = c->d;
   const int H = d.hidden, F = d.ffn, h = d.n_heads, hd = H / h;
   const long long M = (long long)B * S;
-  Runner r(c);
+  cudaStream_t st = (!student_params && !init_steps && c->teacher_stream) ? c->teacher_stream : c->stream;
+  Runner r(c, st);
   const int ok = r.okind();
   const void* cur = x;
   for (int l = 0; l < d.n_layers; ++l) {
@@ -117,7 +118,7 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
       }
       for (int k = 0; k < N_WMAT; ++k) {
         WeightBuf& w = c->wq[l][k];
-        launch_narrow(b.student[kMatParam[k]], w.what, (long long)w.rows * w.cols, c->dt, c->stream);
+        launch_narrow(b.student[kMatParam[k]], w.what, (long long)w.rows * w.cols, c->dt, st);
         b.teacher[kMatParam[k]] = w.what;
       }
     }
@@ -130,12 +131,12 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
       for (int seg = 0; seg < 3; ++seg) init_site(c, b, S_Q + seg, r.at(c->t_qkv, seg * H), 3 * H, M, H);
     if (attention_fwd_supported(S, hd, c->dt)) {
       r.note(launch_attention_fwd(c->t_qkv, B, S, h, H, len, 1.f / sqrtf((float)hd), nullptr, nullptr, nullptr, nullptr,
-                                  nullptr, 0, 0, c->t_P, nullptr, c->t_ctx, nullptr, 0, nullptr, nullptr, c->status, c->stream),
+                                  nullptr, 0, 0, c->t_P, nullptr, c->t_ctx, nullptr, 0, nullptr, nullptr, c->status, st),
              "attention launch failed");
     } else {
       r.gemm(view(c->t_qkv, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(c->t_qkv, H), 3 * H, 0, hd, (long long)S * 3 * H),
              S, S, hd, h, B, Epi(c->scores, OUT_F32, S, (long long)S * S, (long long)h * S * S).alpha(1.f / sqrtf((float)hd)).e);
-      launch_softmax_fwd(c->scores, len, B, h, S, c->t_P, nullptr, nullptr, 0, 0, nullptr, c->dt, c->stream);
+      launch_softmax_fwd(c->scores, len, B, h, S, c->t_P, nullptr, nullptr, 0, 0, nullptr, c->dt, st);
       r.gemm(view(c->t_P, S, 0, (long long)S * S, (long long)h * S * S), view(r.at(c->t_qkv, 2 * H), 3 * H, 1, hd, (long long)S * 3 * H),
              S, hd, S, h, B, Epi(c->t_ctx, ok, H, hd, (long long)S * H).e);
     }
@@ -144,7 +145,7 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
     r.gemm(view(c->t_ctx, H), view(b.teacher[MREM_WO], H), (int)M, H, H, 1, 1,
            Epi(c->t_y1, ok, H).colbias((float*)b.teacher[MREM_BO]).residual(cur).e);
     launch_layernorm_fwd(c->t_y1, (float*)b.teacher[MREM_LN1_G], (float*)b.teacher[MREM_LN1_B], d.ln_eps, M, H, c->t_a,
-                         nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, c->stream);
+                         nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, st);
     if (init_steps) init_site(c, b, S_A, c->t_a, H, M, H);
     r.gemm(view(c->t_a, H), view(b.teacher[MREM_W1], H), (int)M, F, H, 1, 1,
            Epi(c->t_g, ok, F).colbias((float*)b.teacher[MREM_B1]).gelu().e);
@@ -152,7 +153,7 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
     r.gemm(view(c->t_g, F), view(b.teacher[MREM_W2], F), (int)M, H, F, 1, 1,
            Epi(c->t_y2, ok, H).colbias((float*)b.teacher[MREM_B2]).residual(c->t_a).e);
     launch_layernorm_fwd(c->t_y2, (float*)b.teacher[MREM_LN2_G], (float*)b.teacher[MREM_LN2_B], d.ln_eps, M, H, out,
-                         nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, c->stream);
+                         nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, st);
     cur = out;
   }
   if (r.rc != MREM_OK) return r.rc;
