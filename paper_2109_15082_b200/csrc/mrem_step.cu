@@ -282,32 +282,33 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     // second LayerNorm: total gradient at the layer output = loss term + what the next layer sent back
     launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, carry ? c->d_sum : nullptr, c->dt, st);
     // LayerNorm parameter gradients and the bias gradient of FFN2 (y2 = G_hat W2_hat^T + b2 + a) in one pass
+    // (column sums feed only the update and the weight-gradient epilogue: side stream)
+    fork();
     launch_col_reduce(carry ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, c->d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
-                      g.p[MREM_B2], c->col_scratch, c->col_counters, c->dt, st);
+                      g.p[MREM_B2], c->col_scratch, c->col_counters, c->dt, side);
     r.gemm(view(c->d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
     {
       Epi e(g.p[MREM_W2], OUT_F32, F);
       e.alpha(1.f, b.a_steps[S_G]);
-      if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], c->rowbias, H, st); e.rowbias(c->rowbias); }
-      fork();
+      if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], c->rowbias, H, side); e.rowbias(c->rowbias); }
       rw.gemm(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, 1, 1, e.e);
     }
     launch_gelu_bwd(s.u, c->d_ghat, c->d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
                     part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
     // FFN1:  u = A_hat W1_hat^T + b1
-    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
-    r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
     fork();
+    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, side);
+    r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
     rw.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
                    part + S_A * RED_BLOCKS, nullptr, c->dt, st);
     // first LayerNorm
     launch_layernorm_bwd(c->d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, c->d_y1, nullptr, c->dt, st);
     // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x  (its bias gradient rides along)
-    launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
-                      c->col_scratch, c->col_counters, c->dt, st);
-    r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
     fork();
+    launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
+                      c->col_scratch, c->col_counters, c->dt, side);
+    r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
     rw.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
                    part + S_C * RED_BLOCKS, nullptr, c->dt, st);
@@ -332,9 +333,9 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
                        b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, part + (S_Q + seg) * RED_BLOCKS, nullptr, c->dt, st);
     }
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
-    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, st);
-    r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
     fork();
+    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, side);
+    r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
     rw.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
     void* next_carry = c->carry[l & 1];
     launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
