@@ -22,6 +22,12 @@ void launch_quantize_act(const void* x, int dt, long long rows, int cols, long l
                          const float* offset, int lo, int hi, int8_t* q8, long long ld_q8, void* qt,
                          long long ld_qt, cudaStream_t st);
 
+// Three adjacent column segments of width seg_cols (Q | K | V of the fused projection), each with its own
+// symmetric step, in one pass; codes as storage-type numbers.
+void launch_quantize_act3(const void* x, int dt, long long rows, int seg_cols, long long ld_x, const float* step0,
+                          const float* step1, const float* step2, int lo, int hi, void* qt, long long ld_qt,
+                          cudaStream_t st);
+
 // dst[i] = (float)src[i] for a bfloat16 source
 void launch_widen_bf16(const void* src, float* dst, long long n, cudaStream_t st);
 

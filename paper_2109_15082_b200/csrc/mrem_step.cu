@@ -183,12 +183,12 @@ int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S
     void* out = r.at(outs, (long long)l * M * H);
     const ActRange rx = site_range(d, S_X), rp = site_range(d, S_P), rg = site_range(d, S_G);
 
-    launch_quantize_act(cur, c->dt, M, H, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi, s.x_q8, H, s.x_qt, H, c->stream);
+    // (layers above the first get the codes of their input from the LayerNorm that produced it)
+    if (l == 0) launch_quantize_act(cur, c->dt, M, H, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi, s.x_q8, H, s.x_qt, H, c->stream);
     r.gemm_i8(s.x_q8, 0, w[W_QKV].codes, (int)M, 3 * H, H,
               Epi(s.qkv, ok, 3 * H).alpha(1.f, b.a_steps[S_X]).colscale(w[W_QKV].scale).colbias(b.student[MREM_BQKV]).e);
-    for (int seg = 0; seg < 3; ++seg)
-      launch_quantize_act(r.at(s.qkv, seg * H), c->dt, M, H, 3 * H, b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, nullptr, 0,
-                          r.at(s.qkv_qt, seg * H), 3 * H, c->stream);
+    launch_quantize_act3(s.qkv, c->dt, M, H, 3 * H, b.a_steps[S_Q], b.a_steps[S_K], b.a_steps[S_V], rx.lo, rx.hi, s.qkv_qt,
+                         3 * H, c->stream);
     if (attention_fwd_supported(S, hd, c->dt)) {
       r.note(launch_attention_fwd(s.qkv_qt, B, S, h, H, len, 1.f / sqrtf((float)hd), b.a_steps[S_Q], b.a_steps[S_K],
                                   b.a_steps[S_P], b.a_steps[S_V], b.a_steps[S_P], rp.lo, rp.hi, s.P, s.P_qt, s.ctx,
@@ -217,8 +217,12 @@ int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S
     }
     r.gemm_i8(s.g_q8, rg.asym ? 1 : 0, w[W_2].codes, (int)M, H, F,
               Epi(s.y2, ok, H).alpha(1.f, b.a_steps[S_G]).colscale(w[W_2].scale).colbias(bias2).residual(s.a).e);
-    launch_layernorm_fwd(s.y2, b.student[MREM_LN2_G], b.student[MREM_LN2_B], d.ln_eps, M, H, out, s.mean2, s.rstd2,
-                         nullptr, 0, nullptr, nullptr, c->dt, c->stream);
+    if (l + 1 < d.n_layers)
+      launch_layernorm_fwd(s.y2, b.student[MREM_LN2_G], b.student[MREM_LN2_B], d.ln_eps, M, H, out, s.mean2, s.rstd2,
+                           c->bind[l + 1].a_steps[S_X], rx.hi, c->stash[l + 1].x_q8, c->stash[l + 1].x_qt, c->dt, c->stream);
+    else
+      launch_layernorm_fwd(s.y2, b.student[MREM_LN2_G], b.student[MREM_LN2_B], d.ln_eps, M, H, out, s.mean2, s.rstd2,
+                           nullptr, 0, nullptr, nullptr, c->dt, c->stream);
     cur = out;
   }
   if (r.rc != MREM_OK) return r.rc;

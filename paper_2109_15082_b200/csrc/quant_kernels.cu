@@ -61,10 +61,13 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
                                                            long long ld_x, const float* __restrict__ step,
                                                            const float* __restrict__ offset, float lo, float hi,
                                                            int8_t* __restrict__ q8, long long ld_q8,
-                                                           T* __restrict__ qt, long long ld_qt) {
+                                                           T* __restrict__ qt, long long ld_qt, int seg_cols,
+                                                           const float* __restrict__ step1,
+                                                           const float* __restrict__ step2) {
   pdl_trigger();
   pdl_wait();
-  const float s = *step;
+  // seg_cols > 0: three column segments of that width (a multiple of V), each with its own step
+  const float s0 = *step, s1 = seg_cols ? *step1 : s0, s2 = seg_cols ? *step2 : s0;
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
   const int vcols = cols / V;
@@ -74,6 +77,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
     const int c = (int)(i - r * vcols) * V;
     float v[V];
     load_vec<T, V>(x + r * ld_x + c, v);
+    const float s = !seg_cols || c < seg_cols ? s0 : (c < 2 * seg_cols ? s1 : s2);
     int q[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) q[j] = act_code(v[j], s, off, has_off, lo, hi);
@@ -257,14 +261,15 @@ void launch_quantize_weight(const float* w, int rows, int cols, const float* ste
 
 template <typename T>
 static void quantize_act_t(const T* x, long long rows, int cols, long long ld_x, const float* step, const float* offset,
-                           int lo, int hi, int8_t* q8, long long ld_q8, T* qt, long long ld_qt, cudaStream_t st) {
+                           int lo, int hi, int8_t* q8, long long ld_q8, T* qt, long long ld_qt, int seg_cols,
+                           const float* step1, const float* step2, cudaStream_t st) {
   constexpr int V = 16 / (int)sizeof(T);
-  const bool v = vec_ok<T>(x, ld_x, cols) && vec_ok<T>(qt, ld_qt, cols) &&
+  const bool v = vec_ok<T>(x, ld_x, cols) && vec_ok<T>(qt, ld_qt, cols) && seg_cols % V == 0 &&
                  (q8 == nullptr || ((reinterpret_cast<uintptr_t>(q8) % V) == 0 && ld_q8 % V == 0));
   if (v)
-    launch_k(quantize_act_kernel<T, V>, grid_for(rows * cols / V), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
+    launch_k(quantize_act_kernel<T, V>, grid_for(rows * cols / V), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt, seg_cols, step1, step2);
   else
-    launch_k(quantize_act_kernel<T, 1>, grid_for(rows * cols), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt);
+    launch_k(quantize_act_kernel<T, 1>, grid_for(rows * cols), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt, seg_cols, step1, step2);
 }
 
 void launch_quantize_act(const void* x, int dt, long long rows, int cols, long long ld_x, const float* step,
@@ -272,8 +277,17 @@ void launch_quantize_act(const void* x, int dt, long long rows, int cols, long l
                          long long ld_qt, cudaStream_t st) {
   if (rows <= 0 || cols <= 0) return;
   Scope sc("quantize_act", (double)rows * cols * ((dt == 1 ? 2.0 : 4.0) * (qt ? 2 : 1) + (q8 ? 1 : 0)), 0, st);
-  if (dt == 1) quantize_act_t<bf16>((const bf16*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (bf16*)qt, ld_qt, st);
-  else quantize_act_t<float>((const float*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (float*)qt, ld_qt, st);
+  if (dt == 1) quantize_act_t<bf16>((const bf16*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (bf16*)qt, ld_qt, 0, nullptr, nullptr, st);
+  else quantize_act_t<float>((const float*)x, rows, cols, ld_x, step, offset, lo, hi, q8, ld_q8, (float*)qt, ld_qt, 0, nullptr, nullptr, st);
+}
+
+void launch_quantize_act3(const void* x, int dt, long long rows, int seg_cols, long long ld_x, const float* step0,
+                          const float* step1, const float* step2, int lo, int hi, void* qt, long long ld_qt,
+                          cudaStream_t st) {
+  if (rows <= 0 || seg_cols <= 0) return;
+  Scope sc("quantize_act", (double)rows * 3 * seg_cols * (dt == 1 ? 2.0 : 4.0) * 2, 0, st);
+  if (dt == 1) quantize_act_t<bf16>((const bf16*)x, rows, 3 * seg_cols, ld_x, step0, nullptr, lo, hi, nullptr, 0, (bf16*)qt, ld_qt, seg_cols, step1, step2, st);
+  else quantize_act_t<float>((const float*)x, rows, 3 * seg_cols, ld_x, step0, nullptr, lo, hi, nullptr, 0, (float*)qt, ld_qt, seg_cols, step1, step2, st);
 }
 
 void launch_widen_bf16(const void* src, float* dst, long long n, cudaStream_t st) {
