@@ -137,24 +137,27 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     const bool got = mbar_wait(smem_u32(&bar_s), 0);
     if (!__all_sync(0xffffffffu, got) && lane == 0) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_MMA);
     tc_fence_after();
+    // scores in units of log2(e): exp(alpha * a - max) = 2^(alpha2 * a - max2); alpha > 0, so the maximum
+    // can be taken over the raw accumulators
+    const float alpha2 = alpha * 1.4426950408889634f;
     float mx = -INFINITY;
     for (int c = half; c < n_chunks; c += 2) {
       uint32_t a[32];
       tmem_ld32(trow + (uint32_t)(c * 32), a);
 #pragma unroll
       for (int j = 0; j < 32; ++j)
-        if (c * 32 + j < len) mx = fmaxf(mx, alpha * __uint_as_float(a[j]));
+        if (c * 32 + j < len) mx = fmaxf(mx, __uint_as_float(a[j]));
     }
     red[0][half][r] = mx;
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    mx = fmaxf(red[0][0][r], red[0][1][r]);
+    const float mx2 = alpha2 * fmaxf(red[0][0][r], red[0][1][r]);
     float sum = 0.f;
     for (int c = half; c < n_chunks; c += 2) {            // exp once: kept in TMEM in place of the score
       uint32_t a[32];
       tmem_ld32(trow + (uint32_t)(c * 32), a);
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        const float e = c * 32 + j < len ? expf(alpha * __uint_as_float(a[j]) - mx) : 0.f;
+        const float e = c * 32 + j < len ? exp2f(fmaf(alpha2, __uint_as_float(a[j]), -mx2)) : 0.f;
         sum += e;
         a[j] = __float_as_uint(e);
       }
@@ -163,6 +166,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     red[1][half][r] = sum;
     asm volatile("bar.sync 1, 256;" ::: "memory");
     sum = red[1][0][r] + red[1][1][r];
+    const float inv_sum = __frcp_rn(sum);
     const long long prow = (((long long)b * p.h + head) * p.S + q) * p.S;
     for (int c = half; c < 2 * p.n_kb; c += 2) {          // 32-key chunks up to the padded key count
       uint32_t pw[16], cw[16];                            // 32 probabilities / codes packed as bf16 pairs
@@ -171,7 +175,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
         tmem_ld32(trow + (uint32_t)(c * 32), a);
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
-          const float v0 = __fdiv_rn(__uint_as_float(a[j]), sum), v1 = __fdiv_rn(__uint_as_float(a[j + 1]), sum);
+          const float v0 = __uint_as_float(a[j]) * inv_sum, v1 = __uint_as_float(a[j + 1]) * inv_sum;
           const __nv_bfloat162 pb = __floats2bfloat162_rn(v0, v1);
           pw[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
           if (quant) {
