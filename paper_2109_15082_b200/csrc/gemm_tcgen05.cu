@@ -77,7 +77,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
         const TileCoord t = decode_tile(p, tile);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (*vabort || !mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u)) {
+          if (!mbar_wait_or_abort(smem_u32(&empty_bar[stage]), phase ^ 1u, vabort)) {
             if (!*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
             ok = false;
             break;
@@ -112,32 +112,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
-      const uint32_t adv_a = p.a_mn ? 2048u : 32u, adv_b = p.b_mn ? 2048u : 32u;
-      const uint32_t lbo_a = p.a_mn ? 8192u : 16u, lbo_b = p.b_mn ? 8192u : 16u;
+      // descriptor words: high word fixed (stride between 8-row groups, version, 128-byte swizzle); low word =
+      // address >> 4 plus the leading-dimension offset field, advanced per 16-deep step and per stage
+      const uint32_t adv_a = (p.a_mn ? 2048u : 32u) >> 4, adv_b = (p.b_mn ? 2048u : 32u) >> 4;
+      const uint64_t proto_a = smem_desc(tiles_base, p.a_mn ? 8192u : 16u, 1024u);
+      const uint64_t proto_b = smem_desc(tiles_base + A_STAGE_BYTES, p.b_mn ? 8192u : 16u, 1024u);
+      const uint32_t a_hi = (uint32_t)(proto_a >> 32), b_hi = (uint32_t)(proto_b >> 32);
+      const uint32_t a_lo0 = (uint32_t)proto_a, b_lo0 = (uint32_t)proto_b, stage_adv = (uint32_t)p.stage_bytes >> 4;
+      uint32_t a_lo = a_lo0, b_lo = b_lo0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-        if (*vabort || !mbar_wait(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u)) {
+        if (!mbar_wait_or_abort(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, vabort)) {
           if (!*vabort) fail(p, DEV_TIMEOUT_EPI, vabort);
           break;
         }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * p.block_n);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (*vabort || !mbar_wait(smem_u32(&full_bar[stage]), phase)) {
+          if (!mbar_wait_or_abort(smem_u32(&full_bar[stage]), phase, vabort)) {
             if (!*vabort) fail(p, DEV_TIMEOUT_TMA, vabort);
             ok = false;
             break;
           }
           tc_fence_after();
-          const uint32_t sa = tiles_base + stage * p.stage_bytes, sb = sa + A_STAGE_BYTES;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint64_t da = smem_desc(sa + k * adv_a, lbo_a, 1024u);
-            const uint64_t db = smem_desc(sb + k * adv_b, lbo_b, 1024u);
-            tc_mma<KIND>(tmem_d, da, db, p.idesc, (uint32_t)((kb | k) != 0));
-          }
+          tc_mma_lohi<KIND>(tmem_d, a_lo, a_hi, b_lo, b_hi, p.idesc, (uint32_t)(kb != 0));
+          tc_mma_lohi<KIND>(tmem_d, a_lo + adv_a, a_hi, b_lo + adv_b, b_hi, p.idesc, 1u);
+          tc_mma_lohi<KIND>(tmem_d, a_lo + 2 * adv_a, a_hi, b_lo + 2 * adv_b, b_hi, p.idesc, 1u);
+          tc_mma_lohi<KIND>(tmem_d, a_lo + 3 * adv_a, a_hi, b_lo + 3 * adv_b, b_hi, p.idesc, 1u);
           tc_commit(smem_u32(&empty_bar[stage]));
-          if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
+          a_lo += stage_adv; b_lo += stage_adv;
+          if (++stage == p.num_stages) { stage = 0; phase ^= 1u; a_lo = a_lo0; b_lo = b_lo0; }
         }
         if (!ok) break;
         tc_commit(smem_u32(&tfull_bar[acc]));
@@ -165,7 +169,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const TileCoord t = decode_tile(p, tile);
       // every lane polls; the decision is made warp-uniform before any .sync.aligned instruction
-      const bool got = !*vabort && mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase);
+      const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0 && !*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
         break;
