@@ -312,3 +312,51 @@ def test_nonfinite_loss_is_reported_in_status():
         assert m.poll_status() == 0                                     # cleared by the poll
     finally:
         p.close()
+
+
+def test_module_sweep_caches_outputs_for_the_next_module():
+    """Two one-layer modules in sequence: after module 0's steps its teacher and student outputs over the
+    calibration set become module 1's inputs (Algorithm 2's outer loop).  Checked against the oracle run
+    on the same bytes: the cached tensors, and module 1's first loss computed from them."""
+    from paper_2109_15082_b200.sweep import ModuleSweep
+    wl = _wl("base3_w4a8", n_layers=1, hidden=128, n_heads=2, ffn=256, seq=32, batch=4, len_lo=8, len_hi=32)
+    n_calib = 8
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        probs = [Problem(wl, seed=s, student_noise=0.002) for s in (0, 5)]
+        try:
+            mods = [p.m for p in probs]
+            x = synth.hidden_states(wl, n_calib, 3)
+            calib = mods[0].to_device(x)
+            vl = synth.valid_lengths(wl, n_calib, 3)
+            vld = torch.from_numpy(vl).to(mods[0].device)
+            order = lambda k, e: synth.permutation(7, f"m{k}e{e}", n_calib)
+            sw = ModuleSweep(mods, calib, vld, wl.batch, order, wl.w_step_rule)
+            opt = B.make_optim(lr=1e-5, step=0, decay_total_steps=4)
+            l0 = sw.run_module(0, 2, opt)
+            assert len(l0) == 2 and all(np.isfinite(l0)) and mods[0].poll_status() == 0
+            sw.cache_outputs(0)
+            # oracle on the same bytes with module 0's parameters and steps as they are now
+            p0 = probs[0]
+            st0 = mods[0].student_numpy()
+            ws, a, off = mods[0].get_steps()
+            steps0 = O.make_steps(ws, a, off)
+            xs = calib.float().cpu().numpy()
+            t_ref = O.teacher_forward(p0.desc, p0.teacher, xs, vl)[-1]
+            s_ref = O.student_forward(p0.desc, st0, steps0, xs, vl)[0][-1]
+            assert rel(sw.x_teacher.float().cpu().numpy(), t_ref) < 1e-3
+            assert rel(sw.x_student.float().cpu().numpy(), s_ref) < 1e-3
+            assert not torch.equal(sw.x_teacher, sw.x_student)
+            # module 1 starts from the cached pair: its first recorded loss is that of its initial state
+            l1 = sw.run_module(1, 1, opt)
+            p1 = probs[1]
+            first = order(1, 0)[: wl.batch]
+            xt1 = sw.x_teacher.float().cpu().numpy()[first]
+            xs1 = sw.x_student.float().cpu().numpy()[first]
+            ws1 = O.init_weight_steps(p1.desc, p1.student, wl.w_step_rule)
+            a1, off1 = O.init_act_steps(p1.desc, p1.student, xs1, vl[first])
+            r = O.forward_loss_backward(p1.desc, p1.teacher, p1.student, O.make_steps(ws1, a1, off1), xt1, xs1, vl[first], 0.0)
+            assert abs(l1[0] - r["loss"]) / r["loss"] < GRAD_TOL, (l1[0], r["loss"])
+        finally:
+            for p in probs:
+                p.close()
