@@ -145,6 +145,10 @@ def run_reference(args, wl):
 
 # ----------------------------------------------------------------------------- GPU leg
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over two whole steps
+NCU_DRAM_BYTES_PER_LAUNCH = {("large6_w4a8", "gemm_bf16_tcgen05"): 28.05e6}
+
+
 def build_problem(wl, rank, torch, calib_n):
     from paper_2109_15082_b200 import synth
     from paper_2109_15082_b200.session import ReconModule
@@ -315,8 +319,12 @@ def main():
                         "us_per_launch": 1e3 * per_launch_ms, "bound": bound, "achieved": ach, "peak": peak,
                         "unit": unit, "frac": ach / peak})
     top = kernels[0]
+    # DRAM bytes per launch of the dominant kernel from the committed ncu capture of this workload
+    # (profiles/tc_gemm_dram_large6_w4a8.md); known only for that kernel on that workload
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, top["name"]))
     roofline = {"kernel": top["name"], "bound": top["bound"], "achieved": top["achieved"], "peak": top["peak"],
-                "unit": top["unit"], "frac": top["frac"], "traffic": None,
+                "unit": top["unit"], "frac": top["frac"], "traffic": traffic,
+                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, ncu)" if traffic else None,
                 "peak_source": pk["source"] + (" bf16 sustained" if top["bound"] == "tensor" else " copy bandwidth"),
                 "timed": f"CUDA events around each launch of {n_trace} eager steps"}
 
