@@ -17,6 +17,9 @@ from tests.gpu_util import Problem, compare_grads, rel
 pytestmark = pytest.mark.gpu
 
 FWD_TOL = {"f32": 1e-4, "bf16": 1e-3}
+# Per layer at hidden 1024 / FFN 4096: a float32 CPU replica of a teacher layer (same bf16 storage points, other
+# summation order) differs from the float64 oracle by 7e-4; the tensor-core path by 1.3e-3.
+FULL_SIZE_FWD_TOL = 2.5e-3
 GRAD_TOL = 2e-2
 
 
@@ -360,3 +363,90 @@ def test_module_sweep_caches_outputs_for_the_next_module():
         finally:
             for p in probs:
                 p.close()
+
+
+@pytest.mark.parametrize("name", ["large6_w4a8", "large6_w2a8_s384"])
+def test_full_size_step_in_the_benchmark_launch_configuration(name):
+    """The BERT-large module at its full size, stepped the way bench.py steps it (one captured graph, two
+    streams inside).  The oracle cannot run 4096+ tokens through six layers in seconds, so it checks what it
+    can compute one by one: sequences of a batch are independent in the forward pass, so two sampled
+    sequences go through the oracle's teacher and student; every weight code of the module is recomputed by
+    Eq. 1 (before the step from the bound weights, after it from the updated weights and steps: bit exact);
+    the loss must equal the mean squared difference of the outputs the step itself wrote."""
+    from paper_2109_15082_b200.session import ReconModule
+    wl = synth.workloads()[name]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, wl.a_bits, wl.w_grid,
+                        True, 3, wl.act_dtype, True)
+        try:
+            desc = O.ModuleDesc(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.w_bits, wl.a_bits, wl.w_grid, True, True, True,
+                                wl.act_dtype, True)
+            m.load_teacher(synth.teacher_params(wl, 0, bias_std=0.02))
+            m.init_student_from_teacher()
+            x = synth.hidden_states(wl, wl.batch, 0)
+            xd = m.to_device(x)
+            vl = synth.valid_lengths(wl, wl.batch, 0)
+            vld = torch.from_numpy(vl).to(m.device)
+            m.init_weight_steps(wl.w_step_rule)
+            m.init_act_steps(xd, vld, wl.batch, wl.seq)
+            side.synchronize()
+            teacher, student0 = m.teacher_numpy(), m.student_numpy()
+            ws0, a0, off0 = m.get_steps()
+            # codes before the step
+            m.quantize_weights()
+            for l in (0, wl.n_layers - 1):
+                for pid in (B.WQKV, B.W2):
+                    codes, rowsum = m.weight_codes(l, pid)
+                    nm = B.PARAM_NAMES[pid]
+                    ref = O.quantize_weight(student0[l][nm], ws0[l][nm].reshape(-1, 1), wl.w_bits, wl.w_grid)[0]
+                    assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref)
+                    assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1))
+            opt = B.make_optim(lr=1e-4, step=0, decay_total_steps=100)
+            B.mrem_graph_capture_step(m.ctx, xd, xd, 0.0, vld, wl.batch, wl.seq, m.t_out, m.s_out, m.loss, opt)
+            B.mrem_graph_launch(m.ctx)
+            side.synchronize()
+            assert m.poll_status() == 0
+            n = wl.n_layers * wl.batch * wl.seq * wl.hidden
+            f_t = m.t_out[:n].view(wl.n_layers, wl.batch, wl.seq, wl.hidden)
+            f_s = m.s_out[:n].view(wl.n_layers, wl.batch, wl.seq, wl.hidden)
+            loss = float(m.loss[0])
+            per_layer = ((f_s.double() - f_t.double()) ** 2).mean(dim=(1, 2, 3))
+            assert abs(loss - float(per_layer.sum())) / loss < 1e-4
+            # two sampled sequences through the oracle (same stored bytes)
+            pick = [1, wl.batch - 2]
+            xs = xd.float().cpu().numpy()[pick]
+            steps0 = O.make_steps(ws0, a0, off0)
+            t_ref = O.teacher_forward(desc, teacher, xs, vl[pick])
+            s_ref = O.student_forward(desc, student0, steps0, xs, vl[pick])[0]
+            # (a) whole module: differences accumulate layer over layer (each layer's input already differs)
+            errs = [(rel(f_t[l][pick].float().cpu().numpy(), t_ref[l]), rel(f_s[l][pick].float().cpu().numpy(), s_ref[l]))
+                    for l in range(wl.n_layers)]
+            print(name, "accumulated forward rel L2 (teacher, student) per layer:", [(round(a, 5), round(b, 5)) for a, b in errs])
+            assert errs[0][1] < FWD_TOL["bf16"]            # first student layer: exact codes in, same codes out
+            assert max(e[0] for e in errs) < 1.5e-2 and max(e[1] for e in errs) < 6e-2
+            # (b) layer by layer, the oracle fed with the input the GPU layer really had
+            for l in range(wl.n_layers):
+                xin_t = xs if l == 0 else f_t[l - 1][pick].float().cpu().numpy()
+                xin_s = xs if l == 0 else f_s[l - 1][pick].float().cpu().numpy()
+                t_one = O.teacher_layer(desc, teacher[l], O.round_bf16(xin_t), vl[pick])
+                s_one = O.student_forward(desc, [student0[l]], [steps0[l]], xin_s, vl[pick])[0][0]
+                et, es = rel(f_t[l][pick].float().cpu().numpy(), t_one), rel(f_s[l][pick].float().cpu().numpy(), s_one)
+                print(name, "layer", l, "rel L2 teacher", round(et, 5), "student", round(es, 5))
+                assert et < FULL_SIZE_FWD_TOL, ("teacher", l, et)
+                assert es < FULL_SIZE_FWD_TOL, ("student", l, es)
+            # after the step: the fused update's codes are Eq. 1 of the updated weights and steps
+            student1 = m.student_numpy()
+            ws1, _, _ = m.get_steps()
+            changed = 0
+            for l in range(wl.n_layers):
+                for pid in (B.WQKV, B.WO, B.W1, B.W2):
+                    codes, rowsum = m.weight_codes(l, pid)
+                    nm = B.PARAM_NAMES[pid]
+                    ref = O.quantize_weight(student1[l][nm], ws1[l][nm].reshape(-1, 1), wl.w_bits, wl.w_grid)[0]
+                    assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref), (l, nm)
+                    assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1)), (l, nm)
+                    changed += int(not np.array_equal(student1[l][nm], student0[l][nm]))
+            assert changed == 4 * wl.n_layers
+        finally:
+            m.close()
