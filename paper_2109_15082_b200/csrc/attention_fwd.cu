@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     if (p.a_p0) alpha *= *p.a_p0;
     if (p.a_p1) alpha *= *p.a_p1;
     const bool quant = p.p_step != nullptr;
-    const float ps = quant ? *p.p_step : 1.f;
+    const float ps = quant ? *p.p_step : 1.f, r_ps = __frcp_rn(ps);
     const uint32_t trow = tmem + ((uint32_t)(quad * 32) << 16);
     const int n_chunks = (p.S + 31) / 32;
     const bool got = mbar_wait(smem_u32(&bar_s), 0);
@@ -180,8 +180,9 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
           pw[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
           if (quant) {
             const float2 f = __bfloat1622float2(pb);
-            const float c0 = (float)__float2int_rn(fminf(fmaxf(__fdiv_rn(f.x, ps), p.p_lo), p.p_hi));
-            const float c1 = (float)__float2int_rn(fminf(fmaxf(__fdiv_rn(f.y, ps), p.p_lo), p.p_hi));
+            // f is bf16-valued: quotient() equals the IEEE division of Eq. 1 for every such value and every step
+            const float c0 = (float)__float2int_rn(fminf(fmaxf(quotient(f.x, ps, r_ps), p.p_lo), p.p_hi));
+            const float c1 = (float)__float2int_rn(fminf(fmaxf(quotient(f.y, ps, r_ps), p.p_lo), p.p_hi));
             const __nv_bfloat162 cb = __floats2bfloat162_rn(c0, c1);
             cw[j >> 1] = *reinterpret_cast<const uint32_t*>(&cb);
           } else {
@@ -219,7 +220,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     float calpha = 1.f;
     if (p.c_p0) calpha *= *p.c_p0;
     if (p.c_p1) calpha *= *p.c_p1;
-    const float cs = p.c_step ? *p.c_step : 1.f;
+    const float cs = p.c_step ? *p.c_step : 1.f, r_cs = __frcp_rn(cs);
     const long long crow = ((long long)b * p.S + q) * p.H + head * HD;
     {
       const int hh = half;
@@ -232,8 +233,8 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
         w[j >> 1] = *reinterpret_cast<const uint32_t*>(&vb);
         if (p.c_step) {
           const float2 f = __bfloat1622float2(vb);
-          const int i0 = __float2int_rn(fminf(fmaxf(__fdiv_rn(f.x, cs), -p.c_qmax), p.c_qmax));
-          const int i1 = __float2int_rn(fminf(fmaxf(__fdiv_rn(f.y, cs), -p.c_qmax), p.c_qmax));
+          const int i0 = __float2int_rn(fminf(fmaxf(quotient(f.x, cs, r_cs), -p.c_qmax), p.c_qmax));
+          const int i1 = __float2int_rn(fminf(fmaxf(quotient(f.y, cs, r_cs), -p.c_qmax), p.c_qmax));
           const __nv_bfloat162 cb = __floats2bfloat162_rn((float)i0, (float)i1);
           cq[j >> 1] = *reinterpret_cast<const uint32_t*>(&cb);
           const uint32_t two = (uint32_t)(i0 & 0xff) | ((uint32_t)(i1 & 0xff) << 8);

@@ -103,9 +103,12 @@ __device__ __forceinline__ float rcp_approx(float x) {
 
 // x / s from r_s = RN(1/s): one product, the exact residual by FMA, one correction.  Equals the correctly
 // rounded quotient except where x/s lies within ~2^-48 (relative) of the midpoint of two floats; a value
-// sitting exactly on a clipping boundary gets the same side as the quantizer's IEEE division.  Used where
-// the quotient feeds a straight-through factor (a surrogate gradient); the codes themselves are always
-// produced with the IEEE division of Eq. 1.
+// sitting exactly on a clipping boundary gets the same side as the quantizer's IEEE division.  For
+// bfloat16-valued x (8 significant bits) it IS the correctly rounded quotient for every float32 s:
+// checked over all 128 x 2^23 significand pairs (the exponents do not enter while x/s, 1/s and the
+// residual stay in the normal range, which holds for activations and steps by many orders of magnitude).
+// Used for the straight-through factors (a surrogate gradient) and, in the fused attention kernel, for the
+// codes of bfloat16-stored tensors; every other code is produced with the division instruction.
 __device__ __forceinline__ float quotient(float x, float s, float r_s) {
   const float z0 = __fmul_rn(x, r_s);
   return __fmaf_rn(__fmaf_rn(-z0, s, x), r_s, z0);
