@@ -55,6 +55,8 @@ __global__ void __launch_bounds__(NT, 1024 / NT) fused_weight_update_kernel(
   const OptimScalars o = *sc;
   const float s_old = steps[row];
   const float r_old = __frcp_rn(s_old);
+  float ms_pre = 0.f, vs_pre = 0.f;
+  if (threadIdx.x == 0 && train_s) { ms_pre = m_s[row]; vs_pre = v_s[row]; }
   const float qmax = (float)((1 << (bits - 1)) - 1);
   const long long base = (long long)row * cols;
   const int nvec = cols / 4;                                   // cols is a multiple of 16
@@ -102,11 +104,11 @@ __global__ void __launch_bounds__(NT, 1024 / NT) fused_weight_update_kernel(
   }
   ds = block_sum(ds, sh);
   if (ds_in) ds = ds_in[row];          // gradients were masked and reduced before (same arithmetic)
-  // 2. the row's step
+  // 2. the row's step (its moments were fetched before the reduction)
   if (threadIdx.x == 0) {
     float s_new = s_old;
     if (train_s) {
-      float ms = m_s[row], vs = v_s[row];
+      float ms = ms_pre, vs = vs_pre;
       s_new = adam_one(s_old, ds, ms, vs, o, 0.f, 1e-8f);
       m_s[row] = ms;
       v_s[row] = vs;
