@@ -41,7 +41,7 @@ __device__ __forceinline__ void store_what4<bf16>(bf16* p, float a, float b, flo
 // NT threads per row, NV float4 vectors per thread kept in registers: (256, 1) for rows up to 1024 wide,
 // (512, 2) up to 4096; wider rows are re-read.
 template <typename T, int NV, int NT>
-__global__ void __launch_bounds__(NT, 1024 / NT) fused_weight_update_kernel(
+__global__ void __launch_bounds__(NT, NT == 256 ? 6 : 2) fused_weight_update_kernel(
     float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v,
     float* __restrict__ steps, const float* __restrict__ ds_in, float* __restrict__ m_s, float* __restrict__ v_s,
     const OptimScalars* __restrict__ sc, int cols, int bits, int grid, int train_w, int train_s,
