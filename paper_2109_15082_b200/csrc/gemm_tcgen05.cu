@@ -161,6 +161,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     bool vec_ok = (e.ldc % vec_elems == 0) && (e.c_b0 % vec_elems == 0) && (e.c_b1 % vec_elems == 0) &&
                   ((reinterpret_cast<uintptr_t>(e.out) & 15) == 0);
     if (e.residual) vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(e.residual) & 15) == 0);
+    vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(e.col_scale) & 15) == 0) && ((reinterpret_cast<uintptr_t>(e.col_bias) & 15) == 0);
     uint32_t* stg = reinterpret_cast<uint32_t*>(smem_raw + (tiles_base - smem_u32(smem_raw)) +
                                                 (size_t)p.num_stages * p.stage_bytes) + (warp - 2) * STAGING_WORDS;
     const int cols_per_round = (e.out_kind == OUT_BF16) ? 64 : 32;
