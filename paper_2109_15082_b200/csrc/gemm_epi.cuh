@@ -139,6 +139,9 @@ __device__ __forceinline__ void epilogue_round(const TcParams& p, uint32_t taddr
   const int vec_elems = is_bf16 ? 8 : 4;
   const int sub = lane >> 3, seg = lane & 7;             // 4 rows per instruction, 8 lanes per row
   uint4* stg4 = reinterpret_cast<uint4*>(stg);
+  uint32_t r0[32], r1[32];
+  tmem_ld32_issue(taddr, r0);                           // in flight while the residual is fetched and transposed
+  if (is_bf16) tmem_ld32_issue(taddr + 32u, r1);
   uint32_t res[32];
   if (e.residual) {
 #pragma unroll
@@ -161,9 +164,6 @@ __device__ __forceinline__ void epilogue_round(const TcParams& p, uint32_t taddr
   }
   const int row = row0 + lane;
   const float rb = (e.row_bias && row < p.M) ? e.row_bias[row] : 0.f;
-  uint32_t r0[32], r1[32];
-  tmem_ld32_issue(taddr, r0);
-  if (is_bf16) tmem_ld32_issue(taddr + 32u, r1);
   tmem_ld_wait();
   tmem_ld_pin(r0);
   if (is_bf16) tmem_ld_pin(r1);
