@@ -571,3 +571,52 @@ def recon_step(desc, teacher, student, steps, state, x_t, x_s, valid_len=None, l
             steps[l]["a"] = np.maximum(upd((l, "a"), steps[l]["a"], g["a"], 0.0), MIN_STEP).astype(np.float32)
             steps[l]["a_off"] = upd((l, "a_off"), steps[l]["a_off"], g["a_off"], 0.0).astype(np.float32)
     return r
+
+
+# ----------------------------------------------------------------------------- Algorithm 1: modules trained in parallel from input queues
+
+def mremp_run(descs, teachers, students, steps, batches, draws, t0, T, T0, lr0, lr_total=0, log=None, **adam):
+    """Algorithm 1 (Sec. 4.2) on N modules, one module after the other inside a step (the result does not
+    depend on the order: a module only reads what its predecessor produced in EARLIER steps, except while the
+    queues are being filled).
+
+    descs, teachers, students, steps: per module n = 0 .. N-1 (students and steps are updated in place)
+    batches: batches[t] = (x [B,S,H], valid_len or None), the calibration batch module 0 takes at step t
+    draws:   draws[t][n] in [0, t0): which of the t0 most recent queue entries module n >= 1 samples at step
+             t >= t0 (0 = the most recent); the same entry is taken from the teacher-side and the
+             student-side queue, so both modules see the same sequences
+    t0:      staleness threshold = queue length.  In the first t0 steps every module is computed one after
+             another and module n takes what module n-1 produced in the SAME step (filling the queues)
+    T, T0:   steps per module; teacher forcing lambda_t = max(1 - t/T0, 0) for t < T0, none afterwards (Alg. 2)
+    lr0, lr_total: AdamW learning rate, linearly decayed over lr_total steps when lr_total > 0
+    Queue entries are (f_t, f_hat_t, valid_len) of the forward pass of step t (before that step's update),
+    kept first-in-first-out.  Returns losses[n][t]; `log`, if a list, receives (t, n, entry index or None).
+    """
+    N = len(descs)
+    queues = [[] for _ in range(N)]                      # queues[n]: most recent first, at most t0 entries
+    states = [dict() for _ in range(N)]
+    losses = [[] for _ in range(N)]
+    for t in range(T):
+        lam = teacher_forcing_lambda(t, T0) if t < T0 else 0.0
+        lr = linear_decay_lr(lr0, t, lr_total) if lr_total > 0 else lr0
+        produced = []
+        for n in range(N):
+            if n == 0:
+                x_t, vl = batches[t]
+                x_s, k = x_t, None
+            elif t < t0:
+                x_t, x_s, vl = produced[n - 1]           # filling: the predecessor's output of this very step
+                k = None
+            else:
+                k = int(draws[t][n])
+                assert 0 <= k < len(queues[n - 1])
+                x_t, x_s, vl = queues[n - 1][k]
+            if log is not None:
+                log.append((t, n, k))
+            r = recon_step(descs[n], teachers[n], students[n], steps[n], states[n], x_t, x_s, vl, lam, lr=lr, **adam)
+            losses[n].append(r["loss"])
+            produced.append((r["f_t"][-1], r["f_s"][-1], vl))
+        for n in range(N):                               # first in, first out
+            queues[n].insert(0, produced[n])
+            del queues[n][t0:]
+    return losses

@@ -328,3 +328,63 @@ def test_recon_step_reduces_loss_on_repeated_batch():
     for t in range(40):
         losses.append(O.recon_step(desc, params, student, steps, state, x, x, lr=3e-5)["loss"])
     assert np.mean(losses[-5:]) < 0.7 * losses[0]
+
+
+# ----------------------------------------------------------------------------- Algorithm 1 (modules in parallel from input queues)
+
+def _mremp_setup(n_modules, seed=0):
+    wl = synth.shrink(synth.workloads()["tiny"], hidden=32, ffn=64, seq=8, batch=2, n_heads=2)
+    descs, teachers, students, steps = [], [], [], []
+    x0 = synth.hidden_states(wl, 2, seed)
+    for n in range(n_modules):
+        desc = O.ModuleDesc(1, 32, 2, 64, 4, 8, act_dtype="f32")
+        params = synth.teacher_params(wl, seed + 10 * n)
+        student = [{k: v.copy() for k, v in params[0].items()}]
+        ws = O.init_weight_steps(desc, student, 0)
+        a, off = O.init_act_steps(desc, student, x0)
+        descs.append(desc); teachers.append(params); students.append(student); steps.append(O.make_steps(ws, a, off))
+    return wl, descs, teachers, students, steps
+
+
+def test_mremp_single_module_is_the_plain_step_loop():
+    wl, descs, teachers, students, steps = _mremp_setup(1)
+    batches = [(synth.hidden_states(wl, 2, 100 + t), None) for t in range(4)]
+    ref_student = [{k: v.copy() for k, v in students[0][0].items()}]
+    ref_steps = O.make_steps([s["w"] for s in steps[0]], np.stack([s["a"] for s in steps[0]]), np.stack([s["a_off"] for s in steps[0]]))
+    got = O.mremp_run(descs, teachers, students, steps, batches, draws=np.zeros((4, 1), int), t0=2, T=4, T0=0, lr0=1e-4)
+    state, want = {}, []
+    for t in range(4):
+        want.append(O.recon_step(descs[0], teachers[0], ref_student, ref_steps, state, batches[t][0], batches[t][0], lr=1e-4)["loss"])
+    assert got[0] == want
+    assert all(np.array_equal(students[0][0][k], ref_student[0][k]) for k in O.PARAMS)
+
+
+def test_mremp_queue_is_fifo_fill_phase_is_sequential_and_lambda_follows_the_schedule(monkeypatch):
+    """Replace the step by a recorder: what each module is fed pins the schedule of Algorithm 1 on its own."""
+    calls = []
+
+    def fake_step(desc, teacher, student, steps, state, x_t, x_s, vl, lam, lr=None, **kw):
+        n = desc                                    # the 'descs' passed below are just the module indices
+        t = state["t"] = state.get("t", -1) + 1
+        calls.append((t, n, float(x_t), float(x_s), lam, lr))
+        # teacher output = 1000 * (n + 1) + t, student output = its negative: recognisable stamps
+        return dict(loss=0.0, f_t=[np.float64(1000 * (n + 1) + t)], f_s=[-np.float64(1000 * (n + 1) + t)])
+
+    monkeypatch.setattr(O, "recon_step", fake_step)
+    T, t0, T0, N = 7, 3, 4, 3
+    batches = [(np.float64(t), None) for t in range(T)]
+    draws = np.array([[0, (t + n) % t0, (2 * t + n) % t0] for t in range(T) for n in (0,)]).reshape(T, 3)
+    log = []
+    O.mremp_run(list(range(N)), [None] * N, [None] * N, [None] * N, batches, draws, t0, T, T0, lr0=1.0, lr_total=10, log=log)
+    for (t, n, x_t, x_s, lam, lr) in calls:
+        assert lam == (max(1 - t / T0, 0.0) if t < T0 else 0.0)          # Alg. 2: lambda_t, none after T0
+        assert lr == pytest.approx(1.0 - t / 10)                          # linear decay
+        if n == 0:
+            assert x_t == t and x_s == t                                  # calibration batch of step t
+        elif t < t0:
+            assert x_t == 1000 * n + t and x_s == -(1000 * n + t)         # filling: predecessor's output of the same step
+        else:
+            k = draws[t][n]
+            assert x_t == 1000 * n + (t - 1 - k) and x_s == -x_t          # k-th most recent entry, same entry on both sides
+            assert 0 <= k < t0                                            # never older than t0 steps (first in, first out)
+    assert len(calls) == T * N and [c[:2] for c in calls] == [(t, n) for t in range(T) for n in range(N)]
