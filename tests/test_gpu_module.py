@@ -450,3 +450,52 @@ def test_full_size_step_in_the_benchmark_launch_configuration(name):
             assert changed == 4 * wl.n_layers
         finally:
             m.close()
+
+
+def test_parallel_modules_follow_algorithm_1():
+    """Three one-layer modules trained side by side from input queues (Algorithm 1) with annealed teacher forcing:
+    every module's loss at every step against the oracle's run of the same schedule on the same bytes."""
+    from paper_2109_15082_b200.parallel import ParallelModules
+    from paper_2109_15082_b200.session import ReconModule
+    wl = _wl("base3_w4a8", n_layers=1, hidden=128, n_heads=2, ffn=256, seq=32, batch=4, len_lo=8, len_hi=32)
+    N, n_calib, T, t0, T0, lr0 = 3, 16, 6, 2, 4, 2e-5
+    x = synth.hidden_states(wl, n_calib, 3)
+    vl = synth.valid_lengths(wl, n_calib, 3)
+    ids = lambda t: synth.permutation(11, f"step{t}", n_calib)[: wl.batch]
+    draws = np.array([[0, (t + 1) % t0, (2 * t + 1) % t0] for t in range(T)])
+    mods, descs, teachers = [], [], []
+    try:
+        for n in range(N):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, wl.a_bits, wl.w_grid,
+                                True, 3, wl.act_dtype, True)
+            m.load_teacher(synth.teacher_params(wl, 20 + n, bias_std=0.02))
+            m.init_student_from_teacher()
+            mods.append(m)
+            descs.append(O.ModuleDesc(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.w_bits, wl.a_bits, wl.w_grid, True, True, True,
+                                      wl.act_dtype, True))
+        torch.cuda.synchronize()
+        calib = mods[0].to_device(x)
+        vld = torch.from_numpy(vl).to(mods[0].device)
+        torch.cuda.synchronize()
+        pm = ParallelModules(mods, calib, vld, wl.batch, ids, draws, t0, T0)
+        pm.init_steps(wl.w_step_rule)
+        teachers = [m.teacher_numpy() for m in mods]
+        students = [m.student_numpy() for m in mods]
+        steps = [O.make_steps(*m.get_steps()) for m in mods]
+        opt = B.make_optim(lr=lr0, step=0, decay_total_steps=10)
+        got = pm.run(T, lambda t: opt)
+        for m in mods:
+            assert m.poll_status() == 0
+        xs = calib.float().cpu().numpy()
+        batches = [(xs[ids(t)], vl[ids(t)]) for t in range(T)]
+        want = O.mremp_run(descs, teachers, students, steps, batches, draws, t0, T, T0, lr0, lr_total=10)
+        for n in range(N):
+            for t in range(T):
+                assert abs(got[n][t] - want[n][t]) / want[n][t] < 3e-2, (n, t, got[n][t], want[n][t])
+        print("parallel modules, losses", [[round(v, 6) for v in g] for g in got])
+        # the run is reproducible bit for bit: no step reads a queue slot that is being written
+        assert got == [[float(v.item()) for v in log] for log in pm.loss_log]
+    finally:
+        for m in mods:
+            m.close()
