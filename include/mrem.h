@@ -181,10 +181,21 @@ int32_t mrem_backward_and_step(mrem_ctx* ctx, const mrem_optim* optim);
 
 /* The whole step from HOST buffers: copies h_x_teacher / h_x_student ([batch, seq, hidden] act_dtype;
  * h_x_student may equal h_x_teacher) and h_valid_len (may be NULL) to the device, runs quantize_weights,
- * both forwards, loss, backward and step, copies the loss back to *h_loss and blocks until it is there. */
+ * both forwards, loss, backward and step, copies the loss back to *h_loss and blocks until it is there.
+ * With optim->step == 0 (device-side step counter) the step is captured into a CUDA graph on first use and
+ * replayed while batch, seq, lambda, *optim and the presence of h_valid_len stay the same. */
 int32_t mrem_recon_step_host(mrem_ctx* ctx, const void* h_x_teacher, const void* h_x_student,
                              const int32_t* h_valid_len, int32_t batch, int32_t seq, float lambda,
                              const mrem_optim* optim, float* h_loss);
+/* The same step in two halves, so that the copy of the next batch overlaps the step in flight: submit
+ * enqueues the host-to-device copies (on a copy stream the context owns, into one of two staging slots) and
+ * the step, and returns at once; wait blocks until the OLDEST submitted step is done and returns its loss.
+ * At most two steps may be in flight (MREM_ERR_ORDER beyond that).  The host buffers (pinned memory for the
+ * copies to be asynchronous) must stay valid and unchanged until the matching wait has returned. */
+int32_t mrem_recon_step_host_submit(mrem_ctx* ctx, const void* h_x_teacher, const void* h_x_student,
+                                    const int32_t* h_valid_len, int32_t batch, int32_t seq, float lambda,
+                                    const mrem_optim* optim);
+int32_t mrem_recon_step_host_wait(mrem_ctx* ctx, float* h_loss);
 
 /* Process-wide switch (default on): kernels are launched with programmatic stream serialization, i.e. a
  * kernel may be scheduled and run its set-up while its predecessor in the stream is still finishing; each

@@ -32,7 +32,8 @@ EXPORTS = (
     "mrem_import_state", "mrem_graph_capture_step", "mrem_graph_launch", "mrem_gather_rows", "mrem_quantize_act",
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
-    "mrem_set_fused_attention_backward", "mrem_backward_and_step",
+    "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
+    "mrem_recon_step_host_wait",
 )
 
 
@@ -193,6 +194,17 @@ def mrem_recon_step_host(ctx, h_x_teacher, h_x_student, h_valid_len, batch, seq,
     loss = C.c_float(0)
     _check(lib().mrem_recon_step_host(ctx, _p(h_x_teacher), _p(h_x_student), _p(h_valid_len), batch, seq,
                                       C.c_float(lam), C.byref(optim), C.byref(loss)), "mrem_recon_step_host", ctx)
+    return loss.value
+
+
+def mrem_recon_step_host_submit(ctx, h_x_teacher, h_x_student, h_valid_len, batch, seq, lam, optim):
+    _check(lib().mrem_recon_step_host_submit(ctx, _p(h_x_teacher), _p(h_x_student), _p(h_valid_len), batch, seq,
+                                             C.c_float(lam), C.byref(optim)), "mrem_recon_step_host_submit", ctx)
+
+
+def mrem_recon_step_host_wait(ctx) -> float:
+    loss = C.c_float(0)
+    _check(lib().mrem_recon_step_host_wait(ctx, C.byref(loss)), "mrem_recon_step_host_wait", ctx)
     return loss.value
 
 

@@ -81,6 +81,11 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->h2d_xt = A.take(M * H * es);
   c->h2d_xs = A.take(M * H * es);
   c->h2d_len = (int32_t*)A.take(sizeof(int32_t) * d.max_batch);
+  for (int k = 0; k < 2; ++k) {
+    c->stage_x[k][0] = A.take(M * H * es);
+    c->stage_x[k][1] = A.take(M * H * es);
+    c->stage_len[k] = (int32_t*)A.take(sizeof(int32_t) * d.max_batch);
+  }
   c->e2e_t_out = A.take((size_t)L * M * H * es);
   c->e2e_s_out = A.take((size_t)L * M * H * es);
 
@@ -251,7 +256,12 @@ int32_t mrem_create(const mrem_module_desc* desc, void* workspace, size_t worksp
   if (cudaDeviceGetStreamPriorityRange(&pri_lo, &pri_hi) != cudaSuccess ||
       cudaStreamCreateWithPriority(&c->side_stream, cudaStreamNonBlocking, pri_lo) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_h2d[0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_h2d[1], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_host_done[0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_host_done[1], cudaEventDisableTiming) != cudaSuccess) {
     mrem_destroy(c);
     return fail(nullptr, MREM_ERR_CUDA, "stream or event creation failed");
   }
@@ -264,6 +274,13 @@ int32_t mrem_destroy(mrem_ctx* c) {
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   if (c->graph) cudaGraphDestroy(c->graph);
   if (c->h_pinned_loss) cudaFreeHost(c->h_pinned_loss);
+  if (c->host_graph_exec) cudaGraphExecDestroy(c->host_graph_exec);
+  if (c->host_graph) cudaGraphDestroy(c->host_graph);
+  for (int k = 0; k < 2; ++k) {
+    if (c->ev_h2d[k]) cudaEventDestroy(c->ev_h2d[k]);
+    if (c->ev_host_done[k]) cudaEventDestroy(c->ev_host_done[k]);
+  }
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->side_stream) cudaStreamDestroy(c->side_stream);

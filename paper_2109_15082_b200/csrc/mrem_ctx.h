@@ -108,7 +108,14 @@ struct mrem_ctx {
   bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;
-  void *h2d_xt, *h2d_xs; int32_t* h2d_len; float* d_loss_e2e;   // staging of mrem_recon_step_host
+  void *h2d_xt, *h2d_xs; int32_t* h2d_len; float* d_loss_e2e;   // inputs and loss of the host-buffer step (fixed: graph inputs)
+  void* stage_x[2][2]; int32_t* stage_len[2];                   // [slot][teacher|student]: where the copies from the host land
+  cudaStream_t copy_stream = nullptr;                           // host -> device copies of the host-buffer step
+  cudaEvent_t ev_h2d[2] = {nullptr, nullptr}, ev_host_done[2] = {nullptr, nullptr};
+  bool slot_used[2] = {false, false};
+  unsigned host_head = 0, host_tail = 0;                        // submitted / waited-for steps
+  cudaGraph_t host_graph = nullptr; cudaGraphExec_t host_graph_exec = nullptr;
+  struct HostKey { int batch = -1, seq = -1, same = 0, has_len = 0; float lambda = 0.f; mrem_optim optim{}; } host_key;
   void *e2e_t_out, *e2e_s_out;                                  // its layer outputs [L, M, H]
   size_t state_off = 0, state_bytes = 0;                          // optimizer moments: one contiguous range
   bool tables_dirty = true;

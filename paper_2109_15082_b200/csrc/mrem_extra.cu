@@ -1,5 +1,8 @@
 // C-ABI entry points built on the step: activation-step initialisation, the host-buffer
 // step, CUDA-graph capture of a step, and the single operations exposed for verification.
+#include <cstring>
+#include <string>
+
 #include "mrem_ctx.h"
 
 using namespace mrem;
@@ -57,29 +60,109 @@ int32_t mrem_init_act_steps(mrem_ctx* c, const void* x, const int32_t* len, int3
   return rc;
 }
 
+// Captures enqueue_step on the context's stream into (*graph, *exec); any earlier pair is destroyed.
+static int capture_step_graph(mrem_ctx* c, const void* xt, const void* xs, float lambda, const int32_t* len, int batch,
+                              int seq, void* t_out, void* s_out, float* d_loss, const mrem_optim* o, cudaGraph_t* graph,
+                              cudaGraphExec_t* exec, const char* who) {
+  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
+  if (*exec) { cudaGraphExecDestroy(*exec); *exec = nullptr; }
+  if (*graph) { cudaGraphDestroy(*graph); *graph = nullptr; }
+  // quantize once outside the graph: inside it the fused update keeps the codes current
+  { const int qrc = mrem_quantize_weights(c); if (qrc != MREM_OK) return qrc; }
+  if (!c->d.w_step_per_row) c->codes_fresh = false;      // per-matrix steps: every step re-quantizes, inside the graph
+  const bool was_tracing = c->trace_on;
+  c->trace_on = false;              // event pairs are not recorded inside a captured graph
+  struct Restore { mrem_ctx* c; bool v; ~Restore() { c->trace_on = v; } } restore{c, was_tracing};
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();   // clear the sticky-until-read error: the legacy default stream cannot be captured
+    c->err = std::string(who) + ": begin capture failed (the context's stream must not be the legacy default stream)";
+    return MREM_ERR_CUDA;
+  }
+  const int rc = enqueue_step(c, xt, xs, lambda, len, batch, seq, t_out, s_out, d_loss, o);
+  cudaGraph_t g = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+  if (rc != MREM_OK) { if (g) cudaGraphDestroy(g); return rc; }
+  if (e != cudaSuccess || !g) return fail(c, MREM_ERR_CUDA, "graph capture failed at end capture");
+  *graph = g;
+  if (cudaGraphInstantiate(exec, g, 0) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph instantiate failed");
+  return MREM_OK;
+}
+
+int32_t mrem_recon_step_host_submit(mrem_ctx* c, const void* h_xt, const void* h_xs, const int32_t* h_len, int32_t batch,
+                                    int32_t seq, float lambda, const mrem_optim* o) {
+  if (!c || !h_xt || !h_xs || !o) return MREM_ERR_ARG;
+  if (batch < 1 || seq < 1 || batch > c->d.max_batch || seq > c->d.max_seq) return fail(c, MREM_ERR_SHAPE, "recon_step_host: batch/seq outside the context's maximum");
+  if (c->host_head - c->host_tail >= 2) return fail(c, MREM_ERR_ORDER, "recon_step_host_submit: two steps already in flight; call mrem_recon_step_host_wait");
+  const int k = (int)(c->host_head & 1u);
+  const size_t bytes = (size_t)batch * seq * c->d.hidden * c->esz;
+  const bool same = h_xs == h_xt;
+  // copies from the host go to slot k on the copy stream, beside whatever the context's stream is computing
+  if (c->slot_used[k] && cudaStreamWaitEvent(c->copy_stream, c->ev_host_done[k], 0) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: stream wait failed");
+  bool okc = cudaMemcpyAsync(c->stage_x[k][0], h_xt, bytes, cudaMemcpyHostToDevice, c->copy_stream) == cudaSuccess;
+  if (!same) okc = okc && cudaMemcpyAsync(c->stage_x[k][1], h_xs, bytes, cudaMemcpyHostToDevice, c->copy_stream) == cudaSuccess;
+  if (h_len) okc = okc && cudaMemcpyAsync(c->stage_len[k], h_len, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, c->copy_stream) == cudaSuccess;
+  okc = okc && cudaEventRecord(c->ev_h2d[k], c->copy_stream) == cudaSuccess && cudaStreamWaitEvent(c->stream, c->ev_h2d[k], 0) == cudaSuccess;
+  // from the slot into the step's fixed input buffers (device to device: microseconds)
+  okc = okc && cudaMemcpyAsync(c->h2d_xt, c->stage_x[k][0], bytes, cudaMemcpyDeviceToDevice, c->stream) == cudaSuccess;
+  if (!same) okc = okc && cudaMemcpyAsync(c->h2d_xs, c->stage_x[k][1], bytes, cudaMemcpyDeviceToDevice, c->stream) == cudaSuccess;
+  if (h_len) okc = okc && cudaMemcpyAsync(c->h2d_len, c->stage_len[k], sizeof(int32_t) * batch, cudaMemcpyDeviceToDevice, c->stream) == cudaSuccess;
+  if (!okc) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
+  const void* xs = same ? c->h2d_xt : c->h2d_xs;
+  const int32_t* len = h_len ? c->h2d_len : nullptr;
+  int rc;
+  const bool capturable = c->stream != nullptr && c->stream != cudaStreamLegacy;
+  if (o->step > 0 || c->trace_on || !capturable) {
+    // an explicit step number is baked into the launch arguments, traced kernels are timed one by one, and the
+    // legacy default stream cannot be captured: no graph
+    rc = enqueue_step(c, c->h2d_xt, xs, lambda, len, batch, seq, c->e2e_t_out, c->e2e_s_out, c->d_loss_e2e, o);
+  } else {
+    mrem_ctx::HostKey key;
+    key.batch = batch; key.seq = seq; key.same = same; key.has_len = h_len != nullptr; key.lambda = lambda; key.optim = *o;
+    const mrem_ctx::HostKey& old = c->host_key;
+    const bool hit = c->host_graph_exec && old.batch == key.batch && old.seq == key.seq && old.same == key.same &&
+                     old.has_len == key.has_len && old.lambda == key.lambda && memcmp(&old.optim, &key.optim, sizeof(mrem_optim)) == 0;
+    rc = MREM_OK;
+    if (!hit) {
+      rc = capture_step_graph(c, c->h2d_xt, xs, lambda, len, batch, seq, c->e2e_t_out, c->e2e_s_out, c->d_loss_e2e, o,
+                              &c->host_graph, &c->host_graph_exec, "recon_step_host");
+      if (rc == MREM_OK) c->host_key = key;
+    } else if (!c->codes_fresh && c->d.w_step_per_row) {
+      rc = mrem_quantize_weights(c);          // weights or steps were written from outside since the last step
+    }
+    if (rc == MREM_OK && cudaGraphLaunch(c->host_graph_exec, c->stream) != cudaSuccess) rc = fail(c, MREM_ERR_CUDA, "recon_step_host: graph launch failed");
+    if (rc == MREM_OK) {                      // the host-side state the eager call sequence would have left
+      c->t_out = c->e2e_t_out; c->s_out = c->e2e_s_out; c->s_in = xs;
+      c->cur_batch = batch; c->cur_seq = seq; c->cur_len = len;
+      c->have_grads = false; c->have_loss = false; c->have_student = false; c->have_teacher = false;
+      c->codes_fresh = c->d.w_step_per_row != 0;
+      c->weights_quantized = c->codes_fresh;
+    }
+  }
+  if (rc != MREM_OK) return rc;
+  if (cudaMemcpyAsync(c->h_pinned_loss + k, c->d_loss_e2e, sizeof(float), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaEventRecord(c->ev_host_done[k], c->stream) != cudaSuccess)
+    return fail(c, MREM_ERR_CUDA, "recon_step_host: device error");
+  c->slot_used[k] = true;
+  ++c->host_head;
+  return MREM_OK;
+}
+
+int32_t mrem_recon_step_host_wait(mrem_ctx* c, float* h_loss) {
+  if (!c || !h_loss) return MREM_ERR_ARG;
+  if (c->host_tail == c->host_head) return fail(c, MREM_ERR_ORDER, "recon_step_host_wait: no step in flight");
+  const int k = (int)(c->host_tail & 1u);
+  if (cudaEventSynchronize(c->ev_host_done[k]) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host_wait: device error");
+  *h_loss = c->h_pinned_loss[k];
+  ++c->host_tail;
+  return MREM_OK;
+}
+
 int32_t mrem_recon_step_host(mrem_ctx* c, const void* h_xt, const void* h_xs, const int32_t* h_len, int32_t batch,
                              int32_t seq, float lambda, const mrem_optim* o, float* h_loss) {
-  if (!c || !h_xt || !h_xs || !o || !h_loss) return MREM_ERR_ARG;
-  if (batch < 1 || seq < 1 || batch > c->d.max_batch || seq > c->d.max_seq) return fail(c, MREM_ERR_SHAPE, "recon_step_host: batch/seq outside the context's maximum");
-  const size_t bytes = (size_t)batch * seq * c->d.hidden * c->esz;
-  if (cudaMemcpyAsync(c->h2d_xt, h_xt, bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
-  const void* xs = c->h2d_xt;
-  if (h_xs != h_xt) {
-    if (cudaMemcpyAsync(c->h2d_xs, h_xs, bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
-    xs = c->h2d_xs;
-  }
-  const int32_t* len = nullptr;
-  if (h_len) {
-    if (cudaMemcpyAsync(c->h2d_len, h_len, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_step_host: copy failed");
-    len = c->h2d_len;
-  }
-  const int rc = enqueue_step(c, c->h2d_xt, xs, lambda, len, batch, seq, c->e2e_t_out, c->e2e_s_out, c->d_loss_e2e, o);
-  if (rc != MREM_OK) return rc;
-  if (cudaMemcpyAsync(c->h_pinned_loss, c->d_loss_e2e, sizeof(float), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
-      cudaStreamSynchronize(c->stream) != cudaSuccess)
-    return fail(c, MREM_ERR_CUDA, "recon_step_host: device error");
-  *h_loss = *c->h_pinned_loss;
-  return MREM_OK;
+  if (!c || !h_loss) return MREM_ERR_ARG;
+  if (c->host_tail != c->host_head) return fail(c, MREM_ERR_ORDER, "recon_step_host: submitted steps are still in flight; wait for them first");
+  const int rc = mrem_recon_step_host_submit(c, h_xt, h_xs, h_len, batch, seq, lambda, o);
+  return rc != MREM_OK ? rc : mrem_recon_step_host_wait(c, h_loss);
 }
 
 int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, float lambda, const int32_t* len,
@@ -87,26 +170,8 @@ int32_t mrem_graph_capture_step(mrem_ctx* c, const void* xt, const void* xs, flo
                                 const mrem_optim* o) {
   if (!c || !xt || !xs || !t_out || !s_out || !d_loss || !o) return MREM_ERR_ARG;
   if (o->step > 0) return fail(c, MREM_ERR_ARG, "graph_capture_step: optim.step must be 0 (device-side counter)");
-  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
-  if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
-  if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
-  // quantize once outside the graph: inside it the fused update keeps the codes current
-  { const int qrc = mrem_quantize_weights(c); if (qrc != MREM_OK) return qrc; }
-  const bool was_tracing = c->trace_on;
-  c->trace_on = false;              // event pairs are not recorded inside a captured graph
-  struct Restore { mrem_ctx* c; bool v; ~Restore() { c->trace_on = v; } } restore{c, was_tracing};
-  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-    cudaGetLastError();   // clear the sticky-until-read error: the legacy default stream cannot be captured
-    return fail(c, MREM_ERR_CUDA, "graph_capture_step: begin capture failed (the context's stream must not be the legacy default stream)");
-  }
-  const int rc = enqueue_step(c, xt, xs, lambda, len, batch, seq, t_out, s_out, d_loss, o);
-  cudaGraph_t g = nullptr;
-  const cudaError_t e = cudaStreamEndCapture(c->stream, &g);
-  if (rc != MREM_OK) { if (g) cudaGraphDestroy(g); return rc; }
-  if (e != cudaSuccess || !g) return fail(c, MREM_ERR_CUDA, "graph_capture_step: end capture failed");
-  c->graph = g;
-  if (cudaGraphInstantiate(&c->graph_exec, g, 0) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "graph_capture_step: instantiate failed");
-  return MREM_OK;
+  return capture_step_graph(c, xt, xs, lambda, len, batch, seq, t_out, s_out, d_loss, o, &c->graph, &c->graph_exec,
+                            "graph_capture_step");
 }
 
 int32_t mrem_graph_num_kernels(mrem_ctx* c, int32_t* n_kernels) {

@@ -200,7 +200,7 @@ def test_graph_replay_and_host_step_equal_eager():
     opt = B.make_optim(lr=1e-4, step=0, decay_total_steps=10)
     results = []
     side = torch.cuda.Stream()                 # the legacy default stream cannot be captured
-    for mode in ("eager", "graph", "host"):
+    for mode in ("eager", "graph", "host", "host_pipelined"):
         with torch.cuda.stream(side):
             p = Problem(wl, **kw)
             try:
@@ -221,8 +221,14 @@ def test_graph_replay_and_host_step_equal_eager():
                         B.mrem_graph_launch(m.ctx)
                         torch.cuda.synchronize()
                         losses.append(float(m.loss[0]))
-                    else:
+                    elif mode == "host":
                         losses.append(B.mrem_recon_step_host(m.ctx, x_host, x_host, vl_host, wl.batch, wl.seq, 0.0, opt))
+                    else:                       # the copy of the next batch is submitted before this step's loss is read
+                        if t == 0:
+                            B.mrem_recon_step_host_submit(m.ctx, x_host, x_host, vl_host, wl.batch, wl.seq, 0.0, opt)
+                        if t < 2:
+                            B.mrem_recon_step_host_submit(m.ctx, x_host, x_host, vl_host, wl.batch, wl.seq, 0.0, opt)
+                        losses.append(B.mrem_recon_step_host_wait(m.ctx))
                 torch.cuda.synchronize()
                 assert m.poll_status() == 0
                 results.append((losses, m.student_numpy()[0]["W1"].copy()))
