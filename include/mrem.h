@@ -151,7 +151,7 @@ int32_t mrem_get_weight_codes(mrem_ctx* ctx, int32_t layer, int32_t tensor_id, c
 /* Runs one module forward.  d_x: [batch, seq, hidden] in act_dtype, this role's own input.
  * STUDENT with lambda != 0: the input becomes lambda * d_x_other + (1 - lambda) * d_x (Eq. 4, d_x_other =
  * the teacher-side input); otherwise d_x_other may be NULL.  d_valid_len: [batch] int32 key lengths
- * (positions >= length are masked out of the attention) or NULL.  d_layer_outputs:
+ * (positions >= length are masked out of the attention; a length below 1 counts as 1, above seq as seq) or NULL.  d_layer_outputs:
  * [n_layers, batch, seq, hidden] act_dtype, written; the last slice is the module output.
  * The student pass needs mrem_quantize_weights first (ERR_ORDER) and keeps d_x and d_layer_outputs
  * borrowed until mrem_module_backward has run. */

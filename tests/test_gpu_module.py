@@ -505,3 +505,50 @@ def test_parallel_modules_follow_algorithm_1():
     finally:
         for m in mods:
             m.close()
+
+
+def test_degenerate_inputs_match_the_oracle():
+    """Degenerate cases of the method: weight rows that are entirely zero (their step is clamped to the minimum,
+    their codes are 0), a sequence with a single valid token and one with every token valid, an all-zero input
+    sequence, and device-side step initialisation on such data."""
+    wl = _wl("base3_w4a8", n_layers=1, hidden=128, n_heads=2, ffn=256, seq=24, batch=3, len_lo=1, len_hi=24)
+    p = Problem(wl, student_noise=0.0)
+    try:
+        m = p.m
+        params = synth.teacher_params(wl, 0, bias_std=0.02)
+        for k in ("Wqkv", "W1", "W2", "Wo"):
+            params[0][k][3, :] = 0.0                         # a dead output row in every matrix
+            params[0][k][7, :] = 0.0
+        m.load_teacher(params)
+        m.init_student_from_teacher()
+        x = synth.hidden_states(wl, wl.batch, 0)
+        x[1] = 0.0                                            # an all-zero sequence
+        p.xd = m.to_device(x)
+        p.x = p.xd.float().cpu().numpy()
+        p.vl = np.array([1, wl.seq, 5], np.int32)
+        p.vld = torch.from_numpy(p.vl).to(m.device)
+        p.teacher, p.student = m.teacher_numpy(), m.student_numpy()
+        # steps initialised on the device, then handed to the oracle
+        m.init_weight_steps(0)
+        m.init_act_steps(p.xd, p.vld, wl.batch, wl.seq)
+        torch.cuda.synchronize()
+        ws, a, off = m.get_steps()
+        ws_ref = O.init_weight_steps(p.desc, p.student, 0)
+        a_ref, off_ref = O.init_act_steps(p.desc, p.student, p.x, p.vl)
+        for k in O.WEIGHTS:
+            assert np.array_equal(ws[0][k], ws_ref[0][k]), k
+            assert ws[0][k][3] == np.float32(O.MIN_STEP) and ws[0][k][7] == np.float32(O.MIN_STEP)
+        assert np.allclose(a, a_ref, rtol=2e-2) and np.allclose(off, off_ref, rtol=2e-2, atol=1e-3)
+        p.ws, p.a, p.off = ws, a, off
+        g = p.run_gpu()
+        r = p.run_oracle()
+        assert rel(g["f_t"][0], r["f_t"][0]) < FWD_TOL["bf16"] and rel(g["f_s"][0], r["f_s"][0]) < FWD_TOL["bf16"]
+        assert np.isfinite(g["loss"]) and abs(g["loss"] - r["loss"]) / r["loss"] < GRAD_TOL
+        for pid, name in ((B.WQKV, "Wqkv"), (B.W2, "W2")):
+            codes, rowsum = m.weight_codes(0, pid)
+            assert not codes[3].any() and not codes[7].any() and rowsum[3] == 0
+        compare_grads(g["grads"], r["grads"], GRAD_TOL, check_offset=False)
+        for k in O.WEIGHTS:                                   # nothing flows into a dead row's weights through the product
+            assert np.all(np.isfinite(g["grads"][0][k]))
+    finally:
+        p.close()
