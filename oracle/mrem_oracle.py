@@ -44,6 +44,7 @@ class ModuleDesc:
     w_bits: int = 4            # 0 = weights not quantized (bypass)
     a_bits: int = 8            # 0 = activations not quantized (bypass)
     w_grid: int = 0            # 0: Omega(b) of Eq. 1; 1: half-integer 2-bit grid {-1.5,-.5,.5,1.5}*s
+    w_twn: bool = False        # 2-bit weights by the closed-form ternary rule (threshold 0.7 mean|w|, scale = mean of the kept |w|) instead of a learnable step
     w_per_row: bool = True     # one step per output row, else one per matrix
     asym_p: bool = True        # softmax output quantized asymmetrically (unsigned codes, offset 0)
     asym_g: bool = True        # GELU output quantized asymmetrically (unsigned codes, learnable offset)
@@ -133,6 +134,24 @@ def quantize_weight(w, s, bits, grid, act_dtype="f32"):
     assert bits == 2
     c = 2 * np.clip(np.floor(z), -2, 1).astype(np.int64) + 1
     return c, s64 * 0.5, z
+
+
+def quantize_weight_twn(w, per_row=True):
+    """Ternary weights with closed-form threshold and scale (the TWN rule the paper names for 2-bit weights,
+    Sec. 5.1): per group (output row or whole matrix) delta = 0.7 * mean|w|, t = sign(w) * 1[|w| > delta],
+    alpha = mean of |w| over the kept entries (0 when none is kept); w_hat = alpha * t.  The means are taken in
+    float64 and the comparison |w| > delta in float32 on float32(delta), the precision in which the kernel
+    decides.  Returns (codes int64 in {-1, 0, 1}, alpha float64 [groups, 1], delta float32 [groups, 1])."""
+    w32 = np.asarray(w, np.float32)
+    a = np.abs(w32.astype(np.float64))
+    g = a if per_row else a.reshape(1, -1)
+    delta = (0.7 * g.mean(-1, keepdims=True)).astype(np.float32)
+    keep = np.abs(w32 if per_row else w32.reshape(1, -1)) > delta
+    cnt = keep.sum(-1, keepdims=True)
+    alpha = (g * keep).sum(-1, keepdims=True) / np.maximum(cnt, 1)
+    alpha = alpha.astype(np.float32).astype(np.float64)
+    t = (np.sign(w32 if per_row else w32.reshape(1, -1)) * keep).astype(np.int64).reshape(w32.shape)
+    return t, alpha, delta
 
 
 def weight_ste(z, codes, bits, grid):
@@ -282,6 +301,9 @@ def _q_act(desc, x, steps, site):
 def _q_w(desc, w, s_w):
     if desc.w_bits == 0:
         return dict(what=np.asarray(w, np.float64), q=None)
+    if desc.w_twn:
+        q, alpha, _ = quantize_weight_twn(w, desc.w_per_row)
+        return dict(what=alpha * q, q=q, z=None, scale=alpha, twn=True)
     s = np.asarray(s_w, np.float32).reshape(-1, 1)
     q, scale, z = quantize_weight(w, s, desc.w_bits, desc.w_grid, desc.act_dtype)
     return dict(what=scale * q, q=q, z=z, scale=scale)
@@ -398,8 +420,8 @@ def _linear_back(desc, qa, qw, dy, name, g, site):
     dy2 = dy.reshape(-1, dy.shape[-1])
     dwhat = dy2.T @ qa["xhat"].reshape(-1, K)
     g["b" + name[1:] if name != "Wqkv" else "bqkv"] = dy2.sum(0)
-    if qw["q"] is None:
-        g[name] = dwhat
+    if qw["q"] is None or qw.get("twn"):
+        g[name] = dwhat                                   # closed-form scales: plain straight-through, nothing to learn
         g["w"][name] = None
     else:
         inside, dwhat_ds = weight_ste(qw["z"], qw["q"], desc.w_bits, desc.w_grid)

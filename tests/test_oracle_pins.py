@@ -388,3 +388,62 @@ def test_mremp_queue_is_fifo_fill_phase_is_sequential_and_lambda_follows_the_sch
             assert x_t == 1000 * n + (t - 1 - k) and x_s == -x_t          # k-th most recent entry, same entry on both sides
             assert 0 <= k < t0                                            # never older than t0 steps (first in, first out)
     assert len(calls) == T * N and [c[:2] for c in calls] == [(t, n) for t in range(T) for n in range(N)]
+
+
+# ----------------------------------------------------------------------------- closed-form ternary weights (TWN rule)
+
+def test_twn_threshold_scale_and_least_squares_property():
+    rng = np.random.default_rng(3)
+    w = (rng.standard_normal((6, 40)) * 0.05).astype(np.float32)
+    w[4] = 0.0                                                  # a dead row: nothing kept, scale 0
+    t, alpha, delta = O.quantize_weight_twn(w, per_row=True)
+    assert set(np.unique(t)) <= {-1, 0, 1} and not t[4].any() and alpha[4, 0] == 0.0
+    for r in range(6):
+        a = np.abs(w[r].astype(np.float64))
+        d = 0.7 * a.mean()
+        assert delta[r, 0] == np.float32(d)
+        keep = np.abs(w[r]) > np.float32(d)
+        assert np.array_equal(t[r], (np.sign(w[r]) * keep).astype(np.int64))
+        if keep.any():
+            assert alpha[r, 0] == pytest.approx(a[keep].mean(), rel=1e-6)
+            # with the support fixed, the mean of the kept magnitudes is the least-squares scale
+            err = lambda al: ((w[r] - al * t[r]) ** 2).sum()
+            assert err(alpha[r, 0]) <= min(err(alpha[r, 0] * 1.01), err(alpha[r, 0] * 0.99))
+    # one group for the whole matrix
+    t1, a1, d1 = O.quantize_weight_twn(w, per_row=False)
+    assert a1.shape == (1, 1) and d1[0, 0] == np.float32(0.7 * np.abs(w.astype(np.float64)).mean())
+
+
+def test_twn_module_matches_torch_autograd_with_plain_straight_through():
+    """The module with closed-form ternary weights: forward = the layers on alpha * t, backward = the gradient
+    with respect to w_hat passed to w unchanged, no weight-step gradient."""
+    wl, desc, params, x = _tiny(w_bits=2, w_twn=True)
+    vl = np.array([4, 5], np.int32)
+    teacher = [{k: v.copy() for k, v in p.items()} for p in params]
+    student = [{k: (v + synth.normal(7, k + str(i), v.shape, 0.01)).astype(np.float32) for k, v in p.items()}
+               for i, p in enumerate(params)]
+    ws = O.init_weight_steps(desc, student, 1)                     # unused by this quantizer
+    a, off = O.init_act_steps(desc, student, x, vl)
+    steps = O.make_steps(ws, (a * 0.8).astype(np.float32), off)
+    r = O.forward_loss_backward(desc, teacher, student, steps, x, x, vl, lam=0.0)
+    tp, ts = _to_torch(student, steps)
+    tt, _ = _to_torch(teacher, [])
+    xs = torch.tensor(x, dtype=torch.float64)
+    cfg = dict(_cfg(desc), w_twn=True, w_per_row=desc.w_per_row)
+    f_t = R.module(xs, tt, [None] * len(tt), cfg, vl, quant=False)
+    f_s = R.module(xs, tp, ts, cfg, vl, quant=True)
+    c = 1.0 / f_s[0].numel()
+    loss = sum(c * ((a_ - b_.detach()) ** 2).sum() for a_, b_ in zip(f_s, f_t))
+    loss.backward()
+    for a_, b_ in zip(r["f_s"], f_s):
+        assert np.allclose(a_, b_.detach().numpy(), rtol=1e-9, atol=1e-11)
+    assert np.isclose(r["loss"], loss.item(), rtol=1e-10)
+    for l, g in enumerate(r["grads"]):
+        for k in O.PARAMS:
+            ref = tp[l][k].grad.numpy()
+            assert np.allclose(g[k], ref, rtol=1e-7, atol=1e-9 * np.abs(ref).max()), (l, k)
+        assert all(g["w"][k] is None for k in O.WEIGHTS)
+        assert np.allclose(g["a"], ts[l]["a"].grad.numpy(), rtol=1e-7, atol=1e-9 * np.abs(ts[l]["a"].grad.numpy()).max())
+    # every row keeps some weights and drops some: the threshold is exercised
+    q = r["caches"][0]["qw"]["W1"]["q"]
+    assert (q == 0).any() and (q != 0).any()

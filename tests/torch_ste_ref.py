@@ -35,6 +35,19 @@ def q_weight(w, s, bits, grid):
     return s * level + inside * (w - (s * z).detach()) + (s - s.detach()) * (-(z * inside)).detach()
 
 
+def q_weight_twn(w, per_row=True):
+    # closed-form ternary weights: value alpha * t, gradient passed to w unchanged
+    a = w.detach().abs()
+    g = a if per_row else a.reshape(1, -1)
+    delta = (0.7 * g.mean(-1, keepdim=True)).float()                 # the comparison is made in float32
+    w32 = (w.detach() if per_row else w.detach().reshape(1, -1)).float()
+    keep = w32.abs() > delta
+    alpha = (g * keep).sum(-1, keepdim=True) / keep.sum(-1, keepdim=True).clamp(min=1)
+    alpha = alpha.float().double()
+    what = (alpha * torch.sign(w32).double() * keep).reshape(w.shape)
+    return w + (what - w).detach()
+
+
 def layer(x, p, st, cfg, pad, quant=True):
     H = x.shape[-1]
     h = cfg["n_heads"]
@@ -53,6 +66,8 @@ def layer(x, p, st, cfg, pad, quant=True):
     def qw(name):
         if not quant or wb == 0:
             return p[name]
+        if cfg.get("w_twn"):
+            return q_weight_twn(p[name], cfg.get("w_per_row", True))
         return q_weight(p[name], st["w"][name], wb, grid)
 
     B, S, _ = x.shape
