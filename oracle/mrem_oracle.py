@@ -44,13 +44,14 @@ class ModuleDesc:
     w_bits: int = 4            # 0 = weights not quantized (bypass)
     a_bits: int = 8            # 0 = activations not quantized (bypass)
     w_grid: int = 0            # 0: Omega(b) of Eq. 1; 1: half-integer 2-bit grid {-1.5,-.5,.5,1.5}*s
-    w_twn: bool = False        # 2-bit weights by the closed-form ternary rule (threshold 0.7 mean|w|, scale = mean of the kept |w|) instead of a learnable step
     w_per_row: bool = True     # one step per output row, else one per matrix
     asym_p: bool = True        # softmax output quantized asymmetrically (unsigned codes, offset 0)
     asym_g: bool = True        # GELU output quantized asymmetrically (unsigned codes, learnable offset)
     act_dtype: str = "f64"
     loss_mean: bool = True     # True: mean over B*S*H per layer; False: the plain sum of Eq. 3
     ln_eps: float = 1e-12
+    w_twn: bool = False        # 2-bit weights by the closed-form ternary rule (threshold 0.7 mean|w|, scale = mean
+                               # of the kept |w|, per output row) instead of a learnable step
 
 
 # ----------------------------------------------------------------------------- storage
