@@ -84,7 +84,10 @@ typedef struct {
   int32_t max_seq, max_batch;  /* the workspace is sized for max_batch * max_seq tokens */
   int32_t w_bits;              /* 2, 4 or 8 */
   int32_t a_bits;              /* 8 or 4 */
-  int32_t w_grid;              /* 0: integer codes Omega(b) of Eq. 1; 1: 2-bit levels {-1.5,-.5,.5,1.5}*step */
+  int32_t w_grid;              /* 0: integer codes Omega(b) of Eq. 1; 1: 2-bit levels {-1.5,-.5,.5,1.5}*step;
+                                  2: 2-bit ternary codes by the closed-form rule named in Sec. 5.1 (per output row:
+                                  threshold 0.7 mean|w|, scale = mean of the kept |w|); no weight steps are bound,
+                                  learnt or reported, the weight gradient passes straight through */
   int32_t w_step_per_row;      /* 1: one step per output row; 0: one per matrix */
   int32_t act_asym_sites;      /* bit 0: softmax output unsigned (offset 0); bit 1: GELU output unsigned with
                                   learnable offset (Sec. 3.1: asymmetric for these two) */

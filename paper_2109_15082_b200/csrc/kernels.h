@@ -15,6 +15,16 @@ constexpr int RED_BLOCKS = 1184;    // grid of every kernel that emits per-block
 void launch_quantize_weight(const float* w, int rows, int cols, const float* steps, int per_row, int bits, int grid,
                             int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt, cudaStream_t st);
 
+// Closed-form ternary weights, one step-free rule per output row (Sec. 5.1 names it for 2-bit weights):
+// delta = 0.7 mean|w|, codes sign(w) 1[|w| > delta], scale = mean of the kept |w|; and the fused update
+// (AdamW with the gradient of w_hat passed through unchanged, then the rule on the new weights).
+void launch_ternary_quantize(const float* w, int rows, int cols, int8_t* codes, int32_t* rowsum, float* scale,
+                             void* what, int dt, cudaStream_t st);
+struct OptimScalars;
+void launch_ternary_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
+                           int train_w, int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt,
+                           cudaStream_t st);
+
 // Activation quantizer over a 2-D view x[rows, cols] with row stride ld_x:
 // z = (x - offset) / step, q = rne(clip(z, lo, hi)).  Writes int8/uint8 codes (row stride
 // ld_q8) and/or the codes as storage-type numbers (row stride ld_qt); either may be null.

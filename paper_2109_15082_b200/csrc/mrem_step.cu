@@ -237,6 +237,11 @@ void enqueue_matrix_updates(mrem_ctx* c, int l, cudaStream_t st) {
     const int pid = kMatParam[k];
     WeightBuf& w = c->wq[l][k];
     LayerGrad& g = c->grad[l];
+    if (d.w_grid == 2) {
+      launch_ternary_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->optim_sc, w.rows, w.cols, train_w,
+                            w.codes, w.rowsum, w.scale, w.what, c->dt, st);
+      continue;
+    }
     launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
                                c->w_ste_done ? g.ws[k] : nullptr, g.m_ws[k], g.v_ws[k], c->optim_sc, w.rows, w.cols,
                                d.w_bits, d.w_grid, train_w, train_s, w.codes, w.rowsum, w.scale, w.what, c->dt, st);
@@ -372,8 +377,12 @@ int32_t mrem_quantize_weights(mrem_ctx* c) {
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) {
       const LayerBind& b = c->bind[l];
-      if (!b.student[kMatParam[k]] || !b.w_steps[k]) return fail(c, MREM_ERR_ORDER, "quantize_weights: weights or steps not bound");
+      if (!b.student[kMatParam[k]] || (!b.w_steps[k] && c->d.w_grid != 2)) return fail(c, MREM_ERR_ORDER, "quantize_weights: weights or steps not bound");
       WeightBuf& w = c->wq[l][k];
+      if (c->d.w_grid == 2) {
+        launch_ternary_quantize(b.student[kMatParam[k]], w.rows, w.cols, w.codes, w.rowsum, w.scale, w.what, c->dt, c->stream);
+        continue;
+      }
       launch_quantize_weight(b.student[kMatParam[k]], w.rows, w.cols, b.w_steps[k], c->d.w_step_per_row, c->d.w_bits,
                              c->d.w_grid, w.codes, w.rowsum, w.scale, w.what, c->dt, c->stream);
     }
@@ -434,7 +443,7 @@ int32_t mrem_module_backward(mrem_ctx* c) {
   TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
   for (int l = 0; l < c->d.n_layers; ++l)
-    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k]) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
+    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k] && c->d.w_grid != 2) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   const int rc = student_backward(c, false);
   if (rc != MREM_OK) return rc;
@@ -454,7 +463,7 @@ int32_t mrem_backward_and_step(mrem_ctx* c, const mrem_optim* o) {
   TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
   for (int l = 0; l < c->d.n_layers; ++l)
-    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k]) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
+    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k] && c->d.w_grid != 2) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
                        o->weight_decay, c->stream);

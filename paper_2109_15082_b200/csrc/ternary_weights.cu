@@ -1,0 +1,215 @@
+// Closed-form ternary weights (the rule the paper names for 2-bit weights, Sec. 5.1), one block per
+// output row:  delta = 0.7 * mean|w|,  t = sign(w) * 1[|w| > delta],  alpha = mean of |w| over the kept
+// entries (0 when none is kept),  w_hat = alpha * t.  Nothing is learnt about the scale: the update is
+// AdamW on the latent weights with the gradient of w_hat passed through unchanged, followed by the same
+// rule on the new weights.  Both means are accumulated in float64 in a fixed order and the comparison
+// |w| > delta is made in float32 on float32(delta), so the codes are a function of the stored weights
+// alone.  Two kernels share the row routine: the stand-alone quantizer and the fused update.
+#include "optim.cuh"
+
+namespace mrem {
+
+namespace {
+
+constexpr int TW_THREADS = 256;
+constexpr int TW_MAXV = 4;                 // float4 vectors per thread kept in registers: rows up to 4096 wide
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double block_sum_d(double v, double* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_sum_d(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  double r = (lane < nw) ? sh[lane] : 0.0;
+  return warp_sum_d(r);
+}
+__device__ __forceinline__ int block_sum_i(int v, int* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_sum_i(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  int r = (lane < nw) ? sh[lane] : 0;
+  return warp_sum_i(r);
+}
+
+template <typename T>
+__device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);
+template <>
+__device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+template <>
+__device__ __forceinline__ void store4<bf16>(bf16* p, float a, float b, float c, float d) {
+  uint2 t;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&t);
+  h[0] = __floats2bfloat162_rn(a, b);
+  h[1] = __floats2bfloat162_rn(c, d);
+  *reinterpret_cast<uint2*>(p) = t;
+}
+
+__device__ __forceinline__ int tern(float w, float delta) { return fabsf(w) > delta ? (w > 0.f ? 1 : -1) : 0; }
+
+// The rule on one row.  `cached`: the row sits in wr[] (vector c = threadIdx.x + i * TW_THREADS), else it is re-read
+// from w_row.  Writes codes, row sum, scale and the dequantized row.
+template <typename T>
+__device__ __forceinline__ void ternary_row(const float4* wr, bool cached, const float* w_row, int cols, int row,
+                                            int8_t* codes_row, int32_t* rowsum, float* scale, T* what_row,
+                                            double* shd, int* shi) {
+  const int nvec = cols / 4;
+  double s = 0.0;
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < TW_MAXV; ++i) {
+      const int c = threadIdx.x + i * TW_THREADS;
+      if (c < nvec) s += (double)fabsf(wr[i].x) + (double)fabsf(wr[i].y) + (double)fabsf(wr[i].z) + (double)fabsf(wr[i].w);
+    }
+  } else {
+    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) {
+      const float4 v = reinterpret_cast<const float4*>(w_row)[c];
+      s += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
+    }
+  }
+  s = block_sum_d(s, shd);
+  const float delta = (float)(0.7 * (s / (double)cols));
+  double ks = 0.0;
+  int cnt = 0;
+  auto acc = [&](float4 v) {
+    if (fabsf(v.x) > delta) { ks += (double)fabsf(v.x); ++cnt; }
+    if (fabsf(v.y) > delta) { ks += (double)fabsf(v.y); ++cnt; }
+    if (fabsf(v.z) > delta) { ks += (double)fabsf(v.z); ++cnt; }
+    if (fabsf(v.w) > delta) { ks += (double)fabsf(v.w); ++cnt; }
+  };
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < TW_MAXV; ++i) {
+      const int c = threadIdx.x + i * TW_THREADS;
+      if (c < nvec) acc(wr[i]);
+    }
+  } else {
+    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) acc(reinterpret_cast<const float4*>(w_row)[c]);
+  }
+  ks = block_sum_d(ks, shd);
+  cnt = block_sum_i(cnt, shi);
+  const float alpha = (float)(ks / (double)(cnt > 0 ? cnt : 1));
+  int sum = 0;
+  auto emit = [&](int c, float4 v) {
+    const int q0 = tern(v.x, delta), q1 = tern(v.y, delta), q2 = tern(v.z, delta), q3 = tern(v.w, delta);
+    *reinterpret_cast<uint32_t*>(codes_row + 4 * c) =
+        (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) | ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
+    if (what_row) store4<T>(what_row + 4 * c, alpha * (float)q0, alpha * (float)q1, alpha * (float)q2, alpha * (float)q3);
+    sum += q0 + q1 + q2 + q3;
+  };
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < TW_MAXV; ++i) {
+      const int c = threadIdx.x + i * TW_THREADS;
+      if (c < nvec) emit(c, wr[i]);
+    }
+  } else {
+    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) emit(c, reinterpret_cast<const float4*>(w_row)[c]);
+  }
+  sum = block_sum_i(sum, shi);
+  if (threadIdx.x == 0) {
+    rowsum[row] = sum;
+    scale[row] = alpha;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(TW_THREADS) ternary_quantize_kernel(const float* __restrict__ w, int cols,
+                                                                      int8_t* __restrict__ codes,
+                                                                      int32_t* __restrict__ rowsum,
+                                                                      float* __restrict__ scale, T* __restrict__ what) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ double shd[32];
+  __shared__ int shi[32];
+  const int row = blockIdx.x;
+  const long long base = (long long)row * cols;
+  const int nvec = cols / 4;
+  const bool cached = nvec <= TW_MAXV * TW_THREADS;
+  float4 wr[TW_MAXV];
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < TW_MAXV; ++i) {
+      const int c = threadIdx.x + i * TW_THREADS;
+      if (c < nvec) wr[i] = reinterpret_cast<const float4*>(w + base)[c];
+    }
+  }
+  ternary_row<T>(wr, cached, w + base, cols, row, codes + base, rowsum, scale, what ? what + base : nullptr, shd, shi);
+}
+
+// AdamW on the row (gradient of w_hat passed through unchanged), then the rule on the new weights.
+template <typename T>
+__global__ void __launch_bounds__(TW_THREADS) ternary_update_kernel(float* __restrict__ w, const float* __restrict__ g,
+                                                                    float* __restrict__ m, float* __restrict__ v,
+                                                                    const OptimScalars* __restrict__ sc, int cols,
+                                                                    int train_w, int8_t* __restrict__ codes,
+                                                                    int32_t* __restrict__ rowsum,
+                                                                    float* __restrict__ scale, T* __restrict__ what) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ double shd[32];
+  __shared__ int shi[32];
+  const int row = blockIdx.x;
+  const OptimScalars o = *sc;
+  const long long base = (long long)row * cols;
+  const int nvec = cols / 4;
+  const bool cached = nvec <= TW_MAXV * TW_THREADS;
+  float4* w4 = reinterpret_cast<float4*>(w + base);
+  const float4* g4 = reinterpret_cast<const float4*>(g + base);
+  float4* m4 = reinterpret_cast<float4*>(m + base);
+  float4* v4 = reinterpret_cast<float4*>(v + base);
+  float4 wr[TW_MAXV];
+  auto upd = [&](int c) {
+    float4 wv = w4[c];
+    if (train_w) {
+      const float4 d = g4[c];
+      float4 mm = m4[c], vv = v4[c];
+      wv.x = adam_one(wv.x, d.x, mm.x, vv.x, o, 1.f, -INFINITY);
+      wv.y = adam_one(wv.y, d.y, mm.y, vv.y, o, 1.f, -INFINITY);
+      wv.z = adam_one(wv.z, d.z, mm.z, vv.z, o, 1.f, -INFINITY);
+      wv.w = adam_one(wv.w, d.w, mm.w, vv.w, o, 1.f, -INFINITY);
+      w4[c] = wv;
+      m4[c] = mm;
+      v4[c] = vv;
+    }
+    return wv;
+  };
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < TW_MAXV; ++i) {
+      const int c = threadIdx.x + i * TW_THREADS;
+      if (c < nvec) wr[i] = upd(c);
+    }
+  } else {
+    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) upd(c);
+    __syncthreads();                     // the row is re-read below by other threads of the block
+  }
+  ternary_row<T>(wr, cached, w + base, cols, row, codes + base, rowsum, scale, what ? what + base : nullptr, shd, shi);
+}
+
+}  // namespace
+
+void launch_ternary_quantize(const float* w, int rows, int cols, int8_t* codes, int32_t* rowsum, float* scale,
+                             void* what, int dt, cudaStream_t st) {
+  Scope sc("quantize_weight", (double)rows * cols * (5.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)) + rows * 8.0, 0, st);
+  if (dt == 1) launch_k(ternary_quantize_kernel<bf16>, rows, TW_THREADS, 0, st, w, cols, codes, rowsum, scale, (bf16*)what);
+  else launch_k(ternary_quantize_kernel<float>, rows, TW_THREADS, 0, st, w, cols, codes, rowsum, scale, (float*)what);
+}
+
+void launch_ternary_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
+                           int train_w, int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt,
+                           cudaStream_t st) {
+  Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
+  if (dt == 1) launch_k(ternary_update_kernel<bf16>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, codes, rowsum, scale, (bf16*)what);
+  else launch_k(ternary_update_kernel<float>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, codes, rowsum, scale, (float*)what);
+}
+
+}  // namespace mrem

@@ -26,8 +26,9 @@ class Problem:
         a_bits = a_bits or wl.a_bits
         self.m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, a_bits,
                              wl.w_grid, w_per_row, asym, wl.act_dtype, loss_mean)
-        self.desc = O.ModuleDesc(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.w_bits, a_bits, wl.w_grid,
-                                 w_per_row, bool(asym & 1), bool(asym & 2), wl.act_dtype, loss_mean)
+        self.twn = wl.w_grid == 2                                    # closed-form ternary weights: no weight steps
+        self.desc = O.ModuleDesc(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.w_bits, a_bits, 0 if self.twn else wl.w_grid,
+                                 w_per_row, bool(asym & 1), bool(asym & 2), wl.act_dtype, loss_mean, w_twn=self.twn)
         m = self.m
         m.load_teacher(synth.teacher_params(wl, seed, bias_std=bias_std))
         m.init_student_from_teacher()
@@ -85,7 +86,7 @@ class Problem:
             g["w"] = {}
             for k, pid in enumerate((B.WQKV, B.WO, B.W1, B.W2)):
                 n = m.shapes[pid][0] if m.per_row else 1
-                g["w"][B.PARAM_NAMES[pid]] = m.grad(l, B.GRAD_STEP + k, (n,)).cpu().numpy()
+                g["w"][B.PARAM_NAMES[pid]] = None if self.twn else m.grad(l, B.GRAD_STEP + k, (n,)).cpu().numpy()
             g["a"] = np.array([m.grad(l, B.GRAD_STEP + 4 + s, (1,)).item() for s in range(8)])
             g["a_off"] = np.array([m.grad(l, B.GRAD_OFFSET + 4 + s, (1,)).item() for s in range(8)])
             gs.append(g)
@@ -107,7 +108,7 @@ def compare_grads(gpu, ora, tol, skip_small=1e-12, check_offset=True):
     worst = ("", 0.0)
     for l, (g, r) in enumerate(zip(gpu, ora)):
         items = [(k, g[k], r[k]) for k in O.PARAMS]
-        items += [("s_" + k, g["w"][k], r["w"][k]) for k in O.WEIGHTS]
+        items += [("s_" + k, g["w"][k], r["w"][k]) for k in O.WEIGHTS if r["w"][k] is not None]
         if check_offset:
             items += [("a_off", g["a_off"][7:8], r["a_off"][7:8])]
         # activation step gradients are scalars: compare each one on its own; a scalar that is a

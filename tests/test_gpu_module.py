@@ -552,3 +552,45 @@ def test_degenerate_inputs_match_the_oracle():
             assert np.all(np.isfinite(g["grads"][0][k]))
     finally:
         p.close()
+
+
+def test_closed_form_ternary_weights_match_the_oracle():
+    """w_grid = 2: ternary codes and scales by the closed-form rule.  Codes bit exact before the step and, from the
+    updated weights, after it; forward, loss and every gradient against the oracle; no weight-step gradient."""
+    wl = _wl("base3_w2a8", n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40, w_grid=2)
+    p = Problem(wl, student_noise=0.002)
+    try:
+        m = p.m
+        g = p.run_gpu()
+        r = p.run_oracle()
+        for l in range(wl.n_layers):
+            assert rel(g["f_t"][l], r["f_t"][l]) < FWD_TOL["bf16"] and rel(g["f_s"][l], r["f_s"][l]) < FWD_TOL["bf16"]
+            for pid, name in ((B.WQKV, "Wqkv"), (B.WO, "Wo"), (B.W1, "W1"), (B.W2, "W2")):
+                codes, rowsum = m.weight_codes(l, pid)
+                ref = r["caches"][l]["qw"][name]["q"]
+                assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref)
+                assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1))
+                assert set(np.unique(ref)) == {-1, 0, 1}
+        assert abs(g["loss"] - r["loss"]) / r["loss"] < GRAD_TOL
+        compare_grads(g["grads"], r["grads"], GRAD_TOL, check_offset=False)
+        with pytest.raises(B.MremError):
+            m.grad(0, B.GRAD_STEP + 0, (1,))
+        before = m.student_numpy()
+        grads = p.gpu_grads()
+        opt = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+        m.step(B.make_optim(step=1, **opt))
+        torch.cuda.synchronize()
+        after = m.student_numpy()
+        for l in range(wl.n_layers):
+            for pid, name in ((B.WQKV, "Wqkv"), (B.W2, "W2")):
+                z = np.zeros_like(before[l][name], np.float64)
+                ref_w, _, _ = O.adamw_update(before[l][name], grads[l][name], z, z.copy(), 1, opt["lr"], 0.9, 0.999, 1e-8, 0.01)
+                assert np.allclose(after[l][name], ref_w, rtol=1e-5, atol=2e-3 * opt["lr"])
+                codes, rowsum = m.weight_codes(l, pid)
+                ref = O.quantize_weight_twn(after[l][name], True)[0]
+                assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref), (l, name)
+        # and the next forward runs on the new codes
+        g2 = p.run_gpu()
+        assert np.isfinite(g2["loss"]) and g2["loss"] != g["loss"]
+    finally:
+        p.close()
