@@ -130,8 +130,9 @@ def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    # each step is a bounded sample: the full batch for short runs, a quarter of it for long ones
-    batch = wl.batch if args.steps <= 5 else max(2, wl.batch // 4)
+    # each step is a bounded sample of the batch, sized so that the whole run stays within a few minutes: one
+    # sequence through one layer of the module costs the oracle about 0.2 s on 16 cores
+    batch = max(1, min(wl.batch, 700 // max(args.steps + min(args.warmup, 1), 1)))
     val, threads, sample, sec = oracle_sample(wl, n_steps=max(1, args.steps), warmup=min(args.warmup, 1), batch=batch)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec * wl.n_layers,
