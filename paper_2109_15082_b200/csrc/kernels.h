@@ -113,7 +113,7 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
 // with a2 also out2[c] = sum_r a2[r,c].  One kernel: per-chunk partials in `scratch` (>= 3*COL_CHUNKS*cols
 // floats), summed in index order by the last block of each column group.  `counters` (>= cols/32 + 1 ints)
 // must be zero before the first launch; the kernel leaves them zero.
-constexpr int COL_CHUNKS = 64;
+constexpr int COL_CHUNKS = 32;
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
                        const void* a2, long long ld_a2, long long rows, int cols, float* out0, float* out1,
                        float* out2, float* scratch, int* counters, int dt, cudaStream_t st);
