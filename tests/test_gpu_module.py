@@ -300,6 +300,27 @@ def test_call_order_and_argument_errors():
         with pytest.raises(B.MremError) as e:
             m.step(B.make_optim())
         assert e.value.code == -5
+        with pytest.raises(B.MremError) as e:
+            m.backward_and_step(B.make_optim())                         # no loss of this step yet
+        assert e.value.code == -5
+        # the host-buffer step in two halves: at most two in flight, nothing to wait for when none is
+        with pytest.raises(B.MremError) as e:
+            B.mrem_recon_step_host_wait(m.ctx)
+        assert e.value.code == -5
+        xh = p.xd.cpu().contiguous().pin_memory()
+        vh = torch.from_numpy(p.vl).pin_memory()
+        opt = B.make_optim(lr=1e-5, step=1)                             # explicit step number: the eager form of the step
+        B.mrem_recon_step_host_submit(m.ctx, xh, xh, vh, wl.batch, wl.seq, 0.0, opt)
+        B.mrem_recon_step_host_submit(m.ctx, xh, xh, vh, wl.batch, wl.seq, 0.0, opt)
+        with pytest.raises(B.MremError) as e:
+            B.mrem_recon_step_host_submit(m.ctx, xh, xh, vh, wl.batch, wl.seq, 0.0, opt)
+        assert e.value.code == -5
+        with pytest.raises(B.MremError) as e:
+            B.mrem_recon_step_host(m.ctx, xh, xh, vh, wl.batch, wl.seq, 0.0, opt)   # the blocking form needs an empty queue
+        assert e.value.code == -5
+        l0 = B.mrem_recon_step_host_wait(m.ctx)
+        l1 = B.mrem_recon_step_host_wait(m.ctx)
+        assert np.isfinite(l0) and np.isfinite(l1) and l0 != l1
         torch.cuda.synchronize()
         assert m.poll_status() == 0
     finally:
