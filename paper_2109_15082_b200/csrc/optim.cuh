@@ -26,10 +26,15 @@ __device__ __forceinline__ float adam_one(float p, float g, float& m, float& v, 
 
 // Straight-through factors of the weight quantizer at z = w / s: whether the gradient passes to w,
 // and the level d w_hat / d s is measured from (code on the integer grid, k + 0.5 on the half-integer one).
+// Round to nearest even without the conversion unit: adding and subtracting 1.5 * 2^23 leaves rint(x) for
+// |x| < 2^22 (codes are at most 127 in magnitude); the sum's low mantissa bits are the integer itself.
+constexpr float RINT_MAGIC = 12582912.f;
+__device__ __forceinline__ float rint_small(float x) { return __fsub_rn(__fadd_rn(x, RINT_MAGIC), RINT_MAGIC); }
+
 __device__ __forceinline__ void weight_ste(float z, float qmax, int grid, bool& in, float& level) {
   if (grid == 0) {
     in = z >= -qmax && z <= qmax;
-    level = (float)__float2int_rn(fminf(fmaxf(z, -qmax), qmax));
+    level = rint_small(fminf(fmaxf(z, -qmax), qmax));
   } else {
     in = z >= -2.f && z < 2.f;
     level = fminf(fmaxf(floorf(z), -2.f), 1.f) + 0.5f;

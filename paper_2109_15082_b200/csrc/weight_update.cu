@@ -17,10 +17,18 @@ namespace mrem {
 namespace {
 
 
-__device__ __forceinline__ int weight_code(float w, float s, float qmax, int grid) {
+// Code of Eq. 1 and the same value as a float.  Integer grid: the sum with 1.5 * 2^23 holds the code in its
+// low mantissa bits (two's complement), so neither direction goes through the conversion unit.
+__device__ __forceinline__ int weight_code(float w, float s, float qmax, int grid, float& qf) {
   const float z = __fdiv_rn(w, s);
-  if (grid == 0) return __float2int_rn(fminf(fmaxf(z, -qmax), qmax));
-  return 2 * (int)fminf(fmaxf(floorf(z), -2.f), 1.f) + 1;
+  if (grid == 0) {
+    const float t = __fadd_rn(fminf(fmaxf(z, -qmax), qmax), RINT_MAGIC);
+    qf = __fsub_rn(t, RINT_MAGIC);
+    return (int)(int8_t)(__float_as_uint(t) & 0xffu);
+  }
+  const int q = 2 * (int)fminf(fmaxf(floorf(z), -2.f), 1.f) + 1;
+  qf = (float)q;
+  return q;
 }
 
 template <typename T>
@@ -134,11 +142,12 @@ __global__ void __launch_bounds__(NT, NT == 256 ? 6 : 2) fused_weight_update_ker
       m4[c] = mm;
       v4[c] = vv;
     }
-    const int q0 = weight_code(wv.x, s_new, qmax, grid), q1 = weight_code(wv.y, s_new, qmax, grid);
-    const int q2 = weight_code(wv.z, s_new, qmax, grid), q3 = weight_code(wv.w, s_new, qmax, grid);
+    float f0, f1, f2, f3;
+    const int q0 = weight_code(wv.x, s_new, qmax, grid, f0), q1 = weight_code(wv.y, s_new, qmax, grid, f1);
+    const int q2 = weight_code(wv.z, s_new, qmax, grid, f2), q3 = weight_code(wv.w, s_new, qmax, grid, f3);
     *reinterpret_cast<uint32_t*>(codes + base + 4 * c) =
         (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) | ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
-    if (what) store_what4<T>(what + base + 4 * c, sc_new * (float)q0, sc_new * (float)q1, sc_new * (float)q2, sc_new * (float)q3);
+    if (what) store_what4<T>(what + base + 4 * c, sc_new * f0, sc_new * f1, sc_new * f2, sc_new * f3);
     sum += q0 + q1 + q2 + q3;
   };
   if (cached) {
