@@ -10,7 +10,8 @@ namespace tc {
 
 constexpr int BLOCK_M = 128;
 constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
-constexpr int TILE_SMEM_BUDGET = 196608;              // bytes of operand stages per CTA
+constexpr int TILE_SMEM_BUDGET = 196608;              // bytes of operand stages per CTA (CTA-pair kernel, beside its staging)
+constexpr int SINGLE_CTA_SMEM_BUDGET = 229376;        // bytes of operand stages per CTA (single-CTA kernel: no staging)
 constexpr int MAX_STAGES = 8;
 constexpr int GEMM_THREADS = 320;                    // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_WARPS = 8;
@@ -240,6 +241,192 @@ __device__ __forceinline__ void epilogue_round(const TcParams& p, uint32_t taddr
     }
   }
   __syncwarp();
+}
+
+
+// ------------------------------------------------------------------ register-direct epilogue
+// One warp drains its 32 accumulator rows (TMEM lane = row = lane of the warp) over a range of columns in
+// chunks of 32: tcgen05.ld gives every lane 32 consecutive columns of its row, the lane applies the
+// epilogue and writes its 64 (bf16) or 128 (fp32 / int32) contiguous bytes with 32-byte vector stores, so
+// every store fills whole sectors and nothing passes through shared memory (whose bandwidth the main loop
+// needs).  The load of chunk c + 1 and the fetch of its residual are in flight while chunk c is processed.
+__device__ __forceinline__ void ldg256(const void* p, uint32_t* r) {
+  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "l"(p));
+}
+__device__ __forceinline__ void stg256(void* p, const uint32_t* r) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]),
+               "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+
+// MODE >= 0: bit 0 column scale, bit 1 column bias, bit 2 residual, bit 3 GELU, known at compile time;
+// MODE < 0: the same four read from the Epilogue at run time.
+template <int MODE> struct EpiFlags {
+  bool scale, bias, res, act;
+  __device__ __forceinline__ explicit EpiFlags(const Epilogue& e)
+      : scale(MODE >= 0 ? (MODE & 1) != 0 : e.col_scale != nullptr), bias(MODE >= 0 ? (MODE & 2) != 0 : e.col_bias != nullptr),
+        res(MODE >= 0 ? (MODE & 4) != 0 : e.residual != nullptr), act(MODE >= 0 ? (MODE & 8) != 0 : e.act == 1) {}
+};
+
+// Residual of one chunk of a bf16 output row: 32 values = 64 bytes.
+__device__ __forceinline__ void fetch_res_bf16(const Epilogue& e, long long off, bool row_ok, uint32_t* res) {
+  if (row_ok) {
+    const bf16* src = reinterpret_cast<const bf16*>(e.residual) + off;
+    ldg256(src, res);
+    ldg256(src + 16, res + 8);
+  }
+}
+
+// acc[32] of one row -> out[off .. off + 32).  `n` = global column of acc[0].
+template <int KIND, int OUT, int MODE>
+__device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* r, const uint32_t* res, float alpha, float rb,
+                                             int n, long long off, bool row_ok) {
+  if (OUT == OUT_I32) {
+    if (row_ok) {
+      int* out = reinterpret_cast<int*>(e.out) + off;
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) stg256(out + j, r + j);
+    }
+    return;
+  }
+  const EpiFlags<MODE> f(e);
+  float v[32];
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    float4 sc = make_float4(alpha, alpha, alpha, alpha), bi = make_float4(rb, rb, rb, rb);
+    if (f.scale) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(e.col_scale + n + j));
+      sc.x *= t.x; sc.y *= t.y; sc.z *= t.z; sc.w *= t.w;
+    }
+    if (f.bias) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(e.col_bias + n + j));
+      bi.x += t.x; bi.y += t.y; bi.z += t.z; bi.w += t.w;
+    }
+    const float a0 = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
+    const float a1 = (KIND == 1) ? (float)(int)r[j + 1] : __uint_as_float(r[j + 1]);
+    const float a2 = (KIND == 1) ? (float)(int)r[j + 2] : __uint_as_float(r[j + 2]);
+    const float a3 = (KIND == 1) ? (float)(int)r[j + 3] : __uint_as_float(r[j + 3]);
+    v[j] = a0 * sc.x + bi.x; v[j + 1] = a1 * sc.y + bi.y; v[j + 2] = a2 * sc.z + bi.z; v[j + 3] = a3 * sc.w + bi.w;
+  }
+  if (OUT == OUT_BF16) {
+    if (f.res) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&res[j]));
+        v[2 * j] += t.x;
+        v[2 * j + 1] += t.y;
+      }
+    }
+    if (f.act) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+    }
+    uint32_t o[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      o[j] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    if (row_ok) {
+      bf16* out = reinterpret_cast<bf16*>(e.out) + off;
+      stg256(out, o);
+      stg256(out + 16, o + 8);
+    }
+  } else {
+    if (f.res && row_ok) {
+      const float* src = reinterpret_cast<const float*>(e.residual) + off;
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint32_t t[8];
+        ldg256(src + j, t);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[j + k] += __uint_as_float(t[k]);
+      }
+    }
+    if (f.act) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+    }
+    if (row_ok) {
+      float* out = reinterpret_cast<float*>(e.out) + off;
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint32_t t[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) t[k] = __float_as_uint(v[j + k]);
+        stg256(out + j, t);
+      }
+    }
+  }
+}
+
+// `nchunks` whole chunks starting at accumulator column c0 (tile-relative) / global column n0 + c0.
+// `res0` holds the residual of the first chunk (bf16 output with residual only), fetched by the caller
+// before it waited for the accumulator.
+template <int KIND, int OUT, int MODE>
+__device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb, int n,
+                                             long long off, bool row_ok, uint32_t* res0) {
+  const bool pipelined_res = OUT == OUT_BF16 && EpiFlags<MODE>(e).res;
+  uint32_t ra[32], rb2[32], res1[16];
+  tmem_ld32_issue(taddr, ra);
+  for (int c = 0; c < nchunks; c += 2) {
+    tmem_ld_wait();
+    tmem_ld_pin(ra);
+    const bool more1 = c + 1 < nchunks;
+    if (more1) {
+      tmem_ld32_issue(taddr + 32u * (uint32_t)(c + 1), rb2);
+      if (pipelined_res) fetch_res_bf16(e, off + 32 * (c + 1), row_ok, res1);
+    }
+    finish_chunk<KIND, OUT, MODE>(e, ra, res0, alpha, rb, n + 32 * c, off + 32 * c, row_ok);
+    if (more1) {
+      tmem_ld_wait();
+      tmem_ld_pin(rb2);
+      if (c + 2 < nchunks) {
+        tmem_ld32_issue(taddr + 32u * (uint32_t)(c + 2), ra);
+        if (pipelined_res) fetch_res_bf16(e, off + 32 * (c + 2), row_ok, res0);
+      }
+      finish_chunk<KIND, OUT, MODE>(e, rb2, res1, alpha, rb, n + 32 * (c + 1), off + 32 * (c + 1), row_ok);
+    }
+  }
+}
+
+// MODE >= 0: bf16 output (fp32 with bit 4) with the epilogue terms of MODE; MODE < 0: output kind and terms read
+// at run time.
+template <int KIND, int MODE>
+__device__ __forceinline__ void drain_dispatch(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb, int n,
+                                               long long off, bool row_ok, uint32_t* res0) {
+  if (MODE >= 16) {
+    drain_chunks<KIND, OUT_F32, MODE>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+  } else if (MODE >= 0 || e.out_kind == OUT_BF16) {
+    drain_chunks<KIND, OUT_BF16, MODE>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+  } else if (e.out_kind == OUT_F32) {
+    drain_chunks<KIND, OUT_F32, -1>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+  } else {
+    drain_chunks<KIND, OUT_I32, 0>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+  }
+}
+
+// The epilogue variant a launch takes: bf16 outputs with one of the term sets the encoder uses, and plain fp32
+// outputs (the weight gradients), get a kernel compiled for exactly those terms (bit 0 column scale, bit 1
+// column bias, bit 2 residual, bit 3 GELU, bit 4 fp32 output; alpha and the row bias are always applied);
+// everything else runs the variant that reads them at run time (-1).
+inline int epilogue_mode(int kind, const Epilogue& e) {
+  const int mode = (e.col_scale ? 1 : 0) | (e.col_bias ? 2 : 0) | (e.residual ? 4 : 0) | (e.act == 1 ? 8 : 0);
+  if (e.out_kind == OUT_F32) return (kind == 0 && mode == 0) ? 16 : -1;
+  if (e.out_kind != OUT_BF16) return -1;
+  if (kind == 0) return (mode == 0 || mode == 2 || mode == 6 || mode == 10) ? mode : -1;
+  return (mode == 3 || mode == 7) ? mode : -1;
+}
+
+// True when rows of out (and residual) start on 32-byte boundaries for every row, batch and 32-column chunk,
+// and the column vectors can be fetched as float4.
+__device__ __forceinline__ bool direct_epilogue_ok(const Epilogue& e) {
+  const int per32 = e.out_kind == OUT_BF16 ? 16 : 8;
+  bool ok = (e.ldc % per32 == 0) && (e.c_b0 % per32 == 0) && (e.c_b1 % per32 == 0) && ((reinterpret_cast<uintptr_t>(e.out) & 31) == 0);
+  if (e.residual) ok = ok && ((reinterpret_cast<uintptr_t>(e.residual) & 31) == 0);
+  return ok && ((reinterpret_cast<uintptr_t>(e.col_scale) & 15) == 0) && ((reinterpret_cast<uintptr_t>(e.col_bias) & 15) == 0);
 }
 
 }  // namespace tc

@@ -3,10 +3,10 @@
 // One persistent CTA per SM.  Warp 0 streams operand tiles into a ring of shared-memory
 // stages with TMA (128-byte swizzle), warp 1 issues tcgen05.mma (bf16 -> fp32, or
 // int8 -> int32 with exact accumulation) into one of two TMEM accumulator buffers, and
-// warps 2..9 drain the other buffer with tcgen05.ld, apply the epilogue and write the
-// result through a per-warp shared-memory transpose (each store instruction then covers
-// whole 64- or 128-byte row segments), so the epilogue of tile i overlaps the main loop of
-// tile i+1.
+// warps 2..9 drain the other buffer with tcgen05.ld, apply the epilogue and write their
+// rows straight from registers with 32-byte vector stores (nothing of the epilogue passes
+// through shared memory, whose bandwidth the main loop needs), so the epilogue of tile i
+// overlaps the main loop of tile i+1.
 // Either operand may be stored k-contiguous ("K-major") or m/n-contiguous ("MN-major");
 // the second form serves the backward products (dX = dY * W_hat, dW = dY^T * X_hat) and
 // the attention products without any transposed copy.
@@ -26,7 +26,7 @@ using namespace tc;
 namespace {
 
 // ------------------------------------------------------------------ the kernel
-template <int KIND>
+template <int KIND, int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ TcParams p) {
@@ -150,25 +150,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ---------------- epilogue warps: TMEM lane quadrant = warp % 4, two warps per quadrant
+    // ---------------- epilogue warps: TMEM lane quadrant = warp % 4, two warps per quadrant, each draining
+    // its 32 rows over one half of the tile's columns
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const Epilogue& e = p.epi;
     float alpha = e.alpha_const;
     if (e.alpha_p0) alpha *= *e.alpha_p0;
     if (e.alpha_p1) alpha *= *e.alpha_p1;
-    const int esz = (e.out_kind == OUT_BF16) ? 2 : 4;
-    const int vec_elems = 16 / esz;
-    bool vec_ok = (e.ldc % vec_elems == 0) && (e.c_b0 % vec_elems == 0) && (e.c_b1 % vec_elems == 0) &&
-                  ((reinterpret_cast<uintptr_t>(e.out) & 15) == 0);
-    if (e.residual) vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(e.residual) & 15) == 0);
-    vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(e.col_scale) & 15) == 0) && ((reinterpret_cast<uintptr_t>(e.col_bias) & 15) == 0);
-    uint32_t* stg = reinterpret_cast<uint32_t*>(smem_raw + (tiles_base - smem_u32(smem_raw)) +
-                                                (size_t)p.num_stages * p.stage_bytes) + (warp - 2) * STAGING_WORDS;
-    const int cols_per_round = (e.out_kind == OUT_BF16) ? 64 : 32;
+    const bool direct = direct_epilogue_ok(e);
+    const bool res_bf16 = e.residual != nullptr && e.out_kind == OUT_BF16;
+    const int cols_per_warp = p.block_n >> 1, c_begin = half * cols_per_warp;
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const TileCoord t = decode_tile(p, tile);
+      const int row = t.m0 + quad * 32 + lane, col_begin = t.n0 + c_begin;
+      const bool row_ok = row < p.M;
+      const long long row_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1 + (long long)row * e.ldc;
+      // whole 32-column chunks of this warp's range that lie inside N take the register-direct path
+      int nfull = 0;
+      if (direct && col_begin < p.N) nfull = min((p.N - col_begin) >> 5, cols_per_warp >> 5);
+      uint32_t res0[16];
+      if (nfull > 0 && res_bf16) fetch_res_bf16(e, row_off + col_begin, row_ok, res0);   // in flight during the wait
+      const float rb = (e.row_bias && row_ok) ? e.row_bias[row] : 0.f;
       // every lane polls; the decision is made warp-uniform before any .sync.aligned instruction
       const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort);
       if (!__all_sync(0xffffffffu, got)) {
@@ -176,24 +180,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         break;
       }
       tc_fence_after();
-      const int row0 = t.m0 + quad * 32;
-      const long long tile_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * p.block_n);
-      for (int round = half; round * cols_per_round < p.block_n; round += 2) {
-        const int c0 = round * cols_per_round, col0 = t.n0 + c0;
-        if (col0 >= p.N) break;                          // warp-uniform
-        const bool fast = vec_ok && col0 + cols_per_round <= p.N;
-        if (fast) {
-          epilogue_round<KIND>(p, taddr + (uint32_t)c0, alpha, tile_off, row0, col0, lane, stg);
-        } else {
-          const int row = row0 + lane;
-          const long long row_off = tile_off + (long long)row * e.ldc;
-          for (int c = c0; c < c0 + cols_per_round && t.n0 + c < p.N; c += 32) {
-            uint32_t r[32];
-            tmem_ld32(taddr + (uint32_t)c, r);
-            epilogue_chunk<KIND>(p, r, alpha, row_off, row, t.n0 + c, row < p.M, false);
-          }
-        }
+      if (nfull > 0) drain_dispatch<KIND, MODE>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, col_begin, row_off + col_begin, row_ok, res0);
+      for (int c = c_begin + 32 * nfull; c < c_begin + cols_per_warp && t.n0 + c < p.N; c += 32) {   // ragged or unaligned rest
+        uint32_t r[32];
+        tmem_ld32(taddr + (uint32_t)c, r);
+        epilogue_chunk<KIND>(p, r, alpha, row_off, row, t.n0 + c, row_ok, false);
       }
       tc_fence_before();
       __syncwarp();
@@ -301,7 +293,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   p.k_blocks = (g.K + p.block_k - 1) / p.block_k;
   p.num_tiles = p.m_tiles * p.n_tiles * g.nb0 * g.nb1;
   p.stage_bytes = A_STAGE_BYTES + p.block_n * 128;
-  p.num_stages = TILE_SMEM_BUDGET / p.stage_bytes;
+  p.num_stages = SINGLE_CTA_SMEM_BUDGET / p.stage_bytes;
   if (p.num_stages > MAX_STAGES) p.num_stages = MAX_STAGES;
   p.a_mn = A.mn_contig; p.b_mn = B.mn_contig;
   p.epi = epi;
@@ -329,13 +321,22 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   rc = make_operand_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k);
   if (rc != GEMM_OK) return rc;
 
-  const int smem = p.num_stages * p.stage_bytes + 1024 + STAGING_BYTES;
-  static bool attr_set[2] = {false, false};
-  auto kern = kind == 0 ? tc_gemm_kernel<0> : tc_gemm_kernel<1>;
-  if (!attr_set[kind]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TILE_SMEM_BUDGET + 1024 + STAGING_BYTES) != cudaSuccess)
+  const int smem = p.num_stages * p.stage_bytes + 1024;
+  typedef void (*Kern)(const CUtensorMap, const CUtensorMap, const TcParams);
+  static const struct { int kind, mode; Kern fn; } variants[] = {
+      {0, -1, tc_gemm_kernel<0, -1>}, {0, 0, tc_gemm_kernel<0, 0>}, {0, 2, tc_gemm_kernel<0, 2>}, {0, 6, tc_gemm_kernel<0, 6>},
+      {0, 10, tc_gemm_kernel<0, 10>}, {0, 16, tc_gemm_kernel<0, 16>}, {1, -1, tc_gemm_kernel<1, -1>}, {1, 3, tc_gemm_kernel<1, 3>}, {1, 7, tc_gemm_kernel<1, 7>}};
+  constexpr int n_variants = sizeof(variants) / sizeof(variants[0]);
+  static bool attr_set[n_variants] = {};
+  const int mode = epilogue_mode(kind, epi);
+  int vi = 0;
+  while (vi < n_variants && !(variants[vi].kind == kind && variants[vi].mode == mode)) ++vi;
+  if (vi == n_variants) return GEMM_ERR_ARG;
+  Kern kern = variants[vi].fn;
+  if (!attr_set[vi]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SINGLE_CTA_SMEM_BUDGET + 1024) != cudaSuccess)
       return GEMM_ERR_CUDA;
-    attr_set[kind] = true;
+    attr_set[vi] = true;
   }
   const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
   Scope sc([&] {
