@@ -110,13 +110,14 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
                           cudaStream_t st);
 
 // Column sums over rows: out0[c] = sum_r a[r,c]; with y/mean/rstd also out1[c] = sum_r a[r,c]*(y[r,c]-mean[r])*rstd[r];
-// with a2 also out2[c] = sum_r a2[r,c].  One kernel: per-chunk partials in `scratch` (>= 3*COL_CHUNKS*cols
-// floats), summed in index order by the last block of each column group.  `counters` (>= cols/32 + 1 ints)
-// must be zero before the first launch; the kernel leaves them zero.
-constexpr int COL_CHUNKS = 32;
+// with a2 also out2[c] = sum_r a2[r,c].  One kernel: per-chunk partials in `scratch` (three planes of
+// `plane_floats` floats each, plane_floats >= cols; the launcher takes as many row chunks as a plane holds),
+// summed in a fixed order by the last block of each column group.  `counters` (>= cols/32 + 1 ints) must be
+// zero before the first launch; the kernel leaves them zero.
+constexpr int COL_CHUNKS = 32;      // row chunks a scratch plane holds at the widest tensor
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
                        const void* a2, long long ld_a2, long long rows, int cols, float* out0, float* out1,
-                       float* out2, float* scratch, int* counters, int dt, cudaStream_t st);
+                       float* out2, float* scratch, long long plane_floats, int* counters, int dt, cudaStream_t st);
 
 // Weight STE: dW = dWhat * inside (in place), ds[row] = sum_k dWhat * d what/d s.
 void launch_ste_weight(const float* w, const float* steps, int per_row, int bits, int grid, float* dw, int rows,

@@ -72,7 +72,8 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->minmax = (float*)A.take(256);
   c->d_loss_e2e = (float*)A.take(256);
   c->loss_partial = (float*)A.take(sizeof(float) * RED_BLOCKS * L);
-  c->col_scratch = (float*)A.take(sizeof(float) * 3 * COL_CHUNKS * (3 * H > F ? 3 * H : F));
+  c->col_plane = (long long)COL_CHUNKS * (3 * H > F ? 3 * H : F);
+  c->col_scratch = (float*)A.take(sizeof(float) * 3 * c->col_plane);
   c->col_counters = (int*)A.take(sizeof(int) * ((3 * H > F ? 3 * H : F) / 32 + 2));
   c->rowbias = (float*)A.take(sizeof(float) * (3 * H > F ? 3 * H : F));
   c->reduce_per_layer = N_SITES + 1 + N_WMAT;

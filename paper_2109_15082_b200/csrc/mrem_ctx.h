@@ -89,6 +89,7 @@ struct mrem_ctx {
   void *d_y2, *d_ghat, *d_u, *d_ahat, *d_a, *d_y1, *d_ctxhat, *d_ctx, *d_phat, *d_s, *d_qkvhat, *d_qkv, *d_xhat,
       *d_sum, *carry[2];
   float* col_scratch;
+  long long col_plane = 0;               // floats per plane of col_scratch
   int* col_counters;
   float* rowbias;
   float* loss_partial;

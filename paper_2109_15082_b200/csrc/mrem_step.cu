@@ -294,7 +294,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     // (column sums feed only the update and the weight-gradient epilogue: side stream)
     fork();
     launch_col_reduce(carry ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, c->d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
-                      g.p[MREM_B2], c->col_scratch, c->col_counters, c->dt, side);
+                      g.p[MREM_B2], c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
     {
       Epi e(g.p[MREM_W2], OUT_F32, F);
@@ -306,7 +306,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
                     part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
     // FFN1:  u = A_hat W1_hat^T + b1
     fork();
-    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, side);
+    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
     rw.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
@@ -316,7 +316,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x  (its bias gradient rides along)
     fork();
     launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
-                      c->col_scratch, c->col_counters, c->dt, side);
+                      c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
     rw.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
@@ -343,22 +343,23 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     }
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
     fork();
-    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_counters, c->dt, side);
+    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
     rw.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
     void* next_carry = c->carry[l & 1];
     launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
                    part + S_X * RED_BLOCKS, nullptr, c->dt, st);
     carry = next_carry;
-    // weight quantizers: mask the latent-weight gradients, reduce the step gradients
     // (the weight quantizers' masks and step gradients are applied inside the fused update of mrem_step,
     //  or on demand by mrem_get_grad)
-    launch_reduce_table(c->reduce_table + (size_t)l * c->reduce_per_layer, c->reduce_per_layer, st);
     // the layer below overwrites d_y2, d_u, d_y1, d_qkv and the bias row the weight-gradient products read
     join();
     // nothing below reads what the update writes: the latent weights, moments, row steps and this layer's codes
     if (update_as_you_go) enqueue_matrix_updates(c, l, side);
   }
+  // step-size and offset gradients of every layer's activation quantizers: the per-block partial sums the
+  // kernels above left, added in index order (one launch for the whole module; only the update reads them)
+  launch_reduce_table(c->reduce_table, c->reduce_per_layer * d.n_layers, c->stream);
   join();
   if (sync_failed) return fail(c, MREM_ERR_CUDA, "backward: stream fork/join failed");
   if (rw.rc != MREM_OK) { c->err = "weight-gradient GEMM launch failed"; return rw.rc; }

@@ -199,81 +199,99 @@ __global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout,
 
 // ------------------------------------------------------------------ column sums over rows
 // out0[c] = sum_r a[r,c];  out1[c] = sum_r a[r,c] * (y[r,c] - mean[r]) * rstd[r] (when y);  out2[c] = sum_r a2[r,c]
-// (when a2).  Block (32 x 8) owns 32*V columns of one chunk of rows and adds its 8 row groups in a
-// fixed order; the last block to finish a column group (ticket counter) adds the chunks' partials in
-// index order, so the result does not depend on scheduling.
+// (when a2).  A block of 8 x 32 threads owns 8*V columns (one 128-byte line per row for 16-byte vectors) of
+// one chunk of rows (gridDim.y chunks): a thread keeps four rows' loads in flight and adds them in row
+// order, the block adds its 32 row groups in index order; the last block to finish a column group (ticket
+// counter) adds the chunks' partials in index order, so the result does not depend on scheduling.
+constexpr int COLRED_CT = 8, COLRED_RT = 32;
 template <typename T, int V>
-__global__ void __launch_bounds__(256) col_reduce_kernel(const T* __restrict__ a, long long ld_a,
-                                                         const T* __restrict__ y, const float* __restrict__ mean,
-                                                         const float* __restrict__ rstd, const T* __restrict__ a2,
-                                                         long long ld_a2, long long rows, int cols,
-                                                         float* __restrict__ out0, float* __restrict__ out1,
-                                                         float* __restrict__ out2, float* __restrict__ scratch,
-                                                         int* __restrict__ counters) {
+__global__ void __launch_bounds__(256, 2) col_reduce_kernel(const T* __restrict__ a, long long ld_a,
+                                                            const T* __restrict__ y, const float* __restrict__ mean,
+                                                            const float* __restrict__ rstd, const T* __restrict__ a2,
+                                                            long long ld_a2, long long rows, int cols,
+                                                            float* __restrict__ out0, float* __restrict__ out1,
+                                                            float* __restrict__ out2, float* __restrict__ scratch,
+                                                            long long plane, int* __restrict__ counters) {
   pdl_trigger();
   pdl_wait();
-  __shared__ float sh[3][8][32 * V + 1];
+  constexpr int BC = COLRED_CT * V;                        // columns per block
+  __shared__ float sh[3][COLRED_RT][BC + 1];
   __shared__ int is_last;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int c = (blockIdx.x * 32 + tx) * V;
-  const long long per = (rows + COL_CHUNKS - 1) / COL_CHUNKS;
+  const int tx = threadIdx.x % COLRED_CT, ty = threadIdx.x / COLRED_CT;
+  const int c = blockIdx.x * BC + tx * V;
+  const int chunks = gridDim.y;
+  const long long per = (rows + chunks - 1) / chunks;
   const long long r0 = blockIdx.y * per, r1 = r0 + per < rows ? r0 + per : rows;
   float a0[V], a1[V], a2s[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) a0[j] = a1[j] = a2s[j] = 0.f;
   if (c < cols) {
-    for (long long r = r0 + ty; r < r1; r += 8) {
-      float v[V];
-      load_vec<T, V>(a + r * ld_a + c, v);
+    constexpr int RW = RawWords<T, V>::N;
+    for (long long rb = r0 + ty; rb < r1; rb += 4 * COLRED_RT) {
+      uint32_t v[4][RW], w[4][RW], u[4][RW];
+      float mu[4], rs[4];
 #pragma unroll
-      for (int j = 0; j < V; ++j) a0[j] += v[j];
-      if (y) {
-        float w[V];
-        load_vec<T, V>(y + r * cols + c, w);
-        const float mu = mean[r], rs = rstd[r];
-#pragma unroll
-        for (int j = 0; j < V; ++j) a1[j] += v[j] * (w[j] - mu) * rs;
+      for (int k = 0; k < 4; ++k) {                       // all loads of four rows first (raw words: few registers)
+        const long long r = rb + COLRED_RT * k;
+        if (r < r1) {
+          load_raw<T, V>(a + r * ld_a + c, v[k]);
+          if (y) { load_raw<T, V>(y + r * cols + c, w[k]); mu[k] = mean[r]; rs[k] = rstd[r]; }
+          if (a2) load_raw<T, V>(a2 + r * ld_a2 + c, u[k]);
+        }
       }
-      if (a2) {
-        float w[V];
-        load_vec<T, V>(a2 + r * ld_a2 + c, w);
 #pragma unroll
-        for (int j = 0; j < V; ++j) a2s[j] += w[j];
+      for (int k = 0; k < 4; ++k) {
+        if (rb + COLRED_RT * k < r1) {
+          float fv[V], fw[V];
+          widen_raw<T, V>(v[k], fv);
+#pragma unroll
+          for (int j = 0; j < V; ++j) a0[j] += fv[j];
+          if (y) {
+            widen_raw<T, V>(w[k], fw);
+#pragma unroll
+            for (int j = 0; j < V; ++j) a1[j] += fv[j] * (fw[j] - mu[k]) * rs[k];
+          }
+          if (a2) {
+            widen_raw<T, V>(u[k], fw);
+#pragma unroll
+            for (int j = 0; j < V; ++j) a2s[j] += fw[j];
+          }
+        }
       }
     }
   }
 #pragma unroll
   for (int j = 0; j < V; ++j) { sh[0][ty][tx * V + j] = a0[j]; sh[1][ty][tx * V + j] = a1[j]; sh[2][ty][tx * V + j] = a2s[j]; }
   __syncthreads();
-  const long long plane = (long long)COL_CHUNKS * cols;
-  for (int i = threadIdx.x; i < 32 * V; i += 256) {
-    const int cc = blockIdx.x * 32 * V + i;
-    if (cc >= cols) continue;
-    float t0 = 0.f, t1 = 0.f, t2 = 0.f;
+  const int n_planes = a2 ? 3 : (y ? 2 : 1);
+  for (int i = threadIdx.x; i < n_planes * BC; i += 256) {
+    const int pl = i / BC, col = i - pl * BC, cc = blockIdx.x * BC + col;
+    if (cc >= cols || (pl == 1 && !y)) continue;
+    float t = 0.f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { t0 += sh[0][k][i]; t1 += sh[1][k][i]; t2 += sh[2][k][i]; }
-    scratch[(long long)blockIdx.y * cols + cc] = t0;
-    if (y) scratch[plane + (long long)blockIdx.y * cols + cc] = t1;
-    if (a2) scratch[2 * plane + (long long)blockIdx.y * cols + cc] = t2;
+    for (int k = 0; k < COLRED_RT; ++k) t += sh[pl][k][col];
+    scratch[pl * plane + (long long)blockIdx.y * cols + cc] = t;
   }
   __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) is_last = atomicAdd(&counters[blockIdx.x], 1) == (int)gridDim.y - 1;
+  if (threadIdx.x == 0) is_last = atomicAdd(&counters[blockIdx.x], 1) == chunks - 1;
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  for (int i = threadIdx.x; i < 32 * V; i += 256) {
-    const int cc = blockIdx.x * 32 * V + i;
-    if (cc >= cols) continue;
-    float t0 = 0.f, t1 = 0.f, t2 = 0.f;
-    for (int k = 0; k < COL_CHUNKS; ++k) {
-      t0 += scratch[(long long)k * cols + cc];
-      if (y) t1 += scratch[plane + (long long)k * cols + cc];
-      if (a2) t2 += scratch[2 * plane + (long long)k * cols + cc];
+  for (int i = threadIdx.x; i < n_planes * BC; i += 256) {
+    const int pl = i / BC, col = i - pl * BC, cc = blockIdx.x * BC + col;
+    if (cc >= cols || (pl == 1 && !y)) continue;
+    const float* src = scratch + pl * plane + cc;
+    float t = 0.f;
+    for (int k0 = 0; k0 < chunks; k0 += 8) {               // eight loads in flight, added in index order
+      float q[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) q[k] = k0 + k < chunks ? src[(long long)(k0 + k) * cols] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) t += q[k];
     }
-    out0[cc] = t0;
-    if (y) out1[cc] = t1;
-    if (a2) out2[cc] = t2;
+    float* out = pl == 0 ? out0 : (pl == 1 ? out1 : out2);
+    out[cc] = t;
   }
   if (threadIdx.x == 0) counters[blockIdx.x] = 0;         // ready for the next launch on this stream
 }
@@ -469,10 +487,16 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
 
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
                        const void* a2, long long ld_a2, long long rows, int cols, float* out0, float* out1,
-                       float* out2, float* scratch, int* counters, int dt, cudaStream_t st) {
+                       float* out2, float* scratch, long long plane_floats, int* counters, int dt, cudaStream_t st) {
   Scope sc("col_reduce", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (1 + (y ? 1 : 0) + (a2 ? 1 : 0)), 0, st);
-#define MREM_COLRED(T, V) do { dim3 grid((cols + 32 * V - 1) / (32 * V), COL_CHUNKS); \
-    launch_k(col_reduce_kernel<T, V>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, counters); } while (0)
+  // as many row chunks as one plane of the scratch holds, up to two blocks per SM (one wave) and 128 rows per chunk
+#define MREM_COLRED(T, V) do { const int col_blocks = (cols + COLRED_CT * V - 1) / (COLRED_CT * V); \
+    long long chunks = plane_floats / cols; \
+    if (chunks > 288 / col_blocks) chunks = 288 / col_blocks; \
+    if (chunks > (rows + 4 * COLRED_RT - 1) / (4 * COLRED_RT)) chunks = (rows + 4 * COLRED_RT - 1) / (4 * COLRED_RT); \
+    if (chunks < 1) chunks = 1; \
+    dim3 grid(col_blocks, (unsigned)chunks); \
+    launch_k(col_reduce_kernel<T, V>, grid, 256, 0, st, (const T*)a, ld_a, (const T*)y, mean, rstd, (const T*)a2, ld_a2, rows, cols, out0, out1, out2, scratch, plane_floats, counters); } while (0)
   const bool vec_ok = cols % 8 == 0 && ld_a % 8 == 0 && ld_a2 % 8 == 0 && al16(a) && al16(y) && al16(a2);
   if (dt == 1) { if (vec_ok) MREM_COLRED(bf16, 8); else MREM_COLRED(bf16, 1); }
   else { if (vec_ok) MREM_COLRED(float, 4); else MREM_COLRED(float, 1); }

@@ -33,6 +33,41 @@ __device__ __forceinline__ void load_vec(const T* p, float* v) {
   }
 }
 
+// The same load in two halves: the raw words first (V * sizeof(T) bytes, at most 16, in RAW_WORDS 32-bit
+// registers), widened to float later, so that several loads can be in flight on few registers.
+template <typename T, int V> struct RawWords { static constexpr int N = (V * (int)sizeof(T) + 3) / 4; };
+template <typename T, int V>
+__device__ __forceinline__ void load_raw(const T* p, uint32_t* w) {
+  if constexpr (V * sizeof(T) == 16) {
+    const uint4 t = *reinterpret_cast<const uint4*>(p);
+    w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+  } else if constexpr (V * sizeof(T) == 8) {
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    w[0] = t.x; w[1] = t.y;
+  } else if constexpr (V * sizeof(T) == 4) {
+    w[0] = *reinterpret_cast<const uint32_t*>(p);
+  } else {
+    static_assert(V == 1 && sizeof(T) == 2, "raw loads cover 2, 4, 8 and 16 bytes");
+    w[0] = *reinterpret_cast<const unsigned short*>(p);
+  }
+}
+template <typename T, int V>
+__device__ __forceinline__ void widen_raw(const uint32_t* w, float* v) {
+  if constexpr (sizeof(T) == 4) {
+#pragma unroll
+    for (int i = 0; i < V; ++i) v[i] = __uint_as_float(w[i]);
+  } else if constexpr (V == 1) {
+    v[0] = __uint_as_float(w[0] << 16);
+  } else {
+#pragma unroll
+    for (int i = 0; i < V / 2; ++i) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+      v[2 * i] = f.x;
+      v[2 * i + 1] = f.y;
+    }
+  }
+}
+
 template <typename T, int V>
 __device__ __forceinline__ void store_vec(T* p, const float* v) {
   if constexpr (V == 1) {
