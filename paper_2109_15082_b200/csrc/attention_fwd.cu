@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
             cw[j >> 1] = pw[j >> 1];
           }
         }
-        if (row_ok) {
+        if (row_ok && p.P) {                              // (no P: a pass whose probabilities nobody reads)
           const int ncol = p.S - c * 32;                  // columns of this chunk inside the tensor (S % 8 == 0)
 #pragma unroll
           for (int t = 0; t < 4; ++t)

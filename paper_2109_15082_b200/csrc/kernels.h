@@ -65,7 +65,8 @@ void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h,
 
 // Fused attention forward on the tensor cores (bf16 storage, head size 64, seq <= 384, seq % 8 == 0):
 // scores, masked softmax, quantizer of the probabilities, context product and (student) the context's
-// codes in one kernel.  Returns a GemmRc.  Null p_step / c_step: no quantizer.
+// codes in one kernel.  Returns a GemmRc.  Null p_step / c_step: no quantizer; null P: the probabilities are
+// not written (a full-precision pass whose probabilities nobody reads).
 bool attention_fwd_supported(int S, int head_dim, int dt);
 int launch_attention_fwd(const void* qkv, int B, int S, int h, int H, const int* valid_len, float alpha_const,
                          const float* a_p0, const float* a_p1, const float* c_p0, const float* c_p1,
@@ -108,6 +109,15 @@ void launch_softmax_bwd(const void* P, const void* dphat, void* dS, long long ro
 void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, const float* mean, const float* rstd,
                           const float* gamma, long long rows, int cols, void* dy, void* dsum, int dt,
                           cudaStream_t st);
+
+// The same with the incoming gradient assembled on the fly from a straight-through mask and a skip connection:
+//   dv = dout (or 0 when null) + 1[lo <= x / *step <= hi] * dxhat + add;  dsum = dv;  dy = LayerNorm backward of dv.
+// part_s gets RED_BLOCKS partial sums of the quantizer's step-size gradient.  Returns false (nothing launched)
+// when the row does not fit the register-cached vector path; the caller then runs the separate kernels.
+bool layernorm_bwd_ste_supported(int cols, int dt);      // the row width fits (16-byte aligned tensors assumed)
+bool launch_layernorm_bwd_ste(const void* dout, const void* x, const void* dxhat, const void* add, const float* step,
+                              int lo, int hi, const void* y, const float* mean, const float* rstd, const float* gamma,
+                              long long rows, int cols, void* dy, void* dsum, float* part_s, int dt, cudaStream_t st);
 
 // Column sums over rows: out0[c] = sum_r a[r,c]; with y/mean/rstd also out1[c] = sum_r a[r,c]*(y[r,c]-mean[r])*rstd[r];
 // with a2 also out2[c] = sum_r a2[r,c].  One kernel: per-chunk partials in `scratch` (three planes of

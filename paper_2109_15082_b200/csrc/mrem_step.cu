@@ -130,8 +130,9 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
     if (init_steps)
       for (int seg = 0; seg < 3; ++seg) init_site(c, b, S_Q + seg, r.at(c->t_qkv, seg * H), 3 * H, M, H);
     if (attention_fwd_supported(S, hd, c->dt)) {
+      // (the probabilities of the full-precision pass are read only when the activation steps are initialised)
       r.note(launch_attention_fwd(c->t_qkv, B, S, h, H, len, 1.f / sqrtf((float)hd), nullptr, nullptr, nullptr, nullptr,
-                                  nullptr, 0, 0, c->t_P, nullptr, c->t_ctx, nullptr, 0, nullptr, nullptr, c->status, st),
+                                  nullptr, 0, 0, init_steps ? c->t_P : nullptr, nullptr, c->t_ctx, nullptr, 0, nullptr, nullptr, c->status, st),
              "attention launch failed");
     } else {
       r.gemm(view(c->t_qkv, 3 * H, 0, hd, (long long)S * 3 * H), view(r.at(c->t_qkv, H), 3 * H, 0, hd, (long long)S * 3 * H),
@@ -277,6 +278,9 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
   const int ok = r.okind();
   const float inv_sqrt_d = 1.f / sqrtf((float)hd);
   const void* carry = nullptr;
+  // the straight-through passes that feed a LayerNorm's backward run inside it where the row fits its registers
+  const bool fuse_ln = layernorm_bwd_ste_supported(H, c->dt);
+  struct { const void* x; const float* step; float* part; } pending = {nullptr, nullptr, nullptr};
   for (int l = d.n_layers - 1; l >= 0; --l) {
     const LayerBind& b = c->bind[l];
     LayerStash& s = c->stash[l];
@@ -289,11 +293,26 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     cudaStream_t st = c->stream;
 
     // second LayerNorm: total gradient at the layer output = loss term + what the next layer sent back
-    launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, carry ? c->d_sum : nullptr, c->dt, st);
+    // (with `pending` the layer above left its input gradient unmasked: the straight-through pass of its input
+    //  quantizer and its skip connection are applied while this LayerNorm's backward reads them)
+    bool sent_back = carry != nullptr;
+    if (pending.x) {
+      const bool fused = launch_layernorm_bwd_ste(dF, pending.x, c->d_xhat, c->d_y1, pending.step, rx.lo, rx.hi, s.y2, s.mean2, s.rstd2,
+                                                  b.student[MREM_LN2_G], M, H, c->d_y2, c->d_sum, pending.part, c->dt, st);
+      if (!fused) {
+        launch_ste_act(pending.x, H, c->d_xhat, H, c->d_y1, H, c->carry[0], H, M, H, pending.step, nullptr, rx.lo, rx.hi,
+                       pending.part, nullptr, c->dt, st);
+        launch_layernorm_bwd(dF, c->carry[0], s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, c->d_sum, c->dt, st);
+      }
+      sent_back = true;
+      pending.x = nullptr;
+    } else {
+      launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, carry ? c->d_sum : nullptr, c->dt, st);
+    }
     // LayerNorm parameter gradients and the bias gradient of FFN2 (y2 = G_hat W2_hat^T + b2 + a) in one pass
     // (column sums feed only the update and the weight-gradient epilogue: side stream)
     fork();
-    launch_col_reduce(carry ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, c->d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
+    launch_col_reduce(sent_back ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, c->d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
                       g.p[MREM_B2], c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
     {
@@ -309,10 +328,13 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
     rw.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
-    launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
-                   part + S_A * RED_BLOCKS, nullptr, c->dt, st);
-    // first LayerNorm
-    launch_layernorm_bwd(c->d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, c->d_y1, nullptr, c->dt, st);
+    // straight-through pass of the FFN1 input quantizer + skip connection -> d_a, and the first LayerNorm's backward
+    if (!(fuse_ln && launch_layernorm_bwd_ste(nullptr, s.a, c->d_ahat, c->d_y2, b.a_steps[S_A], rx.lo, rx.hi, s.y1, s.mean1, s.rstd1,
+                                              b.student[MREM_LN1_G], M, H, c->d_y1, c->d_a, part + S_A * RED_BLOCKS, c->dt, st))) {
+      launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
+                     part + S_A * RED_BLOCKS, nullptr, c->dt, st);
+      launch_layernorm_bwd(c->d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, c->d_y1, nullptr, c->dt, st);
+    }
     // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x  (its bias gradient rides along)
     fork();
     launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
@@ -346,10 +368,16 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
     rw.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
-    void* next_carry = c->carry[l & 1];
-    launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
-                   part + S_X * RED_BLOCKS, nullptr, c->dt, st);
-    carry = next_carry;
+    if (fuse_ln && l > 0) {
+      // left to the LayerNorm backward of the layer below, which reads d_xhat and d_y1 before anything overwrites them
+      pending.x = x_in; pending.step = b.a_steps[S_X]; pending.part = part + S_X * RED_BLOCKS;
+      carry = nullptr;
+    } else {
+      void* next_carry = c->carry[l & 1];
+      launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
+                     part + S_X * RED_BLOCKS, nullptr, c->dt, st);
+      carry = next_carry;
+    }
     // (the weight quantizers' masks and step gradients are applied inside the fused update of mrem_step,
     //  or on demand by mrem_get_grad)
     // the layer below overwrites d_y2, d_u, d_y1, d_qkv and the bias row the weight-gradient products read

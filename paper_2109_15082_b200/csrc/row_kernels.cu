@@ -197,6 +197,84 @@ __global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout,
   }
 }
 
+// ------------------------------------------------------------------ LayerNorm backward fed by a straight-through mask
+// The gradient that enters the LayerNorm is assembled on the fly:
+//   dv = dout (when given) + 1[lo <= x / step <= hi] * dxhat + add,
+// i.e. the straight-through pass of the activation quantizer that saw x (Sec. 3.1.1) followed by the skip
+// connection, which the separate kernels write to memory and read back.  dv goes to dsum (the column
+// reductions read it) and, rounded as stored, into the LayerNorm backward.  The quantizer's step-size
+// gradient leaves as one partial sum per block (fixed order; slots beyond the grid are zeroed).
+// Rows up to 32 * V * MAXNV wide, one warp per row, warps stride over the rows.
+template <typename T, int V>
+__global__ void __launch_bounds__(128) ln_bwd_ste_kernel(const T* __restrict__ dout, const T* __restrict__ x,
+                                                         const T* __restrict__ dxhat, const T* __restrict__ add,
+                                                         const float* __restrict__ step, float lo, float hi,
+                                                         const T* __restrict__ y, const float* __restrict__ mean,
+                                                         const float* __restrict__ rstd, const float* __restrict__ gamma,
+                                                         long long rows, int cols, T* __restrict__ dy,
+                                                         T* __restrict__ dsum, float* __restrict__ part_s, int n_slots) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ float sh[4];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const float s = *step, r_s = __frcp_rn(s);
+  float ds = 0.f;
+  for (long long row = blockIdx.x * 4ll + wid; row < rows; row += gridDim.x * 4ll) {
+    const float mu = mean[row], rs = rstd[row];
+    const long long base = row * cols;
+    float d[MAXNV][V], xn[MAXNV][V];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * V;
+      if (c < cols) {
+        float xv[V], e[V];
+        load_vec<T, V>(x + base + c, xv);
+        load_vec<T, V>(dxhat + base + c, d[i]);
+        load_vec<T, V>(add + base + c, e);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          const float z = quotient(xv[j], s, r_s);
+          const bool in = z >= lo && z <= hi;
+          ds += d[i][j] * ((float)__float2int_rn(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
+          d[i][j] = (in ? d[i][j] : 0.f) + e[j];
+        }
+        if (dout) {
+          load_vec<T, V>(dout + base + c, e);
+#pragma unroll
+          for (int j = 0; j < V; ++j) d[i][j] += e[j];
+        }
+        store_vec<T, V>(dsum + base + c, d[i]);
+        load_vec<T, V>(y + base + c, xn[i]);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          xn[i][j] = (xn[i][j] - mu) * rs;
+          d[i][j] = stored<T>(d[i][j]) * gamma[c + j];
+          s1 += d[i][j];
+          s2 += d[i][j] * xn[i][j];
+        }
+      }
+    }
+    s1 = warp_sum(s1) / (float)cols;
+    s2 = warp_sum(s2) / (float)cols;
+#pragma unroll
+    for (int i = 0; i < MAXNV; ++i) {
+      const int c = (lane + 32 * i) * V;
+      if (c < cols) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) d[i][j] = rs * (d[i][j] - s1 - xn[i][j] * s2);
+        store_vec<T, V>(dy + base + c, d[i]);
+      }
+    }
+  }
+  ds = warp_sum(ds);
+  if (lane == 0) sh[wid] = ds;
+  __syncthreads();
+  if (threadIdx.x == 0) part_s[blockIdx.x] = (sh[0] + sh[1]) + (sh[2] + sh[3]);
+  if (blockIdx.x == 0)
+    for (int i = gridDim.x + threadIdx.x; i < n_slots; i += blockDim.x) part_s[i] = 0.f;
+}
+
 // ------------------------------------------------------------------ column sums over rows
 // out0[c] = sum_r a[r,c];  out1[c] = sum_r a[r,c] * (y[r,c] - mean[r]) * rstd[r] (when y);  out2[c] = sum_r a2[r,c]
 // (when a2).  A block of 8 x 32 threads owns 8*V columns (one 128-byte line per row for 16-byte vectors) of
@@ -483,6 +561,32 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
     if (v) launch_k(ln_bwd_kernel<T, V, true>, grid, 128, 0, st, (const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
     else launch_k(ln_bwd_kernel<T, 1, false>, grid, 128, 0, st, (const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
   });
+}
+
+bool layernorm_bwd_ste_supported(int cols, int dt) {
+  const int V = dt == 1 ? 8 : 4;
+  return cols % V == 0 && cols <= 32 * V * MAXNV;
+}
+
+bool launch_layernorm_bwd_ste(const void* dout, const void* x, const void* dxhat, const void* add, const float* step,
+                              int lo, int hi, const void* y, const float* mean, const float* rstd, const float* gamma,
+                              long long rows, int cols, void* dy, void* dsum, float* part_s, int dt, cudaStream_t st) {
+  if (rows <= 0) return false;
+  bool done = false;
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(dout) && al16(x) && al16(dxhat) && al16(add) && al16(y) &&
+                   al16(dy) && al16(dsum);
+    if (v) {
+      Scope sc("layernorm_bwd_ste", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (6 + (dout ? 1 : 0)), 0, st);
+      const long long want = (rows + 3) / 4;
+      const int grid = (int)(want < RED_BLOCKS ? want : RED_BLOCKS);
+      launch_k(ln_bwd_ste_kernel<T, V>, grid, 128, 0, st, (const T*)dout, (const T*)x, (const T*)dxhat, (const T*)add, step,
+               (float)lo, (float)hi, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum, part_s, RED_BLOCKS);
+      done = true;
+    }
+  });
+  return done;
 }
 
 void launch_col_reduce(const void* a, long long ld_a, const void* y, const float* mean, const float* rstd,
