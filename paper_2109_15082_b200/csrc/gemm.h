@@ -19,6 +19,13 @@ bool tc_gemm_pair_eligible(const GemmShape& g, const Epilogue& epi, int block_n)
 int tc_gemm_pair(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
                  const Epilogue& epi, int* d_status, int sm_count, cudaStream_t stream);
 
+// Several bf16 products with plain fp32 outputs (alpha and row bias only) as one persistent launch over the
+// joint tile list: the weight-gradient products of a layer.  Operands as in tc_gemm, one batch each.
+constexpr int MAX_GEMM_GROUP = 4;
+struct GemmGroupItem { OperandDesc A, B; GemmShape g; Epilogue epi; };
+bool tc_gemm_group_eligible(const GemmGroupItem* items, int n);
+int tc_gemm_group(const GemmGroupItem* items, int n, int* d_status, int sm_count, cudaStream_t stream);
+
 // 4-D TMA tensor map (128-byte swizzle) of an operand: (contiguous index, strided index, batch0, batch1).
 // K-major operands get boxes of block_k x tile_mn elements, MN-major ones 64 x block_k.
 int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,

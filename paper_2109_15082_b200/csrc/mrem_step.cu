@@ -61,6 +61,24 @@ struct Runner {
     if (c->dt == 1) note(tc_gemm(0, 0, a, b, g, e, 0, c->status, c->sm_count, st), "bf16 GEMM launch failed");
     else note(simt_gemm_f32(a, b, g, e, st), "f32 GEMM launch failed");
   }
+  // weight-gradient products (bf16 in, fp32 out) of one layer: collected, then launched as one grouped kernel
+  // over the joint tile list where the tensor-core path takes them, else one by one
+  std::vector<GemmGroupItem> deferred;
+  void defer(const View& A, const View& B, int M, int N, int K, const Epilogue& e) {
+    if (c->dt != 1) { gemm(A, B, M, N, K, 1, 1, e); return; }
+    GemmGroupItem it{OperandDesc{A.p, A.ld, A.sb0, A.sb1, A.mn}, OperandDesc{B.p, B.ld, B.sb0, B.sb1, B.mn}, GemmShape{M, N, K, 1, 1}, e};
+    deferred.push_back(it);
+  }
+  void flush_deferred() {
+    if (deferred.empty()) return;
+    if ((int)deferred.size() <= MAX_GEMM_GROUP && tc_gemm_group_eligible(deferred.data(), (int)deferred.size())) {
+      note(tc_gemm_group(deferred.data(), (int)deferred.size(), c->status, c->sm_count, st), "grouped weight-gradient GEMM launch failed");
+    } else {
+      for (const GemmGroupItem& it : deferred)
+        note(tc_gemm(0, 0, it.A, it.B, it.g, it.epi, 0, c->status, c->sm_count, st), "bf16 GEMM launch failed");
+    }
+    deferred.clear();
+  }
   // integer-code product with exact int32 accumulation
   void gemm_i8(const int8_t* A, int a_unsigned, const int8_t* B, int M, int N, int K, const Epilogue& e) {
     OperandDesc a{A, K, 0, 0, 0}, b{B, K, 0, 0, 0};
@@ -319,7 +337,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
       Epi e(g.p[MREM_W2], OUT_F32, F);
       e.alpha(1.f, b.a_steps[S_G]);
       if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], c->rowbias, H, side); e.rowbias(c->rowbias); }
-      rw.gemm(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, 1, 1, e.e);
+      rw.defer(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, e.e);
     }
     launch_gelu_bwd(s.u, c->d_ghat, c->d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
                     part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
@@ -327,7 +345,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     fork();
     launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
-    rw.gemm(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, 1, 1, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
+    rw.defer(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     // straight-through pass of the FFN1 input quantizer + skip connection -> d_a, and the first LayerNorm's backward
     if (!(fuse_ln && launch_layernorm_bwd_ste(nullptr, s.a, c->d_ahat, c->d_y2, b.a_steps[S_A], rx.lo, rx.hi, s.y1, s.mean1, s.rstd1,
                                               b.student[MREM_LN1_G], M, H, c->d_y1, c->d_a, part + S_A * RED_BLOCKS, c->dt, st))) {
@@ -340,7 +358,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
                       c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
-    rw.gemm(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, 1, 1, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
+    rw.defer(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
                    part + S_C * RED_BLOCKS, nullptr, c->dt, st);
     // attention:  ctx = P_hat V_hat,  P = softmax(Q_hat K_hat^T / sqrt(d))
@@ -367,7 +385,8 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     fork();
     launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
     r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
-    rw.gemm(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, 1, 1, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
+    rw.defer(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
+    rw.flush_deferred();                              // the layer's four weight-gradient products, one launch
     if (fuse_ln && l > 0) {
       // left to the LayerNorm backward of the layer below, which reads d_xhat and d_y1 before anything overwrites them
       pending.x = x_in; pending.step = b.a_steps[S_X]; pending.part = part + S_X * RED_BLOCKS;
