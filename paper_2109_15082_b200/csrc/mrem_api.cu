@@ -76,6 +76,7 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->col_scratch = (float*)A.take(sizeof(float) * 3 * c->col_plane);
   c->col_counters = (int*)A.take(sizeof(int) * ((3 * H > F ? 3 * H : F) / 32 + 2));
   c->rowbias = (float*)A.take(sizeof(float) * (3 * H > F ? 3 * H : F));
+  c->alt_rowbias = (float*)A.take(sizeof(float) * (3 * H > F ? 3 * H : F));
   c->reduce_per_layer = N_SITES + 1 + N_WMAT;
   c->reduce_table = (ReduceEntry*)A.take(sizeof(ReduceEntry) * c->reduce_per_layer * L);
   c->adam_table = (AdamEntry*)A.take(sizeof(AdamEntry) * (MREM_N_PARAMS + N_WMAT + N_SITES + 1) * L);
@@ -104,6 +105,8 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->d_qkvhat = A.take(M * 3 * H * es); c->d_qkv = A.take(M * 3 * H * es);
   c->d_xhat = A.take(M * H * es); c->d_sum = A.take(M * H * es);
   c->carry[0] = A.take(M * H * es); c->carry[1] = A.take(M * H * es);
+  c->alt_d_y2 = A.take(M * H * es); c->alt_d_sum = A.take(M * H * es); c->alt_d_u = A.take(M * F * es);
+  c->alt_d_a = A.take(M * H * es); c->alt_d_y1 = A.take(M * H * es); c->alt_d_qkv = A.take(M * 3 * H * es);
 
   c->stash.resize(L); c->wq.assign(L, std::vector<WeightBuf>(N_WMAT)); c->grad.resize(L);
   for (int l = 0; l < L; ++l) {
@@ -259,6 +262,8 @@ int32_t mrem_create(const mrem_module_desc* desc, void* workspace, size_t worksp
       cudaStreamCreateWithPriority(&c->side_stream, cudaStreamNonBlocking, pri_lo) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_layer[0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_layer[1], cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_h2d[0], cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_h2d[1], cudaEventDisableTiming) != cudaSuccess ||
@@ -285,6 +290,7 @@ int32_t mrem_destroy(mrem_ctx* c) {
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
+  for (cudaEvent_t e : c->ev_layer) if (e) cudaEventDestroy(e);
   if (c->side_stream) cudaStreamDestroy(c->side_stream);
   delete c;
   return MREM_OK;

@@ -92,6 +92,10 @@ struct mrem_ctx {
   long long col_plane = 0;               // floats per plane of col_scratch
   int* col_counters;
   float* rowbias;
+  // second copy of the backward buffers the side stream reads (layers alternate between the two copies, so the
+  // main stream may start the layer below while the side stream still works on this one)
+  void *alt_d_y2 = nullptr, *alt_d_sum = nullptr, *alt_d_u = nullptr, *alt_d_a = nullptr, *alt_d_y1 = nullptr, *alt_d_qkv = nullptr;
+  float* alt_rowbias = nullptr;
   float* loss_partial;
   float* minmax;
   int* status;
@@ -105,6 +109,7 @@ struct mrem_ctx {
   // run there while the main stream goes on with the tensor-core work of the layer below
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_layer[2] = {nullptr, nullptr};   // side stream done with the gradient buffers of a layer parity
   cudaStream_t teacher_stream = nullptr;   // set for the duration of a step that runs the teacher pass beside the student's
   bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps

@@ -295,10 +295,16 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
   };
   const int ok = r.okind();
   const float inv_sqrt_d = 1.f / sqrtf((float)hd);
+  // Buffers the side stream reads, two copies used by alternate layers: the main stream starts the layer below while
+  // the side stream still reduces and multiplies this layer's gradients, and waits (ev_layer) only before it
+  // overwrites the copy of the layer two above.
+  struct SideBufs { void *d_y2, *d_sum, *d_u, *d_a, *d_y1, *d_qkv; float* rowbias; };
+  const SideBufs copies[2] = {{c->d_y2, c->d_sum, c->d_u, c->d_a, c->d_y1, c->d_qkv, c->rowbias},
+                              {c->alt_d_y2, c->alt_d_sum, c->alt_d_u, c->alt_d_a, c->alt_d_y1, c->alt_d_qkv, c->alt_rowbias}};
   const void* carry = nullptr;
   // the straight-through passes that feed a LayerNorm's backward run inside it where the row fits its registers
   const bool fuse_ln = layernorm_bwd_ste_supported(H, c->dt);
-  struct { const void* x; const float* step; float* part; } pending = {nullptr, nullptr, nullptr};
+  struct { const void* x; const void* add; const float* step; float* part; } pending = {nullptr, nullptr, nullptr, nullptr};
   for (int l = d.n_layers - 1; l >= 0; --l) {
     const LayerBind& b = c->bind[l];
     LayerStash& s = c->stash[l];
@@ -309,62 +315,64 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     const ActRange rx = site_range(d, S_X), rp = site_range(d, S_P), rg = site_range(d, S_G);
     float* part = s.part;
     cudaStream_t st = c->stream;
+    const SideBufs& q = copies[l & 1];
+    if (two_streams && l + 2 < d.n_layers && cudaStreamWaitEvent(c->stream, c->ev_layer[l & 1], 0) != cudaSuccess) sync_failed = true;
 
     // second LayerNorm: total gradient at the layer output = loss term + what the next layer sent back
     // (with `pending` the layer above left its input gradient unmasked: the straight-through pass of its input
     //  quantizer and its skip connection are applied while this LayerNorm's backward reads them)
     bool sent_back = carry != nullptr;
     if (pending.x) {
-      const bool fused = launch_layernorm_bwd_ste(dF, pending.x, c->d_xhat, c->d_y1, pending.step, rx.lo, rx.hi, s.y2, s.mean2, s.rstd2,
-                                                  b.student[MREM_LN2_G], M, H, c->d_y2, c->d_sum, pending.part, c->dt, st);
+      const bool fused = launch_layernorm_bwd_ste(dF, pending.x, c->d_xhat, pending.add, pending.step, rx.lo, rx.hi, s.y2, s.mean2, s.rstd2,
+                                                  b.student[MREM_LN2_G], M, H, q.d_y2, q.d_sum, pending.part, c->dt, st);
       if (!fused) {
-        launch_ste_act(pending.x, H, c->d_xhat, H, c->d_y1, H, c->carry[0], H, M, H, pending.step, nullptr, rx.lo, rx.hi,
+        launch_ste_act(pending.x, H, c->d_xhat, H, pending.add, H, c->carry[0], H, M, H, pending.step, nullptr, rx.lo, rx.hi,
                        pending.part, nullptr, c->dt, st);
-        launch_layernorm_bwd(dF, c->carry[0], s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, c->d_sum, c->dt, st);
+        launch_layernorm_bwd(dF, c->carry[0], s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, q.d_y2, q.d_sum, c->dt, st);
       }
       sent_back = true;
       pending.x = nullptr;
     } else {
-      launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, c->d_y2, carry ? c->d_sum : nullptr, c->dt, st);
+      launch_layernorm_bwd(dF, carry, s.y2, s.mean2, s.rstd2, b.student[MREM_LN2_G], M, H, q.d_y2, carry ? q.d_sum : nullptr, c->dt, st);
     }
     // LayerNorm parameter gradients and the bias gradient of FFN2 (y2 = G_hat W2_hat^T + b2 + a) in one pass
     // (column sums feed only the update and the weight-gradient epilogue: side stream)
     fork();
-    launch_col_reduce(sent_back ? c->d_sum : dF, H, s.y2, s.mean2, s.rstd2, c->d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
+    launch_col_reduce(sent_back ? q.d_sum : dF, H, s.y2, s.mean2, s.rstd2, q.d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
                       g.p[MREM_B2], c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(c->d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
+    r.gemm(view(q.d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
     {
       Epi e(g.p[MREM_W2], OUT_F32, F);
       e.alpha(1.f, b.a_steps[S_G]);
-      if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], c->rowbias, H, side); e.rowbias(c->rowbias); }
-      rw.defer(view(c->d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, e.e);
+      if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], q.rowbias, H, side); e.rowbias(q.rowbias); }
+      rw.defer(view(q.d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, e.e);
     }
-    launch_gelu_bwd(s.u, c->d_ghat, c->d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
+    launch_gelu_bwd(s.u, c->d_ghat, q.d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
                     part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
     // FFN1:  u = A_hat W1_hat^T + b1
     fork();
-    launch_col_reduce(c->d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(c->d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
-    rw.defer(view(c->d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
+    launch_col_reduce(q.d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
+    r.gemm(view(q.d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
+    rw.defer(view(q.d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     // straight-through pass of the FFN1 input quantizer + skip connection -> d_a, and the first LayerNorm's backward
-    if (!(fuse_ln && launch_layernorm_bwd_ste(nullptr, s.a, c->d_ahat, c->d_y2, b.a_steps[S_A], rx.lo, rx.hi, s.y1, s.mean1, s.rstd1,
-                                              b.student[MREM_LN1_G], M, H, c->d_y1, c->d_a, part + S_A * RED_BLOCKS, c->dt, st))) {
-      launch_ste_act(s.a, H, c->d_ahat, H, c->d_y2, H, c->d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
+    if (!(fuse_ln && launch_layernorm_bwd_ste(nullptr, s.a, c->d_ahat, q.d_y2, b.a_steps[S_A], rx.lo, rx.hi, s.y1, s.mean1, s.rstd1,
+                                              b.student[MREM_LN1_G], M, H, q.d_y1, q.d_a, part + S_A * RED_BLOCKS, c->dt, st))) {
+      launch_ste_act(s.a, H, c->d_ahat, H, q.d_y2, H, q.d_a, H, M, H, b.a_steps[S_A], nullptr, rx.lo, rx.hi,
                      part + S_A * RED_BLOCKS, nullptr, c->dt, st);
-      launch_layernorm_bwd(c->d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, c->d_y1, nullptr, c->dt, st);
+      launch_layernorm_bwd(q.d_a, nullptr, s.y1, s.mean1, s.rstd1, b.student[MREM_LN1_G], M, H, q.d_y1, nullptr, c->dt, st);
     }
     // attention output projection:  y1 = ctx_hat Wo_hat^T + bo + x  (its bias gradient rides along)
     fork();
-    launch_col_reduce(c->d_a, H, s.y1, s.mean1, s.rstd1, c->d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
+    launch_col_reduce(q.d_a, H, s.y1, s.mean1, s.rstd1, q.d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
                       c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(c->d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
-    rw.defer(view(c->d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
+    r.gemm(view(q.d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
+    rw.defer(view(q.d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
                    part + S_C * RED_BLOCKS, nullptr, c->dt, st);
     // attention:  ctx = P_hat V_hat,  P = softmax(Q_hat K_hat^T / sqrt(d))
     if (c->fused_attention_bwd && attention_bwd_supported(S, hd, c->dt, B * h)) {
       r.note(launch_attention_bwd(s.qkv_qt, s.qkv, s.P, c->d_ctx, B, S, h, H, b.a_steps[S_Q], b.a_steps[S_K], b.a_steps[S_V],
-                                  b.a_steps[S_P], rx.lo, rx.hi, rp.lo, rp.hi, c->d_qkv, part + S_Q * RED_BLOCKS,
+                                  b.a_steps[S_P], rx.lo, rx.hi, rp.lo, rp.hi, q.d_qkv, part + S_Q * RED_BLOCKS,
                                   part + S_K * RED_BLOCKS, part + S_V * RED_BLOCKS, part + S_P * RED_BLOCKS, c->status, st),
              "attention backward launch failed");
     } else {
@@ -378,29 +386,29 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
       r.gemm(view(c->d_s, S, 1, sSS, sHSS), view(s.qkv_qt, 3 * H, 1, hd, sQKV), S, hd, S, h, B,
              Epi(r.at(c->d_qkvhat, H), ok, 3 * H, hd, sQKV).alpha(inv_sqrt_d, b.a_steps[S_Q]).e);
       for (int seg = 0; seg < 3; ++seg)
-        launch_ste_act(r.at(s.qkv, seg * H), 3 * H, r.at(c->d_qkvhat, seg * H), 3 * H, nullptr, 0, r.at(c->d_qkv, seg * H), 3 * H, M, H,
+        launch_ste_act(r.at(s.qkv, seg * H), 3 * H, r.at(c->d_qkvhat, seg * H), 3 * H, nullptr, 0, r.at(q.d_qkv, seg * H), 3 * H, M, H,
                        b.a_steps[S_Q + seg], nullptr, rx.lo, rx.hi, part + (S_Q + seg) * RED_BLOCKS, nullptr, c->dt, st);
     }
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
     fork();
-    launch_col_reduce(c->d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(c->d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
-    rw.defer(view(c->d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
+    launch_col_reduce(q.d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
+    r.gemm(view(q.d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
+    rw.defer(view(q.d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
     rw.flush_deferred();                              // the layer's four weight-gradient products, one launch
     if (fuse_ln && l > 0) {
       // left to the LayerNorm backward of the layer below, which reads d_xhat and d_y1 before anything overwrites them
-      pending.x = x_in; pending.step = b.a_steps[S_X]; pending.part = part + S_X * RED_BLOCKS;
+      pending.x = x_in; pending.add = q.d_y1; pending.step = b.a_steps[S_X]; pending.part = part + S_X * RED_BLOCKS;
       carry = nullptr;
     } else {
       void* next_carry = c->carry[l & 1];
-      launch_ste_act(x_in, H, c->d_xhat, H, c->d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
+      launch_ste_act(x_in, H, c->d_xhat, H, q.d_y1, H, next_carry, H, M, H, b.a_steps[S_X], nullptr, rx.lo, rx.hi,
                      part + S_X * RED_BLOCKS, nullptr, c->dt, st);
       carry = next_carry;
     }
     // (the weight quantizers' masks and step gradients are applied inside the fused update of mrem_step,
     //  or on demand by mrem_get_grad)
-    // the layer below overwrites d_y2, d_u, d_y1, d_qkv and the bias row the weight-gradient products read
-    join();
+    // the side stream is done with this layer's copy of the gradient buffers once the grouped products have run
+    if (two_streams && cudaEventRecord(c->ev_layer[l & 1], side) != cudaSuccess) sync_failed = true;
     // nothing below reads what the update writes: the latent weights, moments, row steps and this layer's codes
     if (update_as_you_go) enqueue_matrix_updates(c, l, side);
   }
