@@ -596,6 +596,79 @@ def recon_step(desc, teacher, student, steps, state, x_t, x_s, valid_len=None, l
     return r
 
 
+# ----------------------------------------------------------------------------- Eq. 2: reconstruction error of ONE matrix product
+
+# the activation quantizer that sits at the input of each of a layer's four products
+REM_SITE = {"Wqkv": SITE_X, "Wo": SITE_C, "W1": SITE_A, "W2": SITE_G}
+
+
+def rem_forward_loss_backward(desc, w_teacher, w_student, steps, name, a):
+    """The per-product objective of Eq. 2 for the matrix `name` of one layer:
+        l = c * || Q(w)^T Q(a) - w^T a ||^2   over the rows of a,
+    w the full-precision (teacher) matrix, Q(w) the student's quantized one, Q(a) the
+    input quantizer of that product; c = 1 / (rows * out) when `loss_mean`, else 1 as
+    printed.  No bias on either side (Eq. 2 has none).  `steps` is the layer's step
+    dict (make_steps).  Returns the target, the quantized product, the loss and the
+    gradients w.r.t. the latent matrix, its step(s), the activation step and offset
+    (straight-through estimator of Sec. 3.1.1)."""
+    st = lambda t: store(t, desc.act_dtype)
+    a = np.asarray(a, np.float64)
+    site = REM_SITE[name]
+    target = st(a @ st(w_teacher).T)
+    qa = _q_act(desc, a, steps, site)
+    qw = _q_w(desc, w_student, steps["w"][name])
+    y = st(student_linear(qa, qw, 0.0))
+    diff = y - target
+    c = 1.0 / diff.size if desc.loss_mean else 1.0
+    loss = c * float((diff * diff).sum())
+    dy = 2.0 * c * diff
+    dwhat = dy.T @ qa["xhat"]
+    out = dict(target=target, y=y, loss=loss, qa=qa, qw=qw, d_a_step=0.0, d_a_off=0.0)
+    if qw["q"] is None or qw.get("twn"):
+        out["dW"], out["d_w_step"] = dwhat, None
+    else:
+        inside, dwhat_ds = weight_ste(qw["z"], qw["q"], desc.w_bits, desc.w_grid)
+        out["dW"] = dwhat * inside
+        ds = (dwhat * dwhat_ds).sum(-1)
+        out["d_w_step"] = ds if desc.w_per_row else np.array([ds.sum()])
+    if qa["q"] is not None:
+        dxhat = dy @ qw["what"]
+        inside, dxhat_ds = act_ste(qa["z"], qa["q"], qa["lo"], qa["hi"])
+        out["d_a_step"] = float((dxhat * dxhat_ds).sum())
+        if qa["asym"]:
+            out["d_a_off"] = float((dxhat * (1.0 - inside)).sum())
+    return out
+
+
+def rem_step(desc, w_teacher, w_student, steps, state, name, a, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8,
+             weight_decay=0.01):
+    """One optimisation step of Eq. 2 on one product: gradients as above, then AdamW on
+    the latent matrix (with weight decay), its step(s), the input quantizer's step and
+    offset.  `state`: step count 't' and moments per key.  Returns (record, new matrix);
+    `steps` is updated in place."""
+    r = rem_forward_loss_backward(desc, w_teacher, w_student, steps, name, a)
+    site = REM_SITE[name]
+    state["t"] = state.get("t", 0) + 1
+    t = state["t"]
+
+    def upd(key, p, g, wd):
+        p = np.asarray(p, np.float64)
+        m, v = state.get(key, (np.zeros_like(p), np.zeros_like(p)))
+        p2, m, v = adamw_update(p, np.asarray(g, np.float64), m, v, t, lr, beta1, beta2, eps, wd)
+        state[key] = (m, v)
+        return p2
+
+    w_new = upd(("W", name), w_student, r["dW"], weight_decay).astype(np.float32)
+    if r["d_w_step"] is not None:
+        steps["w"][name] = np.maximum(upd(("s", name), steps["w"][name], r["d_w_step"].reshape(np.shape(steps["w"][name])), 0.0),
+                                      MIN_STEP).astype(np.float32)
+    if desc.a_bits:
+        steps["a"][site] = np.float32(max(float(upd(("a", site), np.array([steps["a"][site]]), np.array([r["d_a_step"]]), 0.0)[0]), MIN_STEP))
+        if r["qa"]["asym"] and site == SITE_G:
+            steps["a_off"][site] = np.float32(upd(("off", site), np.array([steps["a_off"][site]]), np.array([r["d_a_off"]]), 0.0)[0])
+    return r, w_new
+
+
 # ----------------------------------------------------------------------------- Algorithm 1: modules trained in parallel from input queues
 
 def mremp_run(descs, teachers, students, steps, batches, draws, t0, T, T0, lr0, lr_total=0, log=None, **adam):

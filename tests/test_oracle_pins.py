@@ -447,3 +447,104 @@ def test_twn_module_matches_torch_autograd_with_plain_straight_through():
     # every row keeps some weights and drops some: the threshold is exercised
     q = r["caches"][0]["qw"]["W1"]["q"]
     assert (q == 0).any() and (q != 0).any()
+
+
+# ----------------------------------------------------------------------------- Eq. 2 (one product)
+
+def _rem_case(name, asym_g=True, w_bits=4, w_grid=0, a_bits=8, rows=24, h=32, f=48, seed=3, shrink=0.8):
+    rng = np.random.default_rng(seed)
+    shape = {"Wqkv": (3 * h, h), "Wo": (h, h), "W1": (f, h), "W2": (h, f)}[name]
+    desc = O.ModuleDesc(1, h, 2, f, w_bits, a_bits, w_grid, True, True, asym_g, "f64", True)
+    w_t = rng.normal(0, 0.05, shape)
+    w_s = w_t + rng.normal(0, 0.004, shape)
+    a = rng.normal(0.3 if name == "W2" else 0.0, 1.0, (rows, shape[1]))
+    qmax = O.sym_qmax(w_bits)
+    ws = {k: np.ones(1, np.float32) for k in O.WEIGHTS}
+    ws[name] = (shrink * np.abs(w_s).max(1) / qmax if w_grid == 0 else np.abs(w_s).mean(1)).astype(np.float32)
+    a_st = np.ones(O.N_SITES, np.float32)
+    a_off = np.zeros(O.N_SITES, np.float32)
+    site = O.REM_SITE[name]
+    if site == O.SITE_G and asym_g:
+        a_off[site] = np.float32(a.min() + 0.2)                       # some values clip at the lower end
+        a_st[site] = np.float32(shrink * (a.max() - a_off[site]) / (2 ** a_bits - 1))
+    else:
+        a_st[site] = np.float32(shrink * np.abs(a).max() / O.sym_qmax(a_bits))
+    steps = O.make_steps([ws], [a_st], [a_off])[0]
+    return desc, w_t, w_s, steps, a, site
+
+
+@pytest.mark.parametrize("name,asym_g,w_bits,w_grid,a_bits", [("Wqkv", True, 4, 0, 8), ("Wo", True, 2, 1, 8), ("W1", True, 2, 0, 8),
+                                                            ("W2", True, 4, 0, 8), ("W2", False, 4, 0, 4)])
+def test_rem_objective_matches_definition_and_torch_autograd(name, asym_g, w_bits, w_grid, a_bits):
+    """Eq. 2 for one product: the loss is || w_hat^T a_hat - w^T a ||^2 written out with the quantizers of
+    Eq. 1, and every gradient equals library autograd over the detach form of the straight-through estimator."""
+    desc, w_t, w_s, steps, a, site = _rem_case(name, asym_g, w_bits, w_grid, a_bits)
+    r = O.rem_forward_loss_backward(desc, w_t, w_s, steps, name, a)
+    # the definition, written out independently of the oracle's helpers
+    s_w = steps["w"][name].astype(np.float64).reshape(-1, 1)
+    if w_grid == 0:
+        qm = 2 ** (w_bits - 1) - 1
+        w_hat = s_w * np.rint(np.clip((w_s.astype(np.float32) / s_w.astype(np.float32)).astype(np.float64), -qm, qm))
+    else:
+        w_hat = s_w * (np.clip(np.floor((w_s.astype(np.float32) / s_w.astype(np.float32)).astype(np.float64)), -2, 1) + 0.5)
+    s_a, beta = float(steps["a"][site]), float(steps["a_off"][site])
+    if site == O.SITE_G and asym_g:
+        z = ((a.astype(np.float32) - np.float32(beta)) / np.float32(s_a)).astype(np.float64)
+        a_hat = s_a * np.rint(np.clip(z, 0, 2 ** a_bits - 1)) + beta
+    else:
+        qa = 2 ** (a_bits - 1) - 1
+        a_hat = s_a * np.rint(np.clip((a.astype(np.float32) / np.float32(s_a)).astype(np.float64), -qa, qa))
+    diff = a_hat @ w_hat.T - a @ w_t.T
+    assert np.isclose(r["loss"], (diff ** 2).mean(), rtol=1e-10)
+    assert np.allclose(r["target"], a @ w_t.T, rtol=1e-12, atol=0)
+    # autograd
+    tw = torch.tensor(w_s, dtype=torch.float64, requires_grad=True)
+    tsw = torch.tensor(steps["w"][name].astype(np.float64), requires_grad=True)
+    tsa = torch.tensor(float(steps["a"][site]), dtype=torch.float64, requires_grad=True)
+    tb = torch.tensor(float(steps["a_off"][site]), dtype=torch.float64, requires_grad=True)
+    ta = torch.tensor(a, dtype=torch.float64)
+    ah = R.q_asym(ta, tsa, tb, a_bits) if (site == O.SITE_G and asym_g) else R.q_sym(ta, tsa, a_bits)
+    wh = R.q_weight(tw, tsw, w_bits, w_grid)
+    loss = ((ah @ wh.T - ta @ torch.tensor(w_t).T) ** 2).mean()
+    loss.backward()
+    assert np.isclose(r["loss"], loss.item(), rtol=1e-10)
+    assert np.allclose(r["dW"], tw.grad.numpy(), rtol=1e-8, atol=1e-14)
+    assert np.allclose(r["d_w_step"], tsw.grad.numpy(), rtol=1e-8, atol=1e-14)
+    assert np.isclose(r["d_a_step"], tsa.grad.item(), rtol=1e-8, atol=1e-14)
+    if site == O.SITE_G and asym_g:
+        assert abs(tb.grad.item()) > 0                                # the case really clips
+        assert np.isclose(r["d_a_off"], tb.grad.item(), rtol=1e-8, atol=1e-14)
+
+
+def test_rem_bypass_and_high_bit_width():
+    """Without quantizers the two products coincide when the student equals the teacher (loss 0, zero gradients);
+    at 16 bits the reconstruction error of Eq. 2 all but vanishes, and it grows as bits are taken away."""
+    desc, w_t, _, steps, a, site = _rem_case("W1")
+    bypass = O.ModuleDesc(1, desc.hidden, 2, desc.ffn, 0, 0, act_dtype="f64")
+    r = O.rem_forward_loss_backward(bypass, w_t, w_t, steps, "W1", a)
+    assert r["loss"] == 0.0 and not np.any(r["dW"])
+    losses = []
+    for bits in (16, 8, 6, 4):
+        d = O.ModuleDesc(1, desc.hidden, 2, desc.ffn, bits, bits, act_dtype="f64")
+        st = {"w": dict(steps["w"]), "a": steps["a"].copy(), "a_off": steps["a_off"].copy()}
+        st["w"]["W1"] = (np.abs(w_t).max(1) / O.sym_qmax(bits)).astype(np.float32)
+        st["a"][site] = np.float32(np.abs(a).max() / O.sym_qmax(bits))
+        losses.append(O.rem_forward_loss_backward(d, w_t, w_t, st, "W1", a)["loss"])
+    assert losses[0] < 1e-8 * float(((a @ w_t.T) ** 2).mean())
+    assert losses[0] < losses[1] < losses[2] < losses[3]
+
+
+def test_rem_step_reduces_the_reconstruction_error():
+    """Repeating the step of Eq. 2 on one batch lowers its loss (the objective is what the step descends), and the
+    first step moves every weight with a non-zero gradient by lr (AdamW's first step, decay aside)."""
+    desc, w_t, w_s, steps, a, site = _rem_case("Wqkv", shrink=0.6)
+    state, w = {}, w_s.astype(np.float32)
+    r0, w1 = O.rem_step(desc, w_t, w, steps, state, "Wqkv", a, lr=1e-3, weight_decay=0.0)
+    moved = np.abs(w1.astype(np.float64) - w.astype(np.float64))
+    nz = np.abs(r0["dW"]) > 1e-4                                    # lr / (1 + eps / |g|) with eps = 1e-8
+    assert nz.sum() > 100 and np.allclose(moved[nz], 1e-3, rtol=1e-3)
+    w = w1
+    first = r0["loss"]
+    for _ in range(30):
+        r, w = O.rem_step(desc, w_t, w, steps, state, "Wqkv", a, lr=2e-4, weight_decay=0.0)
+    assert r["loss"] < 0.7 * first
