@@ -270,6 +270,31 @@ int32_t mrem_gemm(int32_t dtype, const void* d_a, int32_t a_mn, int64_t lda, int
                   float alpha, float* d_out, int64_t ldc, int64_t c_batch_stride, int32_t block_n, int32_t* d_status,
                   void* cuda_stream);
 
+/* ---- the per-product objective (Eq. 2) ---------------------------------------------------- */
+
+/* One optimisation step on the reconstruction error of ONE matrix product (Eq. 2, Sec. 2.2: the objective
+ * that the module-wise loss of Eq. 3 generalises, and the building block of the layer-by-layer baseline
+ * the paper compares with):
+ *     min over w, s of  c * || Q(w)^T Q(a) - w^T a ||^2   over the rows of a,
+ * w = the teacher's matrix `tensor_id` (MREM_WQKV, MREM_WO, MREM_W1 or MREM_W2) of `layer`, Q(w) = the
+ * student's quantized matrix (Eq. 1, its own latent weights and steps), Q(a) = the activation quantizer
+ * that sits at that product's input in the module (layer input, attention context, FFN1 input, GELU
+ * output: the last one asymmetric with its offset when the context says so); c = 1 / (rows * out) with
+ * loss_mean, else 1.  No bias on either side, as in Eq. 2.  The straight-through gradients (Sec. 3.1.1)
+ * reach the latent matrix, its step(s), the activation step and offset; AdamW (mrem_optim, trainable_mask)
+ * updates exactly those and the matrix is re-quantized.  Biases, LayerNorm parameters and every other
+ * matrix are untouched.
+ *   d_a     [rows, in] activations in the context's storage type, device, 16-byte aligned, 1 <= rows <=
+ *           max_batch * max_seq
+ *   optim   NULL: no update; the gradients of this product (matrix, its steps, the activation step and
+ *           offset) can then be read with mrem_get_grad until the next step of any kind
+ *   d_loss  float32 [1], device: the loss before the update
+ * Needs per-row weight steps or the closed-form ternary weights (MREM_ERR_UNSUPPORTED otherwise), bound
+ * teacher and student parameters and steps (MREM_ERR_ORDER).  Uses the context's workspace and stream;
+ * asynchronous; invalidates the forward / loss / gradient state of a module step in progress. */
+int32_t mrem_rem_step(mrem_ctx* ctx, int32_t layer, int32_t tensor_id, const void* d_a, int32_t rows,
+                      const mrem_optim* optim, float* d_loss);
+
 /* ---- for callers that cannot allocate device memory -------------------------------------- */
 
 /* (The paper has no counterpart to this call; it exists for deployment reasons only.)

@@ -33,7 +33,7 @@ EXPORTS = (
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
-    "mrem_recon_step_host_wait",
+    "mrem_recon_step_host_wait", "mrem_rem_step",
 )
 
 
@@ -188,6 +188,11 @@ def mrem_step(ctx, optim):
 
 def mrem_backward_and_step(ctx, optim):
     _check(lib().mrem_backward_and_step(ctx, C.byref(optim)), "mrem_backward_and_step", ctx)
+
+
+def mrem_rem_step(ctx, layer, tensor_id, d_a, rows, optim, d_loss):
+    _check(lib().mrem_rem_step(ctx, int(layer), int(tensor_id), _p(d_a), int(rows), C.byref(optim) if optim is not None else None, _p(d_loss)),
+           "mrem_rem_step", ctx)
 
 
 def mrem_recon_step_host(ctx, h_x_teacher, h_x_student, h_valid_len, batch, seq, lam, optim) -> float:

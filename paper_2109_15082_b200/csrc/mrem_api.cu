@@ -81,6 +81,7 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->reduce_table = (ReduceEntry*)A.take(sizeof(ReduceEntry) * c->reduce_per_layer * L);
   c->adam_table = (AdamEntry*)A.take(sizeof(AdamEntry) * (MREM_N_PARAMS + N_WMAT + N_SITES + 1) * L);
   c->adam_rest = (AdamEntry*)A.take(sizeof(AdamEntry) * (MREM_N_PARAMS + N_WMAT + N_SITES + 1) * L);
+  c->rem_table = (AdamEntry*)A.take(sizeof(AdamEntry) * 2);
   c->h2d_xt = A.take(M * H * es);
   c->h2d_xs = A.take(M * H * es);
   c->h2d_len = (int32_t*)A.take(sizeof(int32_t) * d.max_batch);

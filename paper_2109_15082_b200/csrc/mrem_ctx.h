@@ -104,6 +104,7 @@ struct mrem_ctx {
   mrem::ReduceEntry* reduce_table;   int reduce_per_layer = 0;
   mrem::AdamEntry* adam_table;       int adam_entries = 0;  long long adam_elems = 0;   // every trainable tensor
   mrem::AdamEntry* adam_rest;        int rest_entries = 0;  long long rest_elems = 0;   // all but matrices and their steps
+  mrem::AdamEntry* rem_table = nullptr;                                                // the two scalar entries of mrem_rem_step
   bool w_ste_done = false;           // the weight gradients have been masked and the step gradients reduced
   // second stream (lowest priority) and its fork/join events: the memory-bound weight updates of a layer
   // run there while the main stream goes on with the tensor-core work of the layer below

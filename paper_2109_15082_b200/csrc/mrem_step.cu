@@ -249,22 +249,23 @@ int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S
 }
 
 // The fused update of one layer's four matrices and their row steps (Algorithm 2: Update(w), Update(s)).
-void enqueue_matrix_updates(mrem_ctx* c, int l, cudaStream_t st) {
+void enqueue_matrix_update(mrem_ctx* c, int l, int k, cudaStream_t st) {
   const mrem_module_desc& d = c->d;
   const int train_w = (d.trainable_mask & MREM_TRAIN_WEIGHTS) != 0, train_s = (d.trainable_mask & MREM_TRAIN_W_STEPS) != 0;
-  for (int k = 0; k < N_WMAT; ++k) {
-    const int pid = kMatParam[k];
-    WeightBuf& w = c->wq[l][k];
-    LayerGrad& g = c->grad[l];
-    if (d.w_grid == 2) {
-      launch_ternary_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->optim_sc, w.rows, w.cols, train_w,
-                            w.codes, w.rowsum, w.scale, w.what, c->dt, st);
-      continue;
-    }
-    launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
-                               c->w_ste_done ? g.ws[k] : nullptr, g.m_ws[k], g.v_ws[k], c->optim_sc, w.rows, w.cols,
-                               d.w_bits, d.w_grid, train_w, train_s, w.codes, w.rowsum, w.scale, w.what, c->dt, st);
+  const int pid = kMatParam[k];
+  WeightBuf& w = c->wq[l][k];
+  LayerGrad& g = c->grad[l];
+  if (d.w_grid == 2) {
+    launch_ternary_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->optim_sc, w.rows, w.cols, train_w,
+                          w.codes, w.rowsum, w.scale, w.what, c->dt, st);
+    return;
   }
+  launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
+                             c->w_ste_done ? g.ws[k] : nullptr, g.m_ws[k], g.v_ws[k], c->optim_sc, w.rows, w.cols,
+                             d.w_bits, d.w_grid, train_w, train_s, w.codes, w.rowsum, w.scale, w.what, c->dt, st);
+}
+void enqueue_matrix_updates(mrem_ctx* c, int l, cudaStream_t st) {
+  for (int k = 0; k < N_WMAT; ++k) enqueue_matrix_update(c, l, k, st);
 }
 
 // ------------------------------------------------------------------ backward
@@ -562,6 +563,112 @@ int32_t mrem_step(mrem_ctx* c, const mrem_optim* o) {
   c->have_grads = false; c->have_loss = false; c->have_student = false; c->have_teacher = false;
   c->codes_fresh = d.w_step_per_row != 0;
   c->weights_quantized = c->codes_fresh;
+  return MREM_OK;
+}
+
+
+// Eq. 2: one optimisation step on the reconstruction error of ONE matrix product of one layer,
+//   min_{w, s} || Q(w)^T Q(a) - w^T a ||^2  over the rows of a,
+// with the same kernels as the module step: the full-precision product on the bf16 (or fp32) path, the
+// quantized one on integer codes, the loss kernel of Eq. 3 on the pair, the straight-through backward of
+// the two quantizers, the fused update of the matrix and AdamW on the input quantizer's step (and offset).
+int32_t mrem_rem_step(mrem_ctx* c, int32_t layer, int32_t tensor_id, const void* a, int32_t rows, const mrem_optim* o,
+                      float* d_loss) {
+  if (!c || !a || !d_loss) return MREM_ERR_ARG;
+  TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
+  const mrem_module_desc& d = c->d;
+  if (layer < 0 || layer >= d.n_layers) return fail(c, MREM_ERR_ARG, "rem_step: layer");
+  int k = -1;
+  for (int i = 0; i < N_WMAT; ++i) if (kMatParam[i] == tensor_id) k = i;
+  if (k < 0) return fail(c, MREM_ERR_ARG, "rem_step: tensor_id must name one of the four weight matrices");
+  if (rows < 1 || rows > c->max_tokens) return fail(c, MREM_ERR_SHAPE, "rem_step: rows outside the context's maximum (max_batch * max_seq)");
+  if (reinterpret_cast<uintptr_t>(a) & 15) return fail(c, MREM_ERR_ALIGN, "rem_step: d_a must be 16-byte aligned");
+  if (!d.w_step_per_row && d.w_grid != 2) return fail(c, MREM_ERR_UNSUPPORTED, "rem_step: needs per-row weight steps or the closed-form ternary weights");
+  const int site = k == W_QKV ? S_X : (k == W_O ? S_C : (k == W_1 ? S_A : S_G));
+  const LayerBind& b = c->bind[layer];
+  if (!b.teacher[tensor_id] || !b.student[tensor_id] || (!b.w_steps[k] && d.w_grid != 2) || !b.a_steps[site])
+    return fail(c, MREM_ERR_ORDER, "rem_step: parameters or steps not bound");
+  const ActRange ar = site_range(d, site);
+  if (ar.asym && !b.a_off[site]) return fail(c, MREM_ERR_ORDER, "rem_step: offset of the GELU-site quantizer not bound");
+  if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
+  int rc = mrem_quantize_weights(c);
+  if (rc != MREM_OK) return rc;
+
+  LayerStash& s = c->stash[layer];
+  LayerGrad& g = c->grad[layer];
+  WeightBuf& w = c->wq[layer][k];
+  const int N = w.rows, K = w.cols, F = d.ffn;
+  const long long M = rows;
+  cudaStream_t st = c->stream;
+  Runner r(c);
+  const int ok = r.okind();
+  // scratch of the module step, by width: codes of the input, the two products, the loss gradient, d a_hat
+  int8_t* q8 = K == F ? s.g_q8 : s.x_q8;
+  void* qt = K == F ? s.g_qt : s.x_qt;
+  void* target = N == F ? c->t_g : c->t_qkv;
+  void* y = N == F ? s.u : s.qkv;
+  void* dy = N == F ? c->d_u : c->d_qkv;
+  void* dxhat = K == F ? c->d_ghat : c->d_ahat;
+  const float* step = b.a_steps[site];
+  const float* off = ar.asym ? b.a_off[site] : nullptr;
+  const int bias_id = tensor_id + 1;                     // the bias follows its matrix in the parameter list
+
+  // w^T a
+  r.gemm(view(a, K), view(b.teacher[tensor_id], K), (int)M, N, K, 1, 1, Epi(target, ok, N).e);
+  // Q(w)^T Q(a): integer codes, exact accumulation, dequantized in the epilogue (offset term as a column bias)
+  launch_quantize_act(a, c->dt, M, K, K, step, off, ar.lo, ar.hi, q8, K, qt, K, st);
+  Epi fe(y, ok, N);
+  fe.alpha(1.f, step).colscale(w.scale);
+  if (ar.asym) {
+    if (cudaMemsetAsync(c->alt_rowbias, 0, sizeof(float) * N, st) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "rem_step: memset failed");
+    launch_effective_bias(c->alt_rowbias, off, w.scale, w.rowsum, w.beff, N, st);
+    fe.colbias(w.beff);
+  }
+  r.gemm_i8(q8, ar.asym ? 1 : 0, w.codes, (int)M, N, K, fe.e);
+  // loss and its gradient
+  const long long n = M * N;
+  const float cc = d.loss_mean ? 1.f / (float)n : 1.f;
+  launch_loss(y, target, 1, n, cc, dy, c->loss_partial, c->status, c->dt, st);
+  launch_loss_finalize(c->loss_partial, 1, cc, d_loss, nullptr, st);
+  // d l / d w_hat = dy^T a_hat, a_hat = step * codes (+ offset: a row bias of offset * column sums of dy)
+  Epi we(g.p[tensor_id], OUT_F32, K);
+  we.alpha(1.f, step);
+  if (ar.asym) {
+    launch_col_reduce(dy, N, nullptr, nullptr, nullptr, nullptr, 0, M, N, g.p[bias_id], nullptr, nullptr, c->col_scratch, c->col_plane,
+                      c->col_counters, c->dt, st);
+    launch_scale_vec(g.p[bias_id], off, c->rowbias, N, st);
+    we.rowbias(c->rowbias);
+  }
+  r.gemm(view(dy, N, 1), view(qt, K, 1), N, K, (int)M, 1, 1, we.e);
+  // d l / d a_hat = dy w_hat, then the straight-through factors of the input quantizer
+  r.gemm(view(dy, N), view(w.what, K, 1), (int)M, K, N, 1, 1, Epi(dxhat, ok, K).e);
+  launch_ste_act(a, K, dxhat, K, nullptr, 0, dxhat, K, M, K, step, off, ar.lo, ar.hi, s.part + site * RED_BLOCKS,
+                 ar.asym ? s.part + N_SITES * RED_BLOCKS : nullptr, c->dt, st);
+  const ReduceEntry* red = c->reduce_table + (size_t)layer * c->reduce_per_layer;
+  launch_reduce_table(red + site, 1, st);
+  if (ar.asym) launch_reduce_table(red + N_SITES, 1, st);
+  c->w_ste_done = false;
+  if (o) {
+    // update: the matrix and its steps (which also re-quantizes it), the input quantizer's step and offset
+    launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
+                         o->weight_decay, st);
+    enqueue_matrix_update(c, layer, k, st);
+    if (d.trainable_mask & MREM_TRAIN_A_STEPS) {
+      AdamEntry host[2];
+      int ne = 0;
+      host[ne++] = AdamEntry{b.a_steps[site], g.a + site, g.m_a + site, g.v_a + site, 1, 0.f, 1e-8f};
+      if (ar.asym) host[ne++] = AdamEntry{b.a_off[site], g.off + site, g.m_off + site, g.v_off + site, 1, 0.f, -INFINITY};
+      if (cudaMemcpyAsync(c->rem_table, host, sizeof(AdamEntry) * ne, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return fail(c, MREM_ERR_CUDA, "rem_step: table upload failed");
+      launch_adamw_table(c->rem_table, ne, ne, c->optim_sc, st);
+    }
+  }
+  if (r.rc != MREM_OK) return r.rc;
+  if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "rem_step: launch failed");
+  c->have_grads = o == nullptr;        // without an update the gradients stay readable (mrem_get_grad)
+  c->have_loss = false; c->have_student = false; c->have_teacher = false;
+  c->codes_fresh = true;
+  c->weights_quantized = true;
   return MREM_OK;
 }
 

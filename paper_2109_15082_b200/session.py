@@ -149,6 +149,12 @@ class ReconModule:
     def step(self, optim):
         B.mrem_step(self.ctx, optim)
 
+    def rem_step(self, layer, tensor_id, a, optim):
+        """One step of Eq. 2 on one matrix product; `a` is a [rows, in] device tensor (optim None: loss and
+        gradients only).  Returns the loss tensor."""
+        B.mrem_rem_step(self.ctx, layer, tensor_id, a, a.shape[0], optim, self.loss)
+        return self.loss[:1]
+
     def backward_and_step(self, optim):
         B.mrem_backward_and_step(self.ctx, optim)
 

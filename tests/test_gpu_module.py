@@ -101,6 +101,95 @@ def test_fused_attention_backward_matches_kernel_per_operation_path(seq, lo):
         p.close()
 
 
+REM_MATRICES = {"Wqkv": (B.WQKV, 0), "Wo": (B.WO, 1), "W1": (B.W1, 2), "W2": (B.W2, 3)}
+
+
+@pytest.mark.parametrize("name,base,asym,a_bits", [("Wqkv", "base3_w4a8", 3, None), ("Wo", "base3_w2a8", 3, None), ("W1", "base3_w4a8", 3, 4),
+                                                  ("W2", "base3_w4a8", 3, None), ("W2", "base3_w4a8", 1, None)])
+def test_rem_step_of_one_product_matches_the_oracle(name, base, asym, a_bits):
+    """Eq. 2 on one matrix product through the C-ABI: the loss and every gradient (matrix, its row steps, the
+    input quantizer's step and offset) against the oracle within the module tests' tolerance on a ragged row
+    count (120 rows: one partial tile); then one real step: the updated matrix, steps and offset against the
+    oracle's AdamW fed with those gradients, the re-quantized codes bit-exact against Eq. 1 on the updated
+    values, and every other parameter untouched."""
+    wl = _wl(base, n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40)
+    p = Problem(wl, step_shrink=0.8, student_noise=0.002, asym=asym, a_bits=a_bits)
+    try:
+        m, layer = p.m, 1
+        pid, k = REM_MATRICES[name]
+        site = O.REM_SITE[name]
+        rows, cols = 120, m.shapes[pid][1]
+        a_np = synth.normal(5, "rem_a" + name, (rows, cols), 1.0) + (0.4 if name == "W2" else 0.0)
+        a_dev = m.to_device(a_np)
+        a = a_dev.float().cpu().numpy()                             # the stored bytes, widened
+        # steps of the product's input quantizer for THIS input, tightened so that some values clip
+        bits = a_bits or wl.a_bits
+        if site == O.SITE_G and (asym & 2):
+            p.off[layer, site] = np.float32(a.min() + 0.3)
+            p.a[layer, site] = np.float32(0.8 * (a.max() - p.off[layer, site]) / (2 ** bits - 1))
+        else:
+            p.a[layer, site] = np.float32(0.8 * np.abs(a).max() / O.sym_qmax(bits))
+        m.set_steps(p.ws, p.a, p.off)
+        steps = p.oracle_steps()[layer]
+        w_t, w_s = p.teacher[layer][name], p.student[layer][name]
+
+        # loss and gradients
+        loss = float(m.rem_step(layer, pid, a_dev, None)[0])
+        gW = m.grad(layer, pid, m.shapes[pid]).cpu().numpy()
+        gS = m.grad(layer, B.GRAD_STEP + k, (m.shapes[pid][0],)).cpu().numpy()
+        gA = m.grad(layer, B.GRAD_STEP + 4 + site, (1,)).item()
+        gOff = m.grad(layer, B.GRAD_OFFSET + 4 + site, (1,)).item()
+        assert m.poll_status() == 0
+        r = O.rem_forward_loss_backward(p.desc, w_t, w_s, steps, name, a)
+        assert abs(loss - r["loss"]) / r["loss"] < GRAD_TOL, (loss, r["loss"])
+        assert rel(gW, r["dW"]) < GRAD_TOL
+        assert rel(gS, r["d_w_step"]) < GRAD_TOL
+        assert abs(gA - r["d_a_step"]) / abs(r["d_a_step"]) < GRAD_TOL, (gA, r["d_a_step"])
+        if site == O.SITE_G and (asym & 2):
+            assert abs(r["d_a_off"]) > 0 and abs(gOff - r["d_a_off"]) / abs(r["d_a_off"]) < GRAD_TOL, (gOff, r["d_a_off"])
+
+        # one step: AdamW of the oracle on the gradients just read
+        before = m.student_numpy()
+        opt = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+        loss2 = float(m.rem_step(layer, pid, a_dev, B.make_optim(step=1, **opt))[0])
+        torch.cuda.synchronize()
+        assert loss2 == loss                                         # same input, same weights: the same bits
+        after = m.student_numpy()
+        w1, a1, off1 = m.get_steps()
+        z = lambda x: np.zeros_like(np.asarray(x, np.float64))
+
+        def expect(p0, grad, wd, clamp=None):
+            p1, _, _ = O.adamw_update(np.asarray(p0, np.float64), np.asarray(grad, np.float64), z(p0), z(p0), 1, opt["lr"], 0.9, 0.999, 1e-8, wd)
+            return np.maximum(p1, clamp) if clamp is not None else p1
+
+        tol = dict(rtol=1e-5, atol=2e-3 * opt["lr"])
+        assert np.allclose(after[layer][name], expect(before[layer][name], gW, 0.01), **tol)
+        assert np.allclose(w1[layer][name], expect(p.ws[layer][name], gS, 0.0, O.MIN_STEP), **tol)
+        assert np.allclose(a1[layer, site], expect(p.a[layer, site:site + 1], [gA], 0.0, O.MIN_STEP), **tol)
+        if site == O.SITE_G and (asym & 2):
+            assert np.allclose(off1[layer, site], expect(p.off[layer, site:site + 1], [gOff], 0.0), **tol)
+        else:
+            assert np.array_equal(off1, p.off)
+        for l in range(wl.n_layers):
+            for key in O.PARAMS:
+                if (l, key) != (layer, name):
+                    assert np.array_equal(after[l][key], before[l][key]), (l, key)
+            for key in O.WEIGHTS:
+                if (l, key) != (layer, name):
+                    assert np.array_equal(w1[l][key], p.ws[l][key]), (l, key)
+        a_mask = np.ones_like(p.a, bool)
+        a_mask[layer, site] = False
+        assert np.array_equal(a1[a_mask], p.a[a_mask])
+        # the matrix was re-quantized by the update: Eq. 1 on the updated weights and steps, bit for bit
+        codes, rowsum = m.weight_codes(layer, pid)
+        q_ref, _, _ = O.quantize_weight(after[layer][name], w1[layer][name].reshape(-1, 1), wl.w_bits, wl.w_grid, wl.act_dtype)
+        assert np.array_equal(codes.cpu().numpy().astype(np.int64), q_ref)
+        assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), q_ref.sum(-1))
+        assert m.poll_status() == 0
+    finally:
+        p.close()
+
+
 def test_teacher_forcing_mix():
     wl, kw = CASES["bf16_small"]
     p = Problem(wl, **kw)
