@@ -557,13 +557,22 @@ def make_steps(w_steps, a, a_off):
             for l in range(len(w_steps))]
 
 
-def forward_loss_backward(desc, teacher, student, steps, x_t, x_s, valid_len=None, lam=0.0):
-    """Teacher output, student output, loss of Eq. 3 and all gradients (no update)."""
+def forward_loss_backward(desc, teacher, student, steps, x_t, x_s, valid_len=None, lam=0.0, head=None):
+    """Teacher output, student output, loss of Eq. 3 and all gradients (no update).  With `head` (the last
+    module of the model) the output-logit term is added to the loss and its gradient enters at the last
+    layer's output beside that layer's own term."""
     f_t = teacher_forward(desc, teacher, x_t, valid_len)
     f_s, caches = student_forward(desc, student, steps, x_s, valid_len, x_teacher=x_t, lam=lam)
     total, per, dF = recon_loss(desc, f_s, f_t)
-    grads = student_backward(desc, student, caches, dF)
-    return dict(f_t=f_t, f_s=f_s, loss=total, loss_per_layer=per, grads=grads, caches=caches)
+    out = dict(f_t=f_t, f_s=f_s, loss_per_layer=per, caches=caches)
+    if head is not None:
+        lz, dFz, z_s, z_t = logit_loss(desc, head, f_s[-1], f_t[-1])
+        total += lz
+        dF[-1] = dF[-1] + dFz
+        out.update(logit_loss=lz, logits_student=z_s, logits_teacher=z_t)
+    out["loss"] = total
+    out["grads"] = student_backward(desc, student, caches, dF)
+    return out
 
 
 def recon_step(desc, teacher, student, steps, state, x_t, x_s, valid_len=None, lam=0.0,
@@ -594,6 +603,34 @@ def recon_step(desc, teacher, student, steps, state, x_t, x_s, valid_len=None, l
             steps[l]["a"] = np.maximum(upd((l, "a"), steps[l]["a"], g["a"], 0.0), MIN_STEP).astype(np.float32)
             steps[l]["a_off"] = upd((l, "a_off"), steps[l]["a_off"], g["a_off"], 0.0).astype(np.float32)
     return r
+
+
+# ----------------------------------------------------------------------------- output logits of the last module (Sec. 4.1)
+
+def head_logits(head, f_last):
+    """Classification head on the last layer's output f_last [B, S, H] (as stored): the first token of every
+    sequence through the pooler (dense + tanh) and the classifier (dense).  The head is not quantized
+    (Sec. 3.1) and is the same on the teacher and the student side.  head: dict Wp [H, H], bp [H],
+    Wc [C, H], bc [C].  Returns (logits [B, C], pooled [B, H])."""
+    cls = np.asarray(f_last, np.float64)[:, 0, :]
+    pooled = np.tanh(cls @ np.asarray(head["Wp"], np.float64).T + np.asarray(head["bp"], np.float64))
+    return pooled @ np.asarray(head["Wc"], np.float64).T + np.asarray(head["bc"], np.float64), pooled
+
+
+def logit_loss(desc, head, f_student_last, f_teacher_last):
+    """The output-logit term of the last module: l_z = c * || z_hat - z ||^2, c = 1 / (B * C) when `loss_mean`
+    (MSE) else 1.  Returns (loss, d l_z / d f_hat_last [B, S, H]: non-zero at the first token only, logits of
+    the student, logits of the teacher)."""
+    z_t, _ = head_logits(head, f_teacher_last)
+    z_s, pooled = head_logits(head, f_student_last)
+    diff = z_s - z_t
+    c = 1.0 / diff.size if desc.loss_mean else 1.0
+    loss = c * float((diff * diff).sum())
+    dz = 2.0 * c * diff
+    dpre = (dz @ np.asarray(head["Wc"], np.float64)) * (1.0 - pooled * pooled)
+    dF = np.zeros(np.shape(f_student_last), np.float64)
+    dF[:, 0, :] = dpre @ np.asarray(head["Wp"], np.float64)
+    return loss, dF, z_s, z_t
 
 
 # ----------------------------------------------------------------------------- Eq. 2: reconstruction error of ONE matrix product

@@ -548,3 +548,73 @@ def test_rem_step_reduces_the_reconstruction_error():
     for _ in range(30):
         r, w = O.rem_step(desc, w_t, w, steps, state, "Wqkv", a, lr=2e-4, weight_decay=0.0)
     assert r["loss"] < 0.7 * first
+
+
+# ----------------------------------------------------------------------------- output logits of the last module
+
+def _head(h, n_classes, seed=11):
+    rng = np.random.default_rng(seed)
+    return dict(Wp=rng.normal(0, 0.3, (h, h)), bp=rng.normal(0, 0.1, h), Wc=rng.normal(0, 0.3, (n_classes, h)),
+                bc=rng.normal(0, 0.1, n_classes))
+
+
+@pytest.mark.parametrize("loss_mean", [True, False])
+def test_logit_loss_matches_torch_head_and_autograd(loss_mean):
+    """Pooler (dense + tanh on the first token) and classifier as library layers; the gradient of the logit MSE
+    with respect to the student's last layer output from library autograd; zero away from the first token."""
+    rng = np.random.default_rng(2)
+    B_, S_, H_, C_ = 3, 5, 16, 4
+    head = _head(H_, C_)
+    f_s, f_t = rng.normal(0, 1, (B_, S_, H_)), rng.normal(0, 1, (B_, S_, H_))
+    desc = O.ModuleDesc(1, H_, 2, 32, loss_mean=loss_mean)
+    loss, dF, z_s, z_t = O.logit_loss(desc, head, f_s, f_t)
+    tp = {k: torch.tensor(v, dtype=torch.float64) for k, v in head.items()}
+    ts = torch.tensor(f_s, dtype=torch.float64, requires_grad=True)
+
+    def logits(f):
+        return torch.nn.functional.linear(torch.tanh(torch.nn.functional.linear(f[:, 0], tp["Wp"], tp["bp"])), tp["Wc"], tp["bc"])
+
+    zs, zt = logits(ts), logits(torch.tensor(f_t, dtype=torch.float64))
+    ref = ((zs - zt) ** 2).mean() if loss_mean else ((zs - zt) ** 2).sum()
+    ref.backward()
+    assert np.allclose(z_s, zs.detach().numpy(), rtol=1e-12) and np.allclose(z_t, zt.numpy(), rtol=1e-12)
+    assert np.isclose(loss, ref.item(), rtol=1e-12)
+    assert np.allclose(dF, ts.grad.numpy(), rtol=1e-10, atol=1e-16)
+    assert not np.any(dF[:, 1:, :]) and np.any(dF[:, 0, :])
+    assert O.logit_loss(desc, head, f_t, f_t)[0] == 0.0             # equal outputs: no logit error
+
+
+def test_module_with_head_adds_the_logit_term_at_the_last_layer_only():
+    """Loss = Eq. 3 + logit term; the extra gradient enters at the last layer's output: against torch autograd of the
+    whole quantized module with the head on top."""
+    wl = synth.shrink(synth.workloads()["tiny"], n_layers=2, hidden=16, n_heads=2, ffn=32, seq=6, batch=3)
+    desc = O.ModuleDesc(2, 16, 2, 32, 4, 8, act_dtype="f64")
+    params = synth.teacher_params(wl, 0, bias_std=0.02)
+    student = [{k: (v + synth.normal(1, f"n{l}{k}", v.shape, 0.003)).astype(np.float32) for k, v in p.items()} for l, p in enumerate(params)]
+    x = synth.hidden_states(wl, wl.batch, 0).astype(np.float64)
+    vl = np.array([6, 4, 5])
+    ws = O.init_weight_steps(desc, student, 0)
+    a, off = O.init_act_steps(desc, student, x, vl)
+    steps = O.make_steps(ws, (a * 0.8).astype(np.float32), off)
+    head = _head(16, 3)
+    base = O.forward_loss_backward(desc, params, student, steps, x, x, vl)
+    r = O.forward_loss_backward(desc, params, student, steps, x, x, vl, head=head)
+    assert np.isclose(r["loss"], base["loss"] + r["logit_loss"], rtol=1e-12) and r["logit_loss"] > 0
+    # autograd over the torch model of the module (detach form of the estimator) with the head on top
+    cfg = dict(n_heads=2, a_bits=8, w_bits=4, w_grid=0, asym_p=True, asym_g=True, ln_eps=desc.ln_eps)
+    tparams = [{k: torch.tensor(v.astype(np.float64), requires_grad=True) for k, v in p.items()} for p in student]
+    tsteps = [dict(w={k: torch.tensor(st["w"][k].astype(np.float64), requires_grad=True) for k in O.WEIGHTS},
+                   a=[torch.tensor(float(v), dtype=torch.float64, requires_grad=True) for v in st["a"]],
+                   a_off=[torch.tensor(float(v), dtype=torch.float64, requires_grad=True) for v in st["a_off"]]) for st in steps]
+    outs = R.module(torch.tensor(x), tparams, tsteps, cfg, vl)
+    tp = {k: torch.tensor(v, dtype=torch.float64) for k, v in head.items()}
+    logits = lambda f: torch.nn.functional.linear(torch.tanh(torch.nn.functional.linear(f[:, 0], tp["Wp"], tp["bp"])), tp["Wc"], tp["bc"])
+    loss = sum(((o - torch.tensor(ft)) ** 2).mean() for o, ft in zip(outs, r["f_t"]))
+    loss = loss + ((logits(outs[-1]) - logits(torch.tensor(r["f_t"][-1]))) ** 2).mean()
+    loss.backward()
+    assert np.isclose(r["loss"], loss.item(), rtol=1e-9)
+    for l in range(2):
+        for k in O.PARAMS:
+            assert np.allclose(r["grads"][l][k], tparams[l][k].grad.numpy(), rtol=1e-6, atol=1e-12), (l, k)
+        assert np.allclose(r["grads"][l]["a"], [t.grad.item() if t.grad is not None else 0.0 for t in tsteps[l]["a"]], rtol=1e-6, atol=1e-12)
+    assert not np.allclose(r["grads"][0]["W1"], base["grads"][0]["W1"], rtol=1e-6, atol=0)   # the term reaches the layers below
