@@ -270,6 +270,23 @@ int32_t mrem_gemm(int32_t dtype, const void* d_a, int32_t a_mn, int64_t lda, int
                   float alpha, float* d_out, int64_t ldc, int64_t c_batch_stride, int32_t block_n, int32_t* d_status,
                   void* cuda_stream);
 
+/* ---- the last module's output logits (Sec. 4.1) -------------------------------------------- */
+
+/* Sec. 4.1: "besides the grouped Transformer layers" the MSE of the output logits is minimised; the
+ * classification head belongs to the last module and is not quantized (Sec. 3.1), so one set of head
+ * parameters serves both sides and is not trained here.  After this call mrem_recon_loss adds
+ *     c_z * || z_hat - z ||^2,   z = Wc tanh(Wp f_L[:, 0, :] + bp) + bc   (pooler and classifier on the first token
+ * of the last layer's output; c_z = 1 / (batch * n_classes) with loss_mean, else 1) to the total loss and the
+ * term's gradient to d loss / d f_hat_L, from where mrem_module_backward carries it through the module.
+ *   d_wp [hidden, hidden], d_bp [hidden], d_wc [n_classes, hidden], d_bc [n_classes]: float32, device,
+ *       caller-owned, borrowed until unbound (d_wp = NULL unbinds) or the context is destroyed
+ *   d_logit_loss  NULL or float32 [1]: the term alone, written by every mrem_recon_loss
+ *   d_logits      NULL or float32 [2, max_batch, n_classes]: student logits, then teacher logits ([2, batch, n_classes]
+ *                 packed for the batch of the call)
+ * hidden <= 2048, n_classes <= 64 (MREM_ERR_SHAPE).  Bind before a step graph is captured. */
+int32_t mrem_bind_head(mrem_ctx* ctx, const float* d_wp, const float* d_bp, const float* d_wc, const float* d_bc,
+                       int32_t n_classes, float* d_logit_loss, float* d_logits);
+
 /* ---- the per-product objective (Eq. 2) ---------------------------------------------------- */
 
 /* One optimisation step on the reconstruction error of ONE matrix product (Eq. 2, Sec. 2.2: the objective

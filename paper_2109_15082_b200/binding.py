@@ -33,7 +33,7 @@ EXPORTS = (
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
-    "mrem_recon_step_host_wait", "mrem_rem_step",
+    "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head",
 )
 
 
@@ -188,6 +188,11 @@ def mrem_step(ctx, optim):
 
 def mrem_backward_and_step(ctx, optim):
     _check(lib().mrem_backward_and_step(ctx, C.byref(optim)), "mrem_backward_and_step", ctx)
+
+
+def mrem_bind_head(ctx, d_wp, d_bp, d_wc, d_bc, n_classes, d_logit_loss=None, d_logits=None):
+    _check(lib().mrem_bind_head(ctx, _p(d_wp), _p(d_bp), _p(d_wc), _p(d_bc), int(n_classes), _p(d_logit_loss), _p(d_logits)),
+           "mrem_bind_head", ctx)
 
 
 def mrem_rem_step(ctx, layer, tensor_id, d_a, rows, optim, d_loss):

@@ -90,6 +90,14 @@ void launch_loss(const void* f_hat, const void* f, int n_layers, long long n_per
 void launch_loss_finalize(const float* partial, int n_layers, float c, float* loss_total, float* loss_per_layer,
                           cudaStream_t st);
 
+// Output-logit term of the last module: pooler (dense + tanh) and classifier on the first token of both last
+// layer outputs [B, S, H]; adds cc * sum (z_hat - z)^2 to *loss_total (and writes it to *logit_loss when non-null),
+// adds its gradient to dF_last at the first tokens; `part` >= B floats of scratch; `logits` null or [2, B, C]
+// (student, teacher).  Returns 0, -1 when hidden / classes do not fit the kernel's shared memory, -2 on a launch error.
+int launch_head_logit_loss(const void* f_s_last, const void* f_t_last, int B, int S, int H, int C, const float* wp,
+                           const float* bp, const float* wc, const float* bc, float cc, void* dF_last, float* part,
+                           float* logits, float* loss_total, float* logit_loss, int dt, cudaStream_t st);
+
 // ---- backward kernels
 // Straight-through backward of an activation quantizer on a 2-D view:
 // dx = dxhat * 1[lo <= z <= hi] (+ add), per-block partials of d l/d step (and d l/d offset).

@@ -429,6 +429,18 @@ int32_t mrem_set_fused_attention_backward(mrem_ctx* c, int32_t on) {
   return MREM_OK;
 }
 
+int32_t mrem_bind_head(mrem_ctx* c, const float* wp, const float* bp, const float* wc, const float* bc, int32_t n_classes,
+                       float* d_logit_loss, float* d_logits) {
+  if (!c) return MREM_ERR_ARG;
+  if (!wp) { c->head = {}; return MREM_OK; }                 // unbind
+  if (!bp || !wc || !bc) return fail(c, MREM_ERR_ARG, "bind_head: NULL tensor");
+  if (n_classes < 1 || n_classes > 64) return fail(c, MREM_ERR_SHAPE, "bind_head: 1 <= n_classes <= 64");
+  if (c->d.hidden > 2048) return fail(c, MREM_ERR_SHAPE, "bind_head: hidden size up to 2048");
+  c->head.wp = wp; c->head.bp = bp; c->head.wc = wc; c->head.bc = bc;
+  c->head.n_classes = n_classes; c->head.logit_loss = d_logit_loss; c->head.logits = d_logits;
+  return MREM_OK;
+}
+
 int32_t mrem_poll_status(mrem_ctx* c, int32_t* h_status) {
   if (!c || !h_status) return MREM_ERR_ARG;
   int v = 0;

@@ -112,6 +112,8 @@ struct mrem_ctx {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   cudaEvent_t ev_layer[2] = {nullptr, nullptr};   // side stream done with the gradient buffers of a layer parity
   cudaStream_t teacher_stream = nullptr;   // set for the duration of a step that runs the teacher pass beside the student's
+  // classification head of the model's last module (null: none): the output-logit term of the loss
+  struct { const float *wp = nullptr, *bp = nullptr, *wc = nullptr, *bc = nullptr; int n_classes = 0; float* logit_loss = nullptr; float* logits = nullptr; } head;
   bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;

@@ -490,6 +490,19 @@ int32_t mrem_recon_loss(mrem_ctx* c, float* loss_total, float* loss_per_layer) {
   const float cc = c->d.loss_mean ? 1.f / (float)n : 1.f;
   launch_loss(c->s_out, c->t_out, c->d.n_layers, n, cc, c->dF, c->loss_partial, c->status, c->dt, c->stream);
   launch_loss_finalize(c->loss_partial, c->d.n_layers, cc, loss_total, loss_per_layer, c->stream);
+  if (c->head.wp) {
+    // last module of the model: the output-logit term, its gradient added to the last layer's loss gradient
+    const int L = c->d.n_layers, C = c->head.n_classes;
+    if (c->cur_batch > RED_BLOCKS) return fail(c, MREM_ERR_SHAPE, "recon_loss: batch too large for the logit term");
+    const float cz = c->d.loss_mean ? 1.f / (float)((long long)c->cur_batch * C) : 1.f;
+    const long long last = (long long)(L - 1) * n;
+    const int hrc = launch_head_logit_loss((const char*)c->s_out + last * c->esz, (const char*)c->t_out + last * c->esz, c->cur_batch,
+                                           c->cur_seq, c->d.hidden, C, c->head.wp, c->head.bp, c->head.wc, c->head.bc, cz,
+                                           (char*)c->dF + last * c->esz, c->loss_partial, c->head.logits, loss_total,
+                                           c->head.logit_loss, c->dt, c->stream);
+    if (hrc == -1) return fail(c, MREM_ERR_SHAPE, "recon_loss: hidden size / class count too large for the logit term");
+    if (hrc != 0) return fail(c, MREM_ERR_CUDA, "recon_loss: launch failed");
+  }
   if (cudaGetLastError() != cudaSuccess) return fail(c, MREM_ERR_CUDA, "recon_loss: launch failed");
   c->have_loss = true;
   return MREM_OK;

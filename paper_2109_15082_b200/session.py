@@ -149,6 +149,19 @@ class ReconModule:
     def step(self, optim):
         B.mrem_step(self.ctx, optim)
 
+    def bind_head(self, head):
+        """head: dict Wp [H, H], bp [H], Wc [C, H], bc [C] (numpy) of the classification head, or None to unbind."""
+        if head is None:
+            B.mrem_bind_head(self.ctx, None, None, None, None, 0)
+            self._head = None
+            return
+        t = {k: torch.from_numpy(np.ascontiguousarray(head[k], dtype=np.float32)).to(self.device) for k in ("Wp", "bp", "Wc", "bc")}
+        C_ = int(t["Wc"].shape[0])
+        self.logit_loss = torch.zeros(1, dtype=torch.float32, device=self.device)
+        self.logits = torch.zeros(2, self.max_batch, C_, dtype=torch.float32, device=self.device)
+        self._head = t                                       # keeps the device tensors alive while bound
+        B.mrem_bind_head(self.ctx, t["Wp"], t["bp"], t["Wc"], t["bc"], C_, self.logit_loss, self.logits)
+
     def rem_step(self, layer, tensor_id, a, optim):
         """One step of Eq. 2 on one matrix product; `a` is a [rows, in] device tensor (optim None: loss and
         gradients only).  Returns the loss tensor."""

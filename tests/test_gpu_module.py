@@ -101,6 +101,50 @@ def test_fused_attention_backward_matches_kernel_per_operation_path(seq, lo):
         p.close()
 
 
+@pytest.mark.parametrize("case", ["bf16_small", "tiny_f32"])
+def test_output_logit_term_of_the_last_module_matches_the_oracle(case):
+    """With a classification head bound the loss gains the MSE of the output logits (pooler + classifier on the
+    first token, not quantized) and its gradient enters at the last layer's output: logits, the term, the total
+    loss and every gradient of the module against the oracle; unbinding gives the plain loss of Eq. 3 back."""
+    wl, kw = CASES[case]
+    p = Problem(wl, **kw)
+    try:
+        rng = np.random.default_rng(7)
+        H, C_ = wl.hidden, 3
+        # float32 storage: a strong head (its gradient dominates) checked tightly, which pins the term's arithmetic;
+        # bf16 storage: a head of ordinary scale and 3e-2 for the scalar step-size gradients (tensors stay at 2e-2): a
+        # gradient concentrated on `batch` rows carries the bf16 rounding of the backward pass into those heavily
+        # cancelling sums with little averaging
+        strong = wl.act_dtype == "f32"
+        gain = 2.0 if strong else 1.0
+        tol = 2e-3 if strong else GRAD_TOL
+        head = dict(Wp=rng.normal(0, gain / np.sqrt(H), (H, H)).astype(np.float32), bp=rng.normal(0, 0.1, H).astype(np.float32),
+                    Wc=rng.normal(0, 2.0 * gain / np.sqrt(H), (C_, H)).astype(np.float32), bc=rng.normal(0, 0.1, C_).astype(np.float32))
+        plain = p.run_gpu()
+        p.m.bind_head(head)
+        g = p.run_gpu()
+        lz = float(p.m.logit_loss[0])
+        logits = p.m.logits[:, : wl.batch].cpu().numpy()
+        r = O.forward_loss_backward(p.desc, p.teacher, p.student, p.oracle_steps(), p.x, p.x, p.vl, head=head)
+        assert r["logit_loss"] > (0.05 if strong else 0.005) * r["loss"]   # the term is not a rounding-level extra
+        assert np.allclose(logits[1], r["logits_teacher"], rtol=2e-2, atol=2e-3) and np.allclose(logits[0], r["logits_student"], rtol=2e-2, atol=2e-3)
+        assert abs(lz - r["logit_loss"]) / r["logit_loss"] < 2 * tol, (lz, r["logit_loss"])
+        assert abs(g["loss"] - r["loss"]) / r["loss"] < tol
+        assert abs((g["loss"] - plain["loss"]) - lz) <= 1e-5 * g["loss"]
+        worst = compare_grads(g["grads"], r["grads"], tol, check_offset=kw.get("step_shrink", 1.0) < 1.0,
+                              scalar_tol=None if strong else 3e-2)
+        print(case, "logit term", lz, r["logit_loss"], "worst grad", worst)
+        assert rel(g["grads"][0]["W1"], plain["grads"][0]["W1"]) > 1e-3   # it reaches the layers below
+        p.m.bind_head(None)
+        again = p.run_gpu()
+        assert again["loss"] == plain["loss"]
+        for a, b in zip(again["grads"], plain["grads"]):
+            for k in O.PARAMS:
+                assert np.array_equal(a[k], b[k]), k
+    finally:
+        p.close()
+
+
 REM_MATRICES = {"Wqkv": (B.WQKV, 0), "Wo": (B.WO, 1), "W1": (B.W1, 2), "W2": (B.W2, 3)}
 
 
