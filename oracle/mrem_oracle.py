@@ -605,6 +605,86 @@ def recon_step(desc, teacher, student, steps, state, x_t, x_s, valid_len=None, l
     return r
 
 
+# ----------------------------------------------------------------------------- embedding layers of the first module (Sec. 4.1)
+
+EMBED_PARAMS = ("word", "pos", "type", "ln_g", "ln_b")
+
+
+def embed_forward(desc, tables, ids, type_ids, word_step=None, e_bits=0):
+    """BERT embedding layers: LayerNorm(word[ids] + pos[0..S) + type[type_ids]) -> [B, S, H].
+    Student side (`e_bits` > 0): the word-embedding table is quantized by Eq. 1 with one learnable step per
+    row (symmetric uniform, Sec. 3.1); position / token-type tables and the LayerNorm are not.  The sum
+    before the LayerNorm and the output are rounded as stored.  Returns (output, cache)."""
+    st = lambda t: store(t, desc.act_dtype)
+    ids = np.asarray(ids)
+    B, S = ids.shape
+    word = np.asarray(tables["word"], np.float64)
+    c = dict(ids=ids, type_ids=np.asarray(type_ids), B=B, S=S)
+    if e_bits:
+        s_rows = np.asarray(word_step, np.float32).reshape(-1, 1)
+        q, scale, z = quantize_weight(tables["word"], s_rows, e_bits, 0, desc.act_dtype)
+        c.update(q=q, z=z)
+        rows = (scale * q)[ids]
+    else:
+        rows = word[ids]
+    y = st(rows + np.asarray(tables["pos"], np.float64)[None, :S, :] + np.asarray(tables["type"], np.float64)[c["type_ids"]])
+    out, xn, rstd = layernorm(y, tables["ln_g"], tables["ln_b"], desc.ln_eps)
+    c.update(y=y, xn=xn, rstd=rstd)
+    return st(out), c
+
+
+def embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids):
+    """MSE between the student's and the teacher's embedding output (Sec. 4.1) and its gradients w.r.t. the
+    student's latent word table (straight-through, rows gathered several times add up), its row steps, the
+    position and token-type tables and the LayerNorm parameters."""
+    e_t, _ = embed_forward(desc, teacher, ids, type_ids)
+    e_s, c = embed_forward(desc, student, ids, type_ids, word_step, e_bits)
+    diff = e_s - e_t
+    cc = 1.0 / diff.size if desc.loss_mean else 1.0
+    loss = cc * float((diff * diff).sum())
+    dE = 2.0 * cc * diff
+    dy, g_ln_g, g_ln_b = layernorm_backward(dE, c["xn"], c["rstd"], student["ln_g"])
+    B, S, H = dy.shape
+    g = dict(ln_g=g_ln_g, ln_b=g_ln_b)
+    g["pos"] = np.zeros(np.shape(student["pos"]), np.float64)
+    g["pos"][:S] = dy.sum(0)
+    g["type"] = np.zeros(np.shape(student["type"]), np.float64)
+    np.add.at(g["type"], c["type_ids"].reshape(-1), dy.reshape(-1, H))
+    dwhat = np.zeros(np.shape(student["word"]), np.float64)
+    np.add.at(dwhat, c["ids"].reshape(-1), dy.reshape(-1, H))
+    if e_bits:
+        inside, dwhat_ds = weight_ste(c["z"], c["q"], e_bits, 0)
+        g["word"] = dwhat * inside
+        g["word_step"] = (dwhat * dwhat_ds).sum(-1)
+    else:
+        g["word"], g["word_step"] = dwhat, None
+    return dict(e_t=e_t, e_s=e_s, loss=loss, grads=g, cache=c)
+
+
+def embed_step(desc, teacher, student, word_step, state, e_bits, ids, type_ids, lr=1e-4, beta1=0.9, beta2=0.999,
+               eps=1e-8, weight_decay=0.01):
+    """One optimisation step of the embedding objective: gradients as above, then AdamW on every student
+    table (the three embedding tables decayed like weight matrices, LayerNorm parameters not) and on the word
+    table's row steps (kept >= MIN_STEP).  Updates `student` and `word_step` in place; returns the record."""
+    r = embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids)
+    state["t"] = state.get("t", 0) + 1
+    t = state["t"]
+
+    def upd(key, p, g, wd):
+        p = np.asarray(p, np.float64)
+        m, v = state.get(key, (np.zeros_like(p), np.zeros_like(p)))
+        p2, m, v = adamw_update(p, np.asarray(g, np.float64), m, v, t, lr, beta1, beta2, eps, wd)
+        state[key] = (m, v)
+        return p2
+
+    for k in EMBED_PARAMS:
+        wd = weight_decay if k in ("word", "pos", "type") else 0.0
+        student[k] = upd(k, student[k], r["grads"][k], wd).astype(np.float32)
+    if r["grads"]["word_step"] is not None:
+        word_step[:] = np.maximum(upd("word_step", word_step, r["grads"]["word_step"], 0.0), MIN_STEP).astype(np.float32)
+    return r
+
+
 # ----------------------------------------------------------------------------- output logits of the last module (Sec. 4.1)
 
 def head_logits(head, f_last):

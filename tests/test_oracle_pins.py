@@ -618,3 +618,63 @@ def test_module_with_head_adds_the_logit_term_at_the_last_layer_only():
             assert np.allclose(r["grads"][l][k], tparams[l][k].grad.numpy(), rtol=1e-6, atol=1e-12), (l, k)
         assert np.allclose(r["grads"][l]["a"], [t.grad.item() if t.grad is not None else 0.0 for t in tsteps[l]["a"]], rtol=1e-6, atol=1e-12)
     assert not np.allclose(r["grads"][0]["W1"], base["grads"][0]["W1"], rtol=1e-6, atol=0)   # the term reaches the layers below
+
+
+# ----------------------------------------------------------------------------- embedding layers of the first module
+
+def _embed_case(e_bits=4, V=40, H=16, P=12, B_=3, S_=7, seed=4, shrink=0.7):
+    rng = np.random.default_rng(seed)
+    teacher = dict(word=rng.normal(0, 0.05, (V, H)), pos=rng.normal(0, 0.02, (P, H)), type=rng.normal(0, 0.02, (2, H)),
+                   ln_g=1 + rng.normal(0, 0.1, H), ln_b=rng.normal(0, 0.05, H))
+    student = {k: (v + rng.normal(0, 0.004, v.shape)).astype(np.float32) for k, v in teacher.items()}
+    ids = rng.integers(0, V, (B_, S_))
+    ids[0, :3] = 5                                                  # one row gathered several times
+    ids[2, 1] = 5
+    tt = (np.arange(S_)[None, :] >= np.array([3, 7, 4])[:, None]).astype(np.int64)
+    step = (shrink * np.abs(student["word"]).max(1) / O.sym_qmax(e_bits)).astype(np.float32)
+    return teacher, student, step, ids, tt
+
+
+@pytest.mark.parametrize("e_bits,loss_mean", [(4, True), (2, True), (8, False)])
+def test_embedding_objective_matches_torch_embedding_layers_and_autograd(e_bits, loss_mean):
+    """Gather, sum of the three embeddings, LayerNorm as library layers over the detach form of the quantized
+    table; the scatter of repeated rows, the row-step gradients and the position / type / LayerNorm gradients
+    from library autograd."""
+    teacher, student, step, ids, tt = _embed_case(e_bits)
+    desc = O.ModuleDesc(1, 16, 2, 32, loss_mean=loss_mean, act_dtype="f64")
+    r = O.embed_loss_backward(desc, teacher, student, step, e_bits, ids, tt)
+    F_ = torch.nn.functional
+    tp = {k: torch.tensor(np.asarray(v, np.float64), requires_grad=True) for k, v in student.items()}
+    ts = torch.tensor(step.astype(np.float64), requires_grad=True)
+    tid, ttt = torch.tensor(ids), torch.tensor(tt)
+    S_ = ids.shape[1]
+
+    def emb(p, table):
+        y = F_.embedding(tid, table) + p["pos"][:S_][None] + F_.embedding(ttt, p["type"])
+        return F_.layer_norm(y, (16,), p["ln_g"], p["ln_b"], desc.ln_eps)
+
+    e_s = emb(tp, R.q_weight(tp["word"], ts, e_bits, 0))
+    tt_ = {k: torch.tensor(np.asarray(v, np.float64)) for k, v in teacher.items()}
+    e_t = emb(tt_, tt_["word"])
+    loss = ((e_s - e_t) ** 2).mean() if loss_mean else ((e_s - e_t) ** 2).sum()
+    loss.backward()
+    assert np.allclose(r["e_t"], e_t.numpy(), rtol=1e-10) and np.allclose(r["e_s"], e_s.detach().numpy(), rtol=1e-10)
+    assert np.isclose(r["loss"], loss.item(), rtol=1e-10)
+    for k in O.EMBED_PARAMS:
+        assert np.allclose(r["grads"][k], tp[k].grad.numpy(), rtol=1e-7, atol=1e-14), k
+    assert np.allclose(r["grads"]["word_step"], ts.grad.numpy(), rtol=1e-7, atol=1e-14)
+    used = np.zeros(40, bool)
+    used[ids.reshape(-1)] = True
+    assert not np.any(r["grads"]["word"][~used]) and np.any(r["grads"]["word"][5])
+
+
+def test_embedding_bypass_is_exact_and_step_reduces_the_loss():
+    teacher, student, step, ids, tt = _embed_case(4)
+    desc = O.ModuleDesc(1, 16, 2, 32, act_dtype="f64")
+    same = {k: np.asarray(v, np.float64) for k, v in teacher.items()}
+    assert O.embed_loss_backward(desc, teacher, same, step, 0, ids, tt)["loss"] == 0.0
+    state = {}
+    first = O.embed_step(desc, teacher, student, step, state, 4, ids, tt, lr=2e-4)["loss"]
+    for _ in range(40):
+        r = O.embed_step(desc, teacher, student, step, state, 4, ids, tt, lr=2e-4)
+    assert r["loss"] < 0.8 * first
