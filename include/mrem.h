@@ -270,6 +270,57 @@ int32_t mrem_gemm(int32_t dtype, const void* d_a, int32_t a_mn, int64_t lda, int
                   float alpha, float* d_out, int64_t ldc, int64_t c_batch_stride, int32_t block_n, int32_t* d_status,
                   void* cuda_stream);
 
+/* ---- the first module's embedding layers (Sec. 4.1) ---------------------------------------- */
+
+/* Sec. 4.1: the embedding layers belong to the first module and the MSE of the Transformer embedding is
+ * minimised beside the layer losses; Sec. 3.1: embeddings are quantized symmetrically like weights (the
+ * "E" of the paper's W-E-A bit settings is the word-embedding width).  One call = one step of
+ *     min  c * || e_hat - e ||^2,
+ *     e     = LayerNorm(word[ids] + pos[0..seq) + type[type_ids])            (teacher tables)
+ *     e_hat = LayerNorm(Q(word)[ids] + pos + type)                           (student tables),
+ * Q = Eq. 1 with e_bits on the student's latent word table, one learnable step per row; position and
+ * token-type tables and the LayerNorm are not quantized.  c = 1 / (batch * seq * hidden) with loss_mean.
+ * Straight-through backward (a row gathered by several tokens gets the sum of their gradients, added in
+ * token order); AdamW on word (with its row steps, kept >= 1e-8; the table is re-quantized in the same
+ * pass), pos, type (decayed like weight matrices) and the LayerNorm parameters (not decayed).
+ * Stateless: every tensor is the caller's; nothing is allocated. */
+typedef struct {
+  uint32_t struct_size;        /* sizeof(mrem_embed_desc) */
+  int32_t vocab, hidden, max_pos, n_types;   /* hidden a multiple of 16 */
+  int32_t e_bits;              /* 2, 4 or 8 */
+  int32_t act_dtype;           /* mrem_dtype of e, e_hat */
+  int32_t loss_mean;
+  float ln_eps;
+} mrem_embed_desc;
+
+typedef struct {               /* device pointers, float32, 16-byte aligned */
+  const float *t_word, *t_pos, *t_type, *t_ln_g, *t_ln_b;   /* teacher: [vocab,H] [max_pos,H] [n_types,H] [H] [H] */
+  float *word, *pos, *type, *ln_g, *ln_b;                   /* student (latent), same shapes, updated */
+  float* word_step;                                         /* [vocab], updated */
+  float *g_word, *g_pos, *g_type, *g_ln_g, *g_ln_b, *g_word_step;   /* gradients, written by every call */
+  float *m_word, *v_word, *m_pos, *v_pos, *m_type, *v_type, *m_ln_g, *v_ln_g, *m_ln_b, *v_ln_b,
+        *m_word_step, *v_word_step;                         /* AdamW moments (zero before the first step); may be NULL when optim is NULL */
+  int32_t* d_step_counter;                                  /* int32 [1], zero before the first step: AdamW's t when optim->step == 0 */
+} mrem_embed_tensors;
+
+int32_t mrem_embed_workspace_bytes(const mrem_embed_desc* desc, int32_t max_tokens, size_t* out_bytes);
+/*   d_ids, d_type_ids  int32 [batch, seq] (d_type_ids NULL: all 0); an index outside its table is clamped and
+ *                      reported in the status word
+ *   requantize         non-zero on the first call and whenever the caller changed word or word_step: the
+ *                      codes of the table (held in the workspace) are rebuilt first; updates keep them current
+ *   d_e_teacher, d_e_student  [batch, seq, hidden] act_dtype, written (16-byte aligned)
+ *   optim              NULL: no update; g_word then holds the MASKED gradient of the latent table and g_word_step
+ *                      the row-step gradients (with an update g_word is the unmasked sum, the mask being applied
+ *                      inside the fused update, and g_word_step is not written)
+ *   d_loss             float32 [1]: the loss before the update
+ *   d_status           int32 [1], zero it once: 0 ok, 4 non-finite loss, 5 index out of range (sticky)
+ * batch * seq <= 24576, seq <= max_pos; workspace 256-byte aligned and at least mrem_embed_workspace_bytes(desc,
+ * batch * seq).  Asynchronous on cuda_stream. */
+int32_t mrem_embed_step(const mrem_embed_desc* desc, const mrem_embed_tensors* tensors, void* workspace,
+                        size_t workspace_bytes, const int32_t* d_ids, const int32_t* d_type_ids, int32_t batch,
+                        int32_t seq, int32_t requantize, void* d_e_teacher, void* d_e_student,
+                        const mrem_optim* optim, float* d_loss, int32_t* d_status, void* cuda_stream);
+
 /* ---- the last module's output logits (Sec. 4.1) -------------------------------------------- */
 
 /* Sec. 4.1: "besides the grouped Transformer layers" the MSE of the output logits is minimised; the

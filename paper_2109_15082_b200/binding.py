@@ -33,7 +33,7 @@ EXPORTS = (
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
-    "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head",
+    "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head", "mrem_embed_workspace_bytes", "mrem_embed_step",
 )
 
 
@@ -188,6 +188,39 @@ def mrem_step(ctx, optim):
 
 def mrem_backward_and_step(ctx, optim):
     _check(lib().mrem_backward_and_step(ctx, C.byref(optim)), "mrem_backward_and_step", ctx)
+
+
+class EmbedDesc(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("vocab", C.c_int32), ("hidden", C.c_int32), ("max_pos", C.c_int32),
+                ("n_types", C.c_int32), ("e_bits", C.c_int32), ("act_dtype", C.c_int32), ("loss_mean", C.c_int32),
+                ("ln_eps", C.c_float)]
+
+
+EMBED_TENSOR_FIELDS = ("t_word", "t_pos", "t_type", "t_ln_g", "t_ln_b", "word", "pos", "type", "ln_g", "ln_b", "word_step",
+                       "g_word", "g_pos", "g_type", "g_ln_g", "g_ln_b", "g_word_step", "m_word", "v_word", "m_pos", "v_pos",
+                       "m_type", "v_type", "m_ln_g", "v_ln_g", "m_ln_b", "v_ln_b", "m_word_step", "v_word_step", "d_step_counter")
+
+
+class EmbedTensors(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in EMBED_TENSOR_FIELDS]
+
+
+def make_embed_desc(vocab, hidden, max_pos, n_types, e_bits, act_dtype=BF16, loss_mean=1, ln_eps=1e-12):
+    return EmbedDesc(C.sizeof(EmbedDesc), vocab, hidden, max_pos, n_types, e_bits, act_dtype, loss_mean, ln_eps)
+
+
+def mrem_embed_workspace_bytes(desc, max_tokens) -> int:
+    out = C.c_size_t(0)
+    _check(lib().mrem_embed_workspace_bytes(C.byref(desc), int(max_tokens), C.byref(out)), "mrem_embed_workspace_bytes")
+    return out.value
+
+
+def mrem_embed_step(desc, tensors, workspace, workspace_bytes, d_ids, d_type_ids, batch, seq, requantize, d_e_teacher,
+                    d_e_student, optim, d_loss, d_status, stream):
+    _check(lib().mrem_embed_step(C.byref(desc), C.byref(tensors), _p(workspace), C.c_size_t(workspace_bytes), _p(d_ids),
+                                 _p(d_type_ids), int(batch), int(seq), int(requantize), _p(d_e_teacher), _p(d_e_student),
+                                 C.byref(optim) if optim is not None else None, _p(d_loss), _p(d_status), _p(stream)),
+           "mrem_embed_step")
 
 
 def mrem_bind_head(ctx, d_wp, d_bp, d_wc, d_bc, n_classes, d_logit_loss=None, d_logits=None):

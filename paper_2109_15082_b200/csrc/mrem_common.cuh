@@ -15,6 +15,7 @@ enum DeviceStatus : int {
   DEV_TIMEOUT_MMA = 2,      // a wait on a tensor-core commit ran out
   DEV_TIMEOUT_EPI = 3,      // a wait on an accumulator hand-over ran out
   DEV_NONFINITE = 4,        // the loss kernel met a non-finite value
+  DEV_BAD_INDEX = 5,        // an embedding index outside its table (clamped)
 };
 
 // ---------------------------------------------------------------- programmatic dependent launch
