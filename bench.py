@@ -168,6 +168,63 @@ def build_problem(wl, rank, torch, calib_n):
     return m, calib, lens
 
 
+def time_extras(m, wl, xbuf, lenbuf, stream, torch, B, pk, reps=10):
+    """Device times (CUDA events, after 3 warm-up calls) of the entry points beside the module step, on the workload's
+    shapes: one step of Eq. 2 per weight matrix of a layer on batch x seq rows, the output-logit term inside
+    mrem_recon_loss, and one embedding step (BERT-large tables when the workload is BERT-large)."""
+    from paper_2109_15082_b200.embedding import EmbeddingStep
+
+    def timed(fn, n=reps):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    out = {}
+    rows = wl.batch * wl.seq
+    opt = B.make_optim(lr=wl.lr, step=0, decay_total_steps=100000)
+    x2 = xbuf.reshape(rows, wl.hidden)
+    g_in = torch.randn(rows, wl.ffn, device=m.device, dtype=torch.float32).abs().to(m.tdtype)     # FFN2 input: non-negative like a GELU output
+    rem = {}
+    for name, pid, a, n_out, n_in in (("Wqkv", B.WQKV, x2, 3 * wl.hidden, wl.hidden), ("Wo", B.WO, x2, wl.hidden, wl.hidden),
+                                      ("W1", B.W1, x2, wl.ffn, wl.hidden), ("W2", B.W2, g_in, wl.hidden, wl.ffn)):
+        ms = timed(lambda: m.rem_step(0, pid, a, opt))
+        flop = 4 * 2.0 * rows * n_out * n_in                   # teacher product, integer product, weight gradient, input gradient
+        rem[name] = {"ms_per_step": ms, "tflops": flop / (ms * 1e-3) / 1e12}
+    out["rem_step"] = {"rows": rows, "per_matrix": rem,
+                       "note": "Eq. 2 on one product: two forward products (bf16, int8), loss, two backward products, fused update"}
+    # output-logit term: mrem_recon_loss with and without a bound head (3 classes)
+    m.quantize_weights()
+    m.forward_teacher(xbuf, lenbuf, wl.batch, wl.seq)
+    m.forward_student(xbuf, lenbuf, wl.batch, wl.seq)
+    plain = timed(lambda: m.recon_loss())
+    rng = np.random.default_rng(0)
+    H = wl.hidden
+    m.bind_head(dict(Wp=rng.normal(0, 1 / np.sqrt(H), (H, H)), bp=np.zeros(H), Wc=rng.normal(0, 1 / np.sqrt(H), (3, H)), bc=np.zeros(3)))
+    with_head = timed(lambda: m.recon_loss())
+    m.bind_head(None)
+    out["logit_term"] = {"recon_loss_ms": plain, "recon_loss_with_head_ms": with_head, "classes": 3}
+    # embedding step
+    V, P = (30522, 512) if wl.hidden >= 768 else (1000, 64)
+    teacher = dict(word=rng.normal(0, 0.05, (V, H)), pos=rng.normal(0, 0.02, (max(P, wl.seq), H)), type=rng.normal(0, 0.02, (2, H)),
+                   ln_g=np.ones(H), ln_b=np.zeros(H))
+    emb = EmbeddingStep(teacher, 4, rows, wl.act_dtype, stream=stream)
+    emb.set_student(None, np.abs(teacher["word"]).max(1) / 7)
+    ids = torch.from_numpy((rng.zipf(1.2, (wl.batch, wl.seq)) % V).astype(np.int32)).to(m.device)
+    ms = timed(lambda: emb.step(ids, None, opt))
+    table_bytes = V * H * (4 + 16 + 12 + 1)                     # gradient cleared; w, g, m, v read; w, m, v, code written
+    out["embed_step"] = {"vocab": V, "tokens": rows, "e_bits": 4, "ms_per_step": ms, "table_gbs": table_bytes / (ms * 1e-3) / 1e9,
+                         "hbm_peak_gbs": pk["hbm_gbs"], "status": int(emb.status[0]),
+                         "note": "whole step; table_gbs counts only the dense pass over the word table (33 B per entry)"}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -178,6 +235,8 @@ def main():
     ap.add_argument("--calib", type=int, default=0, help="calibration sequences (0: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--extras", action="store_true", help="also time the per-product step (Eq. 2), the output-logit term and the "
+                    "embedding step of the first module, and add them to the JSON line as \"extras\"")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches (no programmatic dependent launch)")
     args = ap.parse_args()
 
@@ -295,6 +354,7 @@ def main():
             e2e = {"value": D.whole_job_rate(tokens, ke, world, dt_e2e * 1e3), "unit": UNIT,
                    "h2d_bytes_per_step": row_bytes * wl.batch + len_row_bytes, "d2h_bytes_per_step": 4,
                    "steps": ke}
+        extras = time_extras(m, wl, xbuf, lenbuf, side, torch, B, pk=peaks()) if args.extras and rank == 0 else None
         m.close()
 
     if rank != 0:
@@ -348,6 +408,8 @@ def main():
                              "us_per_launch": 1e3 * e["ms"] / max(e["launches"], 1),
                              "tflops": e["work"] / (e["ms"] * 1e-3) / 1e12} for e in sorted(shapes, key=lambda e: -e["ms"])],
             "loss_last": loss_last, "device_status": status}
+    if extras:
+        line["extras"] = extras
     if world == 1 and not args.no_cpu_baseline:
         val, threads, sample, sec = oracle_sample(wl)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,

@@ -470,11 +470,18 @@ def student_backward(desc, params, caches, dF_list):
     """Backward through the module.  The loss gradient of Eq. 3 enters at every layer
     output; the gradient stops at the module input (it stays local to the module,
     Sec. 4.2).  Returns the list of per-layer gradient dicts."""
+    return student_backward_with_input_grad(desc, params, caches, dF_list)[0]
+
+
+def student_backward_with_input_grad(desc, params, caches, dF_list):
+    """The same, returning also the gradient with respect to the module's input (after the straight-through pass
+    of the first layer's input quantizer and its skip connection): the model's first module hands it to the
+    embedding layers, which belong to that module (Sec. 4.1)."""
     grads = [None] * len(params)
     carry = 0.0
     for l in reversed(range(len(params))):
         carry, grads[l] = student_layer_backward(desc, params[l], caches[l], dF_list[l] + carry)
-    return grads
+    return grads, carry
 
 
 # ----------------------------------------------------------------------------- update (Alg. 2, Update(.) = AdamW)
@@ -571,7 +578,7 @@ def forward_loss_backward(desc, teacher, student, steps, x_t, x_s, valid_len=Non
         dF[-1] = dF[-1] + dFz
         out.update(logit_loss=lz, logits_student=z_s, logits_teacher=z_t)
     out["loss"] = total
-    out["grads"] = student_backward(desc, student, caches, dF)
+    out["grads"], out["d_input"] = student_backward_with_input_grad(desc, student, caches, dF)
     return out
 
 
@@ -633,16 +640,20 @@ def embed_forward(desc, tables, ids, type_ids, word_step=None, e_bits=0):
     return st(out), c
 
 
-def embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids):
+def embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids, d_extra=None):
     """MSE between the student's and the teacher's embedding output (Sec. 4.1) and its gradients w.r.t. the
     student's latent word table (straight-through, rows gathered several times add up), its row steps, the
-    position and token-type tables and the LayerNorm parameters."""
+    position and token-type tables and the LayerNorm parameters.  `d_extra` [B, S, H]: a gradient that arrives
+    at the student's embedding output from the layers it feeds (the first module's input gradient), added to
+    the gradient of the MSE."""
     e_t, _ = embed_forward(desc, teacher, ids, type_ids)
     e_s, c = embed_forward(desc, student, ids, type_ids, word_step, e_bits)
     diff = e_s - e_t
     cc = 1.0 / diff.size if desc.loss_mean else 1.0
     loss = cc * float((diff * diff).sum())
     dE = 2.0 * cc * diff
+    if d_extra is not None:
+        dE = store(dE, desc.act_dtype) + np.asarray(d_extra, np.float64)
     dy, g_ln_g, g_ln_b = layernorm_backward(dE, c["xn"], c["rstd"], student["ln_g"])
     B, S, H = dy.shape
     g = dict(ln_g=g_ln_g, ln_b=g_ln_b)
@@ -662,11 +673,11 @@ def embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids
 
 
 def embed_step(desc, teacher, student, word_step, state, e_bits, ids, type_ids, lr=1e-4, beta1=0.9, beta2=0.999,
-               eps=1e-8, weight_decay=0.01):
+               eps=1e-8, weight_decay=0.01, d_extra=None):
     """One optimisation step of the embedding objective: gradients as above, then AdamW on every student
     table (the three embedding tables decayed like weight matrices, LayerNorm parameters not) and on the word
     table's row steps (kept >= MIN_STEP).  Updates `student` and `word_step` in place; returns the record."""
-    r = embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids)
+    r = embed_loss_backward(desc, teacher, student, word_step, e_bits, ids, type_ids, d_extra)
     state["t"] = state.get("t", 0) + 1
     t = state["t"]
 

@@ -678,3 +678,41 @@ def test_embedding_bypass_is_exact_and_step_reduces_the_loss():
     for _ in range(40):
         r = O.embed_step(desc, teacher, student, step, state, 4, ids, tt, lr=2e-4)
     assert r["loss"] < 0.8 * first
+
+
+def test_embedding_extra_gradient_and_module_input_gradient_match_autograd():
+    """First module of the model: the layers' gradient with respect to their input (the student's embedding output)
+    is added to the embedding MSE's own gradient.  (i) The module's input gradient equals autograd's d loss / d x of
+    the torch model of the module; (ii) an extra gradient g at the embedding output acts like the extra loss
+    term <g, e_hat>."""
+    wl = synth.shrink(synth.workloads()["tiny"], n_layers=1, hidden=16, n_heads=2, ffn=32, seq=7, batch=3)
+    desc = O.ModuleDesc(1, 16, 2, 32, 4, 8, act_dtype="f64")
+    params = synth.teacher_params(wl, 0, bias_std=0.02)
+    student = [{k: (v + synth.normal(1, f"m{l}{k}", v.shape, 0.003)).astype(np.float32) for k, v in p.items()} for l, p in enumerate(params)]
+    x = synth.hidden_states(wl, wl.batch, 0).astype(np.float64)
+    ws = O.init_weight_steps(desc, student, 0)
+    a, off = O.init_act_steps(desc, student, x, None)
+    steps = O.make_steps(ws, (a * 0.8).astype(np.float32), off)
+    r = O.forward_loss_backward(desc, params, student, steps, x, x)
+    cfg = dict(n_heads=2, a_bits=8, w_bits=4, w_grid=0, asym_p=True, asym_g=True, ln_eps=desc.ln_eps)
+    tx = torch.tensor(x, requires_grad=True)
+    tparams = [{k: torch.tensor(v.astype(np.float64)) for k, v in p.items()} for p in student]
+    tsteps = [dict(w={k: torch.tensor(st["w"][k].astype(np.float64)) for k in O.WEIGHTS},
+                   a=[torch.tensor(float(v), dtype=torch.float64) for v in st["a"]],
+                   a_off=[torch.tensor(float(v), dtype=torch.float64) for v in st["a_off"]]) for st in steps]
+    outs = R.module(tx, tparams, tsteps, cfg, None)
+    sum(((o - torch.tensor(ft)) ** 2).mean() for o, ft in zip(outs, r["f_t"])).backward()
+    assert np.allclose(r["d_input"], tx.grad.numpy(), rtol=1e-7, atol=1e-13) and np.any(r["d_input"])
+    # (ii)
+    teacher, est, step, ids, tt = _embed_case(4, H=16, B_=3, S_=7)
+    extra = r["d_input"] * 50
+    re = O.embed_loss_backward(desc, teacher, est, step, 4, ids, tt, d_extra=extra)
+    F_ = torch.nn.functional
+    tp = {k: torch.tensor(np.asarray(v, np.float64), requires_grad=True) for k, v in est.items()}
+    ts = torch.tensor(step.astype(np.float64), requires_grad=True)
+    y = F_.embedding(torch.tensor(ids), R.q_weight(tp["word"], ts, 4, 0)) + tp["pos"][:7][None] + F_.embedding(torch.tensor(tt), tp["type"])
+    e_s = F_.layer_norm(y, (16,), tp["ln_g"], tp["ln_b"], desc.ln_eps)
+    (((e_s - torch.tensor(re["e_t"])) ** 2).mean() + (torch.tensor(extra) * e_s).sum()).backward()
+    for k in O.EMBED_PARAMS:
+        assert np.allclose(re["grads"][k], tp[k].grad.numpy(), rtol=1e-7, atol=1e-13), k
+    assert np.allclose(re["grads"]["word_step"], ts.grad.numpy(), rtol=1e-7, atol=1e-13)
