@@ -169,6 +169,12 @@ int32_t mrem_module_backward(mrem_ctx* ctx);
 /* Borrowed pointer to a gradient (float32, same shape as the parameter / step tensor).  Asking for a weight
  * matrix or a weight step applies the weight quantizers' straight-through masks on the spot. */
 int32_t mrem_get_grad(mrem_ctx* ctx, int32_t layer, int32_t id, const float** d_grad);
+/* Borrowed pointer to d loss / d (student module input), [batch, seq, hidden] in the storage type, after the
+ * straight-through pass of the first layer's input quantizer and its skip connection.  The gradient stays
+ * local to a module (Sec. 4.2) except in the model's first module, whose embedding layers receive it
+ * (mrem_embed_step).  Valid from a backward pass (mrem_module_backward or mrem_backward_and_step) until the next
+ * forward pass on this context (MREM_ERR_ORDER otherwise). */
+int32_t mrem_get_input_grad(mrem_ctx* ctx, const void** d_grad);
 /* AdamW on everything in trainable_mask, steps clamped to >= 1e-8.  With per-row weight steps the update of
  * each matrix also re-quantizes it (Eq. 1 with the new weights and steps), so the next
  * mrem_quantize_weights has nothing left to do. */
@@ -309,17 +315,21 @@ int32_t mrem_embed_workspace_bytes(const mrem_embed_desc* desc, int32_t max_toke
  *   requantize         non-zero on the first call and whenever the caller changed word or word_step: the
  *                      codes of the table (held in the workspace) are rebuilt first; updates keep them current
  *   d_e_teacher, d_e_student  [batch, seq, hidden] act_dtype, written (16-byte aligned)
+ *   d_extra_grad       NULL or [batch, seq, hidden] act_dtype: a gradient with respect to the student's embedding
+ *                      output that arrives from the layers it feeds (mrem_get_input_grad of the first module's
+ *                      context after its backward pass); added to the gradient of the MSE
  *   optim              NULL: no update; g_word then holds the MASKED gradient of the latent table and g_word_step
  *                      the row-step gradients (with an update g_word is the unmasked sum, the mask being applied
  *                      inside the fused update, and g_word_step is not written)
  *   d_loss             float32 [1]: the loss before the update
  *   d_status           int32 [1], zero it once: 0 ok, 4 non-finite loss, 5 index out of range (sticky)
- * batch * seq <= 24576, seq <= max_pos; workspace 256-byte aligned and at least mrem_embed_workspace_bytes(desc,
+ * seq <= max_pos; workspace 256-byte aligned and at least mrem_embed_workspace_bytes(desc,
  * batch * seq).  Asynchronous on cuda_stream. */
 int32_t mrem_embed_step(const mrem_embed_desc* desc, const mrem_embed_tensors* tensors, void* workspace,
                         size_t workspace_bytes, const int32_t* d_ids, const int32_t* d_type_ids, int32_t batch,
                         int32_t seq, int32_t requantize, void* d_e_teacher, void* d_e_student,
-                        const mrem_optim* optim, float* d_loss, int32_t* d_status, void* cuda_stream);
+                        const void* d_extra_grad, const mrem_optim* optim, float* d_loss, int32_t* d_status,
+                        void* cuda_stream);
 
 /* ---- the last module's output logits (Sec. 4.1) -------------------------------------------- */
 

@@ -33,7 +33,7 @@ EXPORTS = (
     "mrem_quantize_weight", "mrem_gemm_i8", "mrem_gemm", "mrem_graph_num_kernels", "mrem_trace_enable",
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
-    "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head", "mrem_embed_workspace_bytes", "mrem_embed_step",
+    "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head", "mrem_embed_workspace_bytes", "mrem_embed_step", "mrem_get_input_grad",
 )
 
 
@@ -215,11 +215,17 @@ def mrem_embed_workspace_bytes(desc, max_tokens) -> int:
     return out.value
 
 
+def mrem_get_input_grad(ctx) -> int:
+    out = C.c_void_p(0)
+    _check(lib().mrem_get_input_grad(ctx, C.byref(out)), "mrem_get_input_grad", ctx)
+    return out.value
+
+
 def mrem_embed_step(desc, tensors, workspace, workspace_bytes, d_ids, d_type_ids, batch, seq, requantize, d_e_teacher,
-                    d_e_student, optim, d_loss, d_status, stream):
+                    d_e_student, d_extra_grad, optim, d_loss, d_status, stream):
     _check(lib().mrem_embed_step(C.byref(desc), C.byref(tensors), _p(workspace), C.c_size_t(workspace_bytes), _p(d_ids),
                                  _p(d_type_ids), int(batch), int(seq), int(requantize), _p(d_e_teacher), _p(d_e_student),
-                                 C.byref(optim) if optim is not None else None, _p(d_loss), _p(d_status), _p(stream)),
+                                 _p(d_extra_grad), C.byref(optim) if optim is not None else None, _p(d_loss), _p(d_status), _p(stream)),
            "mrem_embed_step")
 
 

@@ -45,52 +45,83 @@ __global__ void __launch_bounds__(128) embed_sum_kernel(const float* __restrict_
   }
 }
 
-// g_word[id, :] = sum over the tokens t with ids[t] == id of dy[t, :], in token order.  Block t does the
-// sum for its id when t is the first token with that id, and returns otherwise; rows no token gathered keep
-// the zeros the caller put there.
-template <typename T>
-__global__ void __launch_bounds__(128) embed_scatter_kernel(const T* __restrict__ dy, const int* __restrict__ ids, int M,
-                                                            int H, int vocab, float* __restrict__ g_word) {
+// Occurrence lists of the batch's ids: first[t] = 1 when no earlier token has the id of token t, next[t] = the
+// next later token with that id (-1: none).  One thread per token.
+__global__ void __launch_bounds__(256) embed_links_kernel(const int* __restrict__ ids, int M, int vocab, int* __restrict__ first,
+                                                          int* __restrict__ next) {
   pdl_trigger();
   pdl_wait();
-  extern __shared__ int sh_ids[];
-  for (int i = threadIdx.x; i < M; i += blockDim.x) sh_ids[i] = min(max(ids[i], 0), vocab - 1);
-  __syncthreads();
-  const int t0 = blockIdx.x, id = sh_ids[t0];
-  for (int i = 0; i < t0; ++i)
-    if (sh_ids[i] == id) return;                                    // an earlier token owns this row (block-uniform)
-  for (int c0 = threadIdx.x; c0 < H; c0 += blockDim.x) {
-    float acc = 0.f;
-    for (int i = t0; i < M; ++i)
-      if (sh_ids[i] == id) acc += to_f<T>(dy[(long long)i * H + c0]);
-    g_word[(long long)id * H + c0] = acc;
-  }
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= M) return;
+  const int id = min(max(ids[t], 0), vocab - 1);
+  int nx = -1, fi = 1;
+  for (int i = t + 1; i < M; ++i)
+    if (min(max(ids[i], 0), vocab - 1) == id) { nx = i; break; }
+  for (int i = t - 1; i >= 0; --i)
+    if (min(max(ids[i], 0), vocab - 1) == id) { fi = 0; break; }
+  first[t] = fi;
+  next[t] = nx;
 }
 
-// g_pos[s, c] = sum_b dy[b, s, c];  g_type[k, c] = sum over tokens with type k of dy[t, c] (token order).
+// g_word[id, :] = sum over the tokens t with ids[t] == id of dy[t, :], in token order: the block of the first
+// token with an id walks that id's occurrence list for its 128 columns; rows no token gathered keep the zeros
+// the caller put there.
 template <typename T>
-__global__ void __launch_bounds__(256) embed_pos_type_kernel(const T* __restrict__ dy, const int* __restrict__ type_ids, int B,
-                                                             int S, int H, int max_pos, int n_types,
-                                                             float* __restrict__ g_pos, float* __restrict__ g_type) {
+__global__ void __launch_bounds__(128) embed_scatter_kernel(const T* __restrict__ dy, const int* __restrict__ ids,
+                                                            const int* __restrict__ first, const int* __restrict__ next, int H,
+                                                            int vocab, float* __restrict__ g_word) {
   pdl_trigger();
   pdl_wait();
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  const int t0 = blockIdx.x;
+  if (!first[t0]) return;                                           // block-uniform
+  const int c = blockIdx.y * blockDim.x + threadIdx.x;
   if (c >= H) return;
-  const int row = blockIdx.y;
-  if (row < max_pos) {                                              // one position
-    float acc = 0.f;
-    if (row < S)
-      for (int b = 0; b < B; ++b) acc += to_f<T>(dy[((long long)b * S + row) * H + c]);
-    g_pos[(long long)row * H + c] = acc;
-  } else {                                                          // one token type
-    const int k = row - max_pos;
-    float acc = 0.f;
-    for (long long t = 0; t < (long long)B * S; ++t) {
-      const int tt = type_ids ? min(max(type_ids[t], 0), n_types - 1) : 0;
-      if (tt == k) acc += to_f<T>(dy[t * H + c]);
-    }
-    g_type[(long long)k * H + c] = acc;
+  const int id = min(max(ids[t0], 0), vocab - 1);
+  float acc = 0.f;
+  for (int t = t0; t >= 0; t = next[t]) acc += to_f<T>(dy[(long long)t * H + c]);
+  g_word[(long long)id * H + c] = acc;
+}
+
+// g_pos[s, c] = sum_b dy[b, s, c] (rows of the table beyond seq get zero).
+template <typename T>
+__global__ void __launch_bounds__(256) embed_pos_kernel(const T* __restrict__ dy, int B, int S, int H, float* __restrict__ g_pos) {
+  pdl_trigger();
+  pdl_wait();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x, row = blockIdx.y;
+  if (c >= H) return;
+  float acc = 0.f;
+  if (row < S)
+    for (int b = 0; b < B; ++b) acc += to_f<T>(dy[((long long)b * S + row) * H + c]);
+  g_pos[(long long)row * H + c] = acc;
+}
+
+// Token-type table, two stages with fixed orders: partial[chunk, k, c] = sum over the chunk's tokens of type k (token
+// order), then g_type[k, c] = sum over the chunks in index order.
+constexpr int TYPE_CHUNKS = 64;
+template <typename T>
+__global__ void __launch_bounds__(256) embed_type_partial_kernel(const T* __restrict__ dy, const int* __restrict__ type_ids,
+                                                                 long long M, int H, int n_types, float* __restrict__ partial) {
+  pdl_trigger();
+  pdl_wait();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x, chunk = blockIdx.y, k = blockIdx.z;
+  if (c >= H) return;
+  const long long per = (M + TYPE_CHUNKS - 1) / TYPE_CHUNKS, t0 = chunk * per, t1 = t0 + per < M ? t0 + per : M;
+  float acc = 0.f;
+  for (long long t = t0; t < t1; ++t) {
+    const int tt = type_ids ? min(max(type_ids[t], 0), n_types - 1) : 0;
+    if (tt == k) acc += to_f<T>(dy[t * H + c]);
   }
+  partial[((long long)chunk * n_types + k) * H + c] = acc;
+}
+__global__ void __launch_bounds__(256) embed_type_final_kernel(const float* __restrict__ partial, int H, int n_types,
+                                                               float* __restrict__ g_type) {
+  pdl_trigger();
+  pdl_wait();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x, k = blockIdx.y;
+  if (c >= H) return;
+  float acc = 0.f;
+  for (int chunk = 0; chunk < TYPE_CHUNKS; ++chunk) acc += partial[((long long)chunk * n_types + k) * H + c];
+  g_type[(long long)k * H + c] = acc;
 }
 
 struct Carve {                         // the workspace, cut the same way by the sizing call and by the step
@@ -99,12 +130,13 @@ struct Carve {                         // the workspace, cut the same way by the
   void* take(size_t bytes) { off = (off + 255) & ~size_t(255); void* p = base ? base + off : nullptr; off += bytes; return p; }
 };
 struct EmbedScratch {
-  void *y_t, *y_s, *dE, *dy;
+  void *y_t, *y_s, *dE, *dy, *dsum;
   float *mean, *rstd, *col_scratch, *loss_partial;
   long long col_plane;
   int* col_counters;
   int8_t* codes; int32_t* rowsum; float* scale;
   OptimScalars* optim_sc; AdamEntry* table;
+  int *first, *next; float* type_partial;
   size_t bytes;
 };
 EmbedScratch carve(const mrem_embed_desc& d, long long max_tokens, void* base) {
@@ -112,7 +144,7 @@ EmbedScratch carve(const mrem_embed_desc& d, long long max_tokens, void* base) {
   EmbedScratch s;
   const size_t es = d.act_dtype == MREM_BF16 ? 2 : 4;
   const size_t MH = (size_t)max_tokens * d.hidden;
-  s.y_t = A.take(MH * es); s.y_s = A.take(MH * es); s.dE = A.take(MH * es); s.dy = A.take(MH * es);
+  s.y_t = A.take(MH * es); s.y_s = A.take(MH * es); s.dE = A.take(MH * es); s.dy = A.take(MH * es); s.dsum = A.take(MH * es);
   s.mean = (float*)A.take(4 * max_tokens); s.rstd = (float*)A.take(4 * max_tokens);
   s.col_plane = (long long)COL_CHUNKS * d.hidden;
   s.col_scratch = (float*)A.take(sizeof(float) * 3 * s.col_plane);
@@ -123,6 +155,8 @@ EmbedScratch carve(const mrem_embed_desc& d, long long max_tokens, void* base) {
   s.scale = (float*)A.take(sizeof(float) * d.vocab);
   s.optim_sc = (OptimScalars*)A.take(sizeof(OptimScalars));
   s.table = (AdamEntry*)A.take(sizeof(AdamEntry) * 4);
+  s.first = (int*)A.take(sizeof(int) * max_tokens); s.next = (int*)A.take(sizeof(int) * max_tokens);
+  s.type_partial = (float*)A.take(sizeof(float) * (size_t)TYPE_CHUNKS * d.n_types * d.hidden);
   s.bytes = (A.off + 255) & ~size_t(255);
   return s;
 }
@@ -152,8 +186,8 @@ int32_t mrem_embed_workspace_bytes(const mrem_embed_desc* d, int32_t max_tokens,
 
 int32_t mrem_embed_step(const mrem_embed_desc* d, const mrem_embed_tensors* x, void* workspace, size_t workspace_bytes,
                         const int32_t* d_ids, const int32_t* d_type_ids, int32_t batch, int32_t seq, int32_t requantize,
-                        void* d_e_teacher, void* d_e_student, const mrem_optim* o, float* d_loss, int32_t* d_status,
-                        void* cuda_stream) {
+                        void* d_e_teacher, void* d_e_student, const void* d_extra_grad, const mrem_optim* o, float* d_loss,
+                        int32_t* d_status, void* cuda_stream) {
   int rc = check_desc(d);
   if (rc != MREM_OK) return rc;
   if (!x || !workspace || !d_ids || !d_e_teacher || !d_e_student || !d_loss || !d_status) return MREM_ERR_ARG;
@@ -166,7 +200,6 @@ int32_t mrem_embed_step(const mrem_embed_desc* d, const mrem_embed_tensors* x, v
     return MREM_ERR_ARG;
   const long long M = (long long)batch * seq;
   const int H = d->hidden, V = d->vocab, dt = d->act_dtype == MREM_BF16 ? 1 : 0;
-  if ((size_t)M * sizeof(int) > 96 * 1024) return MREM_ERR_SHAPE;   // the scatter keeps the batch's ids in shared memory
   const EmbedScratch s = carve(*d, M, workspace);
   if (s.bytes > workspace_bytes) return MREM_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(d_e_teacher) & 15) ||
@@ -191,22 +224,23 @@ int32_t mrem_embed_step(const mrem_embed_desc* d, const mrem_embed_tensors* x, v
   launch_loss(d_e_student, d_e_teacher, 1, n, cc, s.dE, s.loss_partial, d_status, dt, st);
   launch_loss_finalize(s.loss_partial, 1, cc, d_loss, nullptr, st);
   // LayerNorm backward and its parameter gradients
-  launch_layernorm_bwd(s.dE, nullptr, s.y_s, s.mean, s.rstd, x->ln_g, M, H, s.dy, nullptr, dt, st);
+  // (with a gradient arriving from the layers the embedding feeds, the LayerNorm sees the sum of the two)
+  if (d_extra_grad && (reinterpret_cast<uintptr_t>(d_extra_grad) & 15)) return MREM_ERR_ALIGN;
+  launch_layernorm_bwd(s.dE, d_extra_grad, s.y_s, s.mean, s.rstd, x->ln_g, M, H, s.dy, d_extra_grad ? s.dsum : nullptr, dt, st);
   if (cudaMemsetAsync(s.col_counters, 0, sizeof(int) * (H / 32 + 2), st) != cudaSuccess) return MREM_ERR_CUDA;
-  launch_col_reduce(s.dE, H, s.y_s, s.mean, s.rstd, nullptr, 0, M, H, x->g_ln_b, x->g_ln_g, nullptr, s.col_scratch, s.col_plane,
+  launch_col_reduce(d_extra_grad ? s.dsum : s.dE, H, s.y_s, s.mean, s.rstd, nullptr, 0, M, H, x->g_ln_b, x->g_ln_g, nullptr, s.col_scratch, s.col_plane,
                     s.col_counters, dt, st);
   // position / token-type tables: sums over the batch; word table: every token's gradient into the row it gathered
   if (cudaMemsetAsync(x->g_word, 0, sizeof(float) * (size_t)V * H, st) != cudaSuccess) return MREM_ERR_CUDA;
-  const size_t ids_smem = sizeof(int) * (size_t)M;
-  if (dt == 1) {
-    if (ids_smem > 48 * 1024) cudaFuncSetAttribute(embed_scatter_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    launch_k(embed_pos_type_kernel<bf16>, dim3((H + 255) / 256, d->max_pos + d->n_types), 256, 0, st, (const bf16*)s.dy, d_type_ids, (int)batch, (int)seq, H, (int)d->max_pos, (int)d->n_types, x->g_pos, x->g_type);
-    launch_k(embed_scatter_kernel<bf16>, (unsigned)M, 128, ids_smem, st, (const bf16*)s.dy, d_ids, (int)M, H, V, x->g_word);
-  } else {
-    if (ids_smem > 48 * 1024) cudaFuncSetAttribute(embed_scatter_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    launch_k(embed_pos_type_kernel<float>, dim3((H + 255) / 256, d->max_pos + d->n_types), 256, 0, st, (const float*)s.dy, d_type_ids, (int)batch, (int)seq, H, (int)d->max_pos, (int)d->n_types, x->g_pos, x->g_type);
-    launch_k(embed_scatter_kernel<float>, (unsigned)M, 128, ids_smem, st, (const float*)s.dy, d_ids, (int)M, H, V, x->g_word);
-  }
+  launch_k(embed_links_kernel, (unsigned)((M + 255) / 256), 256, 0, st, d_ids, (int)M, V, s.first, s.next);
+  const dim3 gcol((H + 255) / 256), gscat((unsigned)M, (H + 127) / 128);
+#define MREM_EMB_BWD(T) do { \
+    launch_k(embed_pos_kernel<T>, dim3(gcol.x, d->max_pos), 256, 0, st, (const T*)s.dy, (int)batch, (int)seq, H, x->g_pos); \
+    launch_k(embed_type_partial_kernel<T>, dim3(gcol.x, TYPE_CHUNKS, d->n_types), 256, 0, st, (const T*)s.dy, d_type_ids, M, H, (int)d->n_types, s.type_partial); \
+    launch_k(embed_scatter_kernel<T>, gscat, 128, 0, st, (const T*)s.dy, d_ids, (const int*)s.first, (const int*)s.next, H, V, x->g_word); } while (0)
+  if (dt == 1) MREM_EMB_BWD(bf16); else MREM_EMB_BWD(float);
+#undef MREM_EMB_BWD
+  launch_k(embed_type_final_kernel, dim3(gcol.x, d->n_types), 256, 0, st, (const float*)s.type_partial, H, (int)d->n_types, x->g_type);
   if (!o) {
     // gradients only: the word table's straight-through mask and its row-step gradients, left in g_word / g_word_step
     launch_ste_weight(x->word, x->word_step, 1, d->e_bits, 0, x->g_word, V, H, x->g_word_step, st);

@@ -92,10 +92,11 @@ void launch_loss_finalize(const float* partial, int n_layers, float c, float* lo
 
 // Output-logit term of the last module: pooler (dense + tanh) and classifier on the first token of both last
 // layer outputs [B, S, H]; adds cc * sum (z_hat - z)^2 to *loss_total (and writes it to *logit_loss when non-null),
-// adds its gradient to dF_last at the first tokens; `part` >= B floats of scratch; `logits` null or [2, B, C]
-// (student, teacher).  Returns 0, -1 when hidden / classes do not fit the kernel's shared memory, -2 on a launch error.
+// adds its gradient to dF_last at the first tokens; `scratch` >= head_scratch_floats(B, H) floats; `logits` null or
+// [2, B, C] (student, teacher).  Returns 0, -1 when hidden / classes do not fit the kernel's shared memory, -2 on a launch error.
+size_t head_scratch_floats(int B, int H);
 int launch_head_logit_loss(const void* f_s_last, const void* f_t_last, int B, int S, int H, int C, const float* wp,
-                           const float* bp, const float* wc, const float* bc, float cc, void* dF_last, float* part,
+                           const float* bp, const float* wc, const float* bc, float cc, void* dF_last, float* scratch,
                            float* logits, float* loss_total, float* logit_loss, int dt, cudaStream_t st);
 
 // ---- backward kernels

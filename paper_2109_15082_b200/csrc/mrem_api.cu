@@ -72,6 +72,7 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->minmax = (float*)A.take(256);
   c->d_loss_e2e = (float*)A.take(256);
   c->loss_partial = (float*)A.take(sizeof(float) * RED_BLOCKS * L);
+  c->head_scratch = (float*)A.take(sizeof(float) * head_scratch_floats(d.max_batch, H));
   c->col_plane = (long long)COL_CHUNKS * (3 * H > F ? 3 * H : F);
   c->col_scratch = (float*)A.take(sizeof(float) * 3 * c->col_plane);
   c->col_counters = (int*)A.take(sizeof(int) * ((3 * H > F ? 3 * H : F) / 32 + 2));
@@ -368,6 +369,13 @@ int32_t mrem_get_grad(mrem_ctx* c, int32_t layer, int32_t id, const float** g) {
   else if (id >= MREM_GRAD_STEP + N_WMAT && id < MREM_GRAD_STEP + MREM_N_QUANTIZERS) *g = G.a + (id - MREM_GRAD_STEP - N_WMAT);
   else if (id >= MREM_GRAD_OFFSET + N_WMAT && id < MREM_GRAD_OFFSET + MREM_N_QUANTIZERS) *g = G.off + (id - MREM_GRAD_OFFSET - N_WMAT);
   else return fail(c, MREM_ERR_ARG, "get_grad: bad id");
+  return MREM_OK;
+}
+
+int32_t mrem_get_input_grad(mrem_ctx* c, const void** g) {
+  if (!c || !g) return MREM_ERR_ARG;
+  if (!c->have_input_grad) return fail(c, MREM_ERR_ORDER, "get_input_grad: no backward pass since the last forward pass");
+  *g = c->carry[0];
   return MREM_OK;
 }
 

@@ -97,6 +97,7 @@ struct mrem_ctx {
   void *alt_d_y2 = nullptr, *alt_d_sum = nullptr, *alt_d_u = nullptr, *alt_d_a = nullptr, *alt_d_y1 = nullptr, *alt_d_qkv = nullptr;
   float* alt_rowbias = nullptr;
   float* loss_partial;
+  float* head_scratch = nullptr;         // pooled vectors, gradient and per-sequence errors of the output-logit term
   float* minmax;
   int* status;
   int* t_counter;
@@ -130,6 +131,7 @@ struct mrem_ctx {
   bool tables_dirty = true;
 
   // per-step state
+  bool have_input_grad = false;      // carry[0] holds d loss / d module input of the last backward pass
   bool weights_quantized = false, have_teacher = false, have_student = false, have_loss = false, have_grads = false;
   const void* s_in = nullptr;  void* s_out = nullptr;  const void* t_out = nullptr;
   const int32_t* cur_len = nullptr;

@@ -417,6 +417,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
   // kernels above left, added in index order (one launch for the whole module; only the update reads them)
   launch_reduce_table(c->reduce_table, c->reduce_per_layer * d.n_layers, c->stream);
   join();
+  c->have_input_grad = true;           // layer 0's straight-through pass wrote it to carry[0]
   if (sync_failed) return fail(c, MREM_ERR_CUDA, "backward: stream fork/join failed");
   if (rw.rc != MREM_OK) { c->err = "weight-gradient GEMM launch failed"; return rw.rc; }
   if (r.rc != MREM_OK) return r.rc;
@@ -478,7 +479,7 @@ int32_t mrem_module_forward(mrem_ctx* c, int32_t role, const void* x, const void
     return fail(c, MREM_ERR_ARG, "forward: role");
   }
   c->cur_batch = batch; c->cur_seq = seq; c->cur_len = len;
-  c->have_loss = false; c->have_grads = false;
+  c->have_loss = false; c->have_grads = false; c->have_input_grad = false;
   return MREM_OK;
 }
 
@@ -493,12 +494,11 @@ int32_t mrem_recon_loss(mrem_ctx* c, float* loss_total, float* loss_per_layer) {
   if (c->head.wp) {
     // last module of the model: the output-logit term, its gradient added to the last layer's loss gradient
     const int L = c->d.n_layers, C = c->head.n_classes;
-    if (c->cur_batch > RED_BLOCKS) return fail(c, MREM_ERR_SHAPE, "recon_loss: batch too large for the logit term");
     const float cz = c->d.loss_mean ? 1.f / (float)((long long)c->cur_batch * C) : 1.f;
     const long long last = (long long)(L - 1) * n;
     const int hrc = launch_head_logit_loss((const char*)c->s_out + last * c->esz, (const char*)c->t_out + last * c->esz, c->cur_batch,
                                            c->cur_seq, c->d.hidden, C, c->head.wp, c->head.bp, c->head.wc, c->head.bc, cz,
-                                           (char*)c->dF + last * c->esz, c->loss_partial, c->head.logits, loss_total,
+                                           (char*)c->dF + last * c->esz, c->head_scratch, c->head.logits, loss_total,
                                            c->head.logit_loss, c->dt, c->stream);
     if (hrc == -1) return fail(c, MREM_ERR_SHAPE, "recon_loss: hidden size / class count too large for the logit term");
     if (hrc != 0) return fail(c, MREM_ERR_CUDA, "recon_loss: launch failed");

@@ -58,11 +58,13 @@ class EmbeddingStep:
             self.word_step.copy_(torch.from_numpy(np.ascontiguousarray(word_step, dtype=np.float32)))
         self.dirty = True
 
-    def step(self, ids, type_ids, optim):
-        """ids, type_ids: int32 device tensors [batch, seq].  optim None: loss and gradients only.  Returns the loss tensor."""
+    def step(self, ids, type_ids, optim, extra_grad=None):
+        """ids, type_ids: int32 device tensors [batch, seq].  optim None: loss and gradients only.  extra_grad: device
+        tensor or address of a gradient at the student's embedding output (the first module's input gradient).
+        Returns the loss tensor."""
         batch, seq = ids.shape
         B.mrem_embed_step(self.desc, self.tensors, self.ws_ptr, self.ws_bytes, ids, type_ids, batch, seq, int(self.dirty),
-                          self.e_teacher, self.e_student, optim, self.loss, self.status, self.stream.cuda_stream)
+                          self.e_teacher, self.e_student, extra_grad, optim, self.loss, self.status, self.stream.cuda_stream)
         self.dirty = False
         return self.loss[:1]
 

@@ -149,6 +149,10 @@ class ReconModule:
     def step(self, optim):
         B.mrem_step(self.ctx, optim)
 
+    def input_grad(self, batch, seq):
+        """d loss / d (student module input) of the last backward pass, [batch, seq, hidden] (a copy)."""
+        return self._ws_view(B.mrem_get_input_grad(self.ctx), batch * seq * self.H, self.tdtype).view(batch, seq, self.H).clone()
+
     def bind_head(self, head):
         """head: dict Wp [H, H], bp [H], Wc [C, H], bc [C] (numpy) of the classification head, or None to unbind."""
         if head is None:

@@ -93,13 +93,41 @@ def test_embedding_step_rejects_and_reports_bad_input():
     d_ids, d_tt = torch.from_numpy(ids).to(e.device), torch.from_numpy(tt).to(e.device)
     with pytest.raises(B.MremError):                                    # longer than the position table
         long_ids = torch.zeros(1, 17, dtype=torch.int32, device=e.device)
-        B.mrem_embed_step(e.desc, e.tensors, e.ws_ptr, e.ws_bytes, long_ids, None, 1, 17, 1, e.e_teacher, e.e_student, None, e.loss,
+        B.mrem_embed_step(e.desc, e.tensors, e.ws_ptr, e.ws_bytes, long_ids, None, 1, 17, 1, e.e_teacher, e.e_student, None, None, e.loss,
                           e.status, e.stream.cuda_stream)
     with pytest.raises(B.MremError):                                    # workspace too small
-        B.mrem_embed_step(e.desc, e.tensors, e.ws_ptr, 1024, d_ids, d_tt, 2, 8, 1, e.e_teacher, e.e_student, None, e.loss, e.status,
+        B.mrem_embed_step(e.desc, e.tensors, e.ws_ptr, 1024, d_ids, d_tt, 2, 8, 1, e.e_teacher, e.e_student, None, None, e.loss, e.status,
                           e.stream.cuda_stream)
     bad = d_ids.clone()
     bad[1, 3] = 64                                                      # one index past the table: clamped, reported
     e.step(bad, d_tt, None)
     torch.cuda.synchronize()
     assert int(e.status[0]) == 5
+
+
+def test_first_module_hands_its_input_gradient_to_the_embedding_step():
+    """The model's first module: the embedding output is the module's input, and the gradient the layers send back to it
+    (mrem_get_input_grad) joins the gradient of the embedding MSE.  The module's input gradient against the oracle's;
+    the embedding gradients with that extra gradient against the oracle's with the same one."""
+    from tests.gpu_util import Problem
+    wl = synth.shrink(synth.workloads()["base3_w4a8"], n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=5, len_lo=10, len_hi=40)
+    p = Problem(wl, step_shrink=0.8, student_noise=0.002)
+    try:
+        p.run_gpu()
+        torch.cuda.synchronize()
+        d_in = p.m.input_grad(wl.batch, wl.seq)
+        r = O.forward_loss_backward(p.desc, p.teacher, p.student, p.oracle_steps(), p.x, p.x, p.vl)
+        assert rel(d_in.float().cpu().numpy(), r["d_input"]) < 2e-2
+        e, desc, teacher, student, step, ids, tt = _problem("bf16", 4, H=128, batch=wl.batch, seq=wl.seq)
+        d_ids, d_tt = torch.from_numpy(ids).to(e.device), torch.from_numpy(tt).to(e.device)
+        extra = (d_in.float() * 20).to(torch.bfloat16).contiguous()      # of the size of the MSE's own gradient
+        e.step(d_ids, d_tt, None, extra_grad=extra)
+        torch.cuda.synchronize()
+        re = O.embed_loss_backward(desc, teacher, student, step, 4, ids, tt, d_extra=extra.float().cpu().numpy())
+        plain = O.embed_loss_backward(desc, teacher, student, step, 4, ids, tt)
+        for k in ("word", "pos", "type", "ln_g", "ln_b", "word_step"):
+            got = e.g[k].cpu().numpy()
+            assert rel(got, re["grads"][k]) < 2e-2, (k, rel(got, re["grads"][k]))
+            assert rel(got, plain["grads"][k]) > 0.1, k                  # the extra gradient is not a rounding-level term
+    finally:
+        p.close()
