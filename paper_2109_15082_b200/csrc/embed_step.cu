@@ -45,40 +45,60 @@ __global__ void __launch_bounds__(128) embed_sum_kernel(const float* __restrict_
   }
 }
 
-// Occurrence lists of the batch's ids: first[t] = 1 when no earlier token has the id of token t, next[t] = the
-// next later token with that id (-1: none).  One thread per token.
-__global__ void __launch_bounds__(256) embed_links_kernel(const int* __restrict__ ids, int M, int vocab, int* __restrict__ first,
-                                                          int* __restrict__ next) {
+// Occurrence lists of the batch's ids, without sorting and without atomics.  Per token t (one thread each):
+//   lead[t] = index of the first token with the id of token t,  rank[t] = number of earlier tokens with that id.
+__global__ void __launch_bounds__(256) embed_lead_kernel(const int* __restrict__ ids, int M, int vocab, int* __restrict__ lead,
+                                                         int* __restrict__ rank) {
   pdl_trigger();
   pdl_wait();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= M) return;
   const int id = min(max(ids[t], 0), vocab - 1);
-  int nx = -1, fi = 1;
-  for (int i = t + 1; i < M; ++i)
-    if (min(max(ids[i], 0), vocab - 1) == id) { nx = i; break; }
+  int first = t, r = 0;
   for (int i = t - 1; i >= 0; --i)
-    if (min(max(ids[i], 0), vocab - 1) == id) { fi = 0; break; }
-  first[t] = fi;
-  next[t] = nx;
+    if (min(max(ids[i], 0), vocab - 1) == id) { first = i; ++r; }
+  lead[t] = first;
+  rank[t] = r;
+}
+// list = the tokens grouped by id (groups ordered by their first token, token order inside a group):
+//   position of token t = number of tokens whose group starts before t's group + rank[t];
+// for the first token of a group also start[t] = that position and count[t] = size of the group (count 0 elsewhere).
+__global__ void __launch_bounds__(256) embed_list_kernel(const int* __restrict__ lead, const int* __restrict__ rank, int M,
+                                                         int* __restrict__ list, int* __restrict__ start, int* __restrict__ count) {
+  pdl_trigger();
+  pdl_wait();
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= M) return;
+  const int mine = lead[t];
+  int before = 0, same = 0;
+  for (int i = 0; i < M; ++i) {
+    const int l = lead[i];
+    before += l < mine;
+    same += l == mine;
+  }
+  list[before + rank[t]] = t;
+  start[t] = before;
+  count[t] = mine == t ? same : 0;
 }
 
 // g_word[id, :] = sum over the tokens t with ids[t] == id of dy[t, :], in token order: the block of the first
-// token with an id walks that id's occurrence list for its 128 columns; rows no token gathered keep the zeros
-// the caller put there.
+// token with an id adds that id's group of the list for its 128 columns (independent loads); rows no token gathered
+// keep the zeros the caller put there.
 template <typename T>
 __global__ void __launch_bounds__(128) embed_scatter_kernel(const T* __restrict__ dy, const int* __restrict__ ids,
-                                                            const int* __restrict__ first, const int* __restrict__ next, int H,
-                                                            int vocab, float* __restrict__ g_word) {
+                                                            const int* __restrict__ list, const int* __restrict__ start,
+                                                            const int* __restrict__ count, int H, int vocab,
+                                                            float* __restrict__ g_word) {
   pdl_trigger();
   pdl_wait();
-  const int t0 = blockIdx.x;
-  if (!first[t0]) return;                                           // block-uniform
+  const int t0 = blockIdx.x, n = count[t0];
+  if (n == 0) return;                                               // block-uniform: not the first token of its id
   const int c = blockIdx.y * blockDim.x + threadIdx.x;
   if (c >= H) return;
   const int id = min(max(ids[t0], 0), vocab - 1);
+  const int* grp = list + start[t0];
   float acc = 0.f;
-  for (int t = t0; t >= 0; t = next[t]) acc += to_f<T>(dy[(long long)t * H + c]);
+  for (int j = 0; j < n; ++j) acc += to_f<T>(dy[(long long)grp[j] * H + c]);
   g_word[(long long)id * H + c] = acc;
 }
 
@@ -136,7 +156,7 @@ struct EmbedScratch {
   int* col_counters;
   int8_t* codes; int32_t* rowsum; float* scale;
   OptimScalars* optim_sc; AdamEntry* table;
-  int *first, *next; float* type_partial;
+  int *lead, *rank, *list, *start, *count; float* type_partial;
   size_t bytes;
 };
 EmbedScratch carve(const mrem_embed_desc& d, long long max_tokens, void* base) {
@@ -155,7 +175,9 @@ EmbedScratch carve(const mrem_embed_desc& d, long long max_tokens, void* base) {
   s.scale = (float*)A.take(sizeof(float) * d.vocab);
   s.optim_sc = (OptimScalars*)A.take(sizeof(OptimScalars));
   s.table = (AdamEntry*)A.take(sizeof(AdamEntry) * 4);
-  s.first = (int*)A.take(sizeof(int) * max_tokens); s.next = (int*)A.take(sizeof(int) * max_tokens);
+  s.lead = (int*)A.take(sizeof(int) * max_tokens); s.rank = (int*)A.take(sizeof(int) * max_tokens);
+  s.list = (int*)A.take(sizeof(int) * max_tokens); s.start = (int*)A.take(sizeof(int) * max_tokens);
+  s.count = (int*)A.take(sizeof(int) * max_tokens);
   s.type_partial = (float*)A.take(sizeof(float) * (size_t)TYPE_CHUNKS * d.n_types * d.hidden);
   s.bytes = (A.off + 255) & ~size_t(255);
   return s;
@@ -232,12 +254,13 @@ int32_t mrem_embed_step(const mrem_embed_desc* d, const mrem_embed_tensors* x, v
                     s.col_counters, dt, st);
   // position / token-type tables: sums over the batch; word table: every token's gradient into the row it gathered
   if (cudaMemsetAsync(x->g_word, 0, sizeof(float) * (size_t)V * H, st) != cudaSuccess) return MREM_ERR_CUDA;
-  launch_k(embed_links_kernel, (unsigned)((M + 255) / 256), 256, 0, st, d_ids, (int)M, V, s.first, s.next);
+  launch_k(embed_lead_kernel, (unsigned)((M + 255) / 256), 256, 0, st, d_ids, (int)M, V, s.lead, s.rank);
+  launch_k(embed_list_kernel, (unsigned)((M + 255) / 256), 256, 0, st, (const int*)s.lead, (const int*)s.rank, (int)M, s.list, s.start, s.count);
   const dim3 gcol((H + 255) / 256), gscat((unsigned)M, (H + 127) / 128);
 #define MREM_EMB_BWD(T) do { \
     launch_k(embed_pos_kernel<T>, dim3(gcol.x, d->max_pos), 256, 0, st, (const T*)s.dy, (int)batch, (int)seq, H, x->g_pos); \
     launch_k(embed_type_partial_kernel<T>, dim3(gcol.x, TYPE_CHUNKS, d->n_types), 256, 0, st, (const T*)s.dy, d_type_ids, M, H, (int)d->n_types, s.type_partial); \
-    launch_k(embed_scatter_kernel<T>, gscat, 128, 0, st, (const T*)s.dy, d_ids, (const int*)s.first, (const int*)s.next, H, V, x->g_word); } while (0)
+    launch_k(embed_scatter_kernel<T>, gscat, 128, 0, st, (const T*)s.dy, d_ids, (const int*)s.list, (const int*)s.start, (const int*)s.count, H, V, x->g_word); } while (0)
   if (dt == 1) MREM_EMB_BWD(bf16); else MREM_EMB_BWD(float);
 #undef MREM_EMB_BWD
   launch_k(embed_type_final_kernel, dim3(gcol.x, d->n_types), 256, 0, st, (const float*)s.type_partial, H, (int)d->n_types, x->g_type);
