@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout,
 // gradient leaves as one partial sum per block (fixed order; slots beyond the grid are zeroed).
 // Rows up to 32 * V * MAXNV wide, one warp per row, warps stride over the rows.
 template <typename T, int V>
-__global__ void __launch_bounds__(128) ln_bwd_ste_kernel(const T* __restrict__ dout, const T* __restrict__ x,
+__global__ void __launch_bounds__(128, 7) ln_bwd_ste_kernel(const T* __restrict__ dout, const T* __restrict__ x,
                                                          const T* __restrict__ dxhat, const T* __restrict__ add,
                                                          const float* __restrict__ step, float lo, float hi,
                                                          const T* __restrict__ y, const float* __restrict__ mean,
