@@ -217,7 +217,8 @@ int32_t mrem_set_programmatic_launch(int32_t on);
  * softmax and context products, with the straight-through masks of the Q, K, V, P quantizers) runs as one
  * kernel; off (0) selects the kernel-per-operation path that covers every shape.  Both compute the same
  * quantities; they differ in where intermediates are rounded to the storage type.  Do not change it
- * between the capture and the replay of a graph. */
+ * between a student forward pass and its backward pass (the forward pass writes the codes of the attention
+ * probabilities only for the kernel-per-operation path), nor between the capture and the replay of a graph. */
 int32_t mrem_set_fused_attention_backward(mrem_ctx* ctx, int32_t on);
 
 /* Reads the device status word (blocks on the stream): MREM_OK, MREM_ERR_TIMEOUT or MREM_ERR_NONFINITE in

@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
           for (int t = 0; t < 4; ++t)
             if (t * 8 < ncol) {
               store16(p.P + prow + c * 32 + t * 8, pw + 4 * t);
-              if (quant) store16(p.P_qt + prow + c * 32 + t * 8, cw + 4 * t);
+              if (quant && p.P_qt) store16(p.P_qt + prow + c * 32 + t * 8, cw + 4 * t);
             }
         }
       } else {

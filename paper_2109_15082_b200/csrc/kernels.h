@@ -66,7 +66,7 @@ void launch_softmax_fwd(const float* scores, const int* valid_len, int B, int h,
 // Fused attention forward on the tensor cores (bf16 storage, head size 64, seq <= 384, seq % 8 == 0):
 // scores, masked softmax, quantizer of the probabilities, context product and (student) the context's
 // codes in one kernel.  Returns a GemmRc.  Null p_step / c_step: no quantizer; null P: the probabilities are
-// not written (a full-precision pass whose probabilities nobody reads).
+// not written (a full-precision pass whose probabilities nobody reads); null P_qt: their codes are not written.
 bool attention_fwd_supported(int S, int head_dim, int dt);
 int launch_attention_fwd(const void* qkv, int B, int S, int h, int H, const int* valid_len, float alpha_const,
                          const float* a_p0, const float* a_p1, const float* c_p0, const float* c_p1,

@@ -209,8 +209,11 @@ int student_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S
     launch_quantize_act3(s.qkv, c->dt, M, H, 3 * H, b.a_steps[S_Q], b.a_steps[S_K], b.a_steps[S_V], rx.lo, rx.hi, s.qkv_qt,
                          3 * H, c->stream);
     if (attention_fwd_supported(S, hd, c->dt)) {
+      // (the single-kernel attention backward takes the codes of the probabilities from the probabilities themselves:
+      //  they are written out only for the kernel-per-operation backward)
+      const bool codes_needed = !(c->fused_attention_bwd && attention_bwd_supported(S, hd, c->dt, B * h));
       r.note(launch_attention_fwd(s.qkv_qt, B, S, h, H, len, 1.f / sqrtf((float)hd), b.a_steps[S_Q], b.a_steps[S_K],
-                                  b.a_steps[S_P], b.a_steps[S_V], b.a_steps[S_P], rp.lo, rp.hi, s.P, s.P_qt, s.ctx,
+                                  b.a_steps[S_P], b.a_steps[S_V], b.a_steps[S_P], rp.lo, rp.hi, s.P, codes_needed ? s.P_qt : nullptr, s.ctx,
                                   b.a_steps[S_C], rx.hi, s.ctx_q8, s.ctx_qt, c->status, c->stream),
              "attention launch failed");
     } else {
