@@ -222,6 +222,38 @@ def time_extras(m, wl, xbuf, lenbuf, stream, torch, B, pk, reps=10):
     out["embed_step"] = {"vocab": V, "tokens": rows, "e_bits": 4, "ms_per_step": ms, "table_gbs": table_bytes / (ms * 1e-3) / 1e9,
                          "hbm_peak_gbs": pk["hbm_gbs"], "status": int(emb.status[0]),
                          "note": "whole step; table_gbs counts only the dense pass over the word table (33 B per entry)"}
+    # the whole sequential sweep of the stated BERT-large configuration: 4 modules of the workload's depth one after the
+    # other, 200 steps each over a 1024-sequence calibration set, outputs cached for the next module (wall clock,
+    # synchronised at both ends; includes step initialisation, graph capture and the caching passes)
+    if wl.name == "large6_w4a8":
+        from paper_2109_15082_b200 import synth
+        from paper_2109_15082_b200.session import ReconModule
+        from paper_2109_15082_b200.sweep import ModuleSweep
+        n_mod, steps, n_cal = 4, 200, 1024
+        with torch.cuda.stream(stream):
+            mods = []
+            for k in range(n_mod):
+                mk = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, wl.a_bits, wl.w_grid, True, 3,
+                                 wl.act_dtype, stream=stream)
+                mk.load_teacher(synth.teacher_params(wl, seed=100 + k))
+                mk.init_student_from_teacher()
+                mods.append(mk)
+            calib = torch.randn(n_cal, wl.seq, wl.hidden, device=m.device, dtype=torch.float32).to(m.tdtype)
+            lens = torch.randint(32, wl.seq + 1, (n_cal,), device=m.device, dtype=torch.int32)
+            sweep = ModuleSweep(mods, calib, lens, wl.batch, lambda k, e: synth.permutation(k, f"sweep{e}", n_cal), wl.w_step_rule)
+            stream.synchronize()
+            t0 = time.perf_counter()
+            for k in range(n_mod):
+                sweep.run_module(k, steps, B.make_optim(lr=wl.lr, step=0, decay_total_steps=steps), record_every=50)
+                if k + 1 < n_mod:
+                    sweep.cache_outputs(k)
+            stream.synchronize()
+            dt = time.perf_counter() - t0
+            out["sweep"] = {"modules": n_mod, "layers_per_module": wl.n_layers, "steps_per_module": steps, "calibration_sequences": n_cal,
+                            "seconds": dt, "tokens_per_s": n_mod * steps * rows / dt,
+                            "first_and_last_recorded_loss": [[l[0], l[-1]] for l in sweep.losses]}
+            for mk in mods:
+                mk.close()
     return out
 
 
