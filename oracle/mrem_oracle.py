@@ -52,6 +52,7 @@ class ModuleDesc:
     ln_eps: float = 1e-12
     w_twn: bool = False        # 2-bit weights by the closed-form ternary rule (threshold 0.7 mean|w|, scale = mean
                                # of the kept |w|, per output row) instead of a learnable step
+    w_laq: bool = False        # b-bit weights with the scale refitted by alternating least squares (quantize_weight_laq)
 
 
 # ----------------------------------------------------------------------------- storage
@@ -153,6 +154,46 @@ def quantize_weight_twn(w, per_row=True):
     alpha = alpha.astype(np.float32).astype(np.float64)
     t = (np.sign(w32 if per_row else w32.reshape(1, -1)) * keep).astype(np.int64).reshape(w32.shape)
     return t, alpha, delta
+
+
+LAQ_ROUNDS = 16
+
+
+def quantize_weight_laq(w, bits, per_row=True, rounds=LAQ_ROUNDS, alpha0=None):
+    """b-bit weights whose scale is refitted from the weights instead of learnt (the loss-aware quantizer the paper
+    names for 4-bit weights, Sec. 5.1, read with unit curvature weights): per group (output row or whole matrix)
+    minimise ||w - alpha q||^2 over alpha and q in Omega(b)^n by alternating the two exact half-steps,
+        q     = Pi_Omega(b)(w / alpha)        (alpha fixed: Eq. 1, element by element)
+        alpha = <q, w> / <q, q>               (q fixed: least squares)
+    `rounds` times from alpha_0 = min(3 mean|w|, max|w|) / qmax (a clipping range of 3 mean|w|, about 2.4 standard
+    deviations of a Gaussian row, which does not follow single outliers the way max|w| does; never beyond max|w|, so
+    that the largest weight always gets a non-zero code and no later scale can exceed max|w|; `alpha0` overrides it);
+    w_hat = alpha_rounds * q_rounds.
+    A group of zeros keeps alpha = 0 and codes 0.  Every alpha is rounded to float32 (the type the scale is stored
+    in) and the division w / alpha is the float32 one of Eq. 1; the mean and the two inner products are accumulated
+    in float64.
+    Returns (codes int64, alpha float64 [groups, 1], trace): trace[r] = (alpha_r, q_{r+1}) per round, for tests."""
+    w32 = np.asarray(w, np.float32)
+    g = w32 if per_row else w32.reshape(1, -1)
+    g64 = g.astype(np.float64)
+    qmax = sym_qmax(bits)
+    if alpha0 is None:
+        a = np.abs(g64)
+        alpha = (np.minimum(3.0 * a.mean(-1, keepdims=True), a.max(-1, keepdims=True)) / qmax).astype(np.float32)
+    else:
+        alpha = np.asarray(alpha0, np.float32).reshape(-1, 1)
+    q = np.zeros(g.shape, np.int64)
+    trace = []
+    for _ in range(rounds):
+        live = alpha[:, 0] > 0
+        q = np.zeros(g.shape, np.int64)
+        if live.any():
+            q[live] = quantize_weight(g[live], alpha[live], bits, 0, "f32")[0]
+        trace.append((alpha.astype(np.float64), q.copy()))
+        qq = (q * q).sum(-1, keepdims=True)
+        qw = (q * g64).sum(-1, keepdims=True)
+        alpha = np.where(qq > 0, qw / np.maximum(qq, 1), 0.0).astype(np.float32)
+    return q.reshape(w32.shape), alpha.astype(np.float64), trace
 
 
 def weight_ste(z, codes, bits, grid):
@@ -304,7 +345,11 @@ def _q_w(desc, w, s_w):
         return dict(what=np.asarray(w, np.float64), q=None)
     if desc.w_twn:
         q, alpha, _ = quantize_weight_twn(w, desc.w_per_row)
-        return dict(what=alpha * q, q=q, z=None, scale=alpha, twn=True)
+        return dict(what=alpha * q, q=q, z=None, scale=alpha, closed=True)
+    if desc.w_laq:
+        q, alpha, _ = quantize_weight_laq(w, desc.w_bits, desc.w_per_row)
+        alpha_e = alpha if desc.w_per_row else alpha.reshape(1, 1)
+        return dict(what=alpha_e * q, q=q, z=None, scale=alpha, closed=True)
     s = np.asarray(s_w, np.float32).reshape(-1, 1)
     q, scale, z = quantize_weight(w, s, desc.w_bits, desc.w_grid, desc.act_dtype)
     return dict(what=scale * q, q=q, z=z, scale=scale)
@@ -421,7 +466,7 @@ def _linear_back(desc, qa, qw, dy, name, g, site):
     dy2 = dy.reshape(-1, dy.shape[-1])
     dwhat = dy2.T @ qa["xhat"].reshape(-1, K)
     g["b" + name[1:] if name != "Wqkv" else "bqkv"] = dy2.sum(0)
-    if qw["q"] is None or qw.get("twn"):
+    if qw["q"] is None or qw.get("closed"):
         g[name] = dwhat                                   # closed-form scales: plain straight-through, nothing to learn
         g["w"][name] = None
     else:
@@ -752,7 +797,7 @@ def rem_forward_loss_backward(desc, w_teacher, w_student, steps, name, a):
     dy = 2.0 * c * diff
     dwhat = dy.T @ qa["xhat"]
     out = dict(target=target, y=y, loss=loss, qa=qa, qw=qw, d_a_step=0.0, d_a_off=0.0)
-    if qw["q"] is None or qw.get("twn"):
+    if qw["q"] is None or qw.get("closed"):
         out["dW"], out["d_w_step"] = dwhat, None
     else:
         inside, dwhat_ds = weight_ste(qw["z"], qw["q"], desc.w_bits, desc.w_grid)

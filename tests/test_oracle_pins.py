@@ -449,6 +449,132 @@ def test_twn_module_matches_torch_autograd_with_plain_straight_through():
     assert (q == 0).any() and (q != 0).any()
 
 
+# ----------------------------------------------------------------------------- refitted scales (alternating rule)
+
+def _sq_err(w, alpha, q):
+    return float(((np.asarray(w, np.float64) - alpha * q) ** 2).sum())
+
+
+def test_laq_keeps_a_grid_point_fixed_and_handles_dead_rows():
+    rng = np.random.default_rng(11)
+    for bits in (2, 4, 8):
+        qmax = 2 ** (bits - 1) - 1
+        b0 = rng.integers(-qmax, qmax + 1, (5, 48))
+        a0 = np.float32(2.0 ** -5) * np.array([[1], [3], [5], [7], [9]], np.float32)     # scales exact in float32
+        w = (a0 * b0).astype(np.float32)
+        w[3] = 0.0
+        q, alpha, _ = O.quantize_weight_laq(w, bits, alpha0=a0)      # started at the true scale, the rounds stay there
+        keep = [0, 1, 2, 4]
+        assert np.array_equal(q[keep], b0[keep]) and np.array_equal(alpha[keep, 0], a0[keep, 0].astype(np.float64))
+        assert not q[3].any() and alpha[3, 0] == 0.0
+        q, alpha, _ = O.quantize_weight_laq(w, bits)                  # default start: dead row all the same
+        assert not q[3].any() and alpha[3, 0] == 0.0 and np.all(alpha[keep] > 0)
+        # rows of +-c only: three mean|w| lies beyond every weight, the start falls back on max|w| and nothing collapses
+        flat = np.where(rng.random((3, 32)) < 0.5, -0.25, 0.25).astype(np.float32)
+        q, alpha, _ = O.quantize_weight_laq(flat, bits)
+        assert np.allclose(alpha * q, flat.astype(np.float64), rtol=1e-6, atol=0)
+
+
+def test_laq_half_steps_are_exact_and_the_error_never_rises():
+    rng = np.random.default_rng(5)
+    w = (rng.standard_normal((7, 200)) * 0.04).astype(np.float32)
+    w[:, :3] *= 6.0                                               # a few outliers: the min-max start is far from the fit
+    for bits in (2, 4):
+        qmax = 2 ** (bits - 1) - 1
+        levels = np.arange(-qmax, qmax + 1)
+        q, alpha, trace = O.quantize_weight_laq(w, bits)
+        assert len(trace) == O.LAQ_ROUNDS and np.array_equal(trace[-1][1], q)
+        assert np.array_equal(trace[0][0][:, 0], (np.minimum(3 * np.abs(w.astype(np.float64)).mean(1), np.abs(w.astype(np.float64)).max(1)) / qmax).astype(np.float32))
+        for r in range(7):
+            prev = None
+            for i, (a_r, q_r) in enumerate(trace):
+                a_r = a_r[r, 0]
+                # projection: every code is the nearest level of alpha_r * Omega(b), by brute force over the levels
+                d = np.abs(w[r].astype(np.float64)[:, None] - a_r * levels[None, :])
+                best = levels[d.argmin(1)]
+                clear = np.sort(d, 1)[:, 1] - np.sort(d, 1)[:, 0] > 1e-9 * a_r      # not a tie
+                assert np.array_equal(q_r[r][clear], best[clear])
+                # scale: the least-squares solution of q * alpha = w from the library solver
+                a_next = trace[i + 1][0][r, 0] if i + 1 < len(trace) else alpha[r, 0]
+                ls = np.linalg.lstsq(q_r[r].astype(np.float64)[:, None], w[r].astype(np.float64), rcond=None)[0][0]
+                assert a_next == pytest.approx(ls, rel=2e-7)
+                e0, e1 = _sq_err(w[r], a_r, q_r[r]), _sq_err(w[r], a_next, q_r[r])
+                assert e1 <= e0 * (1 + 1e-6)
+                if prev is not None:
+                    assert e0 <= prev * (1 + 1e-6)
+                prev = e1
+            # 15 levels: below the min-max scale, which follows the outliers (with 3 levels either local optimum,
+            # the bulk or the outliers, can be the better one)
+            mm = np.float32(np.abs(w[r]).max() / qmax)
+            assert bits == 2 or _sq_err(w[r], alpha[r, 0], q[r]) < _sq_err(w[r], mm, O.quantize_weight(w[r:r + 1], mm.reshape(1, 1), bits, 0, "f32")[0][0])
+
+
+def test_laq_against_exhaustive_search_on_tiny_rows():
+    """2-bit rows of 5 weights: all 3^5 code vectors with their least-squares scale.  The alternating rule never
+    beats the global optimum, never ends above its start, and finds the optimum on most rows."""
+    import itertools
+    rng = np.random.default_rng(2)
+    w = rng.standard_normal((60, 5)).astype(np.float32)
+    q, alpha, trace = O.quantize_weight_laq(w, 2)
+    hits = 0
+    for r in range(60):
+        best = np.inf
+        for c in itertools.product((-1, 0, 1), repeat=5):
+            c = np.array(c, np.float64)
+            if c.any():
+                a = (c @ w[r].astype(np.float64)) / (c @ c)
+                best = min(best, _sq_err(w[r], a, c))
+        e = _sq_err(w[r], alpha[r, 0], q[r])
+        assert e >= best * (1 - 1e-6) and e <= _sq_err(w[r], trace[0][0][r, 0], trace[0][1][r]) * (1 + 1e-6)
+        hits += e <= best * (1 + 1e-5)
+    assert hits >= 45, hits
+
+
+def test_laq_step_on_gaussian_rows_is_the_uniform_quantizer_optimum():
+    """The mean-square-optimal uniform quantizer of a unit Gaussian has a step of 0.335 sigma with 16 levels and of
+    1.22 sigma with 3 (Max 1960, uniform-quantizer table); the 15-level fit must land just above the first (one level
+    fewer), the 3-level fit on the second."""
+    rng = np.random.default_rng(9)
+    w = rng.standard_normal((4, 1 << 16)).astype(np.float32)
+    _, a4, _ = O.quantize_weight_laq(w, 4)
+    _, a2, _ = O.quantize_weight_laq(w, 2)
+    assert np.all((a4 > 0.335) & (a4 < 0.365)), a4.ravel()
+    assert np.all((a2 > 1.20) & (a2 < 1.25)), a2.ravel()
+    one, a1, _ = O.quantize_weight_laq(w, 4, per_row=False)
+    assert a1.shape == (1, 1) and one.shape == w.shape and 0.335 < a1[0, 0] < 0.365
+
+
+def test_laq_module_matches_torch_autograd_with_plain_straight_through():
+    wl, desc, params, x = _tiny(w_bits=4, w_laq=True)
+    vl = np.array([4, 5], np.int32)
+    teacher = [{k: v.copy() for k, v in p.items()} for p in params]
+    student = [{k: (v + synth.normal(7, k + str(i), v.shape, 0.01)).astype(np.float32) for k, v in p.items()}
+               for i, p in enumerate(params)]
+    ws = O.init_weight_steps(desc, student, 0)                     # unused by this quantizer
+    a, off = O.init_act_steps(desc, student, x, vl)
+    steps = O.make_steps(ws, (a * 0.8).astype(np.float32), off)
+    r = O.forward_loss_backward(desc, teacher, student, steps, x, x, vl, lam=0.0)
+    tp, ts = _to_torch(student, steps)
+    tt, _ = _to_torch(teacher, [])
+    xs = torch.tensor(x, dtype=torch.float64)
+    cfg = dict(_cfg(desc), w_laq=True, w_per_row=desc.w_per_row)
+    f_t = R.module(xs, tt, [None] * len(tt), cfg, vl, quant=False)
+    f_s = R.module(xs, tp, ts, cfg, vl, quant=True)
+    c = 1.0 / f_s[0].numel()
+    loss = sum(c * ((a_ - b_.detach()) ** 2).sum() for a_, b_ in zip(f_s, f_t))
+    loss.backward()
+    for a_, b_ in zip(r["f_s"], f_s):
+        assert np.allclose(a_, b_.detach().numpy(), rtol=1e-9, atol=1e-11)
+    assert np.isclose(r["loss"], loss.item(), rtol=1e-10)
+    for l, g in enumerate(r["grads"]):
+        for k in O.PARAMS:
+            ref = tp[l][k].grad.numpy()
+            assert np.allclose(g[k], ref, rtol=1e-7, atol=1e-9 * np.abs(ref).max()), (l, k)
+        assert all(g["w"][k] is None for k in O.WEIGHTS)
+    q = r["caches"][0]["qw"]["W1"]["q"]
+    assert np.abs(q).max() == 7 and len(np.unique(q)) > 8
+
+
 # ----------------------------------------------------------------------------- Eq. 2 (one product)
 
 def _rem_case(name, asym_g=True, w_bits=4, w_grid=0, a_bits=8, rows=24, h=32, f=48, seed=3, shrink=0.8):

@@ -48,6 +48,22 @@ def q_weight_twn(w, per_row=True):
     return w + (what - w).detach()
 
 
+def q_weight_laq(w, bits, per_row=True, rounds=16):
+    # scale refitted by alternating least squares from min(3 mean|w|, max|w|) / qmax: value alpha * q, gradient passed to w unchanged
+    g = w.detach() if per_row else w.detach().reshape(1, -1)
+    g32 = g.float()                                                   # codes are decided in float32
+    qmax = 2 ** (bits - 1) - 1
+    alpha = (torch.minimum(3.0 * g.abs().mean(-1, keepdim=True), g.abs().amax(-1, keepdim=True)) / qmax).float()
+    q = torch.zeros_like(g)
+    for _ in range(rounds):
+        z = torch.where(alpha > 0, g32 / torch.where(alpha > 0, alpha, torch.ones_like(alpha)), torch.zeros_like(g32))
+        q = torch.clamp(torch.round(z), -qmax, qmax).double()
+        qq = (q * q).sum(-1, keepdim=True)
+        alpha = torch.where(qq > 0, (q * g).sum(-1, keepdim=True) / qq.clamp(min=1), torch.zeros_like(qq)).float()
+    what = (alpha.double() * q).reshape(w.shape)
+    return w + (what - w).detach()
+
+
 def layer(x, p, st, cfg, pad, quant=True):
     H = x.shape[-1]
     h = cfg["n_heads"]
@@ -68,6 +84,8 @@ def layer(x, p, st, cfg, pad, quant=True):
             return p[name]
         if cfg.get("w_twn"):
             return q_weight_twn(p[name], cfg.get("w_per_row", True))
+        if cfg.get("w_laq"):
+            return q_weight_laq(p[name], wb, cfg.get("w_per_row", True))
         return q_weight(p[name], st["w"][name], wb, grid)
 
     B, S, _ = x.shape
