@@ -86,8 +86,13 @@ typedef struct {
   int32_t a_bits;              /* 8 or 4 */
   int32_t w_grid;              /* 0: integer codes Omega(b) of Eq. 1; 1: 2-bit levels {-1.5,-.5,.5,1.5}*step;
                                   2: 2-bit ternary codes by the closed-form rule named in Sec. 5.1 (per output row:
-                                  threshold 0.7 mean|w|, scale = mean of the kept |w|); no weight steps are bound,
-                                  learnt or reported, the weight gradient passes straight through */
+                                  threshold 0.7 mean|w|, scale = mean of the kept |w|);
+                                  3: codes in Omega(w_bits) with the scale refitted from the weights by the loss-aware
+                                  rule Sec. 5.1 names for 4-bit weights, read with unit curvature weights (per output
+                                  row, 16 rounds of q = Pi(w / alpha), alpha = <q, w> / <q, q> from
+                                  alpha_0 = min(3 mean|w|, max|w|) / qmax).
+                                  With 2 and 3 no weight steps are bound, learnt or reported and the weight gradient
+                                  passes straight through; both need w_step_per_row = 1 */
   int32_t w_step_per_row;      /* 1: one step per output row; 0: one per matrix */
   int32_t act_asym_sites;      /* bit 0: softmax output unsigned (offset 0); bit 1: GELU output unsigned with
                                   learnable offset (Sec. 3.1: asymmetric for these two) */

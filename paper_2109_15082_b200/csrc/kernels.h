@@ -15,15 +15,17 @@ constexpr int RED_BLOCKS = 1184;    // grid of every kernel that emits per-block
 void launch_quantize_weight(const float* w, int rows, int cols, const float* steps, int per_row, int bits, int grid,
                             int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt, cudaStream_t st);
 
-// Closed-form ternary weights, one step-free rule per output row (Sec. 5.1 names it for 2-bit weights):
-// delta = 0.7 mean|w|, codes sign(w) 1[|w| > delta], scale = mean of the kept |w|; and the fused update
-// (AdamW with the gradient of w_hat passed through unchanged, then the rule on the new weights).
-void launch_ternary_quantize(const float* w, int rows, int cols, int8_t* codes, int32_t* rowsum, float* scale,
-                             void* what, int dt, cudaStream_t st);
+// Weight codes with a scale recomputed from the weights, one step-free rule per output row (Sec. 5.1 names one for
+// 2-bit and one for 4-bit weights).  rule 2: ternary, delta = 0.7 mean|w|, codes sign(w) 1[|w| > delta], scale =
+// mean of the kept |w|.  rule 3: codes in Omega(bits) and scale by alternating least squares (q = Pi(w / alpha),
+// alpha = <q, w> / <q, q>) from min(3 mean|w|, max|w|) / qmax.  The fused update is AdamW with the gradient of
+// w_hat passed through unchanged, then the rule on the new weights.
+void launch_closed_form_quantize(const float* w, int rows, int cols, int rule, int bits, int8_t* codes, int32_t* rowsum,
+                                 float* scale, void* what, int dt, cudaStream_t st);
 struct OptimScalars;
-void launch_ternary_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
-                           int train_w, int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt,
-                           cudaStream_t st);
+void launch_closed_form_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
+                               int train_w, int rule, int bits, int8_t* codes, int32_t* rowsum, float* scale, void* what,
+                               int dt, cudaStream_t st);
 
 // Activation quantizer over a 2-D view x[rows, cols] with row stride ld_x:
 // z = (x - offset) / step, q = rne(clip(z, lo, hi)).  Writes int8/uint8 codes (row stride

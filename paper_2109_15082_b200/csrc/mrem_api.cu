@@ -51,8 +51,9 @@ static int validate(const mrem_module_desc* d, std::string* why) {
     *why = "bf16 path needs head size multiple of 64 and seq multiple of 8"; return MREM_ERR_SHAPE; }
   if (d->w_bits != 2 && d->w_bits != 4 && d->w_bits != 8) { *why = "w_bits must be 2, 4 or 8"; return MREM_ERR_UNSUPPORTED; }
   if (d->a_bits != 8 && d->a_bits != 4) { *why = "a_bits must be 8 or 4"; return MREM_ERR_UNSUPPORTED; }
-  if (d->w_grid != 0 && !((d->w_grid == 1 || d->w_grid == 2) && d->w_bits == 2)) { *why = "w_grid 1 and 2 need w_bits 2"; return MREM_ERR_UNSUPPORTED; }
-  if (d->w_grid == 2 && !d->w_step_per_row) { *why = "w_grid 2 (closed-form ternary weights) works per output row"; return MREM_ERR_UNSUPPORTED; }
+  if (d->w_grid < 0 || d->w_grid > 3) { *why = "w_grid must be 0, 1, 2 or 3"; return MREM_ERR_UNSUPPORTED; }
+  if ((d->w_grid == 1 || d->w_grid == 2) && d->w_bits != 2) { *why = "w_grid 1 and 2 need w_bits 2"; return MREM_ERR_UNSUPPORTED; }
+  if (closed_form_weights(*d) && !d->w_step_per_row) { *why = "w_grid 2 and 3 (closed-form weight scales) work per output row"; return MREM_ERR_UNSUPPORTED; }
   if ((long long)d->max_batch * d->n_heads > 65535) { *why = "batch * heads too large"; return MREM_ERR_SHAPE; }
   return MREM_OK;
 }
@@ -185,7 +186,7 @@ int build_tables(mrem_ctx* c) {
       adam.push_back({b.student[k], g.p[k], g.m_p[k], g.v_p[k], (long long)r * q, mat ? 1.f : 0.f, -INFINITY});
       if (!mat) rest.push_back(adam.back());
     }
-    if ((d.trainable_mask & MREM_TRAIN_W_STEPS) && d.w_grid != 2)
+    if ((d.trainable_mask & MREM_TRAIN_W_STEPS) && !closed_form_weights(d))
       for (int k = 0; k < N_WMAT; ++k) {
         if (!b.w_steps[k]) return fail(c, MREM_ERR_ORDER, "weight steps not bound");
         adam.push_back({b.w_steps[k], g.ws[k], g.m_ws[k], g.v_ws[k], d.w_step_per_row ? c->wq[l][k].rows : 1, 0.f, 1e-8f});
@@ -345,9 +346,9 @@ int32_t mrem_get_grad(mrem_ctx* c, int32_t layer, int32_t id, const float** g) {
   if (layer < 0 || layer >= c->d.n_layers) return fail(c, MREM_ERR_ARG, "get_grad: bad layer");
   if (!c->have_grads) return fail(c, MREM_ERR_ORDER, "get_grad: no backward has run");
   const bool weight_id = (id >= 0 && id < MREM_N_PARAMS && kParamIsMatrix[id]) || (id >= MREM_GRAD_STEP && id < MREM_GRAD_STEP + N_WMAT);
-  if (c->d.w_grid == 2 && id >= MREM_GRAD_STEP && id < MREM_GRAD_STEP + N_WMAT)
+  if (closed_form_weights(c->d) && id >= MREM_GRAD_STEP && id < MREM_GRAD_STEP + N_WMAT)
     return fail(c, MREM_ERR_UNSUPPORTED, "get_grad: closed-form weight scales have no step gradient");
-  if (weight_id && !c->w_ste_done && c->d.w_grid != 2) {
+  if (weight_id && !c->w_ste_done && !closed_form_weights(c->d)) {
     // The backward leaves the matrices' gradients unmasked for the fused update; a caller who wants
     // to read them gets the straight-through masks and the step gradients applied now.
     TracerGuard tg(nullptr);
@@ -405,7 +406,7 @@ int32_t mrem_init_weight_steps(mrem_ctx* c, int32_t rule) {
   if (!c) return MREM_ERR_ARG;
   TracerGuard tg(nullptr);
   if (rule != 0 && rule != 1) return fail(c, MREM_ERR_ARG, "init_weight_steps: rule");
-  if (c->d.w_grid == 2) return MREM_OK;          // closed-form scales: nothing to initialise
+  if (closed_form_weights(c->d)) return MREM_OK;          // closed-form scales: nothing to initialise
   const float qmax = c->d.w_grid == 0 ? (float)((1 << (c->d.w_bits - 1)) - 1) : 1.5f;
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) {

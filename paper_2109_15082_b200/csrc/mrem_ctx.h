@@ -66,6 +66,9 @@ struct Arena {                          // bump allocator over the workspace (ba
 
 }  // namespace mrem
 
+// w_grid 2 and 3: the weight scales are recomputed from the weights by a fixed rule, no weight steps exist
+inline bool closed_form_weights(const mrem_module_desc& d) { return d.w_grid == 2 || d.w_grid == 3; }
+
 struct mrem_ctx {
   mrem_module_desc d;
   cudaStream_t stream = nullptr;

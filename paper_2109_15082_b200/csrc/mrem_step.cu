@@ -258,9 +258,9 @@ void enqueue_matrix_update(mrem_ctx* c, int l, int k, cudaStream_t st) {
   const int pid = kMatParam[k];
   WeightBuf& w = c->wq[l][k];
   LayerGrad& g = c->grad[l];
-  if (d.w_grid == 2) {
-    launch_ternary_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->optim_sc, w.rows, w.cols, train_w,
-                          w.codes, w.rowsum, w.scale, w.what, c->dt, st);
+  if (closed_form_weights(d)) {
+    launch_closed_form_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->optim_sc, w.rows, w.cols, train_w,
+                              d.w_grid, d.w_bits, w.codes, w.rowsum, w.scale, w.what, c->dt, st);
     return;
   }
   launch_fused_weight_update(c->bind[l].student[pid], g.p[pid], g.m_p[pid], g.v_p[pid], c->bind[l].w_steps[k],
@@ -438,10 +438,11 @@ int32_t mrem_quantize_weights(mrem_ctx* c) {
   for (int l = 0; l < c->d.n_layers; ++l)
     for (int k = 0; k < N_WMAT; ++k) {
       const LayerBind& b = c->bind[l];
-      if (!b.student[kMatParam[k]] || (!b.w_steps[k] && c->d.w_grid != 2)) return fail(c, MREM_ERR_ORDER, "quantize_weights: weights or steps not bound");
+      if (!b.student[kMatParam[k]] || (!b.w_steps[k] && !closed_form_weights(c->d))) return fail(c, MREM_ERR_ORDER, "quantize_weights: weights or steps not bound");
       WeightBuf& w = c->wq[l][k];
-      if (c->d.w_grid == 2) {
-        launch_ternary_quantize(b.student[kMatParam[k]], w.rows, w.cols, w.codes, w.rowsum, w.scale, w.what, c->dt, c->stream);
+      if (closed_form_weights(c->d)) {
+        launch_closed_form_quantize(b.student[kMatParam[k]], w.rows, w.cols, c->d.w_grid, c->d.w_bits, w.codes, w.rowsum,
+                                    w.scale, w.what, c->dt, c->stream);
         continue;
       }
       launch_quantize_weight(b.student[kMatParam[k]], w.rows, w.cols, b.w_steps[k], c->d.w_step_per_row, c->d.w_bits,
@@ -516,7 +517,7 @@ int32_t mrem_module_backward(mrem_ctx* c) {
   TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
   for (int l = 0; l < c->d.n_layers; ++l)
-    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k] && c->d.w_grid != 2) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
+    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k] && !closed_form_weights(c->d)) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   const int rc = student_backward(c, false);
   if (rc != MREM_OK) return rc;
@@ -536,7 +537,7 @@ int32_t mrem_backward_and_step(mrem_ctx* c, const mrem_optim* o) {
   TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_student || !c->have_loss) return fail(c, MREM_ERR_ORDER, "backward: needs forward(student) and recon_loss of this step");
   for (int l = 0; l < c->d.n_layers; ++l)
-    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k] && c->d.w_grid != 2) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
+    for (int k = 0; k < N_WMAT; ++k) if (!c->bind[l].w_steps[k] && !closed_form_weights(c->d)) return fail(c, MREM_ERR_ORDER, "backward: weight steps not bound");
   if (c->tables_dirty) { const int rc = build_tables(c); if (rc != MREM_OK) return rc; }
   launch_optim_prepare(c->optim_sc, c->t_counter, o->step, o->lr, o->decay_total_steps, o->beta1, o->beta2, o->eps,
                        o->weight_decay, c->stream);
@@ -599,10 +600,10 @@ int32_t mrem_rem_step(mrem_ctx* c, int32_t layer, int32_t tensor_id, const void*
   if (k < 0) return fail(c, MREM_ERR_ARG, "rem_step: tensor_id must name one of the four weight matrices");
   if (rows < 1 || rows > c->max_tokens) return fail(c, MREM_ERR_SHAPE, "rem_step: rows outside the context's maximum (max_batch * max_seq)");
   if (reinterpret_cast<uintptr_t>(a) & 15) return fail(c, MREM_ERR_ALIGN, "rem_step: d_a must be 16-byte aligned");
-  if (!d.w_step_per_row && d.w_grid != 2) return fail(c, MREM_ERR_UNSUPPORTED, "rem_step: needs per-row weight steps or the closed-form ternary weights");
+  if (!d.w_step_per_row && !closed_form_weights(d)) return fail(c, MREM_ERR_UNSUPPORTED, "rem_step: needs per-row weight steps or closed-form weight scales");
   const int site = k == W_QKV ? S_X : (k == W_O ? S_C : (k == W_1 ? S_A : S_G));
   const LayerBind& b = c->bind[layer];
-  if (!b.teacher[tensor_id] || !b.student[tensor_id] || (!b.w_steps[k] && d.w_grid != 2) || !b.a_steps[site])
+  if (!b.teacher[tensor_id] || !b.student[tensor_id] || (!b.w_steps[k] && !closed_form_weights(d)) || !b.a_steps[site])
     return fail(c, MREM_ERR_ORDER, "rem_step: parameters or steps not bound");
   const ActRange ar = site_range(d, site);
   if (ar.asym && !b.a_off[site]) return fail(c, MREM_ERR_ORDER, "rem_step: offset of the GELU-site quantizer not bound");

@@ -1,10 +1,17 @@
-// Closed-form ternary weights (the rule the paper names for 2-bit weights, Sec. 5.1), one block per
-// output row:  delta = 0.7 * mean|w|,  t = sign(w) * 1[|w| > delta],  alpha = mean of |w| over the kept
+// Weight codes whose scale is recomputed from the weights instead of learnt (Sec. 5.1 names one such rule for 2-bit
+// and one for 4-bit weights), one block per output row.
+//
+// Ternary rule (2-bit):  delta = 0.7 * mean|w|,  t = sign(w) * 1[|w| > delta],  alpha = mean of |w| over the kept
 // entries (0 when none is kept),  w_hat = alpha * t.  Nothing is learnt about the scale: the update is
 // AdamW on the latent weights with the gradient of w_hat passed through unchanged, followed by the same
 // rule on the new weights.  Both means are accumulated in float64 in a fixed order and the comparison
 // |w| > delta is made in float32 on float32(delta), so the codes are a function of the stored weights
 // alone.  Two kernels share the row routine: the stand-alone quantizer and the fused update.
+//
+// Refitted scale (b-bit, the loss-aware rule read with unit curvature weights): minimise ||w - alpha q||^2 over
+// alpha and q in Omega(b)^n by alternating the two exact half-steps  q = Pi_Omega(b)(w / alpha)  (Eq. 1, float32
+// division)  and  alpha = <q, w> / <q, q>  (float64 sums in a fixed order, alpha rounded to float32), LAQ_ROUNDS
+// times from alpha_0 = min(3 mean|w|, max|w|) / qmax; a row of zeros keeps alpha = 0 and codes 0.
 #include "optim.cuh"
 
 namespace mrem {
@@ -121,15 +128,105 @@ __device__ __forceinline__ void ternary_row(const float4* wr, bool cached, const
   }
 }
 
+constexpr int LAQ_ROUNDS = 16;
+
+__device__ __forceinline__ int laq_code(float w, float alpha, float qmax) {
+  return __float2int_rn(fminf(fmaxf(__fdiv_rn(w, alpha), -qmax), qmax));
+}
+
+// Block-wide sums of two doubles and the maximum of a float in one pass.  Every thread gets the results.
+__device__ __forceinline__ void block_sum2_d(double& a, double& b, double* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  a = warp_sum_d(a);
+  b = warp_sum_d(b);
+  __syncthreads();
+  if (lane == 0) { sh[w] = a; sh[32 + w] = b; }
+  __syncthreads();
+  a = warp_sum_d(lane < nw ? sh[lane] : 0.0);
+  b = warp_sum_d(lane < nw ? sh[32 + lane] : 0.0);
+}
+
+// The alternating rule on one row (same conventions as ternary_row).
 template <typename T>
-__global__ void __launch_bounds__(TW_THREADS) ternary_quantize_kernel(const float* __restrict__ w, int cols,
+__device__ __forceinline__ void laq_row(const float4* wr, bool cached, const float* w_row, int cols, int row, int bits,
+                                        int8_t* codes_row, int32_t* rowsum, float* scale, T* what_row, double* shd,
+                                        int* shi, float* shf) {
+  const int nvec = cols / 4;
+  const float qmax = (float)((1 << (bits - 1)) - 1);
+  auto for_row = [&](auto&& f) {
+    if (cached) {
+#pragma unroll
+      for (int i = 0; i < TW_MAXV; ++i) {
+        const int c = threadIdx.x + i * TW_THREADS;
+        if (c < nvec) f(c, wr[i]);
+      }
+    } else {
+      for (int c = threadIdx.x; c < nvec; c += TW_THREADS) f(c, reinterpret_cast<const float4*>(w_row)[c]);
+    }
+  };
+  double s = 0.0;
+  float mx = 0.f;
+  for_row([&](int, float4 v) {
+    s += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
+    mx = fmaxf(fmaxf(mx, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+  });
+  s = block_sum_d(s, shd);
+  mx = block_max(mx, shf);
+  float alpha = (float)(fmin(3.0 * (s / (double)cols), (double)mx) / (double)qmax);
+  for (int r = 0; r < LAQ_ROUNDS; ++r) {
+    double qw = 0.0, qq = 0.0;
+    if (alpha > 0.f) {
+      for_row([&](int, float4 v) {
+        const int q0 = laq_code(v.x, alpha, qmax), q1 = laq_code(v.y, alpha, qmax), q2 = laq_code(v.z, alpha, qmax),
+                  q3 = laq_code(v.w, alpha, qmax);
+        qw += (double)q0 * (double)v.x + (double)q1 * (double)v.y + (double)q2 * (double)v.z + (double)q3 * (double)v.w;
+        qq += (double)(q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3);
+      });
+    }
+    block_sum2_d(qw, qq, shd);
+    const float next = qq > 0.0 ? (float)(qw / qq) : 0.f;
+    if (r + 1 < LAQ_ROUNDS) { alpha = next; continue; }
+    // last round: the codes of this alpha go out with the refitted scale
+    int sum = 0;
+    const float a_in = alpha;
+    for_row([&](int c, float4 v) {
+      int q0 = 0, q1 = 0, q2 = 0, q3 = 0;
+      if (a_in > 0.f) {
+        q0 = laq_code(v.x, a_in, qmax); q1 = laq_code(v.y, a_in, qmax);
+        q2 = laq_code(v.z, a_in, qmax); q3 = laq_code(v.w, a_in, qmax);
+      }
+      *reinterpret_cast<uint32_t*>(codes_row + 4 * c) =
+          (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) | ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
+      if (what_row) store4<T>(what_row + 4 * c, next * (float)q0, next * (float)q1, next * (float)q2, next * (float)q3);
+      sum += q0 + q1 + q2 + q3;
+    });
+    sum = block_sum_i(sum, shi);
+    if (threadIdx.x == 0) {
+      rowsum[row] = sum;
+      scale[row] = next;
+    }
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void closed_form_row(int rule, const float4* wr, bool cached, const float* w_row, int cols,
+                                                int row, int bits, int8_t* codes_row, int32_t* rowsum, float* scale,
+                                                T* what_row, double* shd, int* shi, float* shf) {
+  if (rule == 3) laq_row<T>(wr, cached, w_row, cols, row, bits, codes_row, rowsum, scale, what_row, shd, shi, shf);
+  else ternary_row<T>(wr, cached, w_row, cols, row, codes_row, rowsum, scale, what_row, shd, shi);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(TW_THREADS) closed_form_quantize_kernel(const float* __restrict__ w, int cols,
+                                                                      int rule, int bits,
                                                                       int8_t* __restrict__ codes,
                                                                       int32_t* __restrict__ rowsum,
                                                                       float* __restrict__ scale, T* __restrict__ what) {
   pdl_trigger();
   pdl_wait();
-  __shared__ double shd[32];
+  __shared__ double shd[64];
   __shared__ int shi[32];
+  __shared__ float shf[32];
   const int row = blockIdx.x;
   const long long base = (long long)row * cols;
   const int nvec = cols / 4;
@@ -142,21 +239,24 @@ __global__ void __launch_bounds__(TW_THREADS) ternary_quantize_kernel(const floa
       if (c < nvec) wr[i] = reinterpret_cast<const float4*>(w + base)[c];
     }
   }
-  ternary_row<T>(wr, cached, w + base, cols, row, codes + base, rowsum, scale, what ? what + base : nullptr, shd, shi);
+  closed_form_row<T>(rule, wr, cached, w + base, cols, row, bits, codes + base, rowsum, scale,
+                     what ? what + base : nullptr, shd, shi, shf);
 }
 
 // AdamW on the row (gradient of w_hat passed through unchanged), then the rule on the new weights.
 template <typename T>
-__global__ void __launch_bounds__(TW_THREADS) ternary_update_kernel(float* __restrict__ w, const float* __restrict__ g,
+__global__ void __launch_bounds__(TW_THREADS) closed_form_update_kernel(float* __restrict__ w, const float* __restrict__ g,
                                                                     float* __restrict__ m, float* __restrict__ v,
                                                                     const OptimScalars* __restrict__ sc, int cols,
-                                                                    int train_w, int8_t* __restrict__ codes,
+                                                                    int train_w, int rule, int bits,
+                                                                    int8_t* __restrict__ codes,
                                                                     int32_t* __restrict__ rowsum,
                                                                     float* __restrict__ scale, T* __restrict__ what) {
   pdl_trigger();
   pdl_wait();
-  __shared__ double shd[32];
+  __shared__ double shd[64];
   __shared__ int shi[32];
+  __shared__ float shf[32];
   const int row = blockIdx.x;
   const OptimScalars o = *sc;
   const long long base = (long long)row * cols;
@@ -192,24 +292,25 @@ __global__ void __launch_bounds__(TW_THREADS) ternary_update_kernel(float* __res
     for (int c = threadIdx.x; c < nvec; c += TW_THREADS) upd(c);
     __syncthreads();                     // the row is re-read below by other threads of the block
   }
-  ternary_row<T>(wr, cached, w + base, cols, row, codes + base, rowsum, scale, what ? what + base : nullptr, shd, shi);
+  closed_form_row<T>(rule, wr, cached, w + base, cols, row, bits, codes + base, rowsum, scale,
+                     what ? what + base : nullptr, shd, shi, shf);
 }
 
 }  // namespace
 
-void launch_ternary_quantize(const float* w, int rows, int cols, int8_t* codes, int32_t* rowsum, float* scale,
-                             void* what, int dt, cudaStream_t st) {
+void launch_closed_form_quantize(const float* w, int rows, int cols, int rule, int bits, int8_t* codes, int32_t* rowsum,
+                                 float* scale, void* what, int dt, cudaStream_t st) {
   Scope sc("quantize_weight", (double)rows * cols * (5.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)) + rows * 8.0, 0, st);
-  if (dt == 1) launch_k(ternary_quantize_kernel<bf16>, rows, TW_THREADS, 0, st, w, cols, codes, rowsum, scale, (bf16*)what);
-  else launch_k(ternary_quantize_kernel<float>, rows, TW_THREADS, 0, st, w, cols, codes, rowsum, scale, (float*)what);
+  if (dt == 1) launch_k(closed_form_quantize_kernel<bf16>, rows, TW_THREADS, 0, st, w, cols, rule, bits, codes, rowsum, scale, (bf16*)what);
+  else launch_k(closed_form_quantize_kernel<float>, rows, TW_THREADS, 0, st, w, cols, rule, bits, codes, rowsum, scale, (float*)what);
 }
 
-void launch_ternary_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
-                           int train_w, int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt,
+void launch_closed_form_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
+                               int train_w, int rule, int bits, int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt,
                            cudaStream_t st) {
   Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
-  if (dt == 1) launch_k(ternary_update_kernel<bf16>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, codes, rowsum, scale, (bf16*)what);
-  else launch_k(ternary_update_kernel<float>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, codes, rowsum, scale, (float*)what);
+  if (dt == 1) launch_k(closed_form_update_kernel<bf16>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, rule, bits, codes, rowsum, scale, (bf16*)what);
+  else launch_k(closed_form_update_kernel<float>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, rule, bits, codes, rowsum, scale, (float*)what);
 }
 
 }  // namespace mrem

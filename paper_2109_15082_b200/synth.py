@@ -87,7 +87,7 @@ class Workload:
     batch: int
     w_bits: int = 4
     a_bits: int = 8
-    w_grid: int = 0            # 0: integer grid Omega(b) of Eq. 1; 1: half-integer 2-bit grid
+    w_grid: int = 0            # 0: integer grid Omega(b) of Eq. 1; 1: half-integer 2-bit grid; 2 / 3: closed-form scales
     act_dtype: str = "bf16"    # storage type of activations
     outlier_channels: int = 4  # channels of the input scaled by outlier_scale
     outlier_scale: float = 20.0

@@ -26,9 +26,10 @@ class Problem:
         a_bits = a_bits or wl.a_bits
         self.m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, wl.w_bits, a_bits,
                              wl.w_grid, w_per_row, asym, wl.act_dtype, loss_mean)
-        self.twn = wl.w_grid == 2                                    # closed-form ternary weights: no weight steps
+        self.twn = wl.w_grid in (2, 3)                               # closed-form weight scales: no weight steps
         self.desc = O.ModuleDesc(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.w_bits, a_bits, 0 if self.twn else wl.w_grid,
-                                 w_per_row, bool(asym & 1), bool(asym & 2), wl.act_dtype, loss_mean, w_twn=self.twn)
+                                 w_per_row, bool(asym & 1), bool(asym & 2), wl.act_dtype, loss_mean,
+                                 w_twn=wl.w_grid == 2, w_laq=wl.w_grid == 3)
         m = self.m
         m.load_teacher(synth.teacher_params(wl, seed, bias_std=bias_std))
         m.init_student_from_teacher()

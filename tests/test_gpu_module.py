@@ -708,25 +708,43 @@ def test_degenerate_inputs_match_the_oracle():
         p.close()
 
 
-def test_closed_form_ternary_weights_match_the_oracle():
-    """w_grid = 2: ternary codes and scales by the closed-form rule.  Codes bit exact before the step and, from the
-    updated weights, after it; forward, loss and every gradient against the oracle; no weight-step gradient."""
-    wl = _wl("base3_w2a8", n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40, w_grid=2)
+_BF16_SMALL = dict(n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40)
+_refit = lambda w, bits: O.quantize_weight_laq(w, bits, True)[0]
+# name: (workload, its changes, the code values that must occur, the oracle's quantizer, gradient bound, scalar bound).
+# The float32-storage case holds every gradient to 2e-3: the arithmetic is the oracle's.  With bf16 storage the
+# refitted scales leave a much smaller reconstruction error than the threshold rule or a min-max step, so the rounding
+# of the stored activations weighs more in the heavily cancelling sums behind the activation-step gradients (scalars).
+CLOSED_FORM = {
+    "ternary": ("base3_w2a8", dict(_BF16_SMALL, w_grid=2), {-1, 0, 1}, lambda w, bits: O.quantize_weight_twn(w, True)[0], GRAD_TOL, None),
+    "refit_w4": ("base3_w2a8", dict(_BF16_SMALL, w_grid=3, w_bits=4), set(range(-7, 8)), _refit, GRAD_TOL, 0.1),
+    "refit_w2": ("base3_w2a8", dict(_BF16_SMALL, w_grid=3, w_bits=2), {-1, 0, 1}, _refit, GRAD_TOL, 0.1),
+    "refit_w4_f32": ("tiny", dict(n_layers=2, batch=3, len_lo=9, len_hi=32, w_grid=3, w_bits=4), set(range(-7, 8)), _refit, 2e-3, None),
+}
+
+
+@pytest.mark.parametrize("case", sorted(CLOSED_FORM))
+def test_closed_form_weight_scales_match_the_oracle(case):
+    """w_grid = 2 (ternary codes by the threshold rule) and w_grid = 3 (codes in Omega(b) with the scale refitted by
+    alternating least squares).  Codes and row sums bit exact before the step and, from the updated weights, after
+    it; scales, forward, loss and every gradient against the oracle; no weight-step gradient."""
+    base, kw, levels, quantizer, tol, scalar_tol = CLOSED_FORM[case]
+    wl = _wl(base, **kw)
     p = Problem(wl, student_noise=0.002)
     try:
         m = p.m
         g = p.run_gpu()
         r = p.run_oracle()
         for l in range(wl.n_layers):
-            assert rel(g["f_t"][l], r["f_t"][l]) < FWD_TOL["bf16"] and rel(g["f_s"][l], r["f_s"][l]) < FWD_TOL["bf16"]
+            assert rel(g["f_t"][l], r["f_t"][l]) < FWD_TOL[wl.act_dtype] and rel(g["f_s"][l], r["f_s"][l]) < FWD_TOL[wl.act_dtype]
             for pid, name in ((B.WQKV, "Wqkv"), (B.WO, "Wo"), (B.W1, "W1"), (B.W2, "W2")):
                 codes, rowsum = m.weight_codes(l, pid)
                 ref = r["caches"][l]["qw"][name]["q"]
                 assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref)
                 assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1))
-                assert set(np.unique(ref)) == {-1, 0, 1}
-        assert abs(g["loss"] - r["loss"]) / r["loss"] < GRAD_TOL
-        compare_grads(g["grads"], r["grads"], GRAD_TOL, check_offset=False)
+                assert set(np.unique(ref)) == levels
+        assert abs(g["loss"] - r["loss"]) / r["loss"] < tol
+        worst = compare_grads(g["grads"], r["grads"], tol, check_offset=False, scalar_tol=scalar_tol)
+        print(case, "loss", g["loss"], r["loss"], "worst grad", worst)
         with pytest.raises(B.MremError):
             m.grad(0, B.GRAD_STEP + 0, (1,))
         before = m.student_numpy()
@@ -741,8 +759,9 @@ def test_closed_form_ternary_weights_match_the_oracle():
                 ref_w, _, _ = O.adamw_update(before[l][name], grads[l][name], z, z.copy(), 1, opt["lr"], 0.9, 0.999, 1e-8, 0.01)
                 assert np.allclose(after[l][name], ref_w, rtol=1e-5, atol=2e-3 * opt["lr"])
                 codes, rowsum = m.weight_codes(l, pid)
-                ref = O.quantize_weight_twn(after[l][name], True)[0]
+                ref = quantizer(after[l][name], wl.w_bits)
                 assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref), (l, name)
+                assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1))
         # and the next forward runs on the new codes
         g2 = p.run_gpu()
         assert np.isfinite(g2["loss"]) and g2["loss"] != g["loss"]
