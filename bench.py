@@ -222,6 +222,23 @@ def time_extras(m, wl, xbuf, lenbuf, stream, torch, B, pk, reps=10):
     out["embed_step"] = {"vocab": V, "tokens": rows, "e_bits": 4, "ms_per_step": ms, "table_gbs": table_bytes / (ms * 1e-3) / 1e9,
                          "hbm_peak_gbs": pk["hbm_gbs"], "status": int(emb.status[0]),
                          "note": "whole step; table_gbs counts only the dense pass over the word table (33 B per entry)"}
+    # the module step with weight scales recomputed from the weights (w_grid 3: refitted W4 scales; w_grid 2: ternary)
+    from paper_2109_15082_b200 import synth as _synth
+    from paper_2109_15082_b200.session import ReconModule as _RM
+    cf = {}
+    for label, grid, bits in (("refit_w4", 3, 4), ("ternary_w2", 2, 2)):
+        with torch.cuda.stream(stream):
+            mc = _RM(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, wl.batch, bits, wl.a_bits, grid, True, 3, wl.act_dtype,
+                     stream=stream)
+            mc.load_teacher(_synth.teacher_params(wl, seed=7))
+            mc.init_student_from_teacher()
+            mc.init_act_steps(xbuf, lenbuf, wl.batch, wl.seq)
+            stream.synchronize()
+            B.mrem_graph_capture_step(mc.ctx, xbuf, xbuf, 0.0, lenbuf, wl.batch, wl.seq, mc.t_out, mc.s_out, mc.loss, opt)
+            ms = timed(lambda: B.mrem_graph_launch(mc.ctx), n=20)
+            cf[label] = {"ms_per_step": ms, "tokens_per_s": rows / (ms * 1e-3), "loss": float(mc.loss[:1].item())}
+            mc.close()
+    out["closed_form_scales"] = cf
     # the whole sequential sweep of the stated BERT-large configuration: 4 modules of the workload's depth one after the
     # other, 200 steps each over a 1024-sequence calibration set, outputs cached for the next module (wall clock,
     # synchronised at both ends; includes step initialisation, graph capture and the caching passes)

@@ -18,8 +18,12 @@ namespace mrem {
 
 namespace {
 
+// Threads per row (NT) and float4 vectors per thread kept in registers (MAXV): a block of 256 threads with 4 vectors
+// each holds rows up to 4096 wide; the alternating rule takes one warp with 8 vectors per lane for rows up to 1024
+// wide, where its 16 dependent reductions then need no block barrier.
 constexpr int TW_THREADS = 256;
-constexpr int TW_MAXV = 4;                 // float4 vectors per thread kept in registers: rows up to 4096 wide
+constexpr int TW_MAXV = 4;
+constexpr int TW_WARP_MAXV = 8;
 
 __device__ __forceinline__ double warp_sum_d(double v) {
 #pragma unroll
@@ -62,9 +66,9 @@ __device__ __forceinline__ void store4<bf16>(bf16* p, float a, float b, float c,
 
 __device__ __forceinline__ int tern(float w, float delta) { return fabsf(w) > delta ? (w > 0.f ? 1 : -1) : 0; }
 
-// The rule on one row.  `cached`: the row sits in wr[] (vector c = threadIdx.x + i * TW_THREADS), else it is re-read
+// The rule on one row.  `cached`: the row sits in wr[] (vector c = threadIdx.x + i * NT), else it is re-read
 // from w_row.  Writes codes, row sum, scale and the dequantized row.
-template <typename T>
+template <typename T, int NT, int MAXV>
 __device__ __forceinline__ void ternary_row(const float4* wr, bool cached, const float* w_row, int cols, int row,
                                             int8_t* codes_row, int32_t* rowsum, float* scale, T* what_row,
                                             double* shd, int* shi) {
@@ -72,12 +76,12 @@ __device__ __forceinline__ void ternary_row(const float4* wr, bool cached, const
   double s = 0.0;
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < TW_MAXV; ++i) {
-      const int c = threadIdx.x + i * TW_THREADS;
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) s += (double)fabsf(wr[i].x) + (double)fabsf(wr[i].y) + (double)fabsf(wr[i].z) + (double)fabsf(wr[i].w);
     }
   } else {
-    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) {
+    for (int c = threadIdx.x; c < nvec; c += NT) {
       const float4 v = reinterpret_cast<const float4*>(w_row)[c];
       s += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
     }
@@ -94,12 +98,12 @@ __device__ __forceinline__ void ternary_row(const float4* wr, bool cached, const
   };
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < TW_MAXV; ++i) {
-      const int c = threadIdx.x + i * TW_THREADS;
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) acc(wr[i]);
     }
   } else {
-    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) acc(reinterpret_cast<const float4*>(w_row)[c]);
+    for (int c = threadIdx.x; c < nvec; c += NT) acc(reinterpret_cast<const float4*>(w_row)[c]);
   }
   ks = block_sum_d(ks, shd);
   cnt = block_sum_i(cnt, shi);
@@ -114,12 +118,12 @@ __device__ __forceinline__ void ternary_row(const float4* wr, bool cached, const
   };
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < TW_MAXV; ++i) {
-      const int c = threadIdx.x + i * TW_THREADS;
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) emit(c, wr[i]);
     }
   } else {
-    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) emit(c, reinterpret_cast<const float4*>(w_row)[c]);
+    for (int c = threadIdx.x; c < nvec; c += NT) emit(c, reinterpret_cast<const float4*>(w_row)[c]);
   }
   sum = block_sum_i(sum, shi);
   if (threadIdx.x == 0) {
@@ -133,21 +137,31 @@ constexpr int LAQ_ROUNDS = 16;
 __device__ __forceinline__ int laq_code(float w, float alpha, float qmax) {
   return __float2int_rn(fminf(fmaxf(__fdiv_rn(w, alpha), -qmax), qmax));
 }
+// The same code from RN(1 / alpha): quotient() differs from the division only where w / alpha lies within 2^-48
+// (relative) of the midpoint of two floats, and the code differs only if that quotient is also next to a half-integer.
+// Used in the rounds that only feed the two sums; the codes that are written out come from the division.
+__device__ __forceinline__ int laq_code_fast(float w, float alpha, float r_alpha, float qmax) {
+  return __float2int_rn(fminf(fmaxf(quotient(w, alpha, r_alpha), -qmax), qmax));
+}
+// (double)q for |q| < 2^31 without the conversion unit: 2^52 + 2^31 + q is exact in the low word of a double.
+__device__ __forceinline__ double int_as_double(int q) {
+  return __hiloint2double(0x43300000, (int)(0x80000000u ^ (unsigned)q)) - 4503601774854144.0;
+}
 
-// Block-wide sums of two doubles and the maximum of a float in one pass.  Every thread gets the results.
-__device__ __forceinline__ void block_sum2_d(double& a, double& b, double* sh) {
+// Block-wide sum of a double and of an int in one pass.  Every thread gets the results.
+__device__ __forceinline__ void block_sum_di(double& a, int& n, double* shd, int* shi) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
   a = warp_sum_d(a);
-  b = warp_sum_d(b);
+  n = __reduce_add_sync(0xffffffffu, n);
   __syncthreads();
-  if (lane == 0) { sh[w] = a; sh[32 + w] = b; }
+  if (lane == 0) { shd[w] = a; shi[w] = n; }
   __syncthreads();
-  a = warp_sum_d(lane < nw ? sh[lane] : 0.0);
-  b = warp_sum_d(lane < nw ? sh[32 + lane] : 0.0);
+  a = warp_sum_d(lane < nw ? shd[lane] : 0.0);
+  n = __reduce_add_sync(0xffffffffu, lane < nw ? shi[lane] : 0);
 }
 
 // The alternating rule on one row (same conventions as ternary_row).
-template <typename T>
+template <typename T, int NT, int MAXV>
 __device__ __forceinline__ void laq_row(const float4* wr, bool cached, const float* w_row, int cols, int row, int bits,
                                         int8_t* codes_row, int32_t* rowsum, float* scale, T* what_row, double* shd,
                                         int* shi, float* shf) {
@@ -156,12 +170,12 @@ __device__ __forceinline__ void laq_row(const float4* wr, bool cached, const flo
   auto for_row = [&](auto&& f) {
     if (cached) {
 #pragma unroll
-      for (int i = 0; i < TW_MAXV; ++i) {
-        const int c = threadIdx.x + i * TW_THREADS;
+      for (int i = 0; i < MAXV; ++i) {
+        const int c = threadIdx.x + i * NT;
         if (c < nvec) f(c, wr[i]);
       }
     } else {
-      for (int c = threadIdx.x; c < nvec; c += TW_THREADS) f(c, reinterpret_cast<const float4*>(w_row)[c]);
+      for (int c = threadIdx.x; c < nvec; c += NT) f(c, reinterpret_cast<const float4*>(w_row)[c]);
     }
   };
   double s = 0.0;
@@ -173,52 +187,83 @@ __device__ __forceinline__ void laq_row(const float4* wr, bool cached, const flo
   s = block_sum_d(s, shd);
   mx = block_max(mx, shf);
   float alpha = (float)(fmin(3.0 * (s / (double)cols), (double)mx) / (double)qmax);
-  for (int r = 0; r < LAQ_ROUNDS; ++r) {
-    double qw = 0.0, qq = 0.0;
+  for (int r = 0; r + 1 < LAQ_ROUNDS; ++r) {
+    double qw = 0.0, qw1 = 0.0, qw2 = 0.0, qw3 = 0.0;
+    int qq = 0;
     if (alpha > 0.f) {
-      for_row([&](int, float4 v) {
-        const int q0 = laq_code(v.x, alpha, qmax), q1 = laq_code(v.y, alpha, qmax), q2 = laq_code(v.z, alpha, qmax),
-                  q3 = laq_code(v.w, alpha, qmax);
-        qw += (double)q0 * (double)v.x + (double)q1 * (double)v.y + (double)q2 * (double)v.z + (double)q3 * (double)v.w;
-        qq += (double)(q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3);
-      });
-    }
-    block_sum2_d(qw, qq, shd);
-    const float next = qq > 0.0 ? (float)(qw / qq) : 0.f;
-    if (r + 1 < LAQ_ROUNDS) { alpha = next; continue; }
-    // last round: the codes of this alpha go out with the refitted scale
-    int sum = 0;
-    const float a_in = alpha;
-    for_row([&](int c, float4 v) {
-      int q0 = 0, q1 = 0, q2 = 0, q3 = 0;
-      if (a_in > 0.f) {
-        q0 = laq_code(v.x, a_in, qmax); q1 = laq_code(v.y, a_in, qmax);
-        q2 = laq_code(v.z, a_in, qmax); q3 = laq_code(v.w, a_in, qmax);
+      const bool fast = alpha > 1e-30f;                      // 1 / alpha and the residual stay in the normal range
+      const float r_alpha = __frcp_rn(alpha);
+      auto code = [&](float w) { return fast ? laq_code_fast(w, alpha, r_alpha, qmax) : laq_code(w, alpha, qmax); };
+      if (cached) {
+#pragma unroll
+        for (int i = 0; i < MAXV; ++i) {
+          if (threadIdx.x + i * NT < nvec) {
+            const int q0 = code(wr[i].x), q1 = code(wr[i].y), q2 = code(wr[i].z), q3 = code(wr[i].w);
+            qw = fma(int_as_double(q0), (double)wr[i].x, qw);        // four independent chains
+            qw1 = fma(int_as_double(q1), (double)wr[i].y, qw1);
+            qw2 = fma(int_as_double(q2), (double)wr[i].z, qw2);
+            qw3 = fma(int_as_double(q3), (double)wr[i].w, qw3);
+            qq += q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
+          }
+        }
+      } else {
+        for (int c = threadIdx.x; c < nvec; c += NT) {
+          const float4 v = reinterpret_cast<const float4*>(w_row)[c];
+          const int q0 = code(v.x), q1 = code(v.y), q2 = code(v.z), q3 = code(v.w);
+          qw = fma(int_as_double(q0), (double)v.x, qw);
+          qw1 = fma(int_as_double(q1), (double)v.y, qw1);
+          qw2 = fma(int_as_double(q2), (double)v.z, qw2);
+          qw3 = fma(int_as_double(q3), (double)v.w, qw3);
+          qq += q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
+        }
       }
-      *reinterpret_cast<uint32_t*>(codes_row + 4 * c) =
-          (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) | ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
-      if (what_row) store4<T>(what_row + 4 * c, next * (float)q0, next * (float)q1, next * (float)q2, next * (float)q3);
-      sum += q0 + q1 + q2 + q3;
-    });
-    sum = block_sum_i(sum, shi);
-    if (threadIdx.x == 0) {
-      rowsum[row] = sum;
-      scale[row] = next;
     }
+    qw = (qw + qw1) + (qw2 + qw3);
+    block_sum_di(qw, qq, shd, shi);
+    alpha = qq > 0 ? (float)(qw / (double)qq) : 0.f;
+  }
+  // last round: the codes of this alpha (by the division of Eq. 1) go out with the scale refitted to them
+  double qw = 0.0;
+  int qq = 0, sum = 0;
+  for_row([&](int c, float4 v) {
+    int q0 = 0, q1 = 0, q2 = 0, q3 = 0;
+    if (alpha > 0.f) {
+      q0 = laq_code(v.x, alpha, qmax); q1 = laq_code(v.y, alpha, qmax);
+      q2 = laq_code(v.z, alpha, qmax); q3 = laq_code(v.w, alpha, qmax);
+    }
+    qw += (double)q0 * (double)v.x + (double)q1 * (double)v.y + (double)q2 * (double)v.z + (double)q3 * (double)v.w;
+    qq += q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
+    sum += q0 + q1 + q2 + q3;
+    *reinterpret_cast<uint32_t*>(codes_row + 4 * c) =
+        (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) | ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
+  });
+  block_sum_di(qw, qq, shd, shi);
+  const float next = qq > 0 ? (float)(qw / (double)qq) : 0.f;
+  if (what_row) {
+    auto unpack = [](uint32_t pk, int j) { return (float)(int)(int8_t)(pk >> (8 * j)); };
+    for (int c = threadIdx.x; c < nvec; c += NT) {        // this thread's own codes, written above
+      const uint32_t pk = *reinterpret_cast<const uint32_t*>(codes_row + 4 * c);
+      store4<T>(what_row + 4 * c, next * unpack(pk, 0), next * unpack(pk, 1), next * unpack(pk, 2), next * unpack(pk, 3));
+    }
+  }
+  sum = block_sum_i(sum, shi);
+  if (threadIdx.x == 0) {
+    rowsum[row] = sum;
+    scale[row] = next;
   }
 }
 
-template <typename T>
-__device__ __forceinline__ void closed_form_row(int rule, const float4* wr, bool cached, const float* w_row, int cols,
+template <typename T, int RULE, int NT, int MAXV>
+__device__ __forceinline__ void closed_form_row(const float4* wr, bool cached, const float* w_row, int cols,
                                                 int row, int bits, int8_t* codes_row, int32_t* rowsum, float* scale,
                                                 T* what_row, double* shd, int* shi, float* shf) {
-  if (rule == 3) laq_row<T>(wr, cached, w_row, cols, row, bits, codes_row, rowsum, scale, what_row, shd, shi, shf);
-  else ternary_row<T>(wr, cached, w_row, cols, row, codes_row, rowsum, scale, what_row, shd, shi);
+  if (RULE == 3) laq_row<T, NT, MAXV>(wr, cached, w_row, cols, row, bits, codes_row, rowsum, scale, what_row, shd, shi, shf);
+  else ternary_row<T, NT, MAXV>(wr, cached, w_row, cols, row, codes_row, rowsum, scale, what_row, shd, shi);
 }
 
-template <typename T>
-__global__ void __launch_bounds__(TW_THREADS) closed_form_quantize_kernel(const float* __restrict__ w, int cols,
-                                                                      int rule, int bits,
+template <typename T, int RULE, int NT, int MAXV>
+__global__ void __launch_bounds__(NT, NT == 32 ? 20 : (RULE == 2 ? 5 : 4)) closed_form_quantize_kernel(const float* __restrict__ w, int cols,
+                                                                      int bits,
                                                                       int8_t* __restrict__ codes,
                                                                       int32_t* __restrict__ rowsum,
                                                                       float* __restrict__ scale, T* __restrict__ what) {
@@ -230,25 +275,25 @@ __global__ void __launch_bounds__(TW_THREADS) closed_form_quantize_kernel(const 
   const int row = blockIdx.x;
   const long long base = (long long)row * cols;
   const int nvec = cols / 4;
-  const bool cached = nvec <= TW_MAXV * TW_THREADS;
-  float4 wr[TW_MAXV];
+  const bool cached = nvec <= MAXV * NT;
+  float4 wr[MAXV];
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < TW_MAXV; ++i) {
-      const int c = threadIdx.x + i * TW_THREADS;
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) wr[i] = reinterpret_cast<const float4*>(w + base)[c];
     }
   }
-  closed_form_row<T>(rule, wr, cached, w + base, cols, row, bits, codes + base, rowsum, scale,
+  closed_form_row<T, RULE, NT, MAXV>(wr, cached, w + base, cols, row, bits, codes + base, rowsum, scale,
                      what ? what + base : nullptr, shd, shi, shf);
 }
 
 // AdamW on the row (gradient of w_hat passed through unchanged), then the rule on the new weights.
-template <typename T>
-__global__ void __launch_bounds__(TW_THREADS) closed_form_update_kernel(float* __restrict__ w, const float* __restrict__ g,
+template <typename T, int RULE, int NT, int MAXV>
+__global__ void __launch_bounds__(NT, NT == 32 ? 20 : (RULE == 2 ? 5 : 4)) closed_form_update_kernel(float* __restrict__ w, const float* __restrict__ g,
                                                                     float* __restrict__ m, float* __restrict__ v,
                                                                     const OptimScalars* __restrict__ sc, int cols,
-                                                                    int train_w, int rule, int bits,
+                                                                    int train_w, int bits,
                                                                     int8_t* __restrict__ codes,
                                                                     int32_t* __restrict__ rowsum,
                                                                     float* __restrict__ scale, T* __restrict__ what) {
@@ -261,12 +306,12 @@ __global__ void __launch_bounds__(TW_THREADS) closed_form_update_kernel(float* _
   const OptimScalars o = *sc;
   const long long base = (long long)row * cols;
   const int nvec = cols / 4;
-  const bool cached = nvec <= TW_MAXV * TW_THREADS;
+  const bool cached = nvec <= MAXV * NT;
   float4* w4 = reinterpret_cast<float4*>(w + base);
   const float4* g4 = reinterpret_cast<const float4*>(g + base);
   float4* m4 = reinterpret_cast<float4*>(m + base);
   float4* v4 = reinterpret_cast<float4*>(v + base);
-  float4 wr[TW_MAXV];
+  float4 wr[MAXV];
   auto upd = [&](int c) {
     float4 wv = w4[c];
     if (train_w) {
@@ -284,15 +329,15 @@ __global__ void __launch_bounds__(TW_THREADS) closed_form_update_kernel(float* _
   };
   if (cached) {
 #pragma unroll
-    for (int i = 0; i < TW_MAXV; ++i) {
-      const int c = threadIdx.x + i * TW_THREADS;
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = threadIdx.x + i * NT;
       if (c < nvec) wr[i] = upd(c);
     }
   } else {
-    for (int c = threadIdx.x; c < nvec; c += TW_THREADS) upd(c);
+    for (int c = threadIdx.x; c < nvec; c += NT) upd(c);
     __syncthreads();                     // the row is re-read below by other threads of the block
   }
-  closed_form_row<T>(rule, wr, cached, w + base, cols, row, bits, codes + base, rowsum, scale,
+  closed_form_row<T, RULE, NT, MAXV>(wr, cached, w + base, cols, row, bits, codes + base, rowsum, scale,
                      what ? what + base : nullptr, shd, shi, shf);
 }
 
@@ -301,16 +346,36 @@ __global__ void __launch_bounds__(TW_THREADS) closed_form_update_kernel(float* _
 void launch_closed_form_quantize(const float* w, int rows, int cols, int rule, int bits, int8_t* codes, int32_t* rowsum,
                                  float* scale, void* what, int dt, cudaStream_t st) {
   Scope sc("quantize_weight", (double)rows * cols * (5.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)) + rows * 8.0, 0, st);
-  if (dt == 1) launch_k(closed_form_quantize_kernel<bf16>, rows, TW_THREADS, 0, st, w, cols, rule, bits, codes, rowsum, scale, (bf16*)what);
-  else launch_k(closed_form_quantize_kernel<float>, rows, TW_THREADS, 0, st, w, cols, rule, bits, codes, rowsum, scale, (float*)what);
+  auto go = [&](auto kernel, int nt, auto* out) { launch_k(kernel, rows, nt, 0, st, w, cols, bits, codes, rowsum, scale, out); };
+  const bool warp_rows = rule == 3 && cols <= 32 * 4 * TW_WARP_MAXV;
+  if (dt == 1) {
+    if (warp_rows) go(closed_form_quantize_kernel<bf16, 3, 32, TW_WARP_MAXV>, 32, (bf16*)what);
+    else if (rule == 3) go(closed_form_quantize_kernel<bf16, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
+    else go(closed_form_quantize_kernel<bf16, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
+  } else {
+    if (warp_rows) go(closed_form_quantize_kernel<float, 3, 32, TW_WARP_MAXV>, 32, (float*)what);
+    else if (rule == 3) go(closed_form_quantize_kernel<float, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
+    else go(closed_form_quantize_kernel<float, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
+  }
 }
 
 void launch_closed_form_update(float* w, const float* g, float* m, float* v, const OptimScalars* sc, int rows, int cols,
-                               int train_w, int rule, int bits, int8_t* codes, int32_t* rowsum, float* scale, void* what, int dt,
-                           cudaStream_t st) {
+                               int train_w, int rule, int bits, int8_t* codes, int32_t* rowsum, float* scale, void* what,
+                               int dt, cudaStream_t st) {
   Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
-  if (dt == 1) launch_k(closed_form_update_kernel<bf16>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, rule, bits, codes, rowsum, scale, (bf16*)what);
-  else launch_k(closed_form_update_kernel<float>, rows, TW_THREADS, 0, st, w, g, m, v, sc, cols, train_w, rule, bits, codes, rowsum, scale, (float*)what);
+  auto go = [&](auto kernel, int nt, auto* out) {
+    launch_k(kernel, rows, nt, 0, st, w, g, m, v, sc, cols, train_w, bits, codes, rowsum, scale, out);
+  };
+  const bool warp_rows = rule == 3 && cols <= 32 * 4 * TW_WARP_MAXV;
+  if (dt == 1) {
+    if (warp_rows) go(closed_form_update_kernel<bf16, 3, 32, TW_WARP_MAXV>, 32, (bf16*)what);
+    else if (rule == 3) go(closed_form_update_kernel<bf16, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
+    else go(closed_form_update_kernel<bf16, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
+  } else {
+    if (warp_rows) go(closed_form_update_kernel<float, 3, 32, TW_WARP_MAXV>, 32, (float*)what);
+    else if (rule == 3) go(closed_form_update_kernel<float, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
+    else go(closed_form_update_kernel<float, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
+  }
 }
 
 }  // namespace mrem
