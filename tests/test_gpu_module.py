@@ -708,6 +708,61 @@ def test_degenerate_inputs_match_the_oracle():
         p.close()
 
 
+@pytest.mark.parametrize("name,grid,w_bits", [("W1", 3, 4), ("W2", 3, 4), ("Wqkv", 2, 2)])
+def test_rem_step_with_closed_form_scales_matches_the_oracle(name, grid, w_bits):
+    """Eq. 2 on one product when the weight scales are recomputed from the weights (w_grid 2 and 3): loss, the matrix
+    gradient (passed straight through) and the input quantizer's step gradient against the oracle; no weight-step
+    gradient; after one step the matrix follows AdamW and its codes are the rule's codes of the updated matrix."""
+    wl = _wl("base3_w2a8", n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40, w_grid=grid,
+             w_bits=w_bits)
+    p = Problem(wl, student_noise=0.002)
+    try:
+        m, layer = p.m, 1
+        pid, k = REM_MATRICES[name]
+        site = O.REM_SITE[name]
+        rows, cols = 120, m.shapes[pid][1]
+        a_np = synth.normal(5, "rem_cf" + name, (rows, cols), 1.0) + (0.4 if name == "W2" else 0.0)
+        a_dev = m.to_device(a_np)
+        a = a_dev.float().cpu().numpy()
+        if site == O.SITE_G:
+            p.off[layer, site] = np.float32(a.min() + 0.3)
+            p.a[layer, site] = np.float32(0.8 * (a.max() - p.off[layer, site]) / (2 ** wl.a_bits - 1))
+        else:
+            p.a[layer, site] = np.float32(0.8 * np.abs(a).max() / O.sym_qmax(wl.a_bits))
+        m.set_steps(p.ws, p.a, p.off)
+        steps = p.oracle_steps()[layer]
+        w_t, w_s = p.teacher[layer][name], p.student[layer][name]
+        loss = float(m.rem_step(layer, pid, a_dev, None)[0])
+        gW = m.grad(layer, pid, m.shapes[pid]).cpu().numpy()
+        gA = m.grad(layer, B.GRAD_STEP + 4 + site, (1,)).item()
+        assert m.poll_status() == 0
+        with pytest.raises(B.MremError):
+            m.grad(layer, B.GRAD_STEP + k, (1,))
+        r = O.rem_forward_loss_backward(p.desc, w_t, w_s, steps, name, a)
+        assert r["d_w_step"] is None
+        assert abs(loss - r["loss"]) / r["loss"] < GRAD_TOL, (loss, r["loss"])
+        assert rel(gW, r["dW"]) < GRAD_TOL
+        assert abs(gA - r["d_a_step"]) / abs(r["d_a_step"]) < GRAD_TOL, (gA, r["d_a_step"])
+        before = m.student_numpy()
+        opt = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+        m.rem_step(layer, pid, a_dev, B.make_optim(step=1, **opt))
+        torch.cuda.synchronize()
+        after = m.student_numpy()
+        z = np.zeros_like(before[layer][name], np.float64)
+        ref_w, _, _ = O.adamw_update(before[layer][name], gW, z, z.copy(), 1, opt["lr"], 0.9, 0.999, 1e-8, 0.01)
+        assert np.allclose(after[layer][name], ref_w, rtol=1e-5, atol=2e-3 * opt["lr"])
+        codes, rowsum = m.weight_codes(layer, pid)
+        ref = (O.quantize_weight_laq(after[layer][name], w_bits, True) if grid == 3 else O.quantize_weight_twn(after[layer][name], True))[0]
+        assert np.array_equal(codes.cpu().numpy().astype(np.int64), ref)
+        assert np.array_equal(rowsum.cpu().numpy().astype(np.int64), ref.sum(-1))
+        for l in range(wl.n_layers):                                # nothing else moved
+            for nm in O.PARAMS:
+                if (l, nm) != (layer, name):
+                    assert np.array_equal(after[l][nm], before[l][nm]), (l, nm)
+    finally:
+        p.close()
+
+
 _BF16_SMALL = dict(n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=3, len_lo=10, len_hi=40)
 _refit = lambda w, bits: O.quantize_weight_laq(w, bits, True)[0]
 # name: (workload, its changes, the code values that must occur, the oracle's quantizer, gradient bound, scalar bound).
