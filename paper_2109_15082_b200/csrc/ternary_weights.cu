@@ -19,11 +19,12 @@ namespace mrem {
 namespace {
 
 // Threads per row (NT) and float4 vectors per thread kept in registers (MAXV): a block of 256 threads with 4 vectors
-// each holds rows up to 4096 wide; the alternating rule takes one warp with 8 vectors per lane for rows up to 1024
-// wide, where its 16 dependent reductions then need no block barrier.
+// each holds rows up to 4096 wide; the alternating rule, whose 16 rounds are a dependent chain per thread, takes 128
+// threads with 2 vectors each for rows up to 1024 wide (measured against 32 x 8 and 256 x 1).
 constexpr int TW_THREADS = 256;
 constexpr int TW_MAXV = 4;
-constexpr int TW_WARP_MAXV = 8;
+constexpr int TW_NARROW_THREADS = 128;   // rows up to 1024 wide under the alternating rule: 2 vectors per thread
+constexpr int TW_NARROW_MAXV = 2;
 
 __device__ __forceinline__ double warp_sum_d(double v) {
 #pragma unroll
@@ -190,10 +191,7 @@ __device__ __forceinline__ void laq_row(const float4* wr, bool cached, const flo
   for (int r = 0; r + 1 < LAQ_ROUNDS; ++r) {
     double qw = 0.0, qw1 = 0.0, qw2 = 0.0, qw3 = 0.0;
     int qq = 0;
-    if (alpha > 0.f) {
-      const bool fast = alpha > 1e-30f;                      // 1 / alpha and the residual stay in the normal range
-      const float r_alpha = __frcp_rn(alpha);
-      auto code = [&](float w) { return fast ? laq_code_fast(w, alpha, r_alpha, qmax) : laq_code(w, alpha, qmax); };
+    auto sums = [&](auto code) {
       if (cached) {
 #pragma unroll
         for (int i = 0; i < MAXV; ++i) {
@@ -217,6 +215,12 @@ __device__ __forceinline__ void laq_row(const float4* wr, bool cached, const flo
           qq += q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
         }
       }
+    };
+    if (alpha > 1e-30f) {                                  // 1 / alpha and the residual stay in the normal range
+      const float r_alpha = __frcp_rn(alpha);
+      sums([&](float w) { return laq_code_fast(w, alpha, r_alpha, qmax); });
+    } else if (alpha > 0.f) {
+      sums([&](float w) { return laq_code(w, alpha, qmax); });
     }
     qw = (qw + qw1) + (qw2 + qw3);
     block_sum_di(qw, qq, shd, shi);
@@ -262,7 +266,7 @@ __device__ __forceinline__ void closed_form_row(const float4* wr, bool cached, c
 }
 
 template <typename T, int RULE, int NT, int MAXV>
-__global__ void __launch_bounds__(NT, NT == 32 ? 20 : (RULE == 2 ? 5 : 4)) closed_form_quantize_kernel(const float* __restrict__ w, int cols,
+__global__ void __launch_bounds__(NT, NT == TW_NARROW_THREADS ? 8 : (RULE == 2 ? 5 : 4)) closed_form_quantize_kernel(const float* __restrict__ w, int cols,
                                                                       int bits,
                                                                       int8_t* __restrict__ codes,
                                                                       int32_t* __restrict__ rowsum,
@@ -290,7 +294,7 @@ __global__ void __launch_bounds__(NT, NT == 32 ? 20 : (RULE == 2 ? 5 : 4)) close
 
 // AdamW on the row (gradient of w_hat passed through unchanged), then the rule on the new weights.
 template <typename T, int RULE, int NT, int MAXV>
-__global__ void __launch_bounds__(NT, NT == 32 ? 20 : (RULE == 2 ? 5 : 4)) closed_form_update_kernel(float* __restrict__ w, const float* __restrict__ g,
+__global__ void __launch_bounds__(NT, NT == TW_NARROW_THREADS ? 8 : (RULE == 2 ? 5 : 4)) closed_form_update_kernel(float* __restrict__ w, const float* __restrict__ g,
                                                                     float* __restrict__ m, float* __restrict__ v,
                                                                     const OptimScalars* __restrict__ sc, int cols,
                                                                     int train_w, int bits,
@@ -347,13 +351,13 @@ void launch_closed_form_quantize(const float* w, int rows, int cols, int rule, i
                                  float* scale, void* what, int dt, cudaStream_t st) {
   Scope sc("quantize_weight", (double)rows * cols * (5.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)) + rows * 8.0, 0, st);
   auto go = [&](auto kernel, int nt, auto* out) { launch_k(kernel, rows, nt, 0, st, w, cols, bits, codes, rowsum, scale, out); };
-  const bool warp_rows = rule == 3 && cols <= 32 * 4 * TW_WARP_MAXV;
+  const bool narrow = rule == 3 && cols <= TW_NARROW_THREADS * 4 * TW_NARROW_MAXV;
   if (dt == 1) {
-    if (warp_rows) go(closed_form_quantize_kernel<bf16, 3, 32, TW_WARP_MAXV>, 32, (bf16*)what);
+    if (narrow) go(closed_form_quantize_kernel<bf16, 3, TW_NARROW_THREADS, TW_NARROW_MAXV>, TW_NARROW_THREADS, (bf16*)what);
     else if (rule == 3) go(closed_form_quantize_kernel<bf16, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
     else go(closed_form_quantize_kernel<bf16, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
   } else {
-    if (warp_rows) go(closed_form_quantize_kernel<float, 3, 32, TW_WARP_MAXV>, 32, (float*)what);
+    if (narrow) go(closed_form_quantize_kernel<float, 3, TW_NARROW_THREADS, TW_NARROW_MAXV>, TW_NARROW_THREADS, (float*)what);
     else if (rule == 3) go(closed_form_quantize_kernel<float, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
     else go(closed_form_quantize_kernel<float, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
   }
@@ -366,13 +370,13 @@ void launch_closed_form_update(float* w, const float* g, float* m, float* v, con
   auto go = [&](auto kernel, int nt, auto* out) {
     launch_k(kernel, rows, nt, 0, st, w, g, m, v, sc, cols, train_w, bits, codes, rowsum, scale, out);
   };
-  const bool warp_rows = rule == 3 && cols <= 32 * 4 * TW_WARP_MAXV;
+  const bool narrow = rule == 3 && cols <= TW_NARROW_THREADS * 4 * TW_NARROW_MAXV;
   if (dt == 1) {
-    if (warp_rows) go(closed_form_update_kernel<bf16, 3, 32, TW_WARP_MAXV>, 32, (bf16*)what);
+    if (narrow) go(closed_form_update_kernel<bf16, 3, TW_NARROW_THREADS, TW_NARROW_MAXV>, TW_NARROW_THREADS, (bf16*)what);
     else if (rule == 3) go(closed_form_update_kernel<bf16, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
     else go(closed_form_update_kernel<bf16, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (bf16*)what);
   } else {
-    if (warp_rows) go(closed_form_update_kernel<float, 3, 32, TW_WARP_MAXV>, 32, (float*)what);
+    if (narrow) go(closed_form_update_kernel<float, 3, TW_NARROW_THREADS, TW_NARROW_MAXV>, TW_NARROW_THREADS, (float*)what);
     else if (rule == 3) go(closed_form_update_kernel<float, 3, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
     else go(closed_form_update_kernel<float, 2, TW_THREADS, TW_MAXV>, TW_THREADS, (float*)what);
   }
