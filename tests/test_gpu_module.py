@@ -774,6 +774,11 @@ CLOSED_FORM = {
     "refit_w4": ("base3_w2a8", dict(_BF16_SMALL, w_grid=3, w_bits=4), set(range(-7, 8)), _refit, GRAD_TOL, 0.1),
     "refit_w2": ("base3_w2a8", dict(_BF16_SMALL, w_grid=3, w_bits=2), {-1, 0, 1}, _refit, GRAD_TOL, 0.1),
     "refit_w4_f32": ("tiny", dict(n_layers=2, batch=3, len_lo=9, len_hi=32, w_grid=3, w_bits=4), set(range(-7, 8)), _refit, 2e-3, None),
+    # rows of the second feed-forward matrix 4096 wide (the 256-thread form of the row kernel, registers full) and 8192
+    # wide (beyond what a block keeps in registers: the row is re-read every round; the bound on the gradients is wider
+    # there: a feed-forward width of 64 x hidden sums 8192 bf16-rounded terms into every output)
+    "refit_w4_wide": ("base3_w2a8", dict(_BF16_SMALL, ffn=4096, w_grid=3, w_bits=4), set(range(-7, 8)), _refit, GRAD_TOL, 0.1),
+    "refit_w4_wider": ("base3_w2a8", dict(_BF16_SMALL, ffn=8192, w_grid=3, w_bits=4), set(range(-7, 8)), _refit, 5e-2, 0.1),
 }
 
 
