@@ -169,7 +169,11 @@ int32_t mrem_module_forward(mrem_ctx* ctx, int32_t role, const void* d_x, const 
  * d_loss_total (float32 [1]) and, when non-NULL, each layer's term to d_loss_per_layer
  * ([n_layers]); stores d loss / d f_hat_l for the backward. */
 int32_t mrem_recon_loss(mrem_ctx* ctx, float* d_loss_total, float* d_loss_per_layer);
-/* Straight-through backward through the student module (gradient local to the module). */
+/* Sec. 3.1.1: back-propagation of the loss of Eq. 3 through the student module with the straight-through
+ * estimator at every quantizer (the gradient passes where x / s lies inside the code range; step sizes and the
+ * GELU-site offset get their own gradients, Sec. 4.1).  The loss gradient enters at every layer output of the
+ * module (Eq. 3 sums over them) and stops at the module input (Sec. 4.2).  Needs the student pass and
+ * mrem_recon_loss of this step (MREM_ERR_ORDER otherwise); fills the gradient buffers mrem_get_grad returns. */
 int32_t mrem_module_backward(mrem_ctx* ctx);
 /* Borrowed pointer to a gradient (float32, same shape as the parameter / step tensor).  Asking for a weight
  * matrix or a weight step applies the weight quantizers' straight-through masks on the spot. */
@@ -180,7 +184,9 @@ int32_t mrem_get_grad(mrem_ctx* ctx, int32_t layer, int32_t id, const float** d_
  * (mrem_embed_step).  Valid from a backward pass (mrem_module_backward or mrem_backward_and_step) until the next
  * forward pass on this context (MREM_ERR_ORDER otherwise). */
 int32_t mrem_get_input_grad(mrem_ctx* ctx, const void** d_grad);
-/* AdamW on everything in trainable_mask, steps clamped to >= 1e-8.  With per-row weight steps the update of
+/* Algorithm 2's Update(w) and Update(s): AdamW (Sec. 4.2; learning rate decayed linearly, Sec. 5.1) on
+ * everything in trainable_mask from the gradients of the last backward pass (MREM_ERR_ORDER without one);
+ * weight decay on the four matrices only, steps clamped to >= 1e-8.  With per-row weight steps the update of
  * each matrix also re-quantizes it (Eq. 1 with the new weights and steps), so the next
  * mrem_quantize_weights has nothing left to do. */
 int32_t mrem_step(mrem_ctx* ctx, const mrem_optim* optim);
@@ -269,8 +275,7 @@ int32_t mrem_quantize_weight(const float* d_w, int32_t rows, int32_t cols, const
                              int32_t bits, int32_t grid, int8_t* d_codes, int32_t* d_rowsum, float* d_scale,
                              void* d_what, int32_t dtype, void* cuda_stream);
 /* acc[m, n] = sum_k a[m, k] * b[n, k] in exact int32 on the int8 tensor cores.  a: [M, K] int8 (or uint8
- * when a_unsigned), b: [N, K] int8, K % 16 == 0, acc: [M, N] int32.  block_n 0 = automatic tile width; 64/128/256 force it;
- * -2 selects the CTA-pair kernel (two SMs per 256 x 256 tile, tcgen05 cta_group::2).
+ * when a_unsigned), b: [N, K] int8, K % 16 == 0, acc: [M, N] int32.  block_n 0 = automatic tile width; 64/128/256 force it.
  * d_status: device int32 receiving a DeviceStatus code on a bounded-wait timeout (0 otherwise). */
 int32_t mrem_gemm_i8(const int8_t* d_a, int32_t a_unsigned, const int8_t* d_b, int32_t M, int32_t N, int32_t K,
                      int32_t* d_acc, int32_t block_n, int32_t* d_status, void* cuda_stream);
@@ -401,7 +406,9 @@ int32_t mrem_rem_step(mrem_ctx* ctx, int32_t layer, int32_t tensor_id, const voi
  * no larger), MREM_ERR_ARG for null pointers, a bad dtype or non-positive sizes, MREM_ERR_CUDA when the
  * device cannot be queried.  The first call on each device looks up the device address of the built-in
  * array (a one-off host-side query, made with that device current); make that first call before entering
- * any stream capture.  All calls on a device share the one array: calls that may overlap on the GPU (two
+ * any stream capture.  The address is remembered per device ordinal: `cuda_stream` must belong to the device
+ * (and primary context) that is current at the call, and after cudaDeviceReset the library must not be
+ * called again on that device.  All calls on a device share the one array: calls that may overlap on the GPU (two
  * streams, two threads) race on it and must be serialised by the caller.  Nothing in the array has to
  * be cleared between calls: each call rewrites every slot it later reads.  The call never allocates or
  * frees memory, on the host side of CUDA or otherwise. */

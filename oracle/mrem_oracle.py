@@ -10,7 +10,10 @@ check and the benchmark's CPU-baseline leg may import this file; it shares no
 code with the CUDA path and imports nothing from it.
 
 Every function is pinned by tests/test_oracle_*.py against something other
-than itself (library autograd, brute force, closed forms, invariants of Eq. 1).
+than itself (library autograd, brute force, closed forms, invariants of Eq. 1;
+the storage roundings, the initial activation steps and a whole step's
+bookkeeping in tests/test_oracle_storage_pins.py against torch layers with the
+roundings written out and torch.optim.AdamW).
 The only part that stays "parity unpinned" by the paper is the multi-step loss
 trajectory, for which the paper prints no numbers (only the qualitative trend
 of its training-loss figure).

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmrem.so")
-SOURCES = ["gemm_tcgen05.cu", "gemm_tcgen05_2cta.cu", "gemm_tcgen05_group.cu", "gemm_simt.cu", "quant_kernels.cu", "layer_kernels.cu", "row_kernels.cu", "weight_update.cu", "ternary_weights.cu", "attention_fwd.cu", "attention_bwd.cu", "no_alloc.cu", "head_kernels.cu", "embed_step.cu",
+SOURCES = ["gemm_tcgen05.cu", "gemm_tcgen05_group.cu", "gemm_simt.cu", "quant_kernels.cu", "layer_kernels.cu", "row_kernels.cu", "weight_update.cu", "ternary_weights.cu", "attention_fwd.cu", "attention_bwd.cu", "no_alloc.cu", "head_kernels.cu", "embed_step.cu",
            "mrem_api.cu", "mrem_step.cu", "mrem_extra.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]

@@ -14,11 +14,6 @@ enum GemmRc : int { GEMM_OK = 0, GEMM_ERR_ARG = -1, GEMM_ERR_ALIGN = -2, GEMM_ER
 int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
             const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream);
 
-// CTA-pair variant (cta_group::2) for single large products; tc_gemm hands eligible calls to it.
-bool tc_gemm_pair_eligible(const GemmShape& g, const Epilogue& epi, int block_n);
-int tc_gemm_pair(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
-                 const Epilogue& epi, int* d_status, int sm_count, cudaStream_t stream);
-
 // Several bf16 products with plain fp32 outputs (alpha and row bias only) as one persistent launch over the
 // joint tile list: the weight-gradient products of a layer.  Operands as in tc_gemm, one batch each.
 constexpr int MAX_GEMM_GROUP = 4;

@@ -1,6 +1,6 @@
 // Shared pieces of the tensor-core GEMM kernels: launch parameters, tile decoding and the epilogue
-// (TMEM accumulators -> scale / bias / residual / activation -> coalesced global stores through a
-// per-warp shared-memory transpose).
+// (TMEM accumulators -> scale / bias / residual / activation -> global stores straight from registers,
+// every lane writing whole 32-byte sectors of its own row).
 #pragma once
 #include "gemm.h"
 #include "tc_ptx.cuh"
@@ -10,13 +10,10 @@ namespace tc {
 
 constexpr int BLOCK_M = 128;
 constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
-constexpr int TILE_SMEM_BUDGET = 196608;              // bytes of operand stages per CTA (CTA-pair kernel, beside its staging)
-constexpr int SINGLE_CTA_SMEM_BUDGET = 229376;        // bytes of operand stages per CTA (single-CTA kernel: no staging)
+constexpr int SINGLE_CTA_SMEM_BUDGET = 229376;        // bytes of operand stages per CTA
 constexpr int MAX_STAGES = 8;
 constexpr int GEMM_THREADS = 320;                    // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_WARPS = 8;
-constexpr int STAGING_WORDS = 32 * 33;               // per epilogue warp: 32 rows x 32 words, padded
-constexpr int STAGING_BYTES = EPI_WARPS * STAGING_WORDS * 4;
 constexpr int TMEM_COLS = 512;
 
 struct TcParams {
@@ -46,7 +43,8 @@ __device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int tile) {
   return t;
 }
 
-// ------------------------------------------------------------------ epilogue of 32 columns of one row
+// ------------------------------------------------------------------ epilogue of 32 columns of one row: ragged
+// or unaligned edges (element-wise bounds checks, run-time terms)
 template <int KIND>
 __device__ __forceinline__ void epilogue_chunk(const TcParams& p, const uint32_t* r, float alpha, long long row_off,
                                                int row, int col0, bool row_ok, bool vec_ok) {
@@ -122,127 +120,6 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, const uint32_t
     }
   }
 }
-
-// ------------------------------------------------------------------ epilogue of a 32-row x 32-word block
-// One warp, one round: 64 bf16 or 32 fp32/int32 output columns of its 32 rows (128 bytes per row).
-// Values go through the warp's staging buffer so that global loads (residual) and stores are issued as
-// 16-byte pieces with 8 lanes covering one contiguous 128-byte row segment.  Staging layout: row r at
-// r * 128 bytes, its 16-byte piece c at position c ^ (r & 7): both the row-per-lane side and the
-// 8-lanes-per-row side move 16 bytes per lane without bank conflicts.  The caller guarantees 16-byte
-// alignment of out, residual, col_scale and col_bias and whole rounds inside N.
-__device__ __forceinline__ uint4 ldg16(const void* p) { return *reinterpret_cast<const uint4*>(p); }
-
-template <int KIND>
-__device__ __forceinline__ void epilogue_round(const TcParams& p, uint32_t taddr, float alpha, long long tile_off,
-                                               int row0, int col0, int lane, uint32_t* stg) {
-  const Epilogue& e = p.epi;
-  const bool is_bf16 = e.out_kind == OUT_BF16;
-  const int vec_elems = is_bf16 ? 8 : 4;
-  const int sub = lane >> 3, seg = lane & 7;             // 4 rows per instruction, 8 lanes per row
-  uint4* stg4 = reinterpret_cast<uint4*>(stg);
-  uint32_t r0[32], r1[32];
-  tmem_ld32_issue(taddr, r0);                           // in flight while the residual is fetched and transposed
-  if (is_bf16) tmem_ld32_issue(taddr + 32u, r1);
-  uint32_t res[32];
-  if (e.residual) {
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int rl = it * 4 + sub, row = row0 + rl;
-      uint4 u = make_uint4(0, 0, 0, 0);
-      if (row < p.M) {
-        const long long off = tile_off + (long long)row * e.ldc + col0 + seg * vec_elems;
-        u = is_bf16 ? ldg16(reinterpret_cast<const bf16*>(e.residual) + off) : ldg16(reinterpret_cast<const float*>(e.residual) + off);
-      }
-      stg4[rl * 8 + (seg ^ (rl & 7))] = u;
-    }
-    __syncwarp();
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 u = stg4[lane * 8 + (c ^ (lane & 7))];
-      res[4 * c] = u.x; res[4 * c + 1] = u.y; res[4 * c + 2] = u.z; res[4 * c + 3] = u.w;
-    }
-    __syncwarp();
-  }
-  const int row = row0 + lane;
-  const float rb = (e.row_bias && row < p.M) ? e.row_bias[row] : 0.f;
-  tmem_ld_wait();
-  tmem_ld_pin(r0);
-  if (is_bf16) tmem_ld_pin(r1);
-  if (e.out_kind == OUT_I32) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) stg4[lane * 8 + (c ^ (lane & 7))] = make_uint4(r0[4 * c], r0[4 * c + 1], r0[4 * c + 2], r0[4 * c + 3]);
-  } else {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      if (h == 1 && !is_bf16) break;
-      const uint32_t* r = h == 0 ? r0 : r1;
-      float v[32];
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) {
-        const int n = col0 + h * 32 + j;
-        float4 sc = make_float4(alpha, alpha, alpha, alpha), bi = make_float4(rb, rb, rb, rb);
-        if (e.col_scale) {
-          const float4 t = *reinterpret_cast<const float4*>(e.col_scale + n);
-          sc.x *= t.x; sc.y *= t.y; sc.z *= t.z; sc.w *= t.w;
-        }
-        if (e.col_bias) {
-          const float4 t = *reinterpret_cast<const float4*>(e.col_bias + n);
-          bi.x += t.x; bi.y += t.y; bi.z += t.z; bi.w += t.w;
-        }
-        const float a0 = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
-        const float a1 = (KIND == 1) ? (float)(int)r[j + 1] : __uint_as_float(r[j + 1]);
-        const float a2 = (KIND == 1) ? (float)(int)r[j + 2] : __uint_as_float(r[j + 2]);
-        const float a3 = (KIND == 1) ? (float)(int)r[j + 3] : __uint_as_float(r[j + 3]);
-        v[j] = a0 * sc.x + bi.x; v[j + 1] = a1 * sc.y + bi.y; v[j + 2] = a2 * sc.z + bi.z; v[j + 3] = a3 * sc.w + bi.w;
-      }
-      if (e.residual) {
-        if (is_bf16) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&res[h * 16 + j]));
-            v[2 * j] += f.x;
-            v[2 * j + 1] += f.y;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(res[j]);
-        }
-      }
-      if (e.act == 1) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-      }
-      if (is_bf16) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint4 u;
-          __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&u);
-#pragma unroll
-          for (int t = 0; t < 4; ++t) h2[t] = __floats2bfloat162_rn(v[8 * c + 2 * t], v[8 * c + 2 * t + 1]);
-          stg4[lane * 8 + ((h * 4 + c) ^ (lane & 7))] = u;
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          stg4[lane * 8 + (c ^ (lane & 7))] = make_uint4(__float_as_uint(v[4 * c]), __float_as_uint(v[4 * c + 1]),
-                                                         __float_as_uint(v[4 * c + 2]), __float_as_uint(v[4 * c + 3]));
-      }
-    }
-  }
-  __syncwarp();
-#pragma unroll
-  for (int it = 0; it < 8; ++it) {
-    const int rl = it * 4 + sub, orow = row0 + rl;
-    if (orow < p.M) {
-      const uint4 u = stg4[rl * 8 + (seg ^ (rl & 7))];
-      const long long off = tile_off + (long long)orow * e.ldc + col0 + seg * vec_elems;
-      if (is_bf16) *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(e.out) + off) = u;
-      else *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(e.out) + off) = u;
-    }
-  }
-  __syncwarp();
-}
-
 
 // ------------------------------------------------------------------ register-direct epilogue
 // One warp drains its 32 accumulator rows (TMEM lane = row = lane of the warp) over a range of columns in

@@ -280,7 +280,6 @@ int pick_block_n(int M, int N, int k_blocks, int batches, int sm_count) {
 int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
             const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.nb0 <= 0 || g.nb1 <= 0) return GEMM_ERR_ARG;
-  if (tc_gemm_pair_eligible(g, epi, block_n)) return tc_gemm_pair(kind, a_unsigned, A, B, g, epi, d_status, sm_count, stream);
   const int es = kind == 0 ? 2 : 1;
   if (kind == 1 && (A.mn_contig || B.mn_contig)) return GEMM_ERR_ARG;
   TcParams p;

@@ -12,7 +12,7 @@ int g_programmatic_launch = 1;
 }
 
 namespace {
-std::string g_create_err;
+thread_local std::string g_create_err;   // mrem_last_error(NULL): the calling thread's last create / workspace-size error
 
 const int kParamIsMatrix[MREM_N_PARAMS] = {1, 0, 1, 0, 0, 0, 1, 0, 1, 0, 0, 0};
 const int kMatParam[N_WMAT] = {MREM_WQKV, MREM_WO, MREM_W1, MREM_W2};

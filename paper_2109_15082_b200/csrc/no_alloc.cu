@@ -2,10 +2,12 @@
 //
 // The regular mrem_recon_loss belongs to a context whose workspace the caller allocated; the
 // per-block partial sums of its two-stage reduction live in that workspace.  Some callers have
-// no way to obtain such a workspace: code that runs inside someone else's stream capture, a
-// plug-in loaded into a process whose memory pool it must not touch, a monitoring hook that
-// may be invoked while the application's allocator is locked.  For them the partial sums live
-// in a fixed array that is part of the library image itself.
+// no way to obtain such a workspace: a plug-in loaded into a process whose memory pool it must
+// not touch, a monitoring hook that may be invoked while the application's allocator is locked,
+// a latency-critical loop that cannot afford cudaMalloc's device-wide synchronisation.  For them
+// the partial sums live in a fixed array that is part of the library image itself.  The first
+// call on a device asks the runtime for the array's device address; that call has to be made
+// outside any stream capture, with the device of `cuda_stream` current.
 #include <mutex>
 
 #include "../../include/mrem.h"
@@ -51,7 +53,8 @@ extern "C" int32_t mrem_recon_loss_noalloc(const void* d_f_student, const void* 
   const float c = loss_mean ? 1.f / (float)n_per_layer : 1.f;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // every (layer, block) slot is rewritten by the first kernel before the second one reads it, so nothing
-  // left over from an earlier call can leak into this one
+  // left over from an earlier call can leak into this one.  A launch that fails leaves its error as the
+  // runtime's last error (a later successful launch does not clear it), which the final query returns.
   mrem::launch_loss(d_f_student, d_f_teacher, n_layers, n_per_layer, c, d_grad, partials, nullptr, dtype, st);
   mrem::launch_loss_finalize(partials, n_layers, c, d_loss_total, d_loss_per_layer, st);
   return cudaGetLastError() == cudaSuccess ? MREM_OK : MREM_ERR_CUDA;

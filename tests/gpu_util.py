@@ -133,3 +133,26 @@ def compare_grads(gpu, ora, tol, skip_small=1e-12, check_offset=True, scalar_tol
 
 def code_flip_rate(codes_gpu, codes_ref):
     return float((np.asarray(codes_gpu) != np.asarray(codes_ref)).mean())
+
+
+def bf16_step(x):
+    """Spacing of bfloat16 numbers at the magnitude of x (8 significand bits): 2^(floor(log2|x|) - 7)."""
+    a = np.maximum(np.abs(np.asarray(x, np.float64)), 2.0 ** -126)
+    return np.exp2(np.floor(np.log2(a)) - 7.0)
+
+
+def bf16_closeness(got, ref, floor_frac=0.125):
+    """Element-wise distance of two bf16-stored tensors of shape [..., hidden], in bfloat16 spacings.
+
+    The unit of element i is the bf16 spacing at max(|ref_i|, floor_frac * rms of its row): two correct
+    implementations differ where a value sat within rounding noise of a bf16 rounding boundary (then by exactly
+    one spacing of that element) and, for elements far below the row's scale, by the noise that a flipped
+    rounding elsewhere in the row sends through the row's mean and variance, which is absolute, not relative.
+    Returns dict(frac_differ, frac_over_1, max_units, rel_l2)."""
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    rms = np.sqrt((ref * ref).mean(-1, keepdims=True))
+    unit = bf16_step(np.maximum(np.abs(ref), floor_frac * rms))
+    d = np.abs(got - ref) / unit
+    return dict(frac_differ=float((got != ref).mean()), frac_over_1=float((d > 1.0 + 1e-9).mean()),
+                max_units=float(d.max()), rel_l2=rel(got, ref))

@@ -100,7 +100,7 @@ I8_SHAPES = [(128, 128, 128), (300, 200, 144), (1000, 520, 1040), (77, 3072, 102
 
 
 @pytest.mark.parametrize("M,N,K", I8_SHAPES)
-@pytest.mark.parametrize("block_n", [0, 64, 128, 256, -2])      # -2: the CTA-pair (cta_group::2) kernel
+@pytest.mark.parametrize("block_n", [0, 64, 128, 256])
 @pytest.mark.parametrize("a_unsigned", [0, 1])
 def test_gemm_i8_exact(M, N, K, block_n, a_unsigned):
     rng = np.random.default_rng(M * 7 + N * 3 + K + a_unsigned)
@@ -182,28 +182,6 @@ def test_gemm_float_layouts(dtype, a_mn, b_mn, M, N, K, nb):
     got = out.cpu().numpy().astype(np.float64)
     rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
     assert rel < 2e-6, rel
-
-
-@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 0), (1, 1)])
-def test_gemm_bf16_cta_pair_kernel(a_mn, b_mn):
-    # the cta_group::2 kernel (block_n = -2): ragged in M and N, every operand layout
-    M, N, K = 648, 520, 200
-    a = synth.normal(7, f"pa{a_mn}", (1, M, K), 1.0)
-    b = synth.normal(7, f"pb{b_mn}", (1, N, K), 1.0)
-    ad = torch.from_numpy(_layout(a, a_mn)).to(DEV).to(torch.bfloat16).contiguous()
-    bd = torch.from_numpy(_layout(b, b_mn)).to(DEV).to(torch.bfloat16).contiguous()
-    a64 = ad.float().cpu().numpy().astype(np.float64)[0]
-    b64 = bd.float().cpu().numpy().astype(np.float64)[0]
-    a64 = a64.T if a_mn else a64
-    b64 = b64.T if b_mn else b64
-    out = torch.zeros(M, N, dtype=torch.float32, device=DEV)
-    st = _status()
-    B.mrem_gemm(B.BF16, ad, a_mn, M if a_mn else K, M * K, bd, b_mn, N if b_mn else K, N * K, M, N, K, 1, 1.0, out,
-                N, M * N, -2, st, _stream())
-    torch.cuda.synchronize()
-    assert int(st[0]) == 0
-    ref = a64 @ b64.T
-    assert np.linalg.norm(out.cpu().numpy() - ref) / np.linalg.norm(ref) < 2e-6
 
 
 @pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1)])
