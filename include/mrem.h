@@ -184,6 +184,23 @@ int32_t mrem_get_grad(mrem_ctx* ctx, int32_t layer, int32_t id, const float** d_
  * (mrem_embed_step).  Valid from a backward pass (mrem_module_backward or mrem_backward_and_step) until the next
  * forward pass on this context (MREM_ERR_ORDER otherwise). */
 int32_t mrem_get_input_grad(mrem_ctx* ctx, const void** d_grad);
+/* Borrowed pointer to a tensor that a forward pass stored on its way through one layer (storage type, row-major;
+ * for verification: each stored tensor is the rounding of one stage of the layer of Sec. 3.1 / Sec. 4.1 applied
+ * to the stored tensors before it).  `which`:
+ *   MREM_ACT_QKV  [tokens, 3*hidden]  input projection + bias
+ *   MREM_ACT_P    [batch, heads, seq, seq]  softmax output (student pass only)
+ *   MREM_ACT_CTX  [tokens, hidden]    attention context
+ *   MREM_ACT_Y1   [tokens, hidden]    output projection + bias + layer input (before the first LayerNorm)
+ *   MREM_ACT_A    [tokens, hidden]    first LayerNorm's output
+ *   MREM_ACT_G    [tokens, ffn]       teacher: GELU output (it never stores the tensor before GELU);
+ *                                     student: the tensor BEFORE GELU (its GELU output is recomputed, not kept)
+ *   MREM_ACT_Y2   [tokens, hidden]    FFN2 + bias + first LayerNorm's output (before the second LayerNorm)
+ * The teacher pass reuses one set of buffers for all layers, so only its last layer can be read
+ * (MREM_ERR_ARG otherwise); the student pass keeps every layer.  Valid until the next forward pass of that role;
+ * MREM_ERR_ORDER when there has been none. */
+enum { MREM_ACT_QKV = 0, MREM_ACT_P = 1, MREM_ACT_CTX = 2, MREM_ACT_Y1 = 3, MREM_ACT_A = 4, MREM_ACT_G = 5, MREM_ACT_Y2 = 6,
+       MREM_ACT_COUNT = 7 };
+int32_t mrem_get_activation(mrem_ctx* ctx, int32_t role, int32_t layer, int32_t which, const void** d_ptr);
 /* Algorithm 2's Update(w) and Update(s): AdamW (Sec. 4.2; learning rate decayed linearly, Sec. 5.1) on
  * everything in trainable_mask from the gradients of the last backward pass (MREM_ERR_ORDER without one);
  * weight decay on the four matrices only, steps clamped to >= 1e-8.  With per-row weight steps the update of

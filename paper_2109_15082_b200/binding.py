@@ -34,6 +34,7 @@ EXPORTS = (
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
     "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head", "mrem_embed_workspace_bytes", "mrem_embed_step", "mrem_get_input_grad",
+    "mrem_get_activation",
 )
 
 
@@ -218,6 +219,15 @@ def mrem_embed_workspace_bytes(desc, max_tokens) -> int:
 def mrem_get_input_grad(ctx) -> int:
     out = C.c_void_p(0)
     _check(lib().mrem_get_input_grad(ctx, C.byref(out)), "mrem_get_input_grad", ctx)
+    return out.value
+
+
+ACT_QKV, ACT_P, ACT_CTX, ACT_Y1, ACT_A, ACT_G, ACT_Y2 = range(7)
+
+
+def mrem_get_activation(ctx, role, layer, which) -> int:
+    out = C.c_void_p(0)
+    _check(lib().mrem_get_activation(ctx, int(role), int(layer), int(which), C.byref(out)), "mrem_get_activation", ctx)
     return out.value
 
 

@@ -380,6 +380,28 @@ int32_t mrem_get_input_grad(mrem_ctx* c, const void** g) {
   return MREM_OK;
 }
 
+int32_t mrem_get_activation(mrem_ctx* c, int32_t role, int32_t layer, int32_t which, const void** ptr) {
+  if (!c || !ptr) return MREM_ERR_ARG;
+  if (layer < 0 || layer >= c->d.n_layers) return fail(c, MREM_ERR_ARG, "get_activation: layer");
+  const void* p = nullptr;
+  if (role == MREM_TEACHER) {
+    if (!c->have_teacher) return fail(c, MREM_ERR_ORDER, "get_activation: no teacher pass to read");
+    if (layer != c->d.n_layers - 1) return fail(c, MREM_ERR_ARG, "get_activation: the teacher pass keeps its last layer's tensors only");
+    const void* t[MREM_ACT_COUNT] = {c->t_qkv, nullptr, c->t_ctx, c->t_y1, c->t_a, c->t_g, c->t_y2};
+    if (which >= 0 && which < MREM_ACT_COUNT) p = t[which];
+  } else if (role == MREM_STUDENT) {
+    if (!c->have_student) return fail(c, MREM_ERR_ORDER, "get_activation: no student pass to read");
+    const LayerStash& s = c->stash[layer];
+    const void* t[MREM_ACT_COUNT] = {s.qkv, s.P, s.ctx, s.y1, s.a, s.u, s.y2};
+    if (which >= 0 && which < MREM_ACT_COUNT) p = t[which];
+  } else {
+    return fail(c, MREM_ERR_ARG, "get_activation: role");
+  }
+  if (!p) return fail(c, MREM_ERR_ARG, "get_activation: this tensor is not kept by that pass");
+  *ptr = p;
+  return MREM_OK;
+}
+
 int32_t mrem_init_student_from_teacher(mrem_ctx* c) {
   if (!c) return MREM_ERR_ARG;
   for (int l = 0; l < c->d.n_layers; ++l)

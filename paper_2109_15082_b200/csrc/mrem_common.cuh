@@ -115,6 +115,21 @@ __device__ __forceinline__ float quotient(float x, float s, float r_s) {
   return __fmaf_rn(__fmaf_rn(-z0, s, x), r_s, z0);
 }
 
+// The integer code of Eq. 1, nearest integer (ties to even) of clip(n / s, lo, hi), bit for bit what the IEEE
+// division gives, at a third of its instructions: the three-instruction quotient is within one ulp of the correctly
+// rounded one (1.5e-5 at |z| <= 255), so the two can round to different integers only when the quotient lies that
+// close to a half-integer; any value within 2^-10 of one is decided by the division instruction instead (about one
+// element in a thousand).  A quotient beyond the range is clipped to the same bound by both.  r_s = RN(1 / s).
+__device__ __forceinline__ int code_of(float n, float s, float r_s, float lo, float hi) {
+  float zc = fminf(fmaxf(quotient(n, s, r_s), lo), hi);
+  float q = rintf(zc);
+  if (fabsf(fabsf(zc - q) - 0.5f) < 9.765625e-4f) {
+    zc = fminf(fmaxf(__fdiv_rn(n, s), lo), hi);
+    q = rintf(zc);
+  }
+  return (int)q;
+}
+
 // GELU(u) = u * Phi(u) with the erf form.  erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x), x >= 0
 // (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7, below half a float32 ulp of 1 + erf for u > 0): one
 // exponential serves both erf and the density needed by the derivative.

@@ -50,10 +50,8 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
 }
 
 // ------------------------------------------------------------------ activation quantizer
-__device__ __forceinline__ int act_code(float x, float s, float off, bool has_off, float lo, float hi) {
-  const float t = has_off ? __fsub_rn(x, off) : x;
-  const float z = __fdiv_rn(t, s);
-  return __float2int_rn(fminf(fmaxf(z, lo), hi));
+__device__ __forceinline__ int act_code(float x, float s, float r_s, float off, bool has_off, float lo, float hi) {
+  return code_of(has_off ? __fsub_rn(x, off) : x, s, r_s, lo, hi);
 }
 
 template <typename T, int V>
@@ -68,6 +66,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
   pdl_wait();
   // seg_cols > 0: three column segments of that width (a multiple of V), each with its own step
   const float s0 = *step, s1 = seg_cols ? *step1 : s0, s2 = seg_cols ? *step2 : s0;
+  const float r0 = __frcp_rn(s0), r1 = __frcp_rn(s1), r2 = __frcp_rn(s2);
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
   const int vcols = cols / V;
@@ -77,10 +76,11 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
     const int c = (int)(i - r * vcols) * V;
     float v[V];
     load_vec<T, V>(x + r * ld_x + c, v);
-    const float s = !seg_cols || c < seg_cols ? s0 : (c < 2 * seg_cols ? s1 : s2);
+    const int seg = !seg_cols || c < seg_cols ? 0 : (c < 2 * seg_cols ? 1 : 2);
+    const float s = seg == 0 ? s0 : (seg == 1 ? s1 : s2), r_s = seg == 0 ? r0 : (seg == 1 ? r1 : r2);
     int q[V];
 #pragma unroll
-    for (int j = 0; j < V; ++j) q[j] = act_code(v[j], s, off, has_off, lo, hi);
+    for (int j = 0; j < V; ++j) q[j] = act_code(v[j], s, r_s, off, has_off, lo, hi);
     if (q8) store_codes<V>(q8 + r * ld_q8 + c, q);
     if (qt) {
 #pragma unroll
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(256) gelu_quant_kernel(const T* __restrict__ u
                                                          int8_t* __restrict__ q8, T* __restrict__ qt) {
   pdl_trigger();
   pdl_wait();
-  const float s = *step;
+  const float s = *step, r_s = __frcp_rn(s);
   const bool has_off = offset != nullptr;
   const float off = has_off ? *offset : 0.f;
   for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(256) gelu_quant_kernel(const T* __restrict__ u
     load_vec<T, V>(u + i, v);
     int q[V];
 #pragma unroll
-    for (int j = 0; j < V; ++j) q[j] = act_code(stored<T>(gelu_erf(v[j])), s, off, has_off, lo, hi);
+    for (int j = 0; j < V; ++j) q[j] = act_code(stored<T>(gelu_erf(v[j])), s, r_s, off, has_off, lo, hi);
     if (q8) store_codes<V>(q8 + i, q);
     if (qt) {
 #pragma unroll

@@ -41,6 +41,21 @@ template <> __device__ __forceinline__ void store4<bf16>(bf16* p, const float* v
   *reinterpret_cast<uint2*>(p) = t;
 }
 
+// V consecutive floats of a per-column vector (16-byte aligned when V % 4 == 0: the vector paths guarantee it)
+template <int V>
+__device__ __forceinline__ void load_cols(const float* __restrict__ p, float* v) {
+  if constexpr (V % 4 == 0) {
+#pragma unroll
+    for (int j = 0; j < V; j += 4) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(p + j));
+      v[j] = t.x; v[j + 1] = t.y; v[j + 2] = t.z; v[j + 3] = t.w;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < V; ++j) v[j] = p[j];
+  }
+}
+
 // ------------------------------------------------------------------ LayerNorm forward
 // CACHED: the row sits in registers (cols <= 32 * V * MAXNV, cols % V == 0); else V == 1 and
 // the row is re-read from L1/L2 in each of the three passes.
@@ -88,15 +103,18 @@ __global__ void __launch_bounds__(128) ln_fwd_kernel(const T* __restrict__ y, co
     if (mean) mean[row] = mu;
     if (rstd) rstd[row] = rs;
   }
-  const float s = step ? *step : 1.f;
+  const float s = step ? *step : 1.f, r_s = __frcp_rn(s);
   auto emit = [&](int c, float* o) {
+    float gm[V], bt[V];
+    load_cols<V>(gamma + c, gm);
+    load_cols<V>(beta + c, bt);
 #pragma unroll
-    for (int j = 0; j < V; ++j) o[j] = (o[j] - mu) * rs * gamma[c + j] + beta[c + j];
+    for (int j = 0; j < V; ++j) o[j] = (o[j] - mu) * rs * gm[j] + bt[j];
     store_vec<T, V>(out + row * cols + c, o);
     if (step) {
       int q[V];
 #pragma unroll
-      for (int j = 0; j < V; ++j) q[j] = qcode(__fdiv_rn(stored<T>(o[j]), s), -qmax, qmax);
+      for (int j = 0; j < V; ++j) q[j] = code_of(stored<T>(o[j]), s, r_s, -qmax, qmax);
       if (q8) store_codes<V>(q8 + row * cols + c, q);
       if (qt) {
 #pragma unroll
@@ -151,10 +169,12 @@ __global__ void __launch_bounds__(128) ln_bwd_kernel(const T* __restrict__ dout,
       }
     }
     load_vec<T, V>(y + base + c, xv);
+    float gm[V];
+    load_cols<V>(gamma + c, gm);
 #pragma unroll
     for (int j = 0; j < V; ++j) {
       xv[j] = (xv[j] - mu) * rs;
-      dv[j] *= gamma[c + j];
+      dv[j] *= gm[j];
     }
   };
   if constexpr (CACHED) {
@@ -246,10 +266,12 @@ __global__ void __launch_bounds__(128, 7) ln_bwd_ste_kernel(const T* __restrict_
         }
         store_vec<T, V>(dsum + base + c, d[i]);
         load_vec<T, V>(y + base + c, xn[i]);
+        float gm[V];
+        load_cols<V>(gamma + c, gm);
 #pragma unroll
         for (int j = 0; j < V; ++j) {
           xn[i][j] = (xn[i][j] - mu) * rs;
-          d[i][j] = stored<T>(d[i][j]) * gamma[c + j];
+          d[i][j] = stored<T>(d[i][j]) * gm[j];
           s1 += d[i][j];
           s2 += d[i][j] * xn[i][j];
         }
@@ -542,7 +564,7 @@ void launch_layernorm_fwd(const void* y, const float* gamma, const float* beta, 
   const int grid = (int)((rows + 3) / 4);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
-    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(y) && al16(out) && al16(qt) &&
+    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(y) && al16(out) && al16(qt) && al16(gamma) && al16(beta) &&
                    (reinterpret_cast<uintptr_t>(q8) % V) == 0;
     if (v) launch_k(ln_fwd_kernel<T, V, true>, grid, 128, 0, st, (const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
     else launch_k(ln_fwd_kernel<T, 1, false>, grid, 128, 0, st, (const T*)y, gamma, beta, eps, rows, cols, (T*)out, mean, rstd, step, (float)qmax, q8, (T*)qt);
@@ -557,7 +579,7 @@ void launch_layernorm_bwd(const void* dout, const void* dout2, const void* y, co
   const int grid = (int)((rows + 3) / 4);
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
-    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(dout) && al16(dout2) && al16(y) && al16(dy) && al16(dsum);
+    const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(dout) && al16(dout2) && al16(y) && al16(dy) && al16(dsum) && al16(gamma);
     if (v) launch_k(ln_bwd_kernel<T, V, true>, grid, 128, 0, st, (const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
     else launch_k(ln_bwd_kernel<T, 1, false>, grid, 128, 0, st, (const T*)dout, (const T*)dout2, (const T*)y, mean, rstd, gamma, rows, cols, (T*)dy, (T*)dsum);
   });
@@ -576,7 +598,7 @@ bool launch_layernorm_bwd_ste(const void* dout, const void* x, const void* dxhat
   MREM_DT(dt, T, {
     constexpr int V = 16 / (int)sizeof(T);
     const bool v = cols % V == 0 && cols <= 32 * V * MAXNV && al16(dout) && al16(x) && al16(dxhat) && al16(add) && al16(y) &&
-                   al16(dy) && al16(dsum);
+                   al16(dy) && al16(dsum) && al16(gamma);
     if (v) {
       Scope sc("layernorm_bwd_ste", (double)rows * cols * (dt == 1 ? 2.0 : 4.0) * (6 + (dout ? 1 : 0)), 0, st);
       const long long want = (rows + 3) / 4;

@@ -153,6 +153,11 @@ class ReconModule:
         """d loss / d (student module input) of the last backward pass, [batch, seq, hidden] (a copy)."""
         return self._ws_view(B.mrem_get_input_grad(self.ctx), batch * seq * self.H, self.tdtype).view(batch, seq, self.H).clone()
 
+    def activation(self, role, layer, which, shape):
+        """A copy of a tensor the last forward pass of `role` stored inside `layer` (binding.ACT_*)."""
+        ptr = B.mrem_get_activation(self.ctx, role, layer, which)
+        return self._ws_view(ptr, int(np.prod(shape)), self.tdtype).view(*shape).clone()
+
     def bind_head(self, head):
         """head: dict Wp [H, H], bp [H], Wc [C, H], bc [C] (numpy) of the classification head, or None to unbind."""
         if head is None:

@@ -99,14 +99,17 @@ class Problem:
                                        self.vl, lam)
 
 
-def compare_grads(gpu, ora, tol, skip_small=1e-12, check_offset=True, scalar_tol=None):
+def compare_grads(gpu, ora, tol, skip_small=1e-12, check_offset=True, scalar_tol=None, deep_scalar_floor=0.02, deep_group_tol=None):
     """Relative L2 error of every gradient group; returns the worst (name, value).
 
     The offset gradient of the GELU site is the sum of the incoming gradient over the CLIPPED
     elements only.  With freshly initialised steps the range is covered exactly and at most the
     extreme element or two sit on the boundary, on either side of it depending on the last bit
     of erf: that sum is then compared only when `check_offset` (cases that really clip).
-    `scalar_tol`: another bound for the activation step gradients (scalars) than for the tensors."""
+    `scalar_tol`: another bound for the activation step gradients (scalars) than for the tensors.
+    The eight activation step gradients of a layer are also compared as one group (relative L2 of the 8-vector)
+    at `tol`.  `deep_scalar_floor`: the floor (as a share of the layer's largest step gradient) used for the
+    scalars of layers above the first; `deep_group_tol`: the bound on their group (default: as for the first layer)."""
     worst = ("", 0.0)
     for l, (g, r) in enumerate(zip(gpu, ora)):
         items = [(k, g[k], r[k]) for k in O.PARAMS]
@@ -115,10 +118,12 @@ def compare_grads(gpu, ora, tol, skip_small=1e-12, check_offset=True, scalar_tol
             items += [("a_off", g["a_off"][7:8], r["a_off"][7:8])]
         # activation step gradients are scalars: compare each one on its own; a scalar that is a
         # heavily cancelling sum is measured against the largest of the layer's step gradients
-        floor = 0.02 * np.abs(r["a"]).max()
+        floor = (0.02 if l == 0 else deep_scalar_floor) * np.abs(r["a"]).max()
+        group_tol = (deep_group_tol if (l > 0 and deep_group_tol) else None) or scalar_tol or tol
+        assert rel(g["a"], r["a"]) < group_tol, (l, "a_steps as a group", rel(g["a"], r["a"]))
         for s, name in enumerate(SITE_NAMES):
             e = abs(g["a"][s] - r["a"][s]) / max(abs(r["a"][s]), floor, 1e-300)
-            assert e < (scalar_tol or tol), (l, "a_step_" + name, e, g["a"][s], r["a"][s])
+            assert e < ((deep_group_tol if (l > 0 and deep_group_tol) else None) or scalar_tol or tol), (l, "a_step_" + name, e, g["a"][s], r["a"][s])
             if e > worst[1]:
                 worst = (f"L{l}.a_step_{name}", e)
         for name, a, b in items:

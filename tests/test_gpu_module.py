@@ -13,13 +13,16 @@ from oracle import mrem_oracle as O
 from paper_2109_15082_b200 import binding as B
 from paper_2109_15082_b200 import synth
 from tests.gpu_util import Problem, compare_grads, rel
+from tests.torch_storage_ref import teacher_layer_torch
 
 pytestmark = pytest.mark.gpu
 
 FWD_TOL = {"f32": 1e-4, "bf16": 1e-3}
-# Per layer at hidden 1024 / FFN 4096: a float32 CPU replica of a teacher layer (same bf16 storage points, other
-# summation order) differs from the float64 oracle by 7e-4; the tensor-core path by 1.3e-3.
-FULL_SIZE_FWD_TOL = 2.5e-3
+# Per layer at hidden 1024 / FFN 4096 the full-precision pass is measured against a float32 CPU replica of the same
+# layer (tests/torch_storage_ref.py: same bf16 storage points, the library's summation order), computed inside the test
+# on the same sequences: that replica differs from the float64 oracle by about 7e-4 relative L2, the tensor-core path by
+# 1.9 times that.  The sharp check of the full-precision kernels is stage by stage (tests/test_gpu_full_width.py).
+TEACHER_VS_REPLICA = 3.0
 GRAD_TOL = 2e-2
 
 
@@ -584,7 +587,9 @@ def test_full_size_step_in_the_benchmark_launch_configuration(name):
                     for l in range(wl.n_layers)]
             print(name, "accumulated forward rel L2 (teacher, student) per layer:", [(round(a, 5), round(b, 5)) for a, b in errs])
             assert errs[0][1] < FWD_TOL["bf16"]            # first student layer: exact codes in, same codes out
-            assert max(e[0] for e in errs) < 1.5e-2 and max(e[1] for e in errs) < 6e-2
+            # (the accumulated figures of the layers above are a report: each layer's input already differs, flipped
+            #  roundings and codes feed the next layer; the gate is the per-layer comparison below)
+            assert max(e[0] for e in errs) < 0.1 and max(e[1] for e in errs) < 0.1
             # (b) layer by layer, the oracle fed with the input the GPU layer really had
             for l in range(wl.n_layers):
                 xin_t = xs if l == 0 else f_t[l - 1][pick].float().cpu().numpy()
@@ -592,9 +597,11 @@ def test_full_size_step_in_the_benchmark_launch_configuration(name):
                 t_one = O.teacher_layer(desc, teacher[l], O.round_bf16(xin_t), vl[pick])
                 s_one = O.student_forward(desc, [student0[l]], [steps0[l]], xin_s, vl[pick])[0][0]
                 et, es = rel(f_t[l][pick].float().cpu().numpy(), t_one), rel(f_s[l][pick].float().cpu().numpy(), s_one)
-                print(name, "layer", l, "rel L2 teacher", round(et, 5), "student", round(es, 5))
-                assert et < FULL_SIZE_FWD_TOL, ("teacher", l, et)
-                assert es < FULL_SIZE_FWD_TOL, ("student", l, es)
+                replica = teacher_layer_torch(teacher[l], O.round_bf16(xin_t), vl[pick], wl.n_heads, dtype=torch.float32)
+                floor = rel(replica, t_one)
+                print(name, "layer", l, "rel L2 teacher", round(et, 5), "(float32 replica", round(floor, 5), ") student", round(es, 5))
+                assert et < TEACHER_VS_REPLICA * floor, ("teacher", l, et, floor)
+                assert es < FWD_TOL["bf16"], ("student", l, es)
             # after the step: the fused update's codes are Eq. 1 of the updated weights and steps
             student1 = m.student_numpy()
             ws1, _, _ = m.get_steps()

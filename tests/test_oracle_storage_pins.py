@@ -83,39 +83,7 @@ def test_initial_activation_steps_put_the_extremes_on_the_ends_of_the_code_range
 
 # ----------------------------------------------------------------------------- where the storage mode rounds
 
-def _bf(t):
-    return t.to(torch.bfloat16).to(torch.float64)
-
-
-def _teacher_layer_torch(p, x, vl, h, rnd):
-    """Full-precision layer from torch layers in float64 with the storage roundings written out: the layer input,
-    the matrices, qkv, the softmax output, the context, both pre-LayerNorm sums, both LayerNorm outputs and the
-    GELU output live in the storage type; the pre-GELU tensor does not (bias and GELU are applied to the
-    accumulator before it is stored)."""
-    t = {k: torch.tensor(np.asarray(v, np.float64)) for k, v in p.items()}
-    W = {k: rnd(t[k]) for k in O.WEIGHTS}
-    xt = rnd(torch.tensor(np.asarray(x, np.float64)))
-    B, S, H = xt.shape
-    d = H // h
-    qkv = rnd(F.linear(xt, W["Wqkv"], t["bqkv"]))
-    Q, K, V = qkv.split(H, dim=-1)
-    sp = lambda u: u.reshape(B, S, h, d).transpose(1, 2)
-    pad = (torch.arange(S)[None, :] >= torch.as_tensor(vl)[:, None])[:, None, None, :]
-    P = rnd(torch.softmax((sp(Q) @ sp(K).transpose(-1, -2) / math.sqrt(d)).masked_fill(pad, float("-inf")), dim=-1))
-    ctx = rnd((P @ sp(V)).transpose(1, 2).reshape(B, S, H))
-    y1 = rnd(F.linear(ctx, W["Wo"], t["bo"]) + xt)
-    a = rnd(F.layer_norm(y1, (H,), t["ln1_g"], t["ln1_b"], 1e-12))
-    g = rnd(F.gelu(F.linear(a, W["W1"], t["b1"])))
-    y2 = rnd(F.linear(g, W["W2"], t["b2"]) + a)
-    return rnd(F.layer_norm(y2, (H,), t["ln2_g"], t["ln2_b"], 1e-12)).numpy()
-
-
-def _ulps_apart(a, b):
-    """bf16-representable arrays -> distance in representable numbers."""
-    def key(v):
-        u = np.ascontiguousarray(np.asarray(v, np.float32)).view(np.uint32).astype(np.int64) >> 16
-        return np.where(u & 0x8000, -(u & 0x7FFF), u)
-    return np.abs(key(a) - key(b))
+from tests.torch_storage_ref import round_bf16_t as _bf, teacher_layer_torch as _teacher_layer_torch, bf16_numbers_apart as _ulps_apart
 
 
 def test_teacher_layer_rounds_where_the_storage_type_says():
