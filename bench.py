@@ -134,20 +134,41 @@ def run_reference(args, wl):
     # sequence through one layer of the module costs the oracle about 0.2 s on 16 cores
     batch = max(1, min(wl.batch, 700 // max(args.steps + min(args.warmup, 1), 1)))
     val, threads, sample, sec = oracle_sample(wl, n_steps=max(1, args.steps), warmup=min(args.warmup, 1), batch=batch)
+    # `value` is the rate of the workload's metric; each timed step really ran `batch` sequences through ONE of the
+    # module's layers (`ms_timed_per_step`), and `ms_per_step` scales that to the whole module and batch
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec * wl.n_layers,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec * wl.n_layers * wl.batch / batch,
+            "ms_timed_per_step": 1e3 * sec, "extrapolated": True,
+            "extrapolation": {"layers_timed": 1, "layers": wl.n_layers, "sequences_timed": batch, "sequences": wl.batch},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "batch": wl.batch, "seq_len": wl.seq, "note": "CPU oracle (numpy float64)"},
+            "config": workload_config(wl, wl.calib or wl.batch * 8, 1),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
 
 
+def workload_config(wl, calib_n, world):
+    """The `config` object of the JSON line; both arms print the same keys."""
+    return {"workload": wl.name, "layers": wl.n_layers, "hidden": wl.hidden, "heads": wl.n_heads,
+            "ffn": wl.ffn, "batch": wl.batch, "seq_len": wl.seq, "bits": f"W{wl.w_bits}A{wl.a_bits}",
+            "calibration_sequences": calib_n, "parallelism": "replicas only" if world > 1 else "1 GPU",
+            "l2": "inputs larger than L2: calibration set, weights and optimizer state exceed 126 MB",
+            "launch": "one CUDA-graph replay per step + 2 gather kernels"}
+
+
 # ----------------------------------------------------------------------------- GPU leg
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over two whole steps
-NCU_DRAM_BYTES_PER_LAUNCH = {("large6_w4a8", "gemm_bf16_tcgen05"): 41.57e6}   # 39.22 MB read + 2.35 MB written
+def ncu_dram_bytes_per_launch(workload, kernel):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` from the committed ncu summary of this
+    workload (profiles/tc_gemm_dram_<workload>.md, line `traffic_bytes_per_launch <kernel> = <bytes>`), or None when
+    there is no such capture.  Returns (bytes, file)."""
+    import re
+    path = os.path.join(ROOT, "profiles", f"tc_gemm_dram_{workload}.md")
+    if not os.path.exists(path):
+        return None, None
+    m = re.search(r"traffic_bytes_per_launch\s+" + re.escape(kernel) + r"\s*=\s*([0-9.eE+]+)", open(path).read())
+    return (float(m.group(1)), os.path.relpath(path, ROOT)) if m else (None, None)
 
 
 def build_problem(wl, rank, torch, calib_n):
@@ -287,6 +308,8 @@ def main():
     ap.add_argument("--extras", action="store_true", help="also time the per-product step (Eq. 2), the output-logit term and the "
                     "embedding step of the first module, and add them to the JSON line as \"extras\"")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches (no programmatic dependent launch)")
+    ap.add_argument("--repeats", type=int, default=0, help="timed blocks of --steps steps each (0: as many as bring the timed "
+                    "region to about 2 s, between 3 and 64); the line reports the median block and the fastest")
     args = ap.parse_args()
 
     from paper_2109_15082_b200 import synth
@@ -315,7 +338,8 @@ def main():
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
         m, calib, lens = build_problem(wl, rank, torch, calib_n)
-        total = W + K
+        max_repeats = args.repeats if args.repeats > 0 else 64
+        total = W + K * min(max_repeats, 8)                           # batches drawn; later blocks start over at W
         n_batches = calib_n // wl.batch
         perm = np.concatenate([synth.permutation(rank, f"epoch{e}", calib_n)[: n_batches * wl.batch]
                                for e in range((total + n_batches - 1) // n_batches + 1)])
@@ -335,36 +359,48 @@ def main():
 
         stage(0)
         m.init_act_steps(xbuf, lenbuf, wl.batch, wl.seq)
-        opt = B.make_optim(lr=wl.lr, step=0, decay_total_steps=max(wl.steps, total))
+        opt = B.make_optim(lr=wl.lr, step=0, decay_total_steps=max(wl.steps, W + K * max_repeats + 64))
         side.synchronize()
         B.mrem_graph_capture_step(m.ctx, xbuf, xbuf, 0.0, lenbuf, wl.batch, wl.seq, m.t_out, m.s_out, m.loss, opt)
         kernels_per_step = B.mrem_graph_num_kernels(m.ctx) + 2
 
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for t in range(W):
+            if t == W - 2:
+                w0.record(side)
             stage(t)
             B.mrem_graph_launch(m.ctx)
+        w1.record(side)
         side.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        # timed blocks of exactly K steps each, every one bracketed by a barrier and a device synchronisation; enough of
+        # them for a timed region of about 2 s (the last two warm-up steps give the estimate)
+        repeats = args.repeats
+        if repeats <= 0:
+            est = D.max_over_ranks(w0.elapsed_time(w1) / 2, m.device)
+            repeats = int(min(64, max(3, np.ceil(2000.0 / max(K * est, 1e-3)))))
         sampler = ClockSampler(local)
-        if rank == 0:
-            sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(side)
-        for t in range(W, W + K):
-            stage(t)
-            B.mrem_graph_launch(m.ctx)
-        e1.record(side)
-        side.synchronize()
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        block_ms = []
+        for r in range(repeats):
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            if r == 0 and rank == 0:
+                sampler.start()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for k in range(K):
+                stage(W + (r * K + k) % (total - W))
+                B.mrem_graph_launch(m.ctx)
+            e1.record(side)
+            side.synchronize()
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            block_ms.append(D.max_over_ranks(e0.elapsed_time(e1), m.device))
         clocks = sampler.stop() if rank == 0 else None
-        ms = e0.elapsed_time(e1)
+        ms = float(statistics.median(block_ms))
         loss_last = float(m.loss[0])
         status = m.poll_status()
-        ms = D.max_over_ranks(ms, m.device)
 
         # ---- per-kernel timing (CUDA events around every launch of a few eager steps)
         B.mrem_trace_enable(m.ctx, 1)
@@ -420,12 +456,16 @@ def main():
         f = folded.setdefault(key, dict(name=key, ms=0.0, work=0.0, launches=0, is_flops=e["is_flops"]))
         f["ms"] += e["ms"]; f["work"] += e["work"]; f["launches"] += e["launches"]
     trace = list(folded.values())
+    # Each launch is event-timed on its own; the denominator for the tensor-bound kernels is the burst figure when the
+    # sampled SM clock sat at its maximum with no power cap (the conditions of a kernel timed alone), else the sustained one
+    at_max = bool(clocks and clocks.get("sm_mhz") and clocks["sm_mhz"] >= 0.98 * clocks["sm_max_mhz"] and "sw_power_cap" not in clocks["reasons"])
+    tensor_peak = "bf16_burst" if at_max else "bf16_sustained"
     kernels = []
     for e in sorted(trace, key=lambda e: -e["ms"]):
         per_launch_ms = e["ms"] / max(e["launches"], 1)
         if e["is_flops"]:
             ach = e["work"] / (e["ms"] * 1e-3) / 1e12
-            peak = pk["bf16_sustained"] * (INT8_OVER_BF16 if "i8" in e["name"] else 1.0)
+            peak = pk[tensor_peak] * (INT8_OVER_BF16 if "i8" in e["name"] else 1.0)
             unit, bound = "TFLOP/s", "tensor"
         else:
             ach = e["work"] / (e["ms"] * 1e-3) / 1e9
@@ -436,21 +476,21 @@ def main():
     top = kernels[0]
     # DRAM bytes per launch of the dominant kernel from the committed ncu capture of this workload
     # (profiles/tc_gemm_dram_large6_w4a8.md); known only for that kernel on that workload
-    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, top["name"]))
+    traffic, traffic_file = ncu_dram_bytes_per_launch(wl.name, top["name"])
     roofline = {"kernel": top["name"], "bound": top["bound"], "achieved": top["achieved"], "peak": top["peak"],
                 "unit": top["unit"], "frac": top["frac"], "traffic": traffic,
-                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, ncu)" if traffic else None,
-                "peak_source": pk["source"] + (" bf16 sustained" if top["bound"] == "tensor" else " copy bandwidth"),
+                "traffic_unit": f"bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, ncu; {traffic_file})" if traffic else None,
+                "peak_source": pk["source"] + ((" bf16 burst (SM clock at maximum, no power cap, during the run)" if at_max else
+                                               " bf16 sustained (SM clock below maximum or power cap active during the run)")
+                                              if top["bound"] == "tensor" else " copy bandwidth"),
+                "int8_peak": "assumed: 2 x the measured bf16 figure (nominal dense ratio), not measured",
                 "timed": f"CUDA events around each launch of {n_trace} eager steps"}
 
     line = {"metric": METRIC, "value": D.whole_job_rate(tokens, K, world, ms), "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "warmup": W, "ms_per_step": ms / K, "repeats": repeats, "ms_per_step_min": min(block_ms) / K,
+            "timed_region_ms": sum(block_ms), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16+int8", "data": "synthetic",
-            "config": {"workload": wl.name, "layers": wl.n_layers, "hidden": wl.hidden, "heads": wl.n_heads,
-                       "ffn": wl.ffn, "batch": wl.batch, "seq_len": wl.seq, "bits": f"W{wl.w_bits}A{wl.a_bits}",
-                       "calibration_sequences": calib_n, "parallelism": "replicas only" if world > 1 else "1 GPU",
-                       "l2": "inputs larger than L2: calibration set, weights and optimizer state exceed 126 MB",
-                       "launch": "one CUDA-graph replay per step + 2 gather kernels"},
+            "config": workload_config(wl, calib_n, world),
             "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_step * K, "roofline": roofline,
             "kernels": kernels,
             "gemm_shapes": [{"shape": e["name"], "launches_per_step": e["launches"] / n_trace,

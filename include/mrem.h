@@ -240,6 +240,36 @@ int32_t mrem_recon_step_host_wait(mrem_ctx* ctx, float* h_loss);
  * Turn it off (0) to get plain stream-ordered launches, e.g. when comparing timings. */
 int32_t mrem_set_programmatic_launch(int32_t on);
 
+/* ---- data-parallel use (Sec. 4.2 trains on several devices; Algorithm 2's step is linear in the batch) ---------
+ *
+ * The loss of Eq. 3 is a sum over the batch, so its gradient is the sum of the gradients of the batch's parts: R
+ * ranks that hold the same parameters and steps, each with batch/R of the sequences, obtain the whole batch's
+ * gradient by adding theirs.  Two hooks make that exact without any arithmetic outside the library:
+ * mrem_set_loss_share: from now on mrem_recon_loss multiplies its scale by `share` in (0, 1] (= this rank's sequences /
+ *   all sequences of the step; default 1), so that the losses and every gradient of the ranks ADD UP to the whole
+ *   batch's under loss_mean as under the plain sum.
+ * mrem_grad_bucket: the contiguous float32 range [*d_ptr, *d_ptr + *n_floats) inside the workspace that holds ALL
+ *   gradients of one layer after mrem_module_backward (the twelve parameters, then the weight-step, activation-step
+ *   and offset gradients; alignment gaps between them hold no data).  Sum that range over the ranks (one all-reduce per
+ *   layer, top layer first: the order in which the backward pass completes them), then call mrem_step.  The weight
+ *   matrices' slots hold the gradient with respect to the QUANTIZED weights; the straight-through mask and the
+ *   weight-step gradients are applied by mrem_step from the summed values (both are linear in it). */
+int32_t mrem_set_loss_share(mrem_ctx* ctx, float share);
+int32_t mrem_grad_bucket(mrem_ctx* ctx, int32_t layer, float** d_ptr, size_t* n_floats);
+
+/* Failure detection.  Every device-side wait of the tensor-core kernels (on a TMA-filled stage, on a tensor-core
+ * commit, on an accumulator hand-over) is bounded in time; a wait that runs out makes its kernel record a code in the
+ * context's status word, stop issuing work, release what it holds and return, so the context stays usable and the host
+ * learns of it through mrem_poll_status (MREM_ERR_TIMEOUT).
+ * mrem_set_wait_limit_ns: process-wide limit of one such wait for all launches made afterwards (default 2 s;
+ * 1 us .. 60 s, MREM_ERR_ARG otherwise).
+ * mrem_selftest_wait_limit: enqueues, on the context's stream, one block whose single wait can never be satisfied (an
+ * mbarrier nothing arrives at), using the library's own bounded wait and the current limit: after the limit the block
+ * reports exactly as a starved product would and returns.  Nothing faults and nothing waits longer than the limit;
+ * meant for checking the reporting path (set a limit of a millisecond or so first). */
+int32_t mrem_set_wait_limit_ns(uint64_t ns);
+int32_t mrem_selftest_wait_limit(mrem_ctx* ctx);
+
 /* Per context (default on): where the shapes allow it (bf16 storage, head size 64, seq <= 128, seq % 8 == 0)
  * the backward of the attention block (Sec. 3.1: the gradients of Q, K, V through the quantized scores,
  * softmax and context products, with the straight-through masks of the Q, K, V, P quantizers) runs as one

@@ -34,7 +34,8 @@ EXPORTS = (
     "mrem_trace_read", "mrem_invalidate_weight_codes", "mrem_recon_loss_noalloc", "mrem_set_programmatic_launch",
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
     "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head", "mrem_embed_workspace_bytes", "mrem_embed_step", "mrem_get_input_grad",
-    "mrem_get_activation",
+    "mrem_get_activation", "mrem_set_wait_limit_ns", "mrem_selftest_wait_limit",
+    "mrem_set_loss_share", "mrem_grad_bucket",
 )
 
 
@@ -220,6 +221,25 @@ def mrem_get_input_grad(ctx) -> int:
     out = C.c_void_p(0)
     _check(lib().mrem_get_input_grad(ctx, C.byref(out)), "mrem_get_input_grad", ctx)
     return out.value
+
+
+def mrem_set_loss_share(ctx, share):
+    _check(lib().mrem_set_loss_share(ctx, C.c_float(float(share))), "mrem_set_loss_share", ctx)
+
+
+def mrem_grad_bucket(ctx, layer):
+    """(device address, float32 count) of the range that holds every gradient of `layer`."""
+    ptr, n = C.c_void_p(0), C.c_size_t(0)
+    _check(lib().mrem_grad_bucket(ctx, int(layer), C.byref(ptr), C.byref(n)), "mrem_grad_bucket", ctx)
+    return ptr.value, n.value
+
+
+def mrem_set_wait_limit_ns(ns):
+    _check(lib().mrem_set_wait_limit_ns(C.c_uint64(int(ns))), "mrem_set_wait_limit_ns")
+
+
+def mrem_selftest_wait_limit(ctx):
+    _check(lib().mrem_selftest_wait_limit(ctx), "mrem_selftest_wait_limit", ctx)
 
 
 ACT_QKV, ACT_P, ACT_CTX, ACT_Y1, ACT_A, ACT_G, ACT_Y2 = range(7)

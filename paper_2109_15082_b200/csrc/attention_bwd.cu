@@ -39,6 +39,7 @@ struct AttnBwdParams {
   float *part_q, *part_k, *part_v, *part_p;   // [red_slots] each: one partial per CTA, the rest zeroed
   int red_slots;
   int* status;
+  unsigned long long wait_ns;  // limit of each wait on an mbarrier
 };
 
 __device__ __forceinline__ void ld16(const void* p, uint32_t* w) {
@@ -129,7 +130,7 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
       tma_load_4d(sV, &map_codes, bar, 0, 0, 2 * p.h + head, b);
       tma_load_4d(sK, &map_codes, bar, 0, 0, p.h + head, b);
       tma_load_4d(sQ, &map_codes, bar, 0, 0, head, b);
-      bool ok = mbar_wait(bar, 0);
+      bool ok = mbar_wait(bar, 0, p.wait_ns);
       if (!ok) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_TMA);
       tc_fence_after();
       if (ok) {      // dP_hat [queries x keys] = dctx [q x d] * V_q^T
@@ -142,14 +143,14 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
       const uint32_t f = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(HD >> 3) << 17) | (8u << 24);
       const uint32_t id_tt = f | (1u << 15) | (1u << 16);     // A and B MN-major
       const uint32_t id_nt = f | (1u << 16);                  // A K-major, B MN-major
-      ok = ok && mbar_wait(smem_u32(&bar_p), 0);
+      ok = ok && mbar_wait(smem_u32(&bar_p), 0, p.wait_ns);
       if (!ok) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_EPI);
       tc_fence_after();
       if (ok)
         for (int ks = 0; ks < ksteps; ++ks)       // dV_hat [keys x d] = P_q^T [keys x q] * dctx [q x d]
           tc_mma<0>(tmem + TMEM_DV, smem_desc(sX + ks * 2048, 16384u, 1024u), smem_desc(sD + ks * 2048, 8192u, 1024u), id_tt, (uint32_t)(ks != 0));
       tc_commit(smem_u32(&bar_b));
-      ok = ok && mbar_wait(smem_u32(&bar_s), 0);
+      ok = ok && mbar_wait(smem_u32(&bar_s), 0, p.wait_ns);
       if (!ok) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_EPI);
       tc_fence_after();
       if (ok) {
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
     const int n_chunks = (p.S + 31) / 32;
     const long long prow = (((long long)b * p.h + head) * p.S + r) * p.S;
     float ds_p = 0.f;
-    bool got = mbar_wait(smem_u32(&bar_a), 0);
+    bool got = mbar_wait(smem_u32(&bar_a), 0, p.wait_ns);
     tc_fence_after();
     // ---- pass A: STE of the P quantizer, row dot product, the codes of P into the operand tile
     float dot = 0.f;
@@ -242,7 +243,7 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
         for (int j = 0; j < 16; ++j) sw[i][j] = 0u;
       }
     }
-    got = mbar_wait(smem_u32(&bar_b), 0) && got;
+    got = mbar_wait(smem_u32(&bar_b), 0, p.wait_ns) && got;
     tc_fence_after();
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
@@ -261,7 +262,7 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
     uint32_t a[32];
     tmem_ld32(trow + (uint32_t)(TMEM_DV + half * 32), a);           // complete since bar_b
     const float ds_v = ste_store(a, row_ok, p.qkv + grow + 2 * p.H, p.dqkv + grow + 2 * p.H, s_p, s_v, p.q_lo, p.q_hi);
-    got = mbar_wait(smem_u32(&bar_o), 0) && got;
+    got = mbar_wait(smem_u32(&bar_o), 0, p.wait_ns) && got;
     if (!__all_sync(0xffffffffu, got) && lane == 0) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_MMA);
     tc_fence_after();
     tmem_ld32(trow + (uint32_t)(TMEM_DQ + half * 32), a);
@@ -313,6 +314,7 @@ int launch_attention_bwd(const void* qkv_codes, const void* qkv, const void* P, 
   p.part_q = part_q; p.part_k = part_k; p.part_v = part_v; p.part_p = part_p;
   p.red_slots = RED_BLOCKS;
   p.status = status;
+  p.wait_ns = g_wait_limit_ns;
   CUtensorMap mc, md;
   OperandDesc oc{qkv_codes, 3LL * H, HD, (long long)S * 3 * H, 0};
   int rc = make_operand_map(&mc, oc, 2, S, HD, 3 * h, B, 128, HD);

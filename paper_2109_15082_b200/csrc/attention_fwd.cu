@@ -38,6 +38,7 @@ struct AttnParams {
   int8_t* ctx_q8;            // [B*S, H]
   bf16* ctx_qt;              // [B*S, H]
   int* status;
+  unsigned long long wait_ns;  // limit of each wait on an mbarrier
 };
 
 __device__ __forceinline__ void store16(void* p, const uint32_t* w) {
@@ -91,7 +92,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
         tma_load_4d(sK + i * 16384, &map_qkv, bar, 0, i * 128, p.h + head, b);
         tma_load_4d(sV + i * 16384, &map_qkv, bar, 0, i * 128, 2 * p.h + head, b);
       }
-      bool ok = mbar_wait(bar, 0);
+      bool ok = mbar_wait(bar, 0, p.wait_ns);
       if (!ok) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_TMA);
       tc_fence_after();
       // ---- scores: [128 x n16] = Q [128 x 64] * K^T, in pieces of at most 256 keys
@@ -107,7 +108,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
       }
       tc_commit(smem_u32(&bar_s));
       // ---- context: [128 x 64] = P [128 x keys] * V [keys x 64]  (V is the MN-major operand)
-      ok = ok && mbar_wait(smem_u32(&bar_p), 0);
+      ok = ok && mbar_wait(smem_u32(&bar_p), 0, p.wait_ns);
       if (!ok) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_EPI);
       tc_fence_after();
       if (ok) {
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     const float ps = quant ? *p.p_step : 1.f, r_ps = __frcp_rn(ps);
     const uint32_t trow = tmem + ((uint32_t)(quad * 32) << 16);
     const int n_chunks = (p.S + 31) / 32;
-    const bool got = mbar_wait(smem_u32(&bar_s), 0);
+    const bool got = mbar_wait(smem_u32(&bar_s), 0, p.wait_ns);
     if (!__all_sync(0xffffffffu, got) && lane == 0) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_MMA);
     tc_fence_after();
     // scores in units of log2(e): exp(alpha * a - max) = 2^(alpha2 * a - max2); alpha > 0, so the maximum
@@ -214,7 +215,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     tc_fence_before();
     mbar_arrive(smem_u32(&bar_p));
     // ---- context row
-    const bool got2 = mbar_wait(smem_u32(&bar_o), 0);
+    const bool got2 = mbar_wait(smem_u32(&bar_o), 0, p.wait_ns);
     if (!__all_sync(0xffffffffu, got2) && lane == 0) atomicCAS(p.status, 0, (int)DEV_TIMEOUT_MMA);
     tc_fence_after();
     float calpha = 1.f;
@@ -283,6 +284,7 @@ int launch_attention_fwd(const void* qkv, int B, int S, int h, int H, const int*
   p.c_step = c_step; p.c_qmax = (float)c_qmax;
   p.P = (bf16*)P; p.P_qt = (bf16*)P_qt; p.ctx = (bf16*)ctx; p.ctx_q8 = ctx_q8; p.ctx_qt = (bf16*)ctx_qt;
   p.status = status;
+  p.wait_ns = g_wait_limit_ns;
   // one map over the [tokens, 3H] tensor: (64 of a head, S rows, 3h head slots, B)
   OperandDesc op{qkv, 3LL * H, HD, (long long)S * 3 * H, 0};
   CUtensorMap map;

@@ -14,6 +14,9 @@ enum GemmRc : int { GEMM_OK = 0, GEMM_ERR_ARG = -1, GEMM_ERR_ALIGN = -2, GEMM_ER
 int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B, const GemmShape& g,
             const Epilogue& epi, int block_n, int* d_status, int sm_count, cudaStream_t stream);
 
+// Verification aid: one block that lets a bounded wait run out (limit_ns) and reports DEV_TIMEOUT_TMA in *d_status.
+cudaError_t launch_wait_probe(int* d_status, unsigned long long limit_ns, cudaStream_t stream);
+
 // Several bf16 products with plain fp32 outputs (alpha and row bias only) as one persistent launch over the
 // joint tile list: the weight-gradient products of a layer.  Operands as in tc_gemm, one batch each.
 constexpr int MAX_GEMM_GROUP = 4;

@@ -24,6 +24,7 @@ struct TcParams {
   uint32_t idesc;
   Epilogue epi;
   int* status;
+  unsigned long long wait_ns;          // limit of each wait on an mbarrier
 };
 
 __device__ __forceinline__ void fail(const TcParams& p, int code, volatile int* abort_flag) {

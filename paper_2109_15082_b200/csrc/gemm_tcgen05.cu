@@ -77,7 +77,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
         const TileCoord t = decode_tile(p, tile);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait_or_abort(smem_u32(&empty_bar[stage]), phase ^ 1u, vabort)) {
+          if (!mbar_wait_or_abort(smem_u32(&empty_bar[stage]), phase ^ 1u, vabort, p.wait_ns)) {
             if (!*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
             ok = false;
             break;
@@ -122,14 +122,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t a_lo = a_lo0, b_lo = b_lo0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-        if (!mbar_wait_or_abort(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, vabort)) {
+        if (!mbar_wait_or_abort(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, vabort, p.wait_ns)) {
           if (!*vabort) fail(p, DEV_TIMEOUT_EPI, vabort);
           break;
         }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * p.block_n);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait_or_abort(smem_u32(&full_bar[stage]), phase, vabort)) {
+          if (!mbar_wait_or_abort(smem_u32(&full_bar[stage]), phase, vabort, p.wait_ns)) {
             if (!*vabort) fail(p, DEV_TIMEOUT_TMA, vabort);
             ok = false;
             break;
@@ -174,7 +174,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (nfull > 0 && res_bf16) fetch_res_bf16(e, row_off + col_begin, row_ok, res0);   // in flight during the wait
       const float rb = (e.row_bias && row_ok) ? e.row_bias[row] : 0.f;
       // every lane polls; the decision is made warp-uniform before any .sync.aligned instruction
-      const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort);
+      const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort, p.wait_ns);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0 && !*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
         break;
@@ -201,6 +201,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+}
+
+// One thread waits, with the library's bounded wait, on an mbarrier that nothing ever arrives at; when the limit runs
+// out it reports through the same status word and code as a product whose operand tile never landed, and returns.
+__global__ void wait_probe_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && !mbar_wait_or_abort(smem_u32(&bar), 0u, &abort_flag, limit_ns)) atomicCAS(status, 0, (int)DEV_TIMEOUT_TMA);
 }
 
 // ------------------------------------------------------------------ host side
@@ -297,6 +311,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   p.a_mn = A.mn_contig; p.b_mn = B.mn_contig;
   p.epi = epi;
   p.status = d_status;
+  p.wait_ns = g_wait_limit_ns;
   // instruction descriptor: D format, A/B formats, majors, N >> 3, M >> 4
   uint32_t idesc = 0;
   if (kind == 0) {
@@ -346,6 +361,10 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   }, 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream, 0);
   if (launch_k(kern, grid, GEMM_THREADS, smem, stream, ma, mb, p) != cudaSuccess) return GEMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
+}
+
+cudaError_t launch_wait_probe(int* d_status, unsigned long long limit_ns, cudaStream_t stream) {
+  return launch_k(wait_probe_kernel, 1, 32, 0, stream, d_status, limit_ns);
 }
 
 }  // namespace mrem

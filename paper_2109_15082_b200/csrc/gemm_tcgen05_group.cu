@@ -88,7 +88,7 @@ tc_gemm_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_consta
         const CUtensorMap* map_b = &maps.b[pi];
         const TileCoord t = decode_tile(p, local);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait_or_abort(smem_u32(&empty_bar[stage]), phase ^ 1u, vabort)) {
+          if (!mbar_wait_or_abort(smem_u32(&empty_bar[stage]), phase ^ 1u, vabort, g.p[0].wait_ns)) {
             if (!*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
             ok = false;
             break;
@@ -135,14 +135,14 @@ tc_gemm_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_consta
         const uint32_t a_hi = (uint32_t)(proto_a >> 32), b_hi = (uint32_t)(proto_b >> 32);
         const uint32_t a_lo0 = (uint32_t)proto_a, b_lo0 = (uint32_t)proto_b;
         uint32_t a_lo = a_lo0 + (uint32_t)stage * stage_adv, b_lo = b_lo0 + (uint32_t)stage * stage_adv;
-        if (!mbar_wait_or_abort(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, vabort)) {
+        if (!mbar_wait_or_abort(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, vabort, g.p[0].wait_ns)) {
           if (!*vabort) fail(p, DEV_TIMEOUT_EPI, vabort);
           break;
         }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * p.block_n);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait_or_abort(smem_u32(&full_bar[stage]), phase, vabort)) {
+          if (!mbar_wait_or_abort(smem_u32(&full_bar[stage]), phase, vabort, g.p[0].wait_ns)) {
             if (!*vabort) fail(p, DEV_TIMEOUT_TMA, vabort);
             ok = false;
             break;
@@ -182,7 +182,7 @@ tc_gemm_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_consta
       const long long row_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1 + (long long)row * e.ldc;
       const int nfull = col_begin < p.N ? min((p.N - col_begin) >> 5, cols_per_warp >> 5) : 0;   // N % 32 == 0 (host)
       const float rb = (e.row_bias && row_ok) ? e.row_bias[row] : 0.f;
-      const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort);
+      const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort, g.p[0].wait_ns);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0 && !*vabort) fail(p, DEV_TIMEOUT_MMA, vabort);
         break;
@@ -244,6 +244,7 @@ int tc_gemm_group(const GemmGroupItem* items, int n, int* d_status, int sm_count
     p.a_mn = it.A.mn_contig; p.b_mn = it.B.mn_contig;
     p.epi = it.epi;
     p.status = d_status;
+    p.wait_ns = g_wait_limit_ns;
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(it.A.mn_contig ? 1 : 0) << 15) |
               ((uint32_t)(it.B.mn_contig ? 1 : 0) << 16) | ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
     int rc = make_operand_map(&maps.a[i], it.A, 2, p.M, p.K, 1, 1, BLOCK_M, block_k);

@@ -78,9 +78,14 @@ __global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, l
   const int vcols = cols / V;
   const long long total = rows * vcols;
   float ds = 0.f, dofs = 0.f;
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    const long long r = i / vcols;
-    const int c = (int)(i - r * vcols) * V;
+  // (row, vector) of this thread's element, advanced by the grid stride without a division per element
+  const long long stride = (long long)gridDim.x * blockDim.x, i0 = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  const long long r_step = stride / vcols;
+  const int v_step = (int)(stride - r_step * vcols);
+  long long r = i0 / vcols;
+  int cv = (int)(i0 - r * vcols);
+  for (long long i = i0; i < total; i += stride) {
+    const int c = cv * V;
     float xv[V], d[V];
     load_vec<T, V>(x + r * ld_x + c, xv);
     load_vec<T, V>(dxhat + r * ld_d + c, d);
@@ -88,7 +93,7 @@ __global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, l
     for (int j = 0; j < V; ++j) {
       const float z = qz(xv[j], s, r_s, off, has_off);
       const bool in = z >= lo && z <= hi;
-      ds += d[j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+      ds += d[j] * (rne_magic(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
       dofs += in ? 0.f : d[j];
       d[j] = in ? d[j] : 0.f;
     }
@@ -99,6 +104,9 @@ __global__ void __launch_bounds__(256) ste_act_kernel(const T* __restrict__ x, l
       for (int j = 0; j < V; ++j) d[j] += e[j];
     }
     store_vec<T, V>(dx + r * ld_dx + c, d);
+    r += r_step;
+    cv += v_step;
+    if (cv >= vcols) { cv -= vcols; ++r; }
   }
   ds = block_sum(ds, sh);
   dofs = block_sum(dofs, sh);
@@ -134,7 +142,7 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
       if (quantized) {
         const float z = qz(stored<T>(uv[j] * cdf), s, r_s, off, has_off);
         const bool in = z >= lo && z <= hi;
-        ds += d[j] * ((float)qcode(z, lo, hi) - (in ? z : 0.f));
+        ds += d[j] * (rne_magic(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
         dofs += in ? 0.f : d[j];
         d[j] = in ? d[j] : 0.f;
       }

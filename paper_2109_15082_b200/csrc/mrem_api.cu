@@ -9,6 +9,7 @@ using namespace mrem;
 namespace mrem {
 thread_local Tracer* g_tracer = nullptr;
 int g_programmatic_launch = 1;
+unsigned long long g_wait_limit_ns = 2000000000ull;   // 2 s
 }
 
 namespace {
@@ -451,6 +452,36 @@ int32_t mrem_invalidate_weight_codes(mrem_ctx* c) {
 
 int32_t mrem_set_programmatic_launch(int32_t on) {
   mrem::g_programmatic_launch = on ? 1 : 0;
+  return MREM_OK;
+}
+
+int32_t mrem_set_loss_share(mrem_ctx* c, float share) {
+  if (!c) return MREM_ERR_ARG;
+  if (!(share > 0.f && share <= 1.f)) return fail(c, MREM_ERR_ARG, "set_loss_share: share outside (0, 1]");
+  c->loss_share = share;
+  return MREM_OK;
+}
+
+int32_t mrem_grad_bucket(mrem_ctx* c, int32_t layer, float** d_ptr, size_t* n_floats) {
+  if (!c || !d_ptr || !n_floats) return MREM_ERR_ARG;
+  if (layer < 0 || layer >= c->d.n_layers) return fail(c, MREM_ERR_ARG, "grad_bucket: layer");
+  const LayerGrad& g = c->grad[layer];
+  // the layer's gradients were carved back to back: parameters, weight steps, activation steps, offsets
+  *d_ptr = g.p[0];
+  *n_floats = (size_t)((g.off + N_SITES) - g.p[0]);
+  return MREM_OK;
+}
+
+int32_t mrem_set_wait_limit_ns(uint64_t ns) {
+  if (ns < 1000ull || ns > 60000000000ull) return MREM_ERR_ARG;       // 1 us .. 60 s
+  mrem::g_wait_limit_ns = ns;
+  return MREM_OK;
+}
+
+int32_t mrem_selftest_wait_limit(mrem_ctx* c) {
+  if (!c) return MREM_ERR_ARG;
+  if (launch_wait_probe(c->status, mrem::g_wait_limit_ns, c->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+    return fail(c, MREM_ERR_CUDA, "selftest_wait_limit: launch failed");
   return MREM_OK;
 }
 

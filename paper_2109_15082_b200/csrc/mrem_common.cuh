@@ -26,6 +26,7 @@ enum DeviceStatus : int {
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+extern unsigned long long g_wait_limit_ns;   // limit of every device-side wait, copied into each launch's parameters
 extern int g_programmatic_launch;      // 1: launch with programmatic stream serialization (default)
 
 template <typename... KArgs, typename... Args>
@@ -115,19 +116,46 @@ __device__ __forceinline__ float quotient(float x, float s, float r_s) {
   return __fmaf_rn(__fmaf_rn(-z0, s, x), r_s, z0);
 }
 
-// The integer code of Eq. 1, nearest integer (ties to even) of clip(n / s, lo, hi), bit for bit what the IEEE
-// division gives, at a third of its instructions: the three-instruction quotient is within one ulp of the correctly
-// rounded one (1.5e-5 at |z| <= 255), so the two can round to different integers only when the quotient lies that
-// close to a half-integer; any value within 2^-10 of one is decided by the division instruction instead (about one
-// element in a thousand).  A quotient beyond the range is clipped to the same bound by both.  r_s = RN(1 / s).
-__device__ __forceinline__ int code_of(float n, float s, float r_s, float lo, float hi) {
-  float zc = fminf(fmaxf(quotient(n, s, r_s), lo), hi);
-  float q = rintf(zc);
-  if (fabsf(fabsf(zc - q) - 0.5f) < 9.765625e-4f) {
-    zc = fminf(fmaxf(__fdiv_rn(n, s), lo), hi);
-    q = rintf(zc);
+// Nearest integer (ties to even) of a float with |z| < 2^22 by adding and subtracting 1.5 * 2^23: two additions on the
+// ordinary pipes instead of two conversions.  `bits` receives the bit pattern of z + 1.5 * 2^23, whose low mantissa bits are
+// the integer in two's complement (its low byte IS the 8-bit code).
+constexpr float ROUND_MAGIC = 12582912.f;
+__device__ __forceinline__ float rne_magic(float z, uint32_t& bits) {
+  const float t = __fadd_rn(z, ROUND_MAGIC);
+  bits = __float_as_uint(t);
+  return __fsub_rn(t, ROUND_MAGIC);
+}
+__device__ __forceinline__ float rne_magic(float z) { uint32_t b; return rne_magic(z, b); }
+
+// The integer code of Eq. 1, nearest integer (ties to even) of clip(n / s, lo, hi), bit for bit what the IEEE division
+// gives, at a fraction of its instructions; returned as a float, with the bit pattern that carries its low byte.
+// r_s = RN(1 / s).  The three-instruction quotient is within one ulp of the correctly rounded one (1.5e-5 at |z| <= 255),
+// so the two can round to different integers only when the quotient lies that close to a half-integer: any value within
+// 2^-10 of one is decided by the division instruction instead (about one element in a thousand).  A quotient beyond the
+// range is clipped to the same bound by both.  EXACT_QUOTIENT: the numerator is a bfloat16 value, for which the quotient
+// IS the correctly rounded one (see quotient()) and no second look is needed.
+template <bool EXACT_QUOTIENT>
+__device__ __forceinline__ float code_f(float n, float s, float r_s, float lo, float hi, uint32_t& bits) {
+  // (the first product is kept inside [lo - 1, hi + 1]: unchanged wherever the code is not simply a bound, and a
+  //  numerator so large that n * r_s overflows then still ends on the bound of its sign instead of a NaN)
+  const float z0 = fminf(fmaxf(__fmul_rn(n, r_s), lo - 1.f), hi + 1.f);
+  float zc = fminf(fmaxf(__fmaf_rn(__fmaf_rn(-z0, s, n), r_s, z0), lo), hi);
+  float q = rne_magic(zc, bits);
+  if constexpr (!EXACT_QUOTIENT) {
+    if (fabsf(fabsf(zc - q) - 0.5f) < 9.765625e-4f) {
+      zc = fminf(fmaxf(__fdiv_rn(n, s), lo), hi);
+      q = rne_magic(zc, bits);
+    }
   }
-  return (int)q;
+  return q;
+}
+__device__ __forceinline__ int code_of(float n, float s, float r_s, float lo, float hi) {
+  uint32_t b;
+  return (int)code_f<false>(n, s, r_s, lo, hi, b);
+}
+// low bytes of four words -> one word (byte i from b_i)
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
+  return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
 }
 
 // GELU(u) = u * Phi(u) with the erf form.  erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x), x >= 0

@@ -492,13 +492,13 @@ int32_t mrem_recon_loss(mrem_ctx* c, float* loss_total, float* loss_per_layer) {
   TracerGuard tg(c->trace_on ? &c->tracer : nullptr);
   if (!c->have_teacher || !c->have_student) return fail(c, MREM_ERR_ORDER, "recon_loss: needs a teacher and a student forward of the same batch");
   const long long n = (long long)c->cur_batch * c->cur_seq * c->d.hidden;
-  const float cc = c->d.loss_mean ? 1.f / (float)n : 1.f;
+  const float cc = (c->d.loss_mean ? 1.f / (float)n : 1.f) * c->loss_share;
   launch_loss(c->s_out, c->t_out, c->d.n_layers, n, cc, c->dF, c->loss_partial, c->status, c->dt, c->stream);
   launch_loss_finalize(c->loss_partial, c->d.n_layers, cc, loss_total, loss_per_layer, c->stream);
   if (c->head.wp) {
     // last module of the model: the output-logit term, its gradient added to the last layer's loss gradient
     const int L = c->d.n_layers, C = c->head.n_classes;
-    const float cz = c->d.loss_mean ? 1.f / (float)((long long)c->cur_batch * C) : 1.f;
+    const float cz = (c->d.loss_mean ? 1.f / (float)((long long)c->cur_batch * C) : 1.f) * c->loss_share;
     const long long last = (long long)(L - 1) * n;
     const int hrc = launch_head_logit_loss((const char*)c->s_out + last * c->esz, (const char*)c->t_out + last * c->esz, c->cur_batch,
                                            c->cur_seq, c->d.hidden, C, c->head.wp, c->head.bp, c->head.wc, c->head.bc, cz,

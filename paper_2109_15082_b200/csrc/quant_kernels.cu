@@ -90,6 +90,47 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const T* __restrict__
   }
 }
 
+// The vector form: TPR threads walk one row's 16-byte vectors (TPR divides the vector count of a row where possible),
+// 256 / TPR rows per block round; no index divisions, codes by code_f, packed stores.
+template <typename T, int V, int TPR>
+__global__ void __launch_bounds__(256) quantize_act_rows_kernel(const T* __restrict__ x, long long rows, int cols,
+                                                                long long ld_x, const float* __restrict__ step,
+                                                                const float* __restrict__ offset, float lo, float hi,
+                                                                int8_t* __restrict__ q8, long long ld_q8,
+                                                                T* __restrict__ qt, long long ld_qt, int seg_cols,
+                                                                const float* __restrict__ step1,
+                                                                const float* __restrict__ step2) {
+  pdl_trigger();
+  pdl_wait();
+  const float s0 = *step, s1 = seg_cols ? *step1 : s0, s2 = seg_cols ? *step2 : s0;
+  const float r0 = __frcp_rn(s0), r1 = __frcp_rn(s1), r2 = __frcp_rn(s2);
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  constexpr int RPB = 256 / TPR;
+  const int tr = threadIdx.x / TPR, tc = threadIdx.x % TPR, vcols = cols / V;
+  for (long long r = blockIdx.x * (long long)RPB + tr; r < rows; r += (long long)gridDim.x * RPB) {
+    const T* xr = x + r * ld_x;
+#pragma unroll 2
+    for (int cv = tc; cv < vcols; cv += TPR) {
+      const int c = cv * V;
+      float v[V];
+      load_vec<T, V>(xr + c, v);
+      const int seg = !seg_cols || c < seg_cols ? 0 : (c < 2 * seg_cols ? 1 : 2);
+      const float s = seg == 0 ? s0 : (seg == 1 ? s1 : s2), r_s = seg == 0 ? r0 : (seg == 1 ? r1 : r2);
+      uint32_t b[V];
+      if (sizeof(T) == 2 && !has_off) {                    // bfloat16 numerators: the quotient is the exact one
+#pragma unroll
+        for (int j = 0; j < V; ++j) v[j] = code_f<true>(v[j], s, r_s, lo, hi, b[j]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < V; ++j) v[j] = code_f<false>(has_off ? __fsub_rn(v[j], off) : v[j], s, r_s, lo, hi, b[j]);
+      }
+      if (q8) store_code_bytes<V>(q8 + r * ld_q8 + c, b);
+      if (qt) store_vec<T, V>(qt + r * ld_qt + c, v);
+    }
+  }
+}
+
 template <typename T, int V>
 __global__ void __launch_bounds__(256) mix_kernel(const T* __restrict__ f, const T* __restrict__ fh, float lam,
                                                   T* __restrict__ out, long long n) {
@@ -119,15 +160,19 @@ __global__ void __launch_bounds__(256) gelu_quant_kernel(const T* __restrict__ u
   for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * V; i < n; i += (long long)gridDim.x * blockDim.x * V) {
     float v[V];
     load_vec<T, V>(u + i, v);
-    int q[V];
+    uint32_t b[V];
+    if (sizeof(T) == 2 && !has_off) {
 #pragma unroll
-    for (int j = 0; j < V; ++j) q[j] = act_code(stored<T>(gelu_erf(v[j])), s, r_s, off, has_off, lo, hi);
-    if (q8) store_codes<V>(q8 + i, q);
-    if (qt) {
+      for (int j = 0; j < V; ++j) v[j] = code_f<true>(stored<T>(gelu_erf(v[j])), s, r_s, lo, hi, b[j]);
+    } else {
 #pragma unroll
-      for (int j = 0; j < V; ++j) v[j] = (float)q[j];
-      store_vec<T, V>(qt + i, v);
+      for (int j = 0; j < V; ++j) {
+        const float g = stored<T>(gelu_erf(v[j]));
+        v[j] = code_f<false>(has_off ? __fsub_rn(g, off) : g, s, r_s, lo, hi, b[j]);
+      }
     }
+    if (q8) store_code_bytes<V>(q8 + i, b);
+    if (qt) store_vec<T, V>(qt + i, v);
   }
 }
 
@@ -266,9 +311,16 @@ static void quantize_act_t(const T* x, long long rows, int cols, long long ld_x,
   constexpr int V = 16 / (int)sizeof(T);
   const bool v = vec_ok<T>(x, ld_x, cols) && vec_ok<T>(qt, ld_qt, cols) && seg_cols % V == 0 &&
                  (q8 == nullptr || ((reinterpret_cast<uintptr_t>(q8) % V) == 0 && ld_q8 % V == 0));
-  if (v)
-    launch_k(quantize_act_kernel<T, V>, grid_for(rows * cols / V), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt, seg_cols, step1, step2);
-  else
+  if (v) {
+    const int vcols = cols / V;
+#define MREM_QROWS(TPR) do { const long long want = (rows + 256 / TPR - 1) / (256 / TPR); \
+      launch_k(quantize_act_rows_kernel<T, V, TPR>, (int)(want < RED_BLOCKS ? want : RED_BLOCKS), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt, seg_cols, step1, step2); } while (0)
+    if (vcols % 128 == 0) MREM_QROWS(128);
+    else if (vcols % 64 == 0) MREM_QROWS(64);
+    else if (vcols >= 128) MREM_QROWS(128);
+    else MREM_QROWS(32);
+#undef MREM_QROWS
+  } else
     launch_k(quantize_act_kernel<T, 1>, grid_for(rows * cols), 256, 0, st, x, rows, cols, ld_x, step, offset, (float)lo, (float)hi, q8, ld_q8, qt, ld_qt, seg_cols, step1, step2);
 }
 

@@ -112,15 +112,11 @@ __global__ void __launch_bounds__(128) ln_fwd_kernel(const T* __restrict__ y, co
     for (int j = 0; j < V; ++j) o[j] = (o[j] - mu) * rs * gm[j] + bt[j];
     store_vec<T, V>(out + row * cols + c, o);
     if (step) {
-      int q[V];
+      uint32_t b[V];
 #pragma unroll
-      for (int j = 0; j < V; ++j) q[j] = code_of(stored<T>(o[j]), s, r_s, -qmax, qmax);
-      if (q8) store_codes<V>(q8 + row * cols + c, q);
-      if (qt) {
-#pragma unroll
-        for (int j = 0; j < V; ++j) o[j] = (float)q[j];
-        store_vec<T, V>(qt + row * cols + c, o);
-      }
+      for (int j = 0; j < V; ++j) o[j] = code_f<sizeof(T) == 2>(stored<T>(o[j]), s, r_s, -qmax, qmax, b[j]);   // bfloat16-valued numerators are exact
+      if (q8) store_code_bytes<V>(q8 + row * cols + c, b);
+      if (qt) store_vec<T, V>(qt + row * cols + c, o);
     }
   };
   if constexpr (CACHED) {
@@ -256,7 +252,7 @@ __global__ void __launch_bounds__(128, 7) ln_bwd_ste_kernel(const T* __restrict_
         for (int j = 0; j < V; ++j) {
           const float z = quotient(xv[j], s, r_s);
           const bool in = z >= lo && z <= hi;
-          ds += d[i][j] * ((float)__float2int_rn(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
+          ds += d[i][j] * (rne_magic(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
           d[i][j] = (in ? d[i][j] : 0.f) + e[j];
         }
         if (dout) {

@@ -7,7 +7,7 @@
 
 namespace mrem {
 
-constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait
+constexpr unsigned long long WAIT_NS = 2000000000ull;  // default limit of one wait: 2 s (the host may set another)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -36,26 +36,27 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: false when the phase did not complete within WAIT_NS.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: false when the phase did not complete within `limit_ns`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns = WAIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > WAIT_NS) return false;
+    if (global_ns() - t0 > limit_ns) return false;
   }
 }
 
 // The same wait for the roles of a pipelined kernel: the abort flag another role raised is looked at only
 // on the slow path, so the common case (phase already complete) costs one try_wait.
-__device__ __forceinline__ bool mbar_wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                   unsigned long long limit_ns = WAIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag || global_ns() - t0 > WAIT_NS) return false;
+    if (*abort_flag || global_ns() - t0 > limit_ns) return false;
   }
 }
 

@@ -83,6 +83,19 @@ __device__ __forceinline__ void store_vec(T* p, const float* v) {
   }
 }
 
+// V codes given as the bit patterns of rne_magic (low byte = the 8-bit code) packed into V bytes.
+template <int V>
+__device__ __forceinline__ void store_code_bytes(int8_t* p, const uint32_t* b) {
+  if constexpr (V == 1) {
+    p[0] = (int8_t)(b[0] & 0xff);
+  } else if constexpr (V == 4) {
+    *reinterpret_cast<uint32_t*>(p) = pack_low_bytes(b[0], b[1], b[2], b[3]);
+  } else {
+    static_assert(V == 8, "code vectors hold 1, 4 or 8 values");
+    *reinterpret_cast<uint2*>(p) = make_uint2(pack_low_bytes(b[0], b[1], b[2], b[3]), pack_low_bytes(b[4], b[5], b[6], b[7]));
+  }
+}
+
 // V integer codes (each fits 8 bits, signed or unsigned) packed into V bytes.
 template <int V>
 __device__ __forceinline__ void store_codes(int8_t* p, const int* q) {

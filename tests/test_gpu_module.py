@@ -480,6 +480,97 @@ def test_nonfinite_loss_is_reported_in_status():
         p.close()
 
 
+def test_bounded_wait_runs_out_is_reported_and_leaves_the_context_usable():
+    """Failure detection without a fault: a block waits, with the library's own bounded wait, on a barrier that nothing
+    arrives at; with the limit set to 1 ms it gives up, the status word reads MREM_ERR_TIMEOUT (once: polling clears
+    it), and the same context then runs a whole step that matches the oracle."""
+    import time
+    wl, kw = CASES["bf16_small"]
+    p = Problem(wl, **kw)
+    try:
+        m = p.m
+        with pytest.raises(B.MremError):
+            B.mrem_set_wait_limit_ns(10)                               # below a microsecond: refused
+        B.mrem_set_wait_limit_ns(1_000_000)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        B.mrem_selftest_wait_limit(m.ctx)
+        torch.cuda.synchronize()
+        waited = time.perf_counter() - t0
+        assert 0.0005 < waited < 0.5, waited                           # it waited for the limit, and not for the default 2 s
+        assert m.poll_status() == -7
+        assert m.poll_status() == 0
+        B.mrem_set_wait_limit_ns(2_000_000_000)
+        g = p.run_gpu()
+        r = p.run_oracle()
+        assert abs(g["loss"] - r["loss"]) / r["loss"] < GRAD_TOL
+        assert rel(g["grads"][0]["W1"], r["grads"][0]["W1"]) < GRAD_TOL
+        assert m.poll_status() == 0
+    finally:
+        B.mrem_set_wait_limit_ns(2_000_000_000)
+        p.close()
+
+
+def test_half_batch_gradient_buckets_add_up_to_the_full_batch():
+    """The data-parallel hooks on one GPU: two contexts with identical parameters take the two halves of a batch with a
+    loss share of 1/2 each; their per-layer gradient buckets (mrem_grad_bucket), added, are the full-batch context's
+    buckets, and so are the losses.  (The ranks of a real run do that sum with one all-reduce per layer; the 2-rank
+    logic is covered on CPU in tests/test_dist_cpu.py.)  Then DataParallelModule without a process group steps exactly
+    like the plain call sequence."""
+    from paper_2109_15082_b200.dist import DataParallelModule
+    wl = _wl("base3_w4a8", n_layers=2, hidden=128, n_heads=2, ffn=256, seq=40, batch=4, len_lo=10, len_hi=40)
+    kw = dict(step_shrink=0.8, student_noise=0.002)
+    full, h0, h1 = Problem(wl, **kw), Problem(wl, **kw), Problem(wl, **kw)
+    try:
+        g_full = full.run_gpu()
+        sums, losses = None, []
+        for p, (lo, hi) in ((h0, (0, 2)), (h1, (2, 4))):
+            m = p.m
+            B.mrem_set_loss_share(m.ctx, 0.5)
+            m.quantize_weights()
+            m.forward_teacher(p.xd[lo:hi].contiguous(), p.vld[lo:hi].contiguous(), 2, wl.seq)
+            m.forward_student(p.xd[lo:hi].contiguous(), p.vld[lo:hi].contiguous(), 2, wl.seq)
+            losses.append(float(m.recon_loss()[0][0]))
+            m.backward()
+            torch.cuda.synchronize()
+            bk = [m._ws_view(*B.mrem_grad_bucket(m.ctx, l), torch.float32).clone() for l in range(wl.n_layers)]
+            sums = bk if sums is None else [a + b for a, b in zip(sums, bk)]
+        assert abs(sum(losses) - g_full["loss"]) / g_full["loss"] < 1e-5
+        m = full.m
+        for l in range(wl.n_layers):
+            ptr, n = B.mrem_grad_bucket(m.ctx, l)
+            ref = m._ws_view(ptr, n, torch.float32)
+            # compare what the bucket holds for: every parameter gradient and the activation step gradients
+            base = ptr
+            for pid in range(len(B.PARAM_NAMES)):
+                off = (B.mrem_get_grad(m.ctx, l, pid) - base) // 4
+                cnt = int(np.prod(m.shapes[pid]))
+                if pid in (B.WQKV, B.WO, B.W1, B.W2):
+                    continue                                   # read below, before any mask is applied
+                a, b = sums[l][off: off + cnt].double(), ref[off: off + cnt].double()
+                assert float((a - b).norm() / b.norm().clamp(min=1e-30)) < 1e-4, (l, pid)
+            off = (B.mrem_get_grad(m.ctx, l, B.GRAD_STEP + 4) - base) // 4
+            a, b = sums[l][off: off + 8].double(), ref[off: off + 8].double()
+            assert float((a - b).norm() / b.norm()) < 1e-3, (l, "a_steps")
+        with pytest.raises(B.MremError):
+            B.mrem_set_loss_share(m.ctx, 0.0)
+        # no process group: the wrapper is the plain call sequence
+        opt = B.make_optim(lr=1e-4, step=1)
+        dp = DataParallelModule(h0.m)
+        assert dp.world == 1 and dp.shard(4) == (0, 4)
+        loss_dp = float(dp.step(h0.xd, h0.xd, h0.vld, wl.batch, wl.batch, wl.seq, opt)[0])
+        full.m.step(opt)
+        torch.cuda.synchronize()
+        assert loss_dp == g_full["loss"]
+        a, b = h0.m.student_numpy(), full.m.student_numpy()
+        for l in range(wl.n_layers):
+            for k in O.PARAMS:
+                assert np.array_equal(a[l][k], b[l][k]), (l, k)
+    finally:
+        for p in (full, h0, h1):
+            p.close()
+
+
 def test_module_sweep_caches_outputs_for_the_next_module():
     """Two one-layer modules in sequence: after module 0's steps its teacher and student outputs over the
     calibration set become module 1's inputs (Algorithm 2's outer loop).  Checked against the oracle run
