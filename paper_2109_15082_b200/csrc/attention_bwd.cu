@@ -73,8 +73,8 @@ __device__ __forceinline__ float ste_store(const uint32_t* a, bool row_ok, const
       const float g0 = scale * __uint_as_float(a[2 * j]), g1 = scale * __uint_as_float(a[2 * j + 1]);
       const float z0 = quotient(xv.x, step, r_step), z1 = quotient(xv.y, step, r_step);
       const bool in0 = z0 >= lo && z0 <= hi, in1 = z1 >= lo && z1 <= hi;
-      const float q0 = (float)__float2int_rn(fminf(fmaxf(z0, lo), hi));
-      const float q1 = (float)__float2int_rn(fminf(fmaxf(z1, lo), hi));
+      const float q0 = rne_magic(fminf(fmaxf(z0, lo), hi));
+      const float q1 = rne_magic(fminf(fmaxf(z1, lo), hi));
       acc += g0 * (q0 - (in0 ? z0 : 0.f)) + g1 * (q1 - (in1 ? z1 : 0.f));
       ow[j] = pack2(in0 ? g0 : 0.f, in1 ? g1 : 0.f);
     }
@@ -192,8 +192,8 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
           float d0 = s_v * __uint_as_float(a[2 * j]), d1 = s_v * __uint_as_float(a[2 * j + 1]);
           const float z0 = quotient(pv.x, s_p, r_p), z1 = quotient(pv.y, s_p, r_p);
           const bool in0 = z0 >= p.p_lo && z0 <= p.p_hi, in1 = z1 >= p.p_lo && z1 <= p.p_hi;
-          const float q0 = (float)__float2int_rn(fminf(fmaxf(z0, p.p_lo), p.p_hi));
-          const float q1 = (float)__float2int_rn(fminf(fmaxf(z1, p.p_lo), p.p_hi));
+          const float q0 = rne_magic(fminf(fmaxf(z0, p.p_lo), p.p_hi));
+          const float q1 = rne_magic(fminf(fmaxf(z1, p.p_lo), p.p_hi));
           const bool v0 = 2 * j < ncol, v1 = 2 * j + 1 < ncol;      // inside the sequence (row and key)
           if (v0) ds_p += d0 * (q0 - (in0 ? z0 : 0.f));
           if (v1) ds_p += d1 * (q1 - (in1 ? z1 : 0.f));

@@ -158,7 +158,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
       tmem_ld32(trow + (uint32_t)(c * 32), a);
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        const float e = c * 32 + j < len ? exp2f(fmaf(alpha2, __uint_as_float(a[j]), -mx2)) : 0.f;
+        const float e = c * 32 + j < len ? exp2_approx(fmaf(alpha2, __uint_as_float(a[j]), -mx2)) : 0.f;
         sum += e;
         a[j] = __float_as_uint(e);
       }
@@ -182,8 +182,8 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
           if (quant) {
             const float2 f = __bfloat1622float2(pb);
             // f is bf16-valued: quotient() equals the IEEE division of Eq. 1 for every such value and every step
-            const float c0 = (float)__float2int_rn(fminf(fmaxf(quotient(f.x, ps, r_ps), p.p_lo), p.p_hi));
-            const float c1 = (float)__float2int_rn(fminf(fmaxf(quotient(f.y, ps, r_ps), p.p_lo), p.p_hi));
+            const float c0 = rne_magic(fminf(fmaxf(quotient(f.x, ps, r_ps), p.p_lo), p.p_hi));
+            const float c1 = rne_magic(fminf(fmaxf(quotient(f.y, ps, r_ps), p.p_lo), p.p_hi));
             const __nv_bfloat162 cb = __floats2bfloat162_rn(c0, c1);
             cw[j >> 1] = *reinterpret_cast<const uint32_t*>(&cb);
           } else {
@@ -234,11 +234,12 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
         w[j >> 1] = *reinterpret_cast<const uint32_t*>(&vb);
         if (p.c_step) {
           const float2 f = __bfloat1622float2(vb);
-          const int i0 = __float2int_rn(fminf(fmaxf(quotient(f.x, cs, r_cs), -p.c_qmax), p.c_qmax));
-          const int i1 = __float2int_rn(fminf(fmaxf(quotient(f.y, cs, r_cs), -p.c_qmax), p.c_qmax));
-          const __nv_bfloat162 cb = __floats2bfloat162_rn((float)i0, (float)i1);
+          uint32_t b0, b1;                                 // rounding words: low byte = the 8-bit code
+          const float i0 = rne_magic(fminf(fmaxf(quotient(f.x, cs, r_cs), -p.c_qmax), p.c_qmax), b0);
+          const float i1 = rne_magic(fminf(fmaxf(quotient(f.y, cs, r_cs), -p.c_qmax), p.c_qmax), b1);
+          const __nv_bfloat162 cb = __floats2bfloat162_rn(i0, i1);
           cq[j >> 1] = *reinterpret_cast<const uint32_t*>(&cb);
-          const uint32_t two = (uint32_t)(i0 & 0xff) | ((uint32_t)(i1 & 0xff) << 8);
+          const uint32_t two = __byte_perm(b0, b1, 0x0040) & 0xffffu;
           if ((j & 2) == 0) c8[j >> 2] = two; else c8[j >> 2] |= two << 16;
         }
       }

@@ -21,6 +21,7 @@ struct TcParams {
   int m_tiles, n_tiles, k_blocks, num_tiles;
   int block_n, block_k, num_stages, stage_bytes;
   int a_mn, b_mn;
+  int b_static;                        // the B operand does not depend on the preceding kernel: prefetch its first tiles
   uint32_t idesc;
   Epilogue epi;
   int* status;

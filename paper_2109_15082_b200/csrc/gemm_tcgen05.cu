@@ -64,6 +64,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // A B operand that the preceding kernel does not write (weights): the producer fetches the B tiles of its first
+  // stages now, while that kernel is still finishing; the matching A tiles follow after the wait.
+  int prefetched = 0;
+  if (threadIdx.x == 0 && p.b_static && (int)blockIdx.x < p.num_tiles) {
+    const TileCoord t = decode_tile(p, blockIdx.x);
+    prefetched = p.k_blocks < p.num_stages ? p.k_blocks : p.num_stages;
+    for (int kb = 0; kb < prefetched; ++kb) {
+      const uint32_t bar = smem_u32(&full_bar[kb]);
+      const uint32_t sb = tiles_base + kb * p.stage_bytes + A_STAGE_BYTES;
+      mbar_expect_tx(bar, (uint32_t)p.stage_bytes);
+      const int k0 = kb * p.block_k;
+      if (!p.b_mn) {
+        tma_load_4d(sb, &map_b, bar, k0, t.n0, t.b0, t.b1);
+      } else {
+        for (int j = 0; j < p.block_n / 64; ++j) tma_load_4d(sb + j * 8192, &map_b, bar, t.n0 + 64 * j, k0, t.b0, t.b1);
+      }
+    }
+  }
   pdl_wait();                            // set-up done; from here on the predecessor's results are needed
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
   volatile int* vabort = &abort_flag;
@@ -84,14 +102,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           const uint32_t bar = smem_u32(&full_bar[stage]);
           const uint32_t sa = tiles_base + stage * p.stage_bytes, sb = sa + A_STAGE_BYTES;
-          mbar_expect_tx(bar, (uint32_t)p.stage_bytes);
+          const bool b_done = tile == (int)blockIdx.x && kb < prefetched;     // fetched (and announced) before the wait
+          if (!b_done) mbar_expect_tx(bar, (uint32_t)p.stage_bytes);
           const int k0 = kb * p.block_k;
           if (!p.a_mn) {
             tma_load_4d(sa, &map_a, bar, k0, t.m0, t.b0, t.b1);
           } else {
             for (int j = 0; j < BLOCK_M / 64; ++j) tma_load_4d(sa + j * 8192, &map_a, bar, t.m0 + 64 * j, k0, t.b0, t.b1);
           }
-          if (!p.b_mn) {
+          if (b_done) {
+          } else if (!p.b_mn) {
             tma_load_4d(sb, &map_b, bar, k0, t.n0, t.b0, t.b1);
           } else {
             for (int j = 0; j < p.block_n / 64; ++j) tma_load_4d(sb + j * 8192, &map_b, bar, t.n0 + 64 * j, k0, t.b0, t.b1);
@@ -309,6 +329,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   p.num_stages = SINGLE_CTA_SMEM_BUDGET / p.stage_bytes;
   if (p.num_stages > MAX_STAGES) p.num_stages = MAX_STAGES;
   p.a_mn = A.mn_contig; p.b_mn = B.mn_contig;
+  p.b_static = B.is_static;
   p.epi = epi;
   p.status = d_status;
   p.wait_ns = g_wait_limit_ns;

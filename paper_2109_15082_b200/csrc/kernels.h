@@ -109,6 +109,13 @@ void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long 
                     const float* offset, int lo, int hi, float* part_s, float* part_o, int dt, cudaStream_t st);
 
 // GELU-site backward: recompute g = stored(gelu(u)), STE of its quantizer, dU = dGhat * inside * gelu'(u).
+// GELU backward of a [rows, cols] tensor with the column sums of its result (the bias gradient of the linear layer
+// before the GELU) in the same pass.  scratch: scratch_floats floats, counters: n_counters zero-initialised ints, both
+// private to this call site.  Returns false (nothing launched) when the shape does not take the vector path.
+bool launch_gelu_bwd_colsum(const void* u, const void* dghat, void* du, long long rows, int cols, const float* step,
+                            const float* offset, int lo, int hi, int quantized, float* part_s, float* part_o,
+                            float* bias_grad, float* scratch, long long scratch_floats, int* counters, int n_counters,
+                            int dt, cudaStream_t st);
 void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, const float* step, const float* offset,
                      int lo, int hi, int quantized, float* part_s, float* part_o, int dt, cudaStream_t st);
 

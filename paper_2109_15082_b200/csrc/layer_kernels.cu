@@ -159,6 +159,105 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
 }
 
 // ------------------------------------------------------------------ STE of the weight quantizer (one block per row)
+// The same pass with the bias gradient of the linear layer before the GELU riding along: b1_grad[c] = sum over rows of
+// du[r, c].  A block of 16 x 16 threads owns 16 vectors of columns of one chunk of rows (gridDim.y chunks): a thread adds
+// its rows in row order, the block adds its 16 row lanes in index order, and the last block to finish a column group
+// (ticket counter) adds the chunks' partials in index order, so the sums do not depend on scheduling.  Block b = y *
+// gridDim.x + x leaves its partial step / offset gradient in slot b; slots from the grid size up to n_slots are zeroed.
+constexpr int GB_TX = 16, GB_TY = 16;
+template <typename T, int V>
+__global__ void __launch_bounds__(256) gelu_bwd_colsum_kernel(const T* __restrict__ u, const T* __restrict__ dghat,
+                                                              T* __restrict__ du, long long rows, int cols,
+                                                              const float* __restrict__ step,
+                                                              const float* __restrict__ offset, float lo, float hi,
+                                                              int quantized, float* __restrict__ part_s,
+                                                              float* __restrict__ part_o, int n_slots,
+                                                              float* __restrict__ bias_grad, float* __restrict__ scratch,
+                                                              int* __restrict__ counters) {
+  pdl_trigger();
+  pdl_wait();
+  constexpr int BC = GB_TX * V;                              // columns per block
+  __shared__ float sh[32];
+  __shared__ float cs[GB_TY][BC + 1];
+  __shared__ int is_last;
+  const float s = quantized ? *step : 1.f, r_s = __frcp_rn(s);
+  const bool has_off = offset != nullptr;
+  const float off = has_off ? *offset : 0.f;
+  const int tx = threadIdx.x % GB_TX, ty = threadIdx.x / GB_TX;
+  const int c = blockIdx.x * BC + tx * V;
+  const int chunks = gridDim.y;
+  const long long per = (rows + chunks - 1) / chunks;
+  const long long r0 = blockIdx.y * per, r1 = r0 + per < rows ? r0 + per : rows;
+  float acc[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) acc[j] = 0.f;
+  float ds = 0.f, dofs = 0.f;
+  if (c < cols) {
+    for (long long r = r0 + ty; r < r1; r += GB_TY) {
+      const long long i = r * cols + c;
+      float uv[V], d[V];
+      load_vec<T, V>(u + i, uv);
+      load_vec<T, V>(dghat + i, d);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        float cdf, pdf;
+        gelu_parts(uv[j], cdf, pdf);
+        if (quantized) {
+          const float z = qz(stored<T>(uv[j] * cdf), s, r_s, off, has_off);
+          const bool in = z >= lo && z <= hi;
+          ds += d[j] * (rne_magic(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
+          dofs += in ? 0.f : d[j];
+          d[j] = in ? d[j] : 0.f;
+        }
+        d[j] *= fmaf(uv[j], pdf, cdf);
+        acc[j] += d[j];
+      }
+      store_vec<T, V>(du + i, d);
+    }
+  }
+  ds = block_sum(ds, sh);
+  dofs = block_sum(dofs, sh);
+  const int bid = blockIdx.y * gridDim.x + blockIdx.x, n_blocks = gridDim.x * gridDim.y;
+  if (threadIdx.x == 0) {
+    if (part_s) part_s[bid] = ds;
+    if (part_o) part_o[bid] = dofs;
+  }
+  if (bid == 0)
+    for (int i = n_blocks + threadIdx.x; i < n_slots; i += blockDim.x) {
+      if (part_s) part_s[i] = 0.f;
+      if (part_o) part_o[i] = 0.f;
+    }
+#pragma unroll
+  for (int j = 0; j < V; ++j) cs[ty][tx * V + j] = acc[j];
+  __syncthreads();
+  const int col = threadIdx.x, cc = blockIdx.x * BC + col;
+  if (col < BC && cc < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int k = 0; k < GB_TY; ++k) t += cs[k][col];
+    scratch[(long long)blockIdx.y * cols + cc] = t;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = atomicAdd(&counters[blockIdx.x], 1) == chunks - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  if (col < BC && cc < cols) {
+    const float* src = scratch + cc;
+    float t = 0.f;
+    for (int k0 = 0; k0 < chunks; k0 += 8) {                 // eight loads in flight, added in index order
+      float q[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) q[k] = k0 + k < chunks ? src[(long long)(k0 + k) * cols] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) t += q[k];
+    }
+    bias_grad[cc] = t;
+  }
+  if (threadIdx.x == 0) counters[blockIdx.x] = 0;           // ready for the next launch
+}
+
 __global__ void __launch_bounds__(256) ste_weight_kernel(const float* __restrict__ w, const float* __restrict__ steps,
                                                          int per_row, int bits, int grid, float* __restrict__ dw,
                                                          int cols, float* __restrict__ ds_rows) {
@@ -289,6 +388,30 @@ void launch_ste_act(const void* x, long long ld_x, const void* dxhat, long long 
     if (v) launch_k(ste_act_kernel<T, V>, RED_BLOCKS, 256, 0, st, (const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
     else launch_k(ste_act_kernel<T, 1>, RED_BLOCKS, 256, 0, st, (const T*)x, ld_x, (const T*)dxhat, ld_d, (const T*)add, ld_add, (T*)dx, ld_dx, rows, cols, step, offset, (float)lo, (float)hi, part_s, part_o);
   });
+}
+
+bool launch_gelu_bwd_colsum(const void* u, const void* dghat, void* du, long long rows, int cols, const float* step,
+                             const float* offset, int lo, int hi, int quantized, float* part_s, float* part_o,
+                             float* bias_grad, float* scratch, long long scratch_floats, int* counters, int n_counters,
+                             int dt, cudaStream_t st) {
+  if (rows <= 0 || cols <= 0) return false;
+  bool done = false;
+  MREM_DT(dt, T, {
+    constexpr int V = 16 / (int)sizeof(T);
+    constexpr int BC = GB_TX * V;
+    const int col_blocks = (cols + BC - 1) / BC;
+    long long chunks = RED_BLOCKS / col_blocks;                       // the grid fills the RED_BLOCKS partial-sum slots
+    if (chunks > (rows + GB_TY - 1) / GB_TY) chunks = (rows + GB_TY - 1) / GB_TY;
+    if (chunks > scratch_floats / cols) chunks = scratch_floats / cols;
+    if (cols % V == 0 && al16(u) && al16(dghat) && al16(du) && chunks >= 1 && col_blocks <= n_counters && col_blocks <= RED_BLOCKS) {
+      Scope sc("gelu_bwd", (double)rows * cols * 3 * (dt == 1 ? 2.0 : 4.0), 0, st);
+      dim3 grid(col_blocks, (unsigned)chunks);
+      launch_k(gelu_bwd_colsum_kernel<T, V>, grid, 256, 0, st, (const T*)u, (const T*)dghat, (T*)du, rows, cols, step, offset,
+               (float)lo, (float)hi, quantized, part_s, part_o, RED_BLOCKS, bias_grad, scratch, counters);
+      done = true;
+    }
+  });
+  return done;
 }
 
 void launch_gelu_bwd(const void* u, const void* dghat, void* du, long long n, const float* step, const float* offset,

@@ -9,6 +9,7 @@ using namespace mrem;
 namespace mrem {
 thread_local Tracer* g_tracer = nullptr;
 int g_programmatic_launch = 1;
+thread_local int g_plain_next_launch = 0;
 unsigned long long g_wait_limit_ns = 2000000000ull;   // 2 s
 }
 
@@ -78,6 +79,10 @@ static void layout(mrem_ctx* c, char* base, size_t* total) {
   c->col_plane = (long long)COL_CHUNKS * (3 * H > F ? 3 * H : F);
   c->col_scratch = (float*)A.take(sizeof(float) * 3 * c->col_plane);
   c->col_counters = (int*)A.take(sizeof(int) * ((3 * H > F ? 3 * H : F) / 32 + 2));
+  c->gb_floats = (long long)(RED_BLOCKS / ((F + 127) / 128) + 1) * F;     // one row of partials per chunk of the GELU backward's grid
+  c->gb_scratch = (float*)A.take(sizeof(float) * c->gb_floats);
+  c->gb_n_counters = F / 32 + 2;
+  c->gb_counters = (int*)A.take(sizeof(int) * c->gb_n_counters);
   c->rowbias = (float*)A.take(sizeof(float) * (3 * H > F ? 3 * H : F));
   c->alt_rowbias = (float*)A.take(sizeof(float) * (3 * H > F ? 3 * H : F));
   c->reduce_per_layer = N_SITES + 1 + N_WMAT;

@@ -28,6 +28,11 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 
 extern unsigned long long g_wait_limit_ns;   // limit of every device-side wait, copied into each launch's parameters
 extern int g_programmatic_launch;      // 1: launch with programmatic stream serialization (default)
+// Set to 1 to make the NEXT launch a plain stream-ordered one (consumed by that launch): such a kernel starts only after
+// everything enqueued before it on its stream has completed, and no later kernel can start before it does.  The first
+// kernel of every forward pass is launched this way, so that whatever an earlier pass or update wrote (weight codes,
+// dequantized weights) is complete for every kernel of the pass, also before its own dependency wait.
+extern thread_local int g_plain_next_launch;
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
@@ -38,7 +43,8 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = g_programmatic_launch ? 1 : 0;
+  attr[0].val.programmaticStreamSerializationAllowed = (g_programmatic_launch && !g_plain_next_launch) ? 1 : 0;
+  g_plain_next_launch = 0;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
@@ -97,6 +103,12 @@ __device__ __forceinline__ float block_max(float v, float* sh) {
 }
 
 // ---------------------------------------------------------------- math
+// 2^x by the special-function unit alone (x <= 0 here: scores minus their maximum); about 2 ulp, flushes to zero below 2^-126
+__device__ __forceinline__ float exp2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float rcp_approx(float x) {
   float y;
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -210,6 +222,8 @@ struct OperandDesc {
   long long ld;                // element stride of the non-contiguous index
   long long s_b0, s_b1;        // element strides of the batch indices
   int mn_contig;
+  int is_static;               // 1: nothing the stream's preceding kernel writes (a weight matrix, codes of the last update):
+                               //    its first tiles may be fetched while that kernel is still finishing (B operand only)
 };
 
 struct GemmShape { int M, N, K, nb0, nb1; };

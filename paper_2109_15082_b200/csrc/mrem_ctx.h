@@ -94,6 +94,10 @@ struct mrem_ctx {
   float* col_scratch;
   long long col_plane = 0;               // floats per plane of col_scratch
   int* col_counters;
+  float* gb_scratch = nullptr;           // chunk partials and tickets of the column sums the GELU backward takes along
+  long long gb_floats = 0;               // (its own: column reductions of the side stream run at the same time)
+  int* gb_counters = nullptr;
+  int gb_n_counters = 0;
   float* rowbias;
   // second copy of the backward buffers the side stream reads (layers alternate between the two copies, so the
   // main stream may start the layer below while the side stream still works on this one)

@@ -20,11 +20,14 @@ enum { W_QKV = 0, W_O = 1, W_1 = 2, W_2 = 3 };
 enum { S_X = 0, S_Q = 1, S_K = 2, S_V = 3, S_P = 4, S_C = 5, S_A = 6, S_G = 7 };
 
 struct View {                      // an operand: pointer, stride of the non-contiguous index, batch strides
-  const void* p; long long ld, sb0, sb1; int mn;
+  const void* p; long long ld, sb0, sb1; int mn; int is_static;
 };
 inline View view(const void* p, long long ld, int mn = 0, long long sb0 = 0, long long sb1 = 0) {
-  return View{p, ld, sb0, sb1, mn};
+  return View{p, ld, sb0, sb1, mn, 0};
 }
+// a weight matrix (or its dequantized form): written by no kernel that directly precedes a product reading it, so the
+// product may fetch its first tiles before its predecessor in the stream has finished
+inline View weights(const void* p, long long ld, int mn = 0) { return View{p, ld, 0, 0, mn, 1}; }
 
 struct Epi {                       // shorthand builder of an Epilogue
   Epilogue e{};
@@ -56,7 +59,7 @@ struct Runner {
   }
   // storage-type product on the tensor cores (bf16) or CUDA cores (f32)
   void gemm(const View& A, const View& B, int M, int N, int K, int nb0, int nb1, const Epilogue& e) {
-    OperandDesc a{A.p, A.ld, A.sb0, A.sb1, A.mn}, b{B.p, B.ld, B.sb0, B.sb1, B.mn};
+    OperandDesc a{A.p, A.ld, A.sb0, A.sb1, A.mn, 0}, b{B.p, B.ld, B.sb0, B.sb1, B.mn, B.is_static};
     GemmShape g{M, N, K, nb0, nb1};
     if (c->dt == 1) note(tc_gemm(0, 0, a, b, g, e, 0, c->status, c->sm_count, st), "bf16 GEMM launch failed");
     else note(simt_gemm_f32(a, b, g, e, st), "f32 GEMM launch failed");
@@ -81,7 +84,7 @@ struct Runner {
   }
   // integer-code product with exact int32 accumulation
   void gemm_i8(const int8_t* A, int a_unsigned, const int8_t* B, int M, int N, int K, const Epilogue& e) {
-    OperandDesc a{A, K, 0, 0, 0}, b{B, K, 0, 0, 0};
+    OperandDesc a{A, K, 0, 0, 0, 0}, b{B, K, 0, 0, 0, 1};      // B: weight codes, written by the last update
     GemmShape g{M, N, K, 1, 1};
     note(tc_gemm(1, a_unsigned, a, b, g, e, 0, c->status, c->sm_count, st), "int8 GEMM launch failed");
   }
@@ -143,7 +146,7 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
     for (int k = 0; k < MREM_N_PARAMS; ++k) if (!b.teacher[k]) return fail(c, MREM_ERR_ORDER, "forward: teacher parameters not bound");
     void* out = r.at(outs, (long long)l * M * H);
     if (init_steps) init_site(c, b, S_X, cur, H, M, H);
-    r.gemm(view(cur, H), view(b.teacher[MREM_WQKV], H), (int)M, 3 * H, H, 1, 1,
+    r.gemm(view(cur, H), (student_params ? view(b.teacher[MREM_WQKV], H) : weights(b.teacher[MREM_WQKV], H)), (int)M, 3 * H, H, 1, 1,
            Epi(c->t_qkv, ok, 3 * H).colbias((float*)b.teacher[MREM_BQKV]).e);
     if (init_steps)
       for (int seg = 0; seg < 3; ++seg) init_site(c, b, S_Q + seg, r.at(c->t_qkv, seg * H), 3 * H, M, H);
@@ -161,15 +164,15 @@ int float_forward(mrem_ctx* c, const void* x, const int32_t* len, int B, int S, 
     }
     if (init_steps) init_site(c, b, S_P, c->t_P, S, (long long)B * h * S, S);
     if (init_steps) init_site(c, b, S_C, c->t_ctx, H, M, H);
-    r.gemm(view(c->t_ctx, H), view(b.teacher[MREM_WO], H), (int)M, H, H, 1, 1,
+    r.gemm(view(c->t_ctx, H), (student_params ? view(b.teacher[MREM_WO], H) : weights(b.teacher[MREM_WO], H)), (int)M, H, H, 1, 1,
            Epi(c->t_y1, ok, H).colbias((float*)b.teacher[MREM_BO]).residual(cur).e);
     launch_layernorm_fwd(c->t_y1, (float*)b.teacher[MREM_LN1_G], (float*)b.teacher[MREM_LN1_B], d.ln_eps, M, H, c->t_a,
                          nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, st);
     if (init_steps) init_site(c, b, S_A, c->t_a, H, M, H);
-    r.gemm(view(c->t_a, H), view(b.teacher[MREM_W1], H), (int)M, F, H, 1, 1,
+    r.gemm(view(c->t_a, H), (student_params ? view(b.teacher[MREM_W1], H) : weights(b.teacher[MREM_W1], H)), (int)M, F, H, 1, 1,
            Epi(c->t_g, ok, F).colbias((float*)b.teacher[MREM_B1]).gelu().e);
     if (init_steps) init_site(c, b, S_G, c->t_g, F, M, F);
-    r.gemm(view(c->t_g, F), view(b.teacher[MREM_W2], F), (int)M, H, F, 1, 1,
+    r.gemm(view(c->t_g, F), (student_params ? view(b.teacher[MREM_W2], F) : weights(b.teacher[MREM_W2], F)), (int)M, H, F, 1, 1,
            Epi(c->t_y2, ok, H).colbias((float*)b.teacher[MREM_B2]).residual(c->t_a).e);
     launch_layernorm_fwd(c->t_y2, (float*)b.teacher[MREM_LN2_G], (float*)b.teacher[MREM_LN2_B], d.ln_eps, M, H, out,
                          nullptr, nullptr, nullptr, 0, nullptr, nullptr, c->dt, st);
@@ -344,19 +347,25 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     fork();
     launch_col_reduce(sent_back ? q.d_sum : dF, H, s.y2, s.mean2, s.rstd2, q.d_y2, H, M, H, g.p[MREM_LN2_B], g.p[MREM_LN2_G],
                       g.p[MREM_B2], c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(q.d_y2, H), view(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
+    r.gemm(view(q.d_y2, H), weights(w[W_2].what, F, 1), (int)M, F, H, 1, 1, Epi(c->d_ghat, ok, F).e);
     {
       Epi e(g.p[MREM_W2], OUT_F32, F);
       e.alpha(1.f, b.a_steps[S_G]);
       if (rg.asym) { launch_scale_vec(g.p[MREM_B2], b.a_off[S_G], q.rowbias, H, side); e.rowbias(q.rowbias); }
       rw.defer(view(q.d_y2, H, 1), view(s.g_qt, F, 1), H, F, (int)M, e.e);
     }
-    launch_gelu_bwd(s.u, c->d_ghat, q.d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
-                    part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
+    // (the bias gradient of FFN1, the column sums of d_u, rides along where the vector path applies)
+    const bool b1_done = launch_gelu_bwd_colsum(s.u, c->d_ghat, q.d_u, M, F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
+                                                part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, g.p[MREM_B1], c->gb_scratch,
+                                                c->gb_floats, c->gb_counters, c->gb_n_counters, c->dt, st);
+    if (!b1_done)
+      launch_gelu_bwd(s.u, c->d_ghat, q.d_u, M * F, b.a_steps[S_G], rg.asym ? b.a_off[S_G] : nullptr, rg.lo, rg.hi, 1,
+                      part + S_G * RED_BLOCKS, part + N_SITES * RED_BLOCKS, c->dt, st);
     // FFN1:  u = A_hat W1_hat^T + b1
     fork();
-    launch_col_reduce(q.d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(q.d_u, F), view(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
+    if (!b1_done)
+      launch_col_reduce(q.d_u, F, nullptr, nullptr, nullptr, nullptr, 0, M, F, g.p[MREM_B1], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
+    r.gemm(view(q.d_u, F), weights(w[W_1].what, H, 1), (int)M, H, F, 1, 1, Epi(c->d_ahat, ok, H).e);
     rw.defer(view(q.d_u, F, 1), view(s.a_qt, H, 1), F, H, (int)M, Epi(g.p[MREM_W1], OUT_F32, H).alpha(1.f, b.a_steps[S_A]).e);
     // straight-through pass of the FFN1 input quantizer + skip connection -> d_a, and the first LayerNorm's backward
     if (!(fuse_ln && launch_layernorm_bwd_ste(nullptr, s.a, c->d_ahat, q.d_y2, b.a_steps[S_A], rx.lo, rx.hi, s.y1, s.mean1, s.rstd1,
@@ -369,7 +378,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     fork();
     launch_col_reduce(q.d_a, H, s.y1, s.mean1, s.rstd1, q.d_y1, H, M, H, g.p[MREM_LN1_B], g.p[MREM_LN1_G], g.p[MREM_BO],
                       c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(q.d_y1, H), view(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
+    r.gemm(view(q.d_y1, H), weights(w[W_O].what, H, 1), (int)M, H, H, 1, 1, Epi(c->d_ctxhat, ok, H).e);
     rw.defer(view(q.d_y1, H, 1), view(s.ctx_qt, H, 1), H, H, (int)M, Epi(g.p[MREM_WO], OUT_F32, H).alpha(1.f, b.a_steps[S_C]).e);
     launch_ste_act(s.ctx, H, c->d_ctxhat, H, nullptr, 0, c->d_ctx, H, M, H, b.a_steps[S_C], nullptr, rx.lo, rx.hi,
                    part + S_C * RED_BLOCKS, nullptr, c->dt, st);
@@ -396,7 +405,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
     // QKV projection:  qkv = X_hat Wqkv_hat^T + bqkv
     fork();
     launch_col_reduce(q.d_qkv, 3 * H, nullptr, nullptr, nullptr, nullptr, 0, M, 3 * H, g.p[MREM_BQKV], nullptr, nullptr, c->col_scratch, c->col_plane, c->col_counters, c->dt, side);
-    r.gemm(view(q.d_qkv, 3 * H), view(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
+    r.gemm(view(q.d_qkv, 3 * H), weights(w[W_QKV].what, H, 1), (int)M, H, 3 * H, 1, 1, Epi(c->d_xhat, ok, H).e);
     rw.defer(view(q.d_qkv, 3 * H, 1), view(s.x_qt, H, 1), 3 * H, H, (int)M, Epi(g.p[MREM_WQKV], OUT_F32, H).alpha(1.f, b.a_steps[S_X]).e);
     rw.flush_deferred();                              // the layer's four weight-gradient products, one launch
     if (fuse_ln && l > 0) {
@@ -463,6 +472,7 @@ int32_t mrem_module_forward(mrem_ctx* c, int32_t role, const void* x, const void
   if (c->have_teacher || c->have_student) {
     if (batch != c->cur_batch || seq != c->cur_seq) { c->have_teacher = c->have_student = false; }
   }
+  mrem::g_plain_next_launch = 1;          // the pass's first kernel is a full barrier towards everything before it
   if (role == MREM_TEACHER) {
     rc = float_forward(c, x, len, batch, seq, outs, false, false);
     if (rc != MREM_OK) return rc;
@@ -630,7 +640,8 @@ int32_t mrem_rem_step(mrem_ctx* c, int32_t layer, int32_t tensor_id, const void*
   const float* off = ar.asym ? b.a_off[site] : nullptr;
   const int bias_id = tensor_id + 1;                     // the bias follows its matrix in the parameter list
 
-  // w^T a
+  // w^T a  (launched as a full barrier: the codes the quantizer above may just have written are complete for all that follows)
+  mrem::g_plain_next_launch = 1;
   r.gemm(view(a, K), view(b.teacher[tensor_id], K), (int)M, N, K, 1, 1, Epi(target, ok, N).e);
   // Q(w)^T Q(a): integer codes, exact accumulation, dequantized in the epilogue (offset term as a column bias)
   launch_quantize_act(a, c->dt, M, K, K, step, off, ar.lo, ar.hi, q8, K, qt, K, st);
