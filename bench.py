@@ -402,6 +402,27 @@ def main():
         loss_last = float(m.loss[0])
         status = m.poll_status()
 
+        # ---- the same step captured on ONE stream (no kernel runs beside another): its replay time is the sum of the
+        #      kernels' own run times plus their launch gaps, the cross-check of the per-kernel figures below
+        serial_ms = None
+        if world == 1:
+            B.mrem_set_two_streams(m.ctx, 0)
+            B.mrem_graph_capture_step(m.ctx, xbuf, xbuf, 0.0, lenbuf, wl.batch, wl.seq, m.t_out, m.s_out, m.loss, opt)
+            for t in range(3):
+                stage(W + t)
+                B.mrem_graph_launch(m.ctx)
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            side.synchronize()
+            s0.record(side)
+            for k in range(K):
+                stage(W + k % (total - W))
+                B.mrem_graph_launch(m.ctx)
+            s1.record(side)
+            side.synchronize()
+            serial_ms = s0.elapsed_time(s1) / K
+            B.mrem_set_two_streams(m.ctx, 1)
+            B.mrem_graph_capture_step(m.ctx, xbuf, xbuf, 0.0, lenbuf, wl.batch, wl.seq, m.t_out, m.s_out, m.loss, opt)
+
         # ---- per-kernel timing (CUDA events around every launch of a few eager steps)
         B.mrem_trace_enable(m.ctx, 1)
         n_trace = 3
@@ -449,6 +470,13 @@ def main():
 
     pk = peaks()
     # products are traced per shape ("gemm_bf16 MxNxK.."); fold them into one row per kernel, keep the shapes
+    # what an event pair measures around a kernel that does nothing: contained in every traced duration
+    overhead_ms = 0.0
+    for e in trace:
+        if e["name"] == "(empty kernel)":
+            overhead_ms = e["ms"] / max(e["launches"], 1)
+    trace = [e for e in trace if e["name"] != "(empty kernel)"]
+    net_ms = lambda e: max(e["ms"] - overhead_ms * e["launches"], 0.25 * e["ms"])
     shapes = [e for e in trace if e["name"].startswith("gemm_")]
     folded = {}
     for e in trace:
@@ -463,16 +491,17 @@ def main():
     kernels = []
     for e in sorted(trace, key=lambda e: -e["ms"]):
         per_launch_ms = e["ms"] / max(e["launches"], 1)
+        e["net"] = net_ms(e)
         if e["is_flops"]:
-            ach = e["work"] / (e["ms"] * 1e-3) / 1e12
+            ach = e["work"] / (e["net"] * 1e-3) / 1e12
             peak = pk[tensor_peak] * (INT8_OVER_BF16 if "i8" in e["name"] else 1.0)
             unit, bound = "TFLOP/s", "tensor"
         else:
-            ach = e["work"] / (e["ms"] * 1e-3) / 1e9
+            ach = e["work"] / (e["net"] * 1e-3) / 1e9
             peak, unit, bound = pk["hbm_gbs"], "GB/s", "hbm"
-        kernels.append({"name": e["name"], "launches_per_step": e["launches"] / n_trace, "ms_per_step": e["ms"] / n_trace,
-                        "us_per_launch": 1e3 * per_launch_ms, "bound": bound, "achieved": ach, "peak": peak,
-                        "unit": unit, "frac": ach / peak})
+        kernels.append({"name": e["name"], "launches_per_step": e["launches"] / n_trace, "ms_per_step": e["net"] / n_trace,
+                        "us_per_launch": 1e3 * e["net"] / max(e["launches"], 1), "us_per_launch_with_event_overhead": 1e3 * per_launch_ms,
+                        "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak})
     top = kernels[0]
     # DRAM bytes per launch of the dominant kernel from the committed ncu capture of this workload
     # (profiles/tc_gemm_dram_large6_w4a8.md); known only for that kernel on that workload
@@ -484,7 +513,12 @@ def main():
                                                " bf16 sustained (SM clock below maximum or power cap active during the run)")
                                               if top["bound"] == "tensor" else " copy bandwidth"),
                 "int8_peak": "assumed: 2 x the measured bf16 figure (nominal dense ratio), not measured",
-                "timed": f"CUDA events around each launch of {n_trace} eager steps"}
+                "timed": f"CUDA events around each launch of {n_trace} eager steps, minus what the same event pair measures around a "
+                         f"kernel that does nothing ({1e3 * overhead_ms:.2f} us, measured in this run); check: the kernels' net times "
+                         f"add up to {sum(k['ms_per_step'] for k in kernels):.3f} ms per step, the step captured on one stream replays in "
+                         f"{serial_ms if serial_ms is None else round(serial_ms, 3)} ms",
+                "event_overhead_us": 1e3 * overhead_ms, "sum_net_ms_per_step": sum(k["ms_per_step"] for k in kernels),
+                "serial_graph_ms_per_step": serial_ms}
 
     line = {"metric": METRIC, "value": D.whole_job_rate(tokens, K, world, ms), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms / K, "repeats": repeats, "ms_per_step_min": min(block_ms) / K,
@@ -494,8 +528,9 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_step * K, "roofline": roofline,
             "kernels": kernels,
             "gemm_shapes": [{"shape": e["name"], "launches_per_step": e["launches"] / n_trace,
-                             "us_per_launch": 1e3 * e["ms"] / max(e["launches"], 1),
-                             "tflops": e["work"] / (e["ms"] * 1e-3) / 1e12} for e in sorted(shapes, key=lambda e: -e["ms"])],
+                             "us_per_launch": 1e3 * net_ms(e) / max(e["launches"], 1),
+                             "us_per_launch_with_event_overhead": 1e3 * e["ms"] / max(e["launches"], 1),
+                             "tflops": e["work"] / (net_ms(e) * 1e-3) / 1e12} for e in sorted(shapes, key=lambda e: -e["ms"])],
             "loss_last": loss_last, "device_status": status}
     if extras:
         line["extras"] = extras

@@ -270,6 +270,12 @@ int32_t mrem_grad_bucket(mrem_ctx* ctx, int32_t layer, float** d_ptr, size_t* n_
 int32_t mrem_set_wait_limit_ns(uint64_t ns);
 int32_t mrem_selftest_wait_limit(mrem_ctx* ctx);
 
+/* Per context (default on): inside a step the teacher pass runs on a second stream beside the student pass, and the
+ * weight-gradient products, column reductions and weight updates of a layer beside the backward pass of the layers
+ * below.  0 keeps everything on the context's stream (same kernels, same results; for timing comparisons: the replay
+ * time of a step captured this way is the sum of its kernels' run times).  Takes effect at the next call or capture. */
+int32_t mrem_set_two_streams(mrem_ctx* ctx, int32_t on);
+
 /* Per context (default on): where the shapes allow it (bf16 storage, head size 64, seq <= 128, seq % 8 == 0)
  * the backward of the attention block (Sec. 3.1: the gradients of Q, K, V through the quantized scores,
  * softmax and context products, with the straight-through masks of the Q, K, V, P quantizers) runs as one
@@ -300,7 +306,10 @@ int32_t mrem_graph_num_kernels(mrem_ctx* ctx, int32_t* n_kernels);
 /* Per-kernel timing of the eager calls (not of graph replays) with CUDA events on the context's stream.
  * `work` is the algorithmic work of all launches of that kernel: FLOPs (is_flops = 1: 2*M*N*K per product)
  * or bytes read plus written once at storage width (is_flops = 0).  mrem_trace_enable resets the totals
- * and blocks on the stream; mrem_trace_read blocks on the stream and fills up to max_entries entries. */
+ * and blocks on the stream; mrem_trace_read blocks on the stream and fills up to max_entries entries.
+ * A bracketed duration holds, beside the kernel's run time, what the event pair costs (event processing, launch and
+ * drain of a grid: several microseconds); turning tracing on therefore launches 32 kernels that do nothing, bracketed
+ * the same way, and reports them as the entry "(empty kernel)": its ms / launches is that overhead. */
 typedef struct { char name[40]; double ms; double work; int64_t launches; int32_t is_flops; int32_t reserved; } mrem_trace_entry;
 int32_t mrem_trace_enable(mrem_ctx* ctx, int32_t on);
 int32_t mrem_trace_read(mrem_ctx* ctx, mrem_trace_entry* out, int32_t max_entries, int32_t* n_entries);

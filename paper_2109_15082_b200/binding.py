@@ -35,7 +35,7 @@ EXPORTS = (
     "mrem_set_fused_attention_backward", "mrem_backward_and_step", "mrem_recon_step_host_submit",
     "mrem_recon_step_host_wait", "mrem_rem_step", "mrem_bind_head", "mrem_embed_workspace_bytes", "mrem_embed_step", "mrem_get_input_grad",
     "mrem_get_activation", "mrem_set_wait_limit_ns", "mrem_selftest_wait_limit",
-    "mrem_set_loss_share", "mrem_grad_bucket",
+    "mrem_set_loss_share", "mrem_grad_bucket", "mrem_set_two_streams",
 )
 
 
@@ -232,6 +232,10 @@ def mrem_grad_bucket(ctx, layer):
     ptr, n = C.c_void_p(0), C.c_size_t(0)
     _check(lib().mrem_grad_bucket(ctx, int(layer), C.byref(ptr), C.byref(n)), "mrem_grad_bucket", ctx)
     return ptr.value, n.value
+
+
+def mrem_set_two_streams(ctx, on):
+    _check(lib().mrem_set_two_streams(ctx, int(bool(on))), "mrem_set_two_streams", ctx)
 
 
 def mrem_set_wait_limit_ns(ns):

@@ -153,6 +153,8 @@ void launch_ste_weight(const float* w, const float* steps, int per_row, int bits
 
 // dst[i] = sum_j src_i[j], j in fixed order, for a table of reductions (one block each).
 struct ReduceEntry { const float* src; int count; float* dst; };
+// n traced launches of a kernel that does nothing: the tracer's own overhead per bracketed launch ("(empty kernel)").
+void launch_trace_calibration(int n, cudaStream_t st);
 void launch_reduce_table(const ReduceEntry* d_table, int n_entries, cudaStream_t st);
 
 // out[i] = scale[0] * in[i]  (small vectors)

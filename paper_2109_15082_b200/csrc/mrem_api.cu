@@ -547,6 +547,17 @@ int32_t mrem_trace_enable(mrem_ctx* c, int32_t on) {
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(c, MREM_ERR_CUDA, "trace_enable: sync failed");
   c->tracer.reset();
   c->trace_on = on != 0;
+  if (c->trace_on) {
+    // what a bracketed launch measures beyond the kernel itself: reported as the entry "(empty kernel)"
+    TracerGuard tg(&c->tracer);
+    launch_trace_calibration(32, c->stream);
+  }
+  return MREM_OK;
+}
+
+int32_t mrem_set_two_streams(mrem_ctx* c, int32_t on) {
+  if (!c) return MREM_ERR_ARG;
+  c->use_side_stream = on != 0;
   return MREM_OK;
 }
 

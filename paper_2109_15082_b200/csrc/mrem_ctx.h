@@ -123,6 +123,7 @@ struct mrem_ctx {
   // classification head of the model's last module (null: none): the output-logit term of the loss
   struct { const float *wp = nullptr, *bp = nullptr, *wc = nullptr, *bc = nullptr; int n_classes = 0; float* logit_loss = nullptr; float* logits = nullptr; } head;
   float loss_share = 1.f;            // this context's share of the whole batch (data parallel: local / global sequences)
+  bool use_side_stream = true;       // run the teacher pass and the weight-gradient / update work on the second stream
   bool fused_attention_bwd = true;   // use the single-kernel attention backward where it applies
   bool codes_fresh = false;          // the weight codes match the current latent weights and steps
   mrem::Tracer tracer;               bool trace_on = false;

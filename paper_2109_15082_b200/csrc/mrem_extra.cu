@@ -22,7 +22,7 @@ int enqueue_step(mrem_ctx* c, const void* xt, const void* xs, float lambda, cons
   // Without teacher forcing the two passes are independent until the loss: the teacher's runs on the side
   // stream beside the student's (its tensor-core products under the student's quantizer kernels).  Only
   // with the fused attention kernel, whose path shares no scratch between the passes.
-  const bool beside = lambda == 0.f && c->side_stream && !c->trace_on && c->d.n_heads > 0 &&
+  const bool beside = lambda == 0.f && c->use_side_stream && c->side_stream && !c->trace_on && c->d.n_heads > 0 &&
                       attention_fwd_supported(seq, c->d.hidden / c->d.n_heads, c->dt);
   if (rc == MREM_OK && beside) {
     if (cudaEventRecord(c->ev_fork, c->stream) != cudaSuccess || cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess)

@@ -288,7 +288,7 @@ int student_backward(mrem_ctx* c, bool update_as_you_go) {
   const long long M = (long long)B * S;
   const long long sSS = (long long)S * S, sHSS = (long long)h * S * S, sQKV = (long long)S * 3 * H;
   Runner r(c);
-  const bool two_streams = c->side_stream && !c->trace_on;
+  const bool two_streams = c->use_side_stream && c->side_stream && !c->trace_on;
   cudaStream_t side = two_streams ? c->side_stream : c->stream;
   Runner rw(c, side);                            // weight-gradient products
   bool sync_failed = false;
