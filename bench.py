@@ -189,6 +189,94 @@ def build_problem(wl, rank, torch, calib_n):
     return m, calib, lens
 
 
+def run_data_parallel(args, wl):
+    """--dp: ONE module on all ranks (identical parameters), every step's batch split over the ranks; per layer one
+    all-reduce (NCCL, sum) of the gradient bucket before the update (paper_2109_15082_b200/dist.py).  Strong scaling:
+    the whole job processes one batch of the workload per step whatever the number of ranks.  Eager call sequence (the
+    update has to wait for the all-reduce, so the step is not one captured graph here)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2109_15082_b200 import binding as B
+    from paper_2109_15082_b200 import dist as D
+    from paper_2109_15082_b200 import synth
+    from paper_2109_15082_b200.session import ReconModule
+    rank, world, local = D.env_rank()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    W, K = max(3, args.warmup), args.steps
+    calib_n = args.calib or wl.calib or wl.batch * 8
+    lo, hi = D.shard_bounds(wl.batch, rank, world)
+    nb = hi - lo
+    if nb < 1:
+        raise RuntimeError("--dp needs at least one sequence of the batch per rank")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        m = ReconModule(wl.n_layers, wl.hidden, wl.n_heads, wl.ffn, wl.seq, nb, wl.w_bits, wl.a_bits, wl.w_grid, True, 3, wl.act_dtype)
+        m.load_teacher(synth.teacher_params(wl, seed=0))              # the same module on every rank
+        m.init_student_from_teacher()
+        m.init_weight_steps(wl.w_step_rule)
+        calib = torch.empty(calib_n, wl.seq, wl.hidden, dtype=m.tdtype, device=m.device)
+        for c0 in range(0, calib_n, 64):
+            n = min(64, calib_n - c0)
+            calib[c0:c0 + n].copy_(torch.from_numpy(synth.hidden_states(wl, n, seed=0, tag=f"calib{c0}")).to(m.device))
+        lens = torch.from_numpy(synth.valid_lengths(wl, calib_n, seed=0)).to(m.device)
+        total = W + K
+        n_batches = calib_n // wl.batch
+        perm = np.concatenate([synth.permutation(0, f"epoch{e}", calib_n)[: n_batches * wl.batch]
+                               for e in range((total + n_batches - 1) // n_batches + 1)])
+        idx = torch.from_numpy(perm[: total * wl.batch].reshape(total, wl.batch)[:, lo:hi].astype(np.int32).copy()).to(m.device)
+        lens_steps = lens[idx.long()].contiguous()
+        xbuf = torch.empty(nb, wl.seq, wl.hidden, dtype=m.tdtype, device=m.device)
+        row_bytes = wl.seq * wl.hidden * xbuf.element_size()
+        dp = D.DataParallelModule(m)
+
+        def step(t):
+            B.mrem_gather_rows(calib, idx[t], nb, row_bytes, xbuf, side.cuda_stream)
+            return dp.step(xbuf, xbuf, lens_steps[t], nb, wl.batch, wl.seq, opt)
+
+        B.mrem_gather_rows(calib, idx[0], nb, row_bytes, xbuf, side.cuda_stream)
+        dp.init_act_steps(xbuf, lens_steps[0], nb, wl.seq)
+        opt = B.make_optim(lr=wl.lr, step=0, decay_total_steps=max(wl.steps, total))
+        for t in range(W):
+            step(t)
+        side.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for t in range(W, W + K):
+            loss = step(t)
+        e1.record(side)
+        side.synchronize()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        clocks = sampler.stop() if rank == 0 else None
+        ms = D.max_over_ranks(e0.elapsed_time(e1), m.device)
+        loss_last = float(loss[0])
+        status = m.poll_status()
+        bucket_bytes = sum(int(b.numel()) * 4 for b in dp.buckets)
+        m.close()
+    if rank == 0:
+        tokens = wl.batch * wl.seq
+        cfg = workload_config(wl, calib_n, world)
+        cfg.update(parallelism=f"dp{world}: batch split over the ranks, one gradient all-reduce per layer",
+                   launch="eager call sequence (the update waits for the all-reduce)", sequences_per_rank=nb,
+                   allreduce_bytes_per_step=bucket_bytes)
+        print(json.dumps({"metric": METRIC, "value": tokens * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                          "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+                          "dtype": "bf16+int8", "data": "synthetic", "config": cfg, "clocks": clocks, "e2e": None,
+                          "gpu_launches": None, "loss_last": loss_last, "device_status": status,
+                          "note": "data-parallel mode; with one rank it is the eager call sequence of the step"}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def time_extras(m, wl, xbuf, lenbuf, stream, torch, B, pk, reps=10):
     """Device times (CUDA events, after 3 warm-up calls) of the entry points beside the module step, on the workload's
     shapes: one step of Eq. 2 per weight matrix of a layer on batch x seq rows, the output-logit term inside
@@ -308,6 +396,8 @@ def main():
     ap.add_argument("--extras", action="store_true", help="also time the per-product step (Eq. 2), the output-logit term and the "
                     "embedding step of the first module, and add them to the JSON line as \"extras\"")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches (no programmatic dependent launch)")
+    ap.add_argument("--dp", action="store_true", help="data parallel: one module, each step's batch split over the ranks, gradients "
+                    "all-reduced per layer (strong scaling); default is one independent replica per rank")
     ap.add_argument("--repeats", type=int, default=0, help="timed blocks of --steps steps each (0: as many as bring the timed "
                     "region to about 2 s, between 3 and 64); the line reports the median block and the fastest")
     args = ap.parse_args()
@@ -316,6 +406,10 @@ def main():
     wl = synth.workloads()[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
+        return
+
+    if args.dp:
+        run_data_parallel(args, wl)
         return
 
     import torch
