@@ -503,7 +503,7 @@ def main():
             B.mrem_set_two_streams(m.ctx, 0)
             B.mrem_graph_capture_step(m.ctx, xbuf, xbuf, 0.0, lenbuf, wl.batch, wl.seq, m.t_out, m.s_out, m.loss, opt)
             for t in range(3):
-                stage(W + t)
+                stage(W + t % (total - W))
                 B.mrem_graph_launch(m.ctx)
             s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             side.synchronize()
