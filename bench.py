@@ -619,7 +619,7 @@ def main():
             "timed_region_ms": sum(block_ms), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16+int8", "data": "synthetic",
             "config": workload_config(wl, calib_n, world),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_step * K, "roofline": roofline,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_step * K * repeats, "roofline": roofline,
             "kernels": kernels,
             "gemm_shapes": [{"shape": e["name"], "launches_per_step": e["launches"] / n_trace,
                              "us_per_launch": 1e3 * net_ms(e) / max(e["launches"], 1),

@@ -19,13 +19,13 @@ namespace {
 
 // Code of Eq. 1 and the same value as a float.  Integer grid: the sum with 1.5 * 2^23 holds the code in its
 // low mantissa bits (two's complement), so neither direction goes through the conversion unit.
-__device__ __forceinline__ int weight_code(float w, float s, float qmax, int grid, float& qf) {
-  const float z = __fdiv_rn(w, s);
-  if (grid == 0) {
-    const float t = __fadd_rn(fminf(fmaxf(z, -qmax), qmax), RINT_MAGIC);
-    qf = __fsub_rn(t, RINT_MAGIC);
-    return (int)(int8_t)(__float_as_uint(t) & 0xffu);
+__device__ __forceinline__ int weight_code(float w, float s, float r_s, float qmax, int grid, float& qf) {
+  if (grid == 0) {      // the exact code without the division instruction (code_f); r_s = RN(1 / s)
+    uint32_t bits;
+    qf = code_f<false>(w, s, r_s, -qmax, qmax, bits);
+    return (int)(int8_t)(bits & 0xffu);
   }
+  const float z = __fdiv_rn(w, s);
   const int q = 2 * (int)fminf(fmaxf(floorf(z), -2.f), 1.f) + 1;
   qf = (float)q;
   return q;
@@ -48,14 +48,17 @@ __device__ __forceinline__ void store_what4<bf16>(bf16* p, float a, float b, flo
 
 // NT threads per row, NV float4 vectors per thread kept in registers: (256, 1) for rows up to 1024 wide,
 // (512, 2) up to 4096; wider rows are re-read.
-template <typename T, int NV, int NT>
+// GRID (the weight grid, 0: Eq. 1's integers, 1: half-integer 2-bit levels) is a template parameter: the per-weight code
+// then holds one of the two rules, not both under predicates.
+template <typename T, int NV, int NT, int GRID>
 __global__ void __launch_bounds__(NT, NT == 256 ? 6 : 2) fused_weight_update_kernel(
     float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v,
     float* __restrict__ steps, const float* __restrict__ ds_in, float* __restrict__ m_s, float* __restrict__ v_s,
-    const OptimScalars* __restrict__ sc, int cols, int bits, int grid, int train_w, int train_s,
+    const OptimScalars* __restrict__ sc, int cols, int bits, int train_w, int train_s,
     int8_t* __restrict__ codes, int32_t* __restrict__ rowsum, float* __restrict__ scale, T* __restrict__ what) {
   pdl_trigger();
   pdl_wait();
+  constexpr int grid = GRID;
   __shared__ float sh[32];
   __shared__ int shi[32];
   __shared__ float s_new_sh;
@@ -125,7 +128,7 @@ __global__ void __launch_bounds__(NT, NT == 256 ? 6 : 2) fused_weight_update_ker
     s_new_sh = s_new;
   }
   __syncthreads();
-  const float s_new = s_new_sh;
+  const float s_new = s_new_sh, r_new = __frcp_rn(s_new);
   const float sc_new = grid == 0 ? s_new : 0.5f * s_new;
   // 3 + 4. weights, then their new codes
   float4* wo = reinterpret_cast<float4*>(w + base);
@@ -143,8 +146,8 @@ __global__ void __launch_bounds__(NT, NT == 256 ? 6 : 2) fused_weight_update_ker
       v4[c] = vv;
     }
     float f0, f1, f2, f3;
-    const int q0 = weight_code(wv.x, s_new, qmax, grid, f0), q1 = weight_code(wv.y, s_new, qmax, grid, f1);
-    const int q2 = weight_code(wv.z, s_new, qmax, grid, f2), q3 = weight_code(wv.w, s_new, qmax, grid, f3);
+    const int q0 = weight_code(wv.x, s_new, r_new, qmax, grid, f0), q1 = weight_code(wv.y, s_new, r_new, qmax, grid, f1);
+    const int q2 = weight_code(wv.z, s_new, r_new, qmax, grid, f2), q3 = weight_code(wv.w, s_new, r_new, qmax, grid, f3);
     *reinterpret_cast<uint32_t*>(codes + base + 4 * c) =
         (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) | ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
     if (what) store_what4<T>(what + base + 4 * c, sc_new * f0, sc_new * f1, sc_new * f2, sc_new * f3);
@@ -191,10 +194,12 @@ void launch_fused_weight_update(float* w, const float* g, float* m, float* v, fl
                                 int train_w, int train_s, int8_t* codes, int32_t* rowsum, float* scale, void* what,
                                 int dt, cudaStream_t st) {
   Scope scope("fused_weight_update", (double)rows * cols * (29.0 + (what ? (dt == 1 ? 2.0 : 4.0) : 0.0)), 0, st);
-#define MREM_FWU(T, NV, NT) launch_k(fused_weight_update_kernel<T, NV, NT>, rows, NT, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, grid, train_w, train_s, codes, rowsum, scale, (T*)what)
+#define MREM_FWU_G(T, NV, NT, G) launch_k(fused_weight_update_kernel<T, NV, NT, G>, rows, NT, 0, st, w, g, m, v, steps, ds_in, m_s, v_s, sc, cols, bits, train_w, train_s, codes, rowsum, scale, (T*)what)
+#define MREM_FWU(T, NV, NT) do { if (grid == 0) MREM_FWU_G(T, NV, NT, 0); else MREM_FWU_G(T, NV, NT, 1); } while (0)
   if (dt == 1) { if (cols <= 1024) MREM_FWU(bf16, 1, 256); else MREM_FWU(bf16, 2, 512); }
   else { if (cols <= 1024) MREM_FWU(float, 1, 256); else MREM_FWU(float, 2, 512); }
 #undef MREM_FWU
+#undef MREM_FWU_G
 }
 
 }  // namespace mrem
