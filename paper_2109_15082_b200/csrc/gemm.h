@@ -26,8 +26,11 @@ int tc_gemm_group(const GemmGroupItem* items, int n, int* d_status, int sm_count
 
 // 4-D TMA tensor map (128-byte swizzle) of an operand: (contiguous index, strided index, batch0, batch1).
 // K-major operands get boxes of block_k x tile_mn elements, MN-major ones 64 x block_k.
+// With `chunked` given, an MN-major 16-bit operand whose MN extent is a multiple of 64 gets a 5-D map instead
+// (64 contiguous elements, k, 64-element chunk index, batch0, batch1) whose box holds ALL 64 x block_k pieces of a tile, so
+// that one TMA instruction loads what otherwise takes tile_mn / 64 of them (same shared-memory layout); *chunked says which.
 int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,
-                     int tile_mn, int block_k);
+                     int tile_mn, int block_k, int* chunked = nullptr);
 
 // Plain fp32 SIMT path, used when activations are stored in float32 (small correctness
 // configurations); same operand and epilogue conventions, no alignment requirements.

@@ -77,6 +77,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int k0 = kb * p.block_k;
       if (!p.b_mn) {
         tma_load_4d(sb, &map_b, bar, k0, t.n0, t.b0, t.b1);
+      } else if (p.b_mn == 2) {
+        tma_load_5d(sb, &map_b, bar, 0, k0, t.n0 >> 6, t.b0, t.b1);
       } else {
         for (int j = 0; j < p.block_n / 64; ++j) tma_load_4d(sb + j * 8192, &map_b, bar, t.n0 + 64 * j, k0, t.b0, t.b1);
       }
@@ -107,12 +109,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int k0 = kb * p.block_k;
           if (!p.a_mn) {
             tma_load_4d(sa, &map_a, bar, k0, t.m0, t.b0, t.b1);
+          } else if (p.a_mn == 2) {
+            tma_load_5d(sa, &map_a, bar, 0, k0, t.m0 >> 6, t.b0, t.b1);
           } else {
             for (int j = 0; j < BLOCK_M / 64; ++j) tma_load_4d(sa + j * 8192, &map_a, bar, t.m0 + 64 * j, k0, t.b0, t.b1);
           }
           if (b_done) {
           } else if (!p.b_mn) {
             tma_load_4d(sb, &map_b, bar, k0, t.n0, t.b0, t.b1);
+          } else if (p.b_mn == 2) {
+            tma_load_5d(sb, &map_b, bar, 0, k0, t.n0 >> 6, t.b0, t.b1);
           } else {
             for (int j = 0; j < p.block_n / 64; ++j) tma_load_4d(sb + j * 8192, &map_b, bar, t.n0 + 64 * j, k0, t.b0, t.b1);
           }
@@ -258,9 +264,28 @@ EncodeTiledFn encode_fn() {
 
 // Tensor map of one operand: 4-D (contiguous index, strided index, batch0, batch1).
 int make_operand_map(CUtensorMap* map, const OperandDesc& op, int elem_bytes, int mn_extent, int K, int nb0, int nb1,
-             int tile_mn, int block_k) {
+             int tile_mn, int block_k, int* chunked) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return GEMM_ERR_CUDA;
+  if (chunked) *chunked = 0;
+  if (chunked && op.mn_contig && elem_bytes == 2 && mn_extent % 64 == 0 && tile_mn % 64 == 0) {
+    // (64 contiguous, k rows, chunk of 64, batch0, batch1): one box = every 64-wide piece of the tile, piece after piece
+    const cuuint64_t s1 = (cuuint64_t)op.ld * 2, rows = (cuuint64_t)K;
+    const cuuint64_t s3 = nb0 > 1 ? (cuuint64_t)op.s_b0 * 2 : s1 * rows;
+    const cuuint64_t s4 = nb1 > 1 ? (cuuint64_t)op.s_b1 * 2 : s3 * (cuuint64_t)nb0;
+    if ((reinterpret_cast<uintptr_t>(op.ptr) & 15) || (s1 & 15) || (s3 & 15) || (s4 & 15)) return GEMM_ERR_ALIGN;
+    if (s1 < (cuuint64_t)mn_extent * 2) return GEMM_ERR_ARG;
+    cuuint64_t dims[5] = {64, rows, (cuuint64_t)(mn_extent / 64), (cuuint64_t)nb0, (cuuint64_t)nb1};
+    cuuint64_t strides[4] = {s1, 128, s3, s4};
+    cuuint32_t box[5] = {64, (cuuint32_t)block_k, (cuuint32_t)(tile_mn / 64), 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(op.ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return GEMM_ERR_CUDA;
+    *chunked = 1;
+    return GEMM_OK;
+  }
   const cuuint64_t inner = op.mn_contig ? (cuuint64_t)mn_extent : (cuuint64_t)K;
   const cuuint64_t rows = op.mn_contig ? (cuuint64_t)K : (cuuint64_t)mn_extent;
   cuuint64_t dims[4] = {inner, rows, (cuuint64_t)nb0, (cuuint64_t)nb1};
@@ -351,10 +376,13 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   p.idesc = idesc;
 
   CUtensorMap ma, mb;
-  int rc = make_operand_map(&ma, A, es, g.M, g.K, g.nb0, g.nb1, BLOCK_M, p.block_k);
+  int a_chunked = 0, b_chunked = 0;           // MN-major operands: one 5-D load per stage where the extent allows it
+  int rc = make_operand_map(&ma, A, es, g.M, g.K, g.nb0, g.nb1, BLOCK_M, p.block_k, &a_chunked);
   if (rc != GEMM_OK) return rc;
-  rc = make_operand_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k);
+  rc = make_operand_map(&mb, B, es, g.N, g.K, g.nb0, g.nb1, p.block_n, p.block_k, &b_chunked);
   if (rc != GEMM_OK) return rc;
+  if (a_chunked) p.a_mn = 2;
+  if (b_chunked) p.b_mn = 2;
 
   const int smem = p.num_stages * p.stage_bytes + 1024;
   typedef void (*Kern)(const CUtensorMap, const CUtensorMap, const TcParams);

@@ -99,11 +99,15 @@ tc_gemm_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_consta
           const int k0 = kb * p.block_k;
           if (!p.a_mn) {
             tma_load_4d(sa, map_a, bar, k0, t.m0, t.b0, t.b1);
+          } else if (p.a_mn == 2) {
+            tma_load_5d(sa, map_a, bar, 0, k0, t.m0 >> 6, t.b0, t.b1);
           } else {
             for (int j = 0; j < BLOCK_M / 64; ++j) tma_load_4d(sa + j * 8192, map_a, bar, t.m0 + 64 * j, k0, t.b0, t.b1);
           }
           if (!p.b_mn) {
             tma_load_4d(sb, map_b, bar, k0, t.n0, t.b0, t.b1);
+          } else if (p.b_mn == 2) {
+            tma_load_5d(sb, map_b, bar, 0, k0, t.n0 >> 6, t.b0, t.b1);
           } else {
             for (int j = 0; j < p.block_n / 64; ++j) tma_load_4d(sb + j * 8192, map_b, bar, t.n0 + 64 * j, k0, t.b0, t.b1);
           }
@@ -247,10 +251,13 @@ int tc_gemm_group(const GemmGroupItem* items, int n, int* d_status, int sm_count
     p.wait_ns = g_wait_limit_ns;
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(it.A.mn_contig ? 1 : 0) << 15) |
               ((uint32_t)(it.B.mn_contig ? 1 : 0) << 16) | ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
-    int rc = make_operand_map(&maps.a[i], it.A, 2, p.M, p.K, 1, 1, BLOCK_M, block_k);
+    int a_chunked = 0, b_chunked = 0;         // MN-major operands: one 5-D load per stage where the extent allows it
+    int rc = make_operand_map(&maps.a[i], it.A, 2, p.M, p.K, 1, 1, BLOCK_M, block_k, &a_chunked);
     if (rc != GEMM_OK) return rc;
-    rc = make_operand_map(&maps.b[i], it.B, 2, p.N, p.K, 1, 1, block_n, block_k);
+    rc = make_operand_map(&maps.b[i], it.B, 2, p.N, p.K, 1, 1, block_n, block_k, &b_chunked);
     if (rc != GEMM_OK) return rc;
+    if (a_chunked) p.a_mn = 2;
+    if (b_chunked) p.b_mn = 2;
     if (i < n) {
       tiles += p.num_tiles;
       flops += 2.0 * p.M * p.N * (double)p.K;

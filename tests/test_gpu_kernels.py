@@ -184,11 +184,14 @@ def test_gemm_float_layouts(dtype, a_mn, b_mn, M, N, K, nb):
     assert rel < 2e-6, rel
 
 
-@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1)])
-def test_gemm_bf16_on_integer_codes_is_exact(a_mn, b_mn):
-    # attention products run on codes held as bf16 numbers: sums stay below 2^24, so fp32 accumulation is exact
+@pytest.mark.parametrize("shape", [(128, 64, 384, 2), (320, 576, 208, 1), (4096, 1024, 128, 1)])
+@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 0), (1, 1)])
+def test_gemm_bf16_on_integer_codes_is_exact(a_mn, b_mn, shape):
+    # attention products run on codes held as bf16 numbers: sums stay below 2^24, so fp32 accumulation is exact.
+    # Extents that are multiples of 64 take the one-load-per-stage form of the m- / n-contiguous operands (a ragged last
+    # tile of 64 in the second shape, many tiles per CTA in the third); every element is checked bit for bit
     rng = np.random.default_rng(11)
-    M, N, K, nb = 128, 64, 384, 2
+    M, N, K, nb = shape
     a = rng.integers(0, 256, (nb, M, K)).astype(np.float32)
     b = rng.integers(-127, 128, (nb, N, K)).astype(np.float32)
     ad = torch.from_numpy(_layout(a, a_mn)).to(DEV).to(torch.bfloat16)
