@@ -10,7 +10,8 @@ namespace tc {
 
 constexpr int BLOCK_M = 128;
 constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
-constexpr int SINGLE_CTA_SMEM_BUDGET = 229376;        // bytes of operand stages per CTA
+constexpr int SINGLE_CTA_SMEM_BUDGET = 221184;        // bytes of operand stages per CTA (the rest: barriers, column terms)
+constexpr int COLVEC = 128;                           // columns one epilogue warp drains per tile, at most
 constexpr int MAX_STAGES = 8;
 constexpr int GEMM_THREADS = 320;                    // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_WARPS = 8;
@@ -158,10 +159,12 @@ __device__ __forceinline__ void fetch_res_bf16(const Epilogue& e, long long off,
   }
 }
 
-// acc[32] of one row -> out[off .. off + 32).  `n` = global column of acc[0].
+// acc[32] of one row -> out[off .. off + 32).  `cv` = the chunk's column terms in shared memory: cv[j] = alpha *
+// col_scale of column j of the chunk, cv[COLVEC + j] = its col_bias (staged by the warp before it waited for the
+// accumulator; every lane reads the same address, one broadcast per load).
 template <int KIND, int OUT, int MODE>
 __device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* r, const uint32_t* res, float alpha, float rb,
-                                             int n, long long off, bool row_ok) {
+                                             const float* cv, long long off, bool row_ok) {
   if (OUT == OUT_I32) {
     if (row_ok) {
       int* out = reinterpret_cast<int*>(e.out) + off;
@@ -175,12 +178,9 @@ __device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* 
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
     float4 sc = make_float4(alpha, alpha, alpha, alpha), bi = make_float4(rb, rb, rb, rb);
-    if (f.scale) {
-      const float4 t = __ldg(reinterpret_cast<const float4*>(e.col_scale + n + j));
-      sc.x *= t.x; sc.y *= t.y; sc.z *= t.z; sc.w *= t.w;
-    }
+    if (f.scale) sc = *reinterpret_cast<const float4*>(cv + j);
     if (f.bias) {
-      const float4 t = __ldg(reinterpret_cast<const float4*>(e.col_bias + n + j));
+      const float4 t = *reinterpret_cast<const float4*>(cv + COLVEC + j);
       bi.x += t.x; bi.y += t.y; bi.z += t.z; bi.w += t.w;
     }
     const float a0 = (KIND == 1) ? (float)(int)r[j] : __uint_as_float(r[j]);
@@ -241,12 +241,12 @@ __device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* 
   }
 }
 
-// `nchunks` whole chunks starting at accumulator column c0 (tile-relative) / global column n0 + c0.
+// `nchunks` whole chunks starting at accumulator column c0 (tile-relative); `cv` = column terms of the first.
 // `res0` holds the residual of the first chunk (bf16 output with residual only), fetched by the caller
 // before it waited for the accumulator.
 template <int KIND, int OUT, int MODE>
-__device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb, int n,
-                                             long long off, bool row_ok, uint32_t* res0) {
+__device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb,
+                                             const float* cv, long long off, bool row_ok, uint32_t* res0) {
   const bool pipelined_res = OUT == OUT_BF16 && EpiFlags<MODE>(e).res;
   uint32_t ra[32], rb2[32], res1[16];
   tmem_ld32_issue(taddr, ra);
@@ -258,7 +258,7 @@ __device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, 
       tmem_ld32_issue(taddr + 32u * (uint32_t)(c + 1), rb2);
       if (pipelined_res) fetch_res_bf16(e, off + 32 * (c + 1), row_ok, res1);
     }
-    finish_chunk<KIND, OUT, MODE>(e, ra, res0, alpha, rb, n + 32 * c, off + 32 * c, row_ok);
+    finish_chunk<KIND, OUT, MODE>(e, ra, res0, alpha, rb, cv + 32 * c, off + 32 * c, row_ok);
     if (more1) {
       tmem_ld_wait();
       tmem_ld_pin(rb2);
@@ -266,24 +266,43 @@ __device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, 
         tmem_ld32_issue(taddr + 32u * (uint32_t)(c + 2), ra);
         if (pipelined_res) fetch_res_bf16(e, off + 32 * (c + 2), row_ok, res0);
       }
-      finish_chunk<KIND, OUT, MODE>(e, rb2, res1, alpha, rb, n + 32 * (c + 1), off + 32 * (c + 1), row_ok);
+      finish_chunk<KIND, OUT, MODE>(e, rb2, res1, alpha, rb, cv + 32 * (c + 1), off + 32 * (c + 1), row_ok);
     }
   }
+}
+
+// One warp stages the column terms of its `ncols` (<= COLVEC) columns from global column n on: 4 per lane, alpha
+// folded into the scale.  Columns at or beyond N are left alone (no whole chunk reaches them).
+template <int MODE>
+__device__ __forceinline__ void stage_col_terms(const Epilogue& e, float* cv, float alpha, int n, int ncols, int N, int lane) {
+  const EpiFlags<MODE> f(e);
+  if (!f.scale && !f.bias) return;
+  __syncwarp();                                   // the previous tile's reads of cv are done
+  const int c = 4 * lane;
+  if (c < ncols && n + c + 3 < N) {
+    if (f.scale) {
+      float4 t = __ldg(reinterpret_cast<const float4*>(e.col_scale + n + c));
+      t.x *= alpha; t.y *= alpha; t.z *= alpha; t.w *= alpha;
+      *reinterpret_cast<float4*>(cv + c) = t;
+    }
+    if (f.bias) *reinterpret_cast<float4*>(cv + COLVEC + c) = __ldg(reinterpret_cast<const float4*>(e.col_bias + n + c));
+  }
+  __syncwarp();
 }
 
 // MODE >= 0: bf16 output (fp32 with bit 4) with the epilogue terms of MODE; MODE < 0: output kind and terms read
 // at run time.
 template <int KIND, int MODE>
-__device__ __forceinline__ void drain_dispatch(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb, int n,
-                                               long long off, bool row_ok, uint32_t* res0) {
+__device__ __forceinline__ void drain_dispatch(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb,
+                                               const float* cv, long long off, bool row_ok, uint32_t* res0) {
   if (MODE >= 16) {
-    drain_chunks<KIND, OUT_F32, MODE>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+    drain_chunks<KIND, OUT_F32, MODE>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
   } else if (MODE >= 0 || e.out_kind == OUT_BF16) {
-    drain_chunks<KIND, OUT_BF16, MODE>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+    drain_chunks<KIND, OUT_BF16, MODE>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
   } else if (e.out_kind == OUT_F32) {
-    drain_chunks<KIND, OUT_F32, -1>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+    drain_chunks<KIND, OUT_F32, -1>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
   } else {
-    drain_chunks<KIND, OUT_I32, 0>(e, taddr, nchunks, alpha, rb, n, off, row_ok, res0);
+    drain_chunks<KIND, OUT_I32, 0>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
   }
 }
 

@@ -37,6 +37,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ __align__(8) uint64_t tempty_bar[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ __align__(16) float col_terms[EPI_WARPS][2 * COLVEC];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -199,6 +200,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t res0[16];
       if (nfull > 0 && res_bf16) fetch_res_bf16(e, row_off + col_begin, row_ok, res0);   // in flight during the wait
       const float rb = (e.row_bias && row_ok) ? e.row_bias[row] : 0.f;
+      float* cv = col_terms[warp - 2];
+      if (nfull > 0) stage_col_terms<MODE>(e, cv, alpha, col_begin, cols_per_warp, p.N, lane);   // before the wait as well
       // every lane polls; the decision is made warp-uniform before any .sync.aligned instruction
       const bool got = mbar_wait_or_abort(smem_u32(&tfull_bar[acc]), acc_phase, vabort, p.wait_ns);
       if (!__all_sync(0xffffffffu, got)) {
@@ -207,7 +210,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * p.block_n);
-      if (nfull > 0) drain_dispatch<KIND, MODE>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, col_begin, row_off + col_begin, row_ok, res0);
+      if (nfull > 0) drain_dispatch<KIND, MODE>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, cv, row_off + col_begin, row_ok, res0);
       for (int c = c_begin + 32 * nfull; c < c_begin + cols_per_warp && t.n0 + c < p.N; c += 32) {   // ragged or unaligned rest
         uint32_t r[32];
         tmem_ld32(taddr + (uint32_t)c, r);
