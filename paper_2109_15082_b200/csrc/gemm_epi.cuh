@@ -1,6 +1,6 @@
 // Shared pieces of the tensor-core GEMM kernels: launch parameters, tile decoding and the epilogue
-// (TMEM accumulators -> scale / bias / residual / activation -> global stores straight from registers,
-// every lane writing whole 32-byte sectors of its own row).
+// (TMEM accumulators -> scale / bias / residual / activation -> bf16 rows through a small shared-memory box and a
+// tiled store, or global stores straight from registers, every lane writing whole 32-byte sectors of its own row).
 #pragma once
 #include "gemm.h"
 #include "tc_ptx.cuh"
@@ -10,8 +10,10 @@ namespace tc {
 
 constexpr int BLOCK_M = 128;
 constexpr int A_STAGE_BYTES = BLOCK_M * 128;          // 128 rows x 128 B
-constexpr int SINGLE_CTA_SMEM_BUDGET = 221184;        // bytes of operand stages per CTA (the rest: barriers, column terms)
+constexpr int SINGLE_CTA_SMEM_BUDGET = 204800;        // bytes of operand stages per CTA (the rest: barriers, column terms,
+                                                      // output boxes)
 constexpr int COLVEC = 128;                           // columns one epilogue warp drains per tile, at most
+constexpr int OUT_BOX_BYTES = 2048;                   // per epilogue warp: 32 rows x 32 bf16 columns
 constexpr int MAX_STAGES = 8;
 constexpr int GEMM_THREADS = 320;                    // TMA warp, MMA warp, 8 epilogue warps
 constexpr int EPI_WARPS = 8;
@@ -23,6 +25,7 @@ struct TcParams {
   int block_n, block_k, num_stages, stage_bytes;
   int a_mn, b_mn;
   int b_static;                        // the B operand does not depend on the preceding kernel: prefetch its first tiles
+  int c_tma;                           // bf16 output written with tiled stores (a tensor map of C was built)
   uint32_t idesc;
   Epilogue epi;
   int* status;
@@ -141,6 +144,18 @@ __device__ __forceinline__ void stg256(void* p, const uint32_t* r) {
                : "memory");
 }
 
+// Where one epilogue warp's bf16 chunks go.  map == nullptr: st.global from registers.  Otherwise every lane writes
+// its 64 bytes into the warp's shared-memory box (32 rows x 64 bytes, 64-byte swizzle: 16-byte piece j of row r sits at
+// piece j ^ ((r >> 1) & 3), so a quarter-warp's 16-byte stores cover all banks) and lane 0 issues one tiled store of the
+// box; rows and columns outside C are clipped by the store.  The global stores of a lane-per-row layout touch 32
+// lines per instruction and hold up the memory pipe that the MMA and TMA warps issue through; the tiled store does not.
+struct StoreCtx {
+  const CUtensorMap* map;
+  uint32_t box;               // shared address of the warp's box (1024-byte aligned)
+  int row0, b0, b1;           // C row of lane 0, batch coordinates
+  int lane;
+};
+
 // MODE >= 0: bit 0 column scale, bit 1 column bias, bit 2 residual, bit 3 GELU, known at compile time;
 // MODE < 0: the same four read from the Epilogue at run time.
 template <int MODE> struct EpiFlags {
@@ -164,7 +179,7 @@ __device__ __forceinline__ void fetch_res_bf16(const Epilogue& e, long long off,
 // accumulator; every lane reads the same address, one broadcast per load).
 template <int KIND, int OUT, int MODE>
 __device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* r, const uint32_t* res, float alpha, float rb,
-                                             const float* cv, long long off, bool row_ok) {
+                                             const float* cv, long long off, bool row_ok, const StoreCtx& sx, int n) {
   if (OUT == OUT_I32) {
     if (row_ok) {
       int* out = reinterpret_cast<int*>(e.out) + off;
@@ -208,7 +223,19 @@ __device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* 
       const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
       o[j] = *reinterpret_cast<const uint32_t*>(&h);
     }
-    if (row_ok) {
+    if (sx.map) {
+      if (sx.lane == 0) tma_store_wait_read<0>();          // the box's previous store has read it
+      __syncwarp();
+      const uint32_t row_addr = sx.box + (uint32_t)sx.lane * 64u, sw = ((uint32_t)sx.lane >> 1) & 3u;
+#pragma unroll
+      for (uint32_t j = 0; j < 4; ++j) sts128(row_addr + ((j ^ sw) << 4), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+      fence_async_shared();
+      __syncwarp();
+      if (sx.lane == 0) {
+        tma_store_4d(sx.map, sx.box, n, sx.row0, sx.b0, sx.b1);
+        tma_store_commit();
+      }
+    } else if (row_ok) {
       bf16* out = reinterpret_cast<bf16*>(e.out) + off;
       stg256(out, o);
       stg256(out + 16, o + 8);
@@ -241,12 +268,14 @@ __device__ __forceinline__ void finish_chunk(const Epilogue& e, const uint32_t* 
   }
 }
 
-// `nchunks` whole chunks starting at accumulator column c0 (tile-relative); `cv` = column terms of the first.
+// `nchunks` whole chunks starting at accumulator column c0 (tile-relative) = global column n; `cv` = column terms of
+// the first.
 // `res0` holds the residual of the first chunk (bf16 output with residual only), fetched by the caller
 // before it waited for the accumulator.
 template <int KIND, int OUT, int MODE>
 __device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb,
-                                             const float* cv, long long off, bool row_ok, uint32_t* res0) {
+                                             const float* cv, long long off, bool row_ok, uint32_t* res0, const StoreCtx& sx,
+                                             int n) {
   const bool pipelined_res = OUT == OUT_BF16 && EpiFlags<MODE>(e).res;
   uint32_t ra[32], rb2[32], res1[16];
   tmem_ld32_issue(taddr, ra);
@@ -258,7 +287,7 @@ __device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, 
       tmem_ld32_issue(taddr + 32u * (uint32_t)(c + 1), rb2);
       if (pipelined_res) fetch_res_bf16(e, off + 32 * (c + 1), row_ok, res1);
     }
-    finish_chunk<KIND, OUT, MODE>(e, ra, res0, alpha, rb, cv + 32 * c, off + 32 * c, row_ok);
+    finish_chunk<KIND, OUT, MODE>(e, ra, res0, alpha, rb, cv + 32 * c, off + 32 * c, row_ok, sx, n + 32 * c);
     if (more1) {
       tmem_ld_wait();
       tmem_ld_pin(rb2);
@@ -266,7 +295,7 @@ __device__ __forceinline__ void drain_chunks(const Epilogue& e, uint32_t taddr, 
         tmem_ld32_issue(taddr + 32u * (uint32_t)(c + 2), ra);
         if (pipelined_res) fetch_res_bf16(e, off + 32 * (c + 2), row_ok, res0);
       }
-      finish_chunk<KIND, OUT, MODE>(e, rb2, res1, alpha, rb, cv + 32 * (c + 1), off + 32 * (c + 1), row_ok);
+      finish_chunk<KIND, OUT, MODE>(e, rb2, res1, alpha, rb, cv + 32 * (c + 1), off + 32 * (c + 1), row_ok, sx, n + 32 * (c + 1));
     }
   }
 }
@@ -294,15 +323,16 @@ __device__ __forceinline__ void stage_col_terms(const Epilogue& e, float* cv, fl
 // at run time.
 template <int KIND, int MODE>
 __device__ __forceinline__ void drain_dispatch(const Epilogue& e, uint32_t taddr, int nchunks, float alpha, float rb,
-                                               const float* cv, long long off, bool row_ok, uint32_t* res0) {
+                                               const float* cv, long long off, bool row_ok, uint32_t* res0,
+                                               const StoreCtx& sx, int n) {
   if (MODE >= 16) {
-    drain_chunks<KIND, OUT_F32, MODE>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
+    drain_chunks<KIND, OUT_F32, MODE>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0, sx, n);
   } else if (MODE >= 0 || e.out_kind == OUT_BF16) {
-    drain_chunks<KIND, OUT_BF16, MODE>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
+    drain_chunks<KIND, OUT_BF16, MODE>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0, sx, n);
   } else if (e.out_kind == OUT_F32) {
-    drain_chunks<KIND, OUT_F32, -1>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
+    drain_chunks<KIND, OUT_F32, -1>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0, sx, n);
   } else {
-    drain_chunks<KIND, OUT_I32, 0>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0);
+    drain_chunks<KIND, OUT_I32, 0>(e, taddr, nchunks, alpha, rb, cv, off, row_ok, res0, sx, n);
   }
 }
 

@@ -29,7 +29,7 @@ namespace {
 template <int KIND, int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ TcParams p) {
+               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
@@ -187,6 +187,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const bool direct = direct_epilogue_ok(e);
     const bool res_bf16 = e.residual != nullptr && e.out_kind == OUT_BF16;
     const int cols_per_warp = p.block_n >> 1, c_begin = half * cols_per_warp;
+    // bf16 rows leave through this warp's shared-memory box (behind the operand stages) and tiled stores
+    const bool boxed = direct && p.c_tma;
+    StoreCtx sx{boxed ? &map_c : nullptr, tiles_base + (uint32_t)(p.num_stages * p.stage_bytes) + (uint32_t)((warp - 2) * OUT_BOX_BYTES),
+                0, 0, 0, lane};
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
@@ -210,7 +214,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * p.block_n);
-      if (nfull > 0) drain_dispatch<KIND, MODE>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, cv, row_off + col_begin, row_ok, res0);
+      sx.row0 = t.m0 + quad * 32; sx.b0 = t.b0; sx.b1 = t.b1;
+      if (nfull > 0) drain_dispatch<KIND, MODE>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, cv, row_off + col_begin, row_ok, res0, sx, col_begin);
       for (int c = c_begin + 32 * nfull; c < c_begin + cols_per_warp && t.n0 + c < p.N; c += 32) {   // ragged or unaligned rest
         uint32_t r[32];
         tmem_ld32(taddr + (uint32_t)c, r);
@@ -222,6 +227,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    if (boxed && lane == 0) tma_store_wait_all();          // the boxes are read and written out before the CTA ends
   }
 
   tc_fence_before();
@@ -386,9 +392,25 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   if (rc != GEMM_OK) return rc;
   if (a_chunked) p.a_mn = 2;
   if (b_chunked) p.b_mn = 2;
+  // bf16 output whose rows and batches start on 16-byte boundaries: tiled stores of 32 x 32 boxes
+  CUtensorMap mc = ma;
+  p.c_tma = 0;
+  if (epi.out_kind == OUT_BF16 && (reinterpret_cast<uintptr_t>(epi.out) & 15) == 0 && epi.ldc % 8 == 0 && epi.ldc >= g.N &&
+      (g.nb0 == 1 || epi.c_b0 % 8 == 0) && (g.nb1 == 1 || epi.c_b1 % 8 == 0)) {
+    const cuuint64_t s1 = (cuuint64_t)epi.ldc * 2;
+    const cuuint64_t s2 = g.nb0 > 1 ? (cuuint64_t)epi.c_b0 * 2 : s1 * (cuuint64_t)g.M;
+    const cuuint64_t s3 = g.nb1 > 1 ? (cuuint64_t)epi.c_b1 * 2 : s2 * (cuuint64_t)g.nb0;
+    cuuint64_t dims[4] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.nb0, (cuuint64_t)g.nb1};
+    cuuint64_t strides[3] = {s1, s2, s3};
+    cuuint32_t box[4] = {32, 32, 1, 1}, estr[4] = {1, 1, 1, 1};
+    EncodeTiledFn fn = encode_fn();
+    if (fn && fn(&mc, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, epi.out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+      p.c_tma = 1;
+  }
 
-  const int smem = p.num_stages * p.stage_bytes + 1024;
-  typedef void (*Kern)(const CUtensorMap, const CUtensorMap, const TcParams);
+  const int smem = p.num_stages * p.stage_bytes + 1024 + EPI_WARPS * OUT_BOX_BYTES;
+  typedef void (*Kern)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcParams);
   static const struct { int kind, mode; Kern fn; } variants[] = {
       {0, -1, tc_gemm_kernel<0, -1>}, {0, 0, tc_gemm_kernel<0, 0>}, {0, 2, tc_gemm_kernel<0, 2>}, {0, 6, tc_gemm_kernel<0, 6>},
       {0, 10, tc_gemm_kernel<0, 10>}, {0, 16, tc_gemm_kernel<0, 16>}, {1, -1, tc_gemm_kernel<1, -1>}, {1, 3, tc_gemm_kernel<1, 3>}, {1, 7, tc_gemm_kernel<1, 7>}};
@@ -400,7 +422,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
   if (vi == n_variants) return GEMM_ERR_ARG;
   Kern kern = variants[vi].fn;
   if (!attr_set[vi]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SINGLE_CTA_SMEM_BUDGET + 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SINGLE_CTA_SMEM_BUDGET + 1024 + EPI_WARPS * OUT_BOX_BYTES) != cudaSuccess)
       return GEMM_ERR_CUDA;
     attr_set[vi] = true;
   }
@@ -411,7 +433,7 @@ int tc_gemm(int kind, int a_unsigned, const OperandDesc& A, const OperandDesc& B
              A.mn_contig ? "T" : "N", B.mn_contig ? "N" : "T", g.nb0 * g.nb1);
     return std::string(buf);
   }, 2.0 * g.M * g.N * (double)g.K * g.nb0 * g.nb1, 1, stream, 0);
-  if (launch_k(kern, grid, GEMM_THREADS, smem, stream, ma, mb, p) != cudaSuccess) return GEMM_ERR_CUDA;
+  if (launch_k(kern, grid, GEMM_THREADS, smem, stream, ma, mb, mc, p) != cudaSuccess) return GEMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? GEMM_OK : GEMM_ERR_CUDA;
 }
 

@@ -194,7 +194,8 @@ tc_gemm_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_consta
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * p.block_n);
       uint32_t res0[16];
-      if (nfull > 0) drain_dispatch<0, 16>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, nullptr, row_off + col_begin, row_ok, res0);
+      if (nfull > 0) drain_dispatch<0, 16>(e, taddr + (uint32_t)c_begin, nfull, alpha, rb, nullptr, row_off + col_begin, row_ok, res0,
+                                       StoreCtx{nullptr, 0u, 0, 0, 0, lane}, col_begin);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
