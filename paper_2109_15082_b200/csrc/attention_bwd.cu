@@ -16,6 +16,8 @@
 #include "kernels.h"
 #include "tc_ptx.cuh"
 
+#include <type_traits>
+
 namespace mrem {
 
 namespace {
@@ -72,10 +74,10 @@ __device__ __forceinline__ float ste_store(const uint32_t* a, bool row_ok, const
       const float2 xv = unpack2(xw[j]);
       const float g0 = scale * __uint_as_float(a[2 * j]), g1 = scale * __uint_as_float(a[2 * j + 1]);
       const float z0 = quotient(xv.x, step, r_step), z1 = quotient(xv.y, step, r_step);
-      const bool in0 = z0 >= lo && z0 <= hi, in1 = z1 >= lo && z1 <= hi;
-      const float q0 = rne_magic(fminf(fmaxf(z0, lo), hi));
-      const float q1 = rne_magic(fminf(fmaxf(z1, lo), hi));
-      acc += g0 * (q0 - (in0 ? z0 : 0.f)) + g1 * (q1 - (in1 ? z1 : 0.f));
+      const float c0 = fminf(fmaxf(z0, lo), hi), c1 = fminf(fmaxf(z1, lo), hi);
+      const bool in0 = c0 == z0, in1 = c1 == z1;              // inside the code range
+      const float q0 = rne_magic(c0), q1 = rne_magic(c1);
+      acc += g0 * (in0 ? q0 - z0 : q0) + g1 * (in1 ? q1 - z1 : q1);
       ow[j] = pack2(in0 ? g0 : 0.f, in1 ? g1 : 0.f);
     }
 #pragma unroll
@@ -186,24 +188,29 @@ __global__ void __launch_bounds__(ATB_THREADS, 2) attention_bwd_kernel(const __g
           if (t * 8 < ncol) ld16(p.P + prow + c * 32 + t * 8, pw + 4 * t);
           else { pw[4 * t] = pw[4 * t + 1] = pw[4 * t + 2] = pw[4 * t + 3] = 0u; }
         }
+        // FULL: every lane's 32 keys lie inside the sequence (the common case), no per-element bounds
+        auto chunk = [&](auto full_tag) {
+          constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float2 pv = unpack2(pw[j]);
-          float d0 = s_v * __uint_as_float(a[2 * j]), d1 = s_v * __uint_as_float(a[2 * j + 1]);
-          const float z0 = quotient(pv.x, s_p, r_p), z1 = quotient(pv.y, s_p, r_p);
-          const bool in0 = z0 >= p.p_lo && z0 <= p.p_hi, in1 = z1 >= p.p_lo && z1 <= p.p_hi;
-          const float q0 = rne_magic(fminf(fmaxf(z0, p.p_lo), p.p_hi));
-          const float q1 = rne_magic(fminf(fmaxf(z1, p.p_lo), p.p_hi));
-          const bool v0 = 2 * j < ncol, v1 = 2 * j + 1 < ncol;      // inside the sequence (row and key)
-          if (v0) ds_p += d0 * (q0 - (in0 ? z0 : 0.f));
-          if (v1) ds_p += d1 * (q1 - (in1 ? z1 : 0.f));
-          d0 = (in0 && v0) ? d0 : 0.f;
-          d1 = (in1 && v1) ? d1 : 0.f;
-          dot += d0 * pv.x + d1 * pv.y;
-          a[2 * j] = __float_as_uint(d0);
-          a[2 * j + 1] = __float_as_uint(d1);
-          cw[j] = pack2(v0 ? q0 : 0.f, v1 ? q1 : 0.f);
-        }
+          for (int j = 0; j < 16; ++j) {
+            const float2 pv = unpack2(pw[j]);
+            float d0 = s_v * __uint_as_float(a[2 * j]), d1 = s_v * __uint_as_float(a[2 * j + 1]);
+            const float z0 = quotient(pv.x, s_p, r_p), z1 = quotient(pv.y, s_p, r_p);
+            const float c0 = fminf(fmaxf(z0, p.p_lo), p.p_hi), c1 = fminf(fmaxf(z1, p.p_lo), p.p_hi);
+            const bool in0 = c0 == z0, in1 = c1 == z1;            // inside the code range
+            const float q0 = rne_magic(c0), q1 = rne_magic(c1);
+            const bool v0 = FULL || 2 * j < ncol, v1 = FULL || 2 * j + 1 < ncol;      // inside the sequence (row and key)
+            if (v0) ds_p += d0 * (in0 ? q0 - z0 : q0);
+            if (v1) ds_p += d1 * (in1 ? q1 - z1 : q1);
+            d0 = (in0 && v0) ? d0 : 0.f;
+            d1 = (in1 && v1) ? d1 : 0.f;
+            dot += d0 * pv.x + d1 * pv.y;
+            a[2 * j] = __float_as_uint(d0);
+            a[2 * j + 1] = __float_as_uint(d1);
+            cw[j] = pack2(v0 ? q0 : 0.f, v1 ? q1 : 0.f);
+          }
+        };
+        if (__all_sync(0xffffffffu, ncol >= 32)) chunk(std::true_type{}); else chunk(std::false_type{});
         tmem_st32(trow + TMEM_DP + (uint32_t)(c * 32), a);        // masked dP kept in place for pass B
       } else {
 #pragma unroll

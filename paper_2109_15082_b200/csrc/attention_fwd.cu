@@ -145,9 +145,14 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     for (int c = half; c < n_chunks; c += 2) {
       uint32_t a[32];
       tmem_ld32(trow + (uint32_t)(c * 32), a);
+      if (c * 32 + 32 <= len) {                          // all 32 keys valid (warp-uniform)
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (c * 32 + j < len) mx = fmaxf(mx, __uint_as_float(a[j]));
+        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(a[j]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (c * 32 + j < len) mx = fmaxf(mx, __uint_as_float(a[j]));
+      }
     }
     red[0][half][r] = mx;
     asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -156,11 +161,20 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_fwd_kernel(const __grid
     for (int c = half; c < n_chunks; c += 2) {            // exp once: kept in TMEM in place of the score
       uint32_t a[32];
       tmem_ld32(trow + (uint32_t)(c * 32), a);
+      if (c * 32 + 32 <= len) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float e = c * 32 + j < len ? exp2_approx(fmaf(alpha2, __uint_as_float(a[j]), -mx2)) : 0.f;
-        sum += e;
-        a[j] = __float_as_uint(e);
+        for (int j = 0; j < 32; ++j) {
+          const float e = exp2_approx(fmaf(alpha2, __uint_as_float(a[j]), -mx2));
+          sum += e;
+          a[j] = __float_as_uint(e);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float e = c * 32 + j < len ? exp2_approx(fmaf(alpha2, __uint_as_float(a[j]), -mx2)) : 0.f;
+          sum += e;
+          a[j] = __float_as_uint(e);
+        }
       }
       tmem_st32(trow + (uint32_t)(c * 32), a);
     }

@@ -137,16 +137,16 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const T* __restrict__ u, 
     load_vec<T, V>(dghat + i, d);
 #pragma unroll
     for (int j = 0; j < V; ++j) {
-      float cdf, pdf;
-      gelu_parts(uv[j], cdf, pdf);
+      float tail, ex;
+      gelu_parts(uv[j], tail, ex);
       if (quantized) {
-        const float z = qz(stored<T>(uv[j] * cdf), s, r_s, off, has_off);
+        const float z = qz(stored<T>(gelu_from_tail(uv[j], tail)), s, r_s, off, has_off);
         const bool in = z >= lo && z <= hi;
         ds += d[j] * (rne_magic(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
         dofs += in ? 0.f : d[j];
         d[j] = in ? d[j] : 0.f;
       }
-      d[j] *= fmaf(uv[j], pdf, cdf);
+      d[j] *= gelu_grad_from_parts(uv[j], tail, ex);
     }
     store_vec<T, V>(du + i, d);
   }
@@ -200,16 +200,16 @@ __global__ void __launch_bounds__(256) gelu_bwd_colsum_kernel(const T* __restric
       load_vec<T, V>(dghat + i, d);
 #pragma unroll
       for (int j = 0; j < V; ++j) {
-        float cdf, pdf;
-        gelu_parts(uv[j], cdf, pdf);
+        float tail, ex;
+        gelu_parts(uv[j], tail, ex);
         if (quantized) {
-          const float z = qz(stored<T>(uv[j] * cdf), s, r_s, off, has_off);
+          const float z = qz(stored<T>(gelu_from_tail(uv[j], tail)), s, r_s, off, has_off);
           const bool in = z >= lo && z <= hi;
           ds += d[j] * (rne_magic(fminf(fmaxf(z, lo), hi)) - (in ? z : 0.f));
           dofs += in ? 0.f : d[j];
           d[j] = in ? d[j] : 0.f;
         }
-        d[j] *= fmaf(uv[j], pdf, cdf);
+        d[j] *= gelu_grad_from_parts(uv[j], tail, ex);
         acc[j] += d[j];
       }
       store_vec<T, V>(du + i, d);

@@ -173,27 +173,34 @@ __device__ __forceinline__ uint32_t pack_low_bytes(uint32_t b0, uint32_t b1, uin
 // GELU(u) = u * Phi(u) with the erf form.  erf(x) = 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x), x >= 0
 // (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7, below half a float32 ulp of 1 + erf for u > 0): one
 // exponential serves both erf and the density needed by the derivative.
-__device__ __forceinline__ void gelu_parts(float u, float& cdf, float& pdf_scaled) {
-  const float x = fabsf(u) * 0.70710678118654752f;
-  const float ex = __expf(-x * x);                          // exp(-u^2 / 2)
-  const float t = rcp_approx(fmaf(0.3275911f, x, 1.f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float tail = 0.5f * poly * t * ex;                  // (1 - erf(x)) / 2
-  cdf = u >= 0.f ? 1.f - tail : tail;
-  pdf_scaled = ex * 0.39894228040143268f;                   // exp(-u^2/2) / sqrt(2 pi)
+//   tail = (1 - erf(|u| / sqrt 2)) / 2 = Phi(-|u|)   (the coefficients below are a_i / 2),   ex = exp(-u^2 / 2)
+__device__ __forceinline__ void gelu_parts(float u, float& tail, float& ex) {
+  const float au = fabsf(u);
+  ex = exp2_approx(u * u * -0.72134752044448170f);          // -log2(e) / 2
+  const float t = rcp_approx(fmaf(0.23164189f, au, 1.f));    // p / sqrt 2
+  float poly = fmaf(0.5307027145f, t, -0.7265760135f);
+  poly = fmaf(poly, t, 0.7107068705f);
+  poly = fmaf(poly, t, -0.142248368f);
+  poly = fmaf(poly, t, 0.127414796f);
+  tail = poly * t * ex;
 }
+// u * Phi(u) = max(u, 0) - |u| * Phi(-|u|): the value both the forward pass and the backward pass (which re-forms it
+// for the quantizer's mask) compute, bit for bit
+__device__ __forceinline__ float gelu_from_tail(float u, float tail) { return fmaf(-fabsf(u), tail, fmaxf(u, 0.f)); }
 __device__ __forceinline__ float gelu_erf(float u) {
-  float cdf, pdf;
-  gelu_parts(u, cdf, pdf);
-  return u * cdf;
+  float tail, ex;
+  gelu_parts(u, tail, ex);
+  return gelu_from_tail(u, tail);
+}
+// d/du (u Phi(u)) = Phi(u) + u phi(u)
+__device__ __forceinline__ float gelu_grad_from_parts(float u, float tail, float ex) {
+  const float cdf = u >= 0.f ? 1.f - tail : tail;
+  return fmaf(u, ex * 0.39894228040143268f, cdf);             // exp(-u^2/2) / sqrt(2 pi)
 }
 __device__ __forceinline__ float gelu_erf_grad(float u) {
-  float cdf, pdf;
-  gelu_parts(u, cdf, pdf);
-  return fmaf(u, pdf, cdf);
+  float tail, ex;
+  gelu_parts(u, tail, ex);
+  return gelu_grad_from_parts(u, tail, ex);
 }
 
 // ---------------------------------------------------------------- GEMM interface (both back ends)
