@@ -127,12 +127,13 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, const uint32_t
   }
 }
 
-// ------------------------------------------------------------------ register-direct epilogue
+// ------------------------------------------------------------------ epilogue of whole 32-column chunks
 // One warp drains its 32 accumulator rows (TMEM lane = row = lane of the warp) over a range of columns in
-// chunks of 32: tcgen05.ld gives every lane 32 consecutive columns of its row, the lane applies the
-// epilogue and writes its 64 (bf16) or 128 (fp32 / int32) contiguous bytes with 32-byte vector stores, so
-// every store fills whole sectors and nothing passes through shared memory (whose bandwidth the main loop
-// needs).  The load of chunk c + 1 and the fetch of its residual are in flight while chunk c is processed.
+// chunks of 32: tcgen05.ld gives every lane 32 consecutive columns of its row and the lane applies the
+// epilogue.  fp32 / int32 rows (128 contiguous bytes per lane) and bf16 rows without a tensor map of C are written
+// with 32-byte vector stores that fill whole sectors; bf16 rows otherwise go through the warp's shared-memory box
+// and a tiled store (StoreCtx).  The load of chunk c + 1 and the fetch of its residual are in flight while chunk c
+// is processed.
 __device__ __forceinline__ void ldg256(const void* p, uint32_t* r) {
   asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])

@@ -3,10 +3,11 @@
 // One persistent CTA per SM.  Warp 0 streams operand tiles into a ring of shared-memory
 // stages with TMA (128-byte swizzle), warp 1 issues tcgen05.mma (bf16 -> fp32, or
 // int8 -> int32 with exact accumulation) into one of two TMEM accumulator buffers, and
-// warps 2..9 drain the other buffer with tcgen05.ld, apply the epilogue and write their
-// rows straight from registers with 32-byte vector stores (nothing of the epilogue passes
-// through shared memory, whose bandwidth the main loop needs), so the epilogue of tile i
-// overlaps the main loop of tile i+1.
+// warps 2..9 drain the other buffer with tcgen05.ld, apply the epilogue (column scale and
+// bias staged in shared memory before the accumulator is ready) and write their rows: bf16
+// through a 2 KB shared-memory box per warp and tiled stores, anything else straight from
+// registers with 32-byte vector stores.  The epilogue of tile i overlaps the main loop of
+// tile i+1.
 // Either operand may be stored k-contiguous ("K-major") or m/n-contiguous ("MN-major");
 // the second form serves the backward products (dX = dY * W_hat, dW = dY^T * X_hat) and
 // the attention products without any transposed copy.
@@ -198,7 +199,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int row = t.m0 + quad * 32 + lane, col_begin = t.n0 + c_begin;
       const bool row_ok = row < p.M;
       const long long row_off = (long long)t.b0 * e.c_b0 + (long long)t.b1 * e.c_b1 + (long long)row * e.ldc;
-      // whole 32-column chunks of this warp's range that lie inside N take the register-direct path
+      // whole 32-column chunks of this warp's range that lie inside N take the vector path
       int nfull = 0;
       if (direct && col_begin < p.N) nfull = min((p.N - col_begin) >> 5, cols_per_warp >> 5);
       uint32_t res0[16];
